@@ -1,0 +1,236 @@
+"""CPU oracle for the per-token, per-FFN-layer path of "LLM in a flash" (arXiv 2312.11514).
+
+TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, deliberately unoptimised statement of
+what the method computes, in float64 over the fp16-stored values.  It shares no code with the
+CUDA library and is imported only by the tests, the smoke check and the benchmark's CPU
+baseline.  The product never calls it.
+
+Per decode step and per layer (paper Sections 3.1-3.3):
+
+1. low-rank predictor: scores = x.A.B + c, neuron i is *active* iff score_i > theta
+   (Section 3.1 "Anticipating ReLU Sparsity", Section 3.1 "The Sliding Window Technique":
+   an active neuron is one with a positive predictor output; Appendix B uses a sigmoid
+   threshold tau, which in the logit domain is theta = ln(tau / (1 - tau)));
+2. sliding window over the last k tokens: neurons not predicted active in any of the last k
+   tokens (the current one included) are deleted, newly needed ones are loaded
+   (Section 3.1 "The Sliding Window Technique");
+3. cache management (Section 3.3): rows to delete are overwritten by the last rows so the
+   used rows stay consecutive, new rows are stacked at the end
+   (rows num_used .. num_used + num_new);
+4. inference (Section 3.3 item 3): matrix[:, :d_model] is the up projection and
+   matrix[:, d_model:] transposed is the down projection of the cached neurons.
+
+Parity pins (tests marked "not gpu"): dense brute force for the FFN, pure-Python loops and
+rank-1 closed forms for the predictor, brute-force set history for the window protocol, and
+the numbers the paper prints for the cost model (tests/golden/).  The *order* of rows inside
+the cache is a convention the paper only draws in a figure: "parity unpinned" for the slot
+order itself (only its invariants are pinned); everything that depends on it (FFN output,
+cached set, bytes fetched) is order-independent and pinned.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+NEVER = -(2 ** 30)          # "never predicted active" stamp
+
+
+# --------------------------------------------------------------------------------------
+# Step 1: low-rank predictor (Section 3.1; Appendix B)
+# --------------------------------------------------------------------------------------
+def predictor_logits(x, A, B, c):
+    """scores[s][i] = sum_j (sum_m x[s][m] A[m][j]) B[j][i] + c[i], float64.
+
+    x: [S][d], A: [d][r], B: [r][F], c: [F].  Two bias-free linear maps with no
+    non-linearity between them, plus a per-neuron offset."""
+    x = np.asarray(x, dtype=np.float64)
+    z = x @ np.asarray(A, dtype=np.float64)              # [S][r]
+    return z @ np.asarray(B, dtype=np.float64) + np.asarray(c, dtype=np.float64)[None, :]
+
+
+def active_set(logits, theta):
+    """Ascending ids of the neurons whose score exceeds theta for at least one stream
+    (score == theta is inactive)."""
+    mask = (np.asarray(logits) > theta).any(axis=0)
+    return np.nonzero(mask)[0].astype(np.int32)
+
+
+def sigmoid_threshold_to_logit(tau):
+    """theta = ln(tau / (1 - tau)); tau = 0.5 is the "positive output" rule."""
+    return float(np.log(tau / (1.0 - tau)))
+
+
+# --------------------------------------------------------------------------------------
+# Steps 2-4: the preallocated neuron cache (Section 3.3)
+# --------------------------------------------------------------------------------------
+class CapacityError(Exception):
+    pass
+
+
+class NeuronCache:
+    """matrix / pointers / bias / num_used / last_k_active of Section 3.3.
+
+    ``last_k_active`` is kept as ``last_active[i]`` = the last step at which neuron i was
+    predicted active, so "still inside the window of k tokens" is last_active[i] > t - k."""
+
+    def __init__(self, d_model, d_ff, capacity, window_k):
+        self.d_model, self.d_ff, self.capacity, self.k = d_model, d_ff, capacity, window_k
+        self.matrix = np.zeros((capacity, 2 * d_model), dtype=np.float16)
+        self.pointers = np.full(capacity, -1, dtype=np.int32)
+        self.bias = np.zeros(capacity, dtype=np.float16)
+        self.slot_of = np.full(d_ff, -1, dtype=np.int32)
+        self.last_active = np.full(d_ff, NEVER, dtype=np.int32)
+        self.num_used = 0
+        self.t = 0
+        self.bytes_fetched = 0
+        self.rows_moved = 0
+
+    # -- delete + plan ------------------------------------------------------------------
+    def window_update(self, act):
+        """One window step for the ascending active list ``act``.  Deletes the neurons that
+        left the window (Section 3.3 item 1), and assigns rows to the ones to bring in
+        (item 2).  Returns the lists; the new rows' weights arrive with ``insert``."""
+        act = np.asarray(act, dtype=np.int32)
+        t, k, n = self.t, self.k, self.num_used
+        in_act = np.zeros(self.d_ff, dtype=bool)
+        in_act[act] = True
+
+        # what would be deleted / loaded, before anything is changed
+        evict_slots = [s for s in range(n)
+                       if not in_act[self.pointers[s]]
+                       and self.last_active[self.pointers[s]] <= t - k]
+        load_ids = [int(i) for i in act if self.slot_of[i] < 0]
+        n_new = n - len(evict_slots)
+        if n_new + len(load_ids) > self.capacity:
+            raise CapacityError(f"need {n_new + len(load_ids)} rows, have {self.capacity}")
+
+        self.last_active[act] = t
+        evict_ids = [int(self.pointers[s]) for s in evict_slots]
+
+        # Deleting: walk the freed rows in ascending order; the current last row replaces
+        # the freed one unless the last row is itself to be deleted, in which case it is
+        # simply dropped.
+        dead = np.zeros(self.capacity, dtype=bool)
+        dead[evict_slots] = True
+        move_src, move_dst = [], []
+        tail = n
+        for hole in evict_slots:
+            while tail > 0 and dead[tail - 1]:
+                tail -= 1                                   # drop deleted rows off the end
+            if hole >= tail:
+                break                                       # every remaining hole was dropped
+            tail -= 1                                       # last surviving row
+            self.matrix[hole] = self.matrix[tail]
+            self.bias[hole] = self.bias[tail]
+            self.pointers[hole] = self.pointers[tail]
+            self.slot_of[self.pointers[hole]] = hole
+            dead[hole] = False
+            move_src.append(tail)
+            move_dst.append(hole)
+        for i in evict_ids:
+            self.slot_of[i] = -1
+        self.pointers[n_new:n] = -1
+        self.num_used = n_new
+        self.rows_moved += len(move_src)
+
+        # Bringing in new neurons: rows num_used .. num_used + num_new, ascending neuron id.
+        load_slots = list(range(n_new, n_new + len(load_ids)))
+        for i, s in zip(load_ids, load_slots):
+            self.pointers[s] = i
+            self.slot_of[i] = s
+        self.num_used = n_new + len(load_ids)
+        self.t = t + 1
+
+        active_slots = self.slot_of[act].astype(np.int32)
+        hit_slots = active_slots[active_slots < n_new]
+        i32 = lambda v: np.asarray(v, dtype=np.int32)
+        return {
+            "evict_ids": i32(evict_ids), "move_src": i32(move_src), "move_dst": i32(move_dst),
+            "load_ids": i32(load_ids), "load_slots": i32(load_slots),
+            "active_slots": active_slots, "hit_slots": i32(hit_slots),
+            "num_used_before": n, "num_kept": n_new, "num_used": self.num_used,
+        }
+
+    # -- insert -------------------------------------------------------------------------
+    def insert(self, lists, bundles, bias_up):
+        """Copy the bundles of the newly needed neurons from the full store into their rows,
+        and their up-projection biases (resident scalars) into ``bias`` (Section 3.3 item 2)."""
+        for i, s in zip(lists["load_ids"], lists["load_slots"]):
+            self.matrix[s] = bundles[i]
+            self.bias[s] = bias_up[i]
+        self.bytes_fetched += len(lists["load_ids"]) * 2 * self.d_model * self.matrix.itemsize
+
+    def cached_ids(self):
+        return set(int(i) for i in self.pointers[: self.num_used])
+
+
+# --------------------------------------------------------------------------------------
+# Step 5: sparse FFN over the cached bundles (Section 3.3 item 3)
+# --------------------------------------------------------------------------------------
+def sparse_ffn(matrix, bias, slots, x, b_down=None):
+    """y[s] = b_down + sum_q relu(<matrix[slots[q], :d], x[s]> + bias[slots[q]]) * matrix[slots[q], d:]
+
+    matrix: [cap][2d] (fp16 values), bias: [cap], slots: row indices, x: [S][d].  float64."""
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[1]
+    rows = np.asarray(matrix)[np.asarray(slots, dtype=np.int64)].astype(np.float64)
+    up, down = rows[:, :d], rows[:, d:]
+    h = np.maximum(x @ up.T + np.asarray(bias, dtype=np.float64)[slots][None, :], 0.0)
+    y = h @ down
+    if b_down is not None:
+        y = y + np.asarray(b_down, dtype=np.float64)[None, :]
+    return y
+
+
+def decode_step(cache, x, A, B, c, theta, bundles, bias_up, b_down=None, whole_cache=False,
+                act=None):
+    """One layer, one token: predict -> window update -> insert -> FFN.  ``act`` overrides the
+    predicted active list (used to follow another implementation's borderline decisions).
+    ``whole_cache`` runs the FFN over every cached row (matrix[:num_used]) instead of only the
+    rows of the currently active neurons."""
+    logits = predictor_logits(x, A, B, c)
+    if act is None:
+        act = active_set(logits, theta)
+    lists = cache.window_update(act)
+    cache.insert(lists, bundles, bias_up)
+    slots = np.arange(cache.num_used) if whole_cache else lists["active_slots"]
+    y = sparse_ffn(cache.matrix, cache.bias, slots, x, b_down)
+    return logits, act, lists, y
+
+
+# --------------------------------------------------------------------------------------
+# The paper's latency / memory accounting (Section 3 intro, Table 1, Appendix C)
+# --------------------------------------------------------------------------------------
+def io_latency_ms(gigabytes, throughput_gb_per_s):
+    """I/O latency = data moved / achieved throughput (Table 1)."""
+    return 1000.0 * gigabytes / throughput_gb_per_s
+
+
+def chunk_bytes(d_model, num_bytes, bundled=True):
+    """Bytes per read: d_model * num_bytes for a lone row or column, doubled by bundling
+    (Section 3.2)."""
+    return (2 if bundled else 1) * d_model * num_bytes
+
+
+def dram_share_percent(fixed_percents, ffn_percent_of_model, ffn_fraction_resident):
+    """Share of the model kept in DRAM = always-resident parts + the cached part of the FFN
+    (Appendix C, per-model paragraphs)."""
+    return float(sum(fixed_percents) + ffn_fraction_resident * ffn_percent_of_model)
+
+
+def flash_to_dram_gb(model_gb, ffn_percent_of_model, fraction_of_ffn_per_token):
+    """Data loaded per token = model size * FFN share * fraction of FFN neurons needed."""
+    return model_gb * ffn_percent_of_model / 100.0 * fraction_of_ffn_per_token
+
+
+def predictor_weight_fraction(rank, d_model, d_ff, non_embedding_per_layer=None):
+    """Predictor parameters r*(d_model + d_ff) relative to a transformer layer's
+    4*d^2 (attention) + 2*d*d_ff (FFN) weights (Appendix B, overhead of predictors)."""
+    if non_embedding_per_layer is None:
+        non_embedding_per_layer = 4 * d_model * d_model + 2 * d_model * d_ff
+    return rank * (d_model + d_ff) / non_embedding_per_layer
+
+
+def kv_cache_fraction(context, d_model, n_layers, model_params):
+    """KV cache elements (context * 2 * d_model per layer) over model parameters
+    (Appendix C footnote)."""
+    return context * 2 * d_model * n_layers / model_params

@@ -1,0 +1,352 @@
+"""Pins for the CPU oracle: each part is checked against something other than itself —
+textbook definitions written as brute-force loops, closed forms, set-history brute force, and
+the numbers the paper prints."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import lif_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "cost_model_paper_values.txt")
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+# ------------------------------------------------------------------ predictor
+def test_predictor_matches_scalar_loops():
+    r = _rng(0)
+    S, d, k, F = 2, 7, 3, 11
+    x, A, B, c = r.normal(size=(S, d)), r.normal(size=(d, k)), r.normal(size=(k, F)), r.normal(size=F)
+    got = O.predictor_logits(x, A, B, c)
+    for s in range(S):
+        for i in range(F):
+            acc = 0.0
+            for j in range(k):
+                z = 0.0
+                for m in range(d):
+                    z += x[s, m] * A[m, j]
+                acc += z * B[j, i]
+            assert got[s, i] == pytest.approx(acc + c[i], rel=1e-12, abs=1e-12)
+
+
+def test_predictor_rank_one_closed_form():
+    # A = u (d x 1), B = v^T (1 x F): score_i = (x.u) v_i + c_i
+    r = _rng(1)
+    d, F = 13, 9
+    x, u, v, c = r.normal(size=(1, d)), r.normal(size=(d, 1)), r.normal(size=(1, F)), r.normal(size=F)
+    got = O.predictor_logits(x, u, v, c)[0]
+    want = float(x[0] @ u[:, 0]) * v[0] + c
+    np.testing.assert_allclose(got, want, rtol=1e-12)
+
+
+def test_predictor_identity_factors_select_coordinates():
+    # A = I, B = [I | 0]: score_i = x_i + c_i for i < d, c_i beyond — catches transposes.
+    d, F = 5, 8
+    x = np.arange(1.0, d + 1)[None, :]
+    B = np.zeros((d, F)); B[:, :d] = np.eye(d)
+    c = 10.0 * np.arange(F)
+    got = O.predictor_logits(x, np.eye(d), B, c)[0]
+    want = c.copy(); want[:d] += x[0]
+    np.testing.assert_array_equal(got, want)
+
+
+def test_active_set_strict_threshold_and_stream_union():
+    logits = np.array([[0.0, 1.0, -1.0, 0.5, 0.0],
+                       [0.5, -2.0, -1.0, 0.5, 0.0]])
+    np.testing.assert_array_equal(O.active_set(logits, 0.0), [0, 1, 3])      # == theta inactive
+    np.testing.assert_array_equal(O.active_set(logits[:1], 0.0), [1, 3])
+    np.testing.assert_array_equal(O.active_set(logits, 0.75), [1])
+    assert O.active_set(logits, np.inf).size == 0
+    assert O.active_set(logits, -np.inf).size == 5
+
+
+def test_sigmoid_threshold():
+    assert O.sigmoid_threshold_to_logit(0.5) == 0.0
+    for tau in (0.4, 0.7):                       # thresholds used in Appendix B
+        th = O.sigmoid_threshold_to_logit(tau)
+        assert 1.0 / (1.0 + math.exp(-th)) == pytest.approx(tau, rel=1e-12)
+
+
+# ------------------------------------------------------------------ sparse FFN
+def _dense_ffn_loops(W_up, b_up, W_down, x, b_down):
+    F, d = W_up.shape
+    y = [b_down[m] for m in range(d)]
+    for i in range(F):
+        pre = b_up[i]
+        for m in range(d):
+            pre += W_up[i, m] * x[m]
+        if pre > 0.0:
+            for m in range(d):
+                y[m] += pre * W_down[m, i]
+    return np.array(y)
+
+
+def _cache_from_dense(W_up, b_up, W_down, ids, cap=None):
+    F, d = W_up.shape
+    cap = cap or len(ids)
+    M = np.zeros((cap, 2 * d)); bias = np.zeros(cap)
+    for s, i in enumerate(ids):
+        M[s, :d] = W_up[i]; M[s, d:] = W_down[:, i]; bias[s] = b_up[i]
+    return M, bias
+
+
+def test_sparse_ffn_with_true_mask_equals_dense_ffn():
+    r = _rng(2)
+    F, d = 23, 6
+    W_up, W_down = r.normal(size=(F, d)), r.normal(size=(d, F))
+    b_up, b_down, x = r.normal(size=F), r.normal(size=d), r.normal(size=d)
+    dense = _dense_ffn_loops(W_up, b_up, W_down, x, b_down)
+    true_active = [i for i in range(F) if W_up[i] @ x + b_up[i] > 0]
+    assert 0 < len(true_active) < F
+    M, bias = _cache_from_dense(W_up, b_up, W_down, true_active)
+    got = O.sparse_ffn(M, bias, np.arange(len(true_active)), x[None, :], b_down)[0]
+    np.testing.assert_allclose(got, dense, rtol=1e-12, atol=1e-12)
+    # every neuron cached (theta = -inf): ReLU zeroes the rest, still the dense FFN
+    M, bias = _cache_from_dense(W_up, b_up, W_down, list(range(F)))
+    got = O.sparse_ffn(M, bias, np.arange(F), x[None, :], b_down)[0]
+    np.testing.assert_allclose(got, dense, rtol=1e-12, atol=1e-12)
+    # library form of the same textbook definition
+    lib = W_down @ np.maximum(W_up @ x + b_up, 0) + b_down
+    np.testing.assert_allclose(got, lib, rtol=1e-12, atol=1e-12)
+
+
+def test_sparse_ffn_row_order_and_empty_and_streams():
+    r = _rng(3)
+    F, d, S = 12, 5, 3
+    W_up, W_down = r.normal(size=(F, d)), r.normal(size=(d, F))
+    b_up, b_down, X = r.normal(size=F), r.normal(size=d), r.normal(size=(S, d))
+    ids = [7, 2, 9, 4]
+    M, bias = _cache_from_dense(W_up, b_up, W_down, ids, cap=6)
+    y0 = O.sparse_ffn(M, bias, [0, 1, 2, 3], X, b_down)
+    perm = [2, 0, 3, 1]                                    # Section 3.3 item 3: order-free
+    M2, bias2 = M.copy(), bias.copy()
+    M2[:4], bias2[:4] = M[perm], bias[perm]
+    np.testing.assert_allclose(O.sparse_ffn(M2, bias2, [0, 1, 2, 3], X, b_down), y0, rtol=1e-12)
+    np.testing.assert_allclose(O.sparse_ffn(M, bias, [3, 1, 0, 2], X, b_down), y0, rtol=1e-12)
+    # no active rows: only the down bias is left; without it, zeros
+    np.testing.assert_array_equal(O.sparse_ffn(M, bias, [], X, b_down), np.tile(b_down, (S, 1)))
+    np.testing.assert_array_equal(O.sparse_ffn(M, bias, [], X), np.zeros((S, d)))
+    # streams are independent rows
+    for s in range(S):
+        np.testing.assert_allclose(O.sparse_ffn(M, bias, [0, 1, 2, 3], X[s:s + 1], b_down)[0], y0[s],
+                                   rtol=1e-12)
+    # a subset of the slots is the dense FFN restricted to those neurons
+    sub = O.sparse_ffn(M, bias, [1, 3], X[:1], None)[0]
+    want = sum(max(W_up[i] @ X[0] + b_up[i], 0.0) * W_down[:, i] for i in (2, 4))
+    np.testing.assert_allclose(sub, want, rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------------ window protocol
+def _random_active_sets(F, T, rate, seed, sticky=0.6):
+    r = _rng(seed)
+    pop = np.clip(rate * np.exp(r.normal(size=F)), 0, 0.9)
+    prev = np.zeros(F, dtype=bool)
+    out = []
+    for _ in range(T):
+        cur = (r.random(F) < pop) | (prev & (r.random(F) < sticky * 0.5))
+        out.append(np.nonzero(cur)[0].astype(np.int32))
+        prev = cur
+    return out
+
+
+def _check_structure(cache):
+    n = cache.num_used
+    ptr = cache.pointers[:n]
+    assert len(set(ptr.tolist())) == n and (ptr >= 0).all()
+    for s in range(n):
+        assert cache.slot_of[ptr[s]] == s
+    assert (cache.slot_of >= 0).sum() == n
+    assert (cache.pointers[n:] == -1).all()
+
+
+@pytest.mark.parametrize("k", [1, 2, 5])
+def test_window_matches_set_history_brute_force(k):
+    F, d, T = 97, 4, 40
+    r = _rng(10 + k)
+    bundles = r.normal(size=(F, 2 * d)).astype(np.float16)
+    bias_up = r.normal(size=F).astype(np.float16)
+    sets = _random_active_sets(F, T, 0.08, seed=k)
+    cache = O.NeuronCache(d, F, capacity=F, window_k=k)
+    total_loaded = 0
+    for t, act in enumerate(sets):
+        before = cache.cached_ids()
+        n_before = cache.num_used
+        rows_before = {int(cache.pointers[s]): cache.matrix[s].copy() for s in range(n_before)}
+        slot_before = cache.slot_of.copy()
+        lists = cache.window_update(act)
+        cache.insert(lists, bundles, bias_up)
+        _check_structure(cache)
+        # cached set = union of the active sets of the last k tokens, current included
+        union = set()
+        for u in range(max(0, t - k + 1), t + 1):
+            union |= set(sets[u].tolist())
+        assert cache.cached_ids() == union
+        # load = needed but absent, ascending; evict = present but outside the window
+        assert lists["load_ids"].tolist() == sorted(set(act.tolist()) - before)
+        assert set(lists["evict_ids"].tolist()) == before - union
+        assert cache.num_used == n_before - len(lists["evict_ids"]) + len(lists["load_ids"])
+        # new rows are stacked at the end: rows num_kept .. num_kept + num_new
+        n_kept = n_before - len(lists["evict_ids"])
+        assert lists["load_slots"].tolist() == list(range(n_kept, n_kept + len(lists["load_ids"])))
+        # deleting rewrites at most one row per deleted neuron, only from the tail into holes
+        assert len(lists["move_src"]) <= len(lists["evict_ids"])
+        assert all(src >= n_kept > dst for src, dst in zip(lists["move_src"], lists["move_dst"]))
+        moved = {int(cache.pointers[dst]) for dst in lists["move_dst"]}
+        for i in before & union:
+            if i not in moved:
+                assert cache.slot_of[i] == slot_before[i]          # untouched rows stay put
+        # every cached row holds exactly its neuron's bundle and bias
+        for s in range(cache.num_used):
+            i = cache.pointers[s]
+            np.testing.assert_array_equal(cache.matrix[s], bundles[i])
+            assert cache.bias[s] == bias_up[i]
+            if i in rows_before:
+                np.testing.assert_array_equal(cache.matrix[s], rows_before[i])
+        # slot lists handed to the FFN
+        assert [int(cache.pointers[s]) for s in lists["active_slots"]] == act.tolist()
+        assert sorted(lists["hit_slots"].tolist() + lists["load_slots"].tolist()) == \
+            sorted(lists["active_slots"].tolist())
+        total_loaded += len(lists["load_ids"])
+        assert cache.bytes_fetched == total_loaded * 2 * d * 2     # |new| x bundle bytes
+    if k == 1:
+        # window of one token: load = A_t \ A_{t-1}
+        c2 = O.NeuronCache(d, F, F, 1)
+        prev = set()
+        for act in sets:
+            ls = c2.window_update(act)
+            assert ls["load_ids"].tolist() == sorted(set(act.tolist()) - prev)
+            prev = set(act.tolist())
+
+
+def test_window_longer_than_sequence_never_evicts_and_growth_slows():
+    F, T = 400, 30
+    sets = _random_active_sets(F, T, 0.05, seed=5, sticky=0.0)
+    cache = O.NeuronCache(2, F, F, window_k=T + 1)
+    used = []
+    for act in sets:
+        ls = cache.window_update(act)
+        assert ls["evict_ids"].size == 0 and ls["move_src"].size == 0
+        used.append(cache.num_used)
+    assert used[-1] == len(set(np.concatenate(sets).tolist()))
+    inc = np.diff([0] + used)
+    # aggregated usage is concave on average (Section 3.1, aggregated neuron usage figure)
+    assert inc[: T // 2].mean() > inc[T // 2:].mean()
+
+
+def test_window_swap_remove_worked_example():
+    # rows [10 11 12 13 14 15]; neurons 11, 14 and 15 leave the window, nothing new arrives.
+    # Holes below the new size: slot 1.  Last surviving row (slot 3, neuron 13) fills it.
+    F, d = 32, 2
+    cache = O.NeuronCache(d, F, 8, window_k=1)
+    bundles = np.arange(F * 2 * d, dtype=np.float16).reshape(F, 2 * d)
+    bias_up = np.arange(F, dtype=np.float16)
+    ls = cache.window_update([10, 11, 12, 13, 14, 15]); cache.insert(ls, bundles, bias_up)
+    assert cache.pointers[:6].tolist() == [10, 11, 12, 13, 14, 15]
+    ls = cache.window_update([10, 12, 13]); cache.insert(ls, bundles, bias_up)
+    assert ls["evict_ids"].tolist() == [11, 14, 15]
+    assert ls["move_src"].tolist() == [3] and ls["move_dst"].tolist() == [1]
+    assert cache.pointers[:3].tolist() == [10, 13, 12] and cache.num_used == 3
+    np.testing.assert_array_equal(cache.matrix[1], bundles[13])
+    assert cache.bias[1] == bias_up[13]
+    assert ls["active_slots"].tolist() == [0, 2, 1]
+    # two holes, two tail survivors: the very last survivor fills the first hole
+    cache = O.NeuronCache(d, F, 8, window_k=1)
+    ls = cache.window_update([1, 2, 3, 4, 5, 6]); cache.insert(ls, bundles, bias_up)
+    ls = cache.window_update([3, 4, 5, 6, 20]); cache.insert(ls, bundles, bias_up)
+    assert ls["move_src"].tolist() == [5, 4] and ls["move_dst"].tolist() == [0, 1]
+    assert cache.pointers[:5].tolist() == [6, 5, 3, 4, 20]
+    assert ls["load_ids"].tolist() == [20] and ls["load_slots"].tolist() == [4]
+    assert ls["hit_slots"].tolist() == [2, 3, 1, 0]
+
+
+def test_window_capacity_error_leaves_state_unchanged():
+    cache = O.NeuronCache(2, 16, capacity=4, window_k=2)
+    cache.window_update([0, 1, 2])
+    snap = (cache.pointers.copy(), cache.slot_of.copy(), cache.last_active.copy(), cache.num_used, cache.t)
+    with pytest.raises(O.CapacityError):
+        cache.window_update([3, 4])
+    assert (cache.pointers == snap[0]).all() and (cache.slot_of == snap[1]).all()
+    assert (cache.last_active == snap[2]).all() and (cache.num_used, cache.t) == snap[3:]
+    cache.window_update([3])                                         # exactly fills: fine
+    assert cache.num_used == 4
+
+
+def test_cold_start_loads_whole_active_set():
+    # the first tokens find an empty cache (Section 4, long-generation figure)
+    cache = O.NeuronCache(2, 50, 50, window_k=3)
+    ls = cache.window_update([4, 8, 15, 16, 23, 42])
+    assert ls["load_ids"].tolist() == [4, 8, 15, 16, 23, 42]
+    assert ls["load_slots"].tolist() == list(range(6)) and ls["hit_slots"].size == 0
+
+
+# ------------------------------------------------------------------ decode step
+def test_decode_step_with_true_mask_predictor_equals_dense_ffn():
+    # A predictor that reproduces the up projection exactly (A = W_up^T, B = I, c = b_up)
+    # predicts the true ReLU mask, so every step's output is the dense FFN, whatever the
+    # cache did in between.
+    r = _rng(7)
+    F, d, T = 40, 8, 12
+    W_up = r.normal(size=(F, d)).astype(np.float16)
+    W_down = r.normal(size=(d, F)).astype(np.float16)
+    b_up = (r.normal(size=F) - 1.0).astype(np.float16)
+    bundles = np.concatenate([W_up, W_down.T], axis=1)
+    cache = O.NeuronCache(d, F, F, window_k=3)
+    x = r.normal(size=(1, d))
+    for _ in range(T):
+        x = (0.8 * x + 0.6 * r.normal(size=(1, d))).astype(np.float16)
+        _, act, lists, y = O.decode_step(cache, x, W_up.T, np.eye(F), b_up, 0.0, bundles, b_up)
+        xd = x[0].astype(np.float64)
+        dense = W_down.astype(np.float64) @ np.maximum(W_up.astype(np.float64) @ xd + b_up, 0.0)
+        np.testing.assert_allclose(y[0], dense, rtol=1e-10, atol=1e-10)
+        # the whole-cache mode adds only rows whose ReLU is zero or that really fire: same y
+        y_all = O.sparse_ffn(cache.matrix, cache.bias, np.arange(cache.num_used), x)
+        np.testing.assert_allclose(y_all[0], dense, rtol=1e-10, atol=1e-10)
+
+
+# ------------------------------------------------------------------ cost model
+def _golden_rows():
+    rows = []
+    with open(GOLDEN) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            kind, inputs, value, tol, cite = [p.strip() for p in line.split("|")]
+            rows.append((kind, inputs, float(value), float(tol), cite))
+    return rows
+
+
+@pytest.mark.parametrize("kind,inputs,value,tol,cite", _golden_rows())
+def test_cost_model_reproduces_paper_values(kind, inputs, value, tol, cite):
+    if kind == "io_ms":
+        gb, thr = map(float, inputs.split(","))
+        got = O.io_latency_ms(gb, thr)
+    elif kind == "chunk_bytes":
+        d, nb = map(int, inputs.split(","))
+        got = O.chunk_bytes(d, nb)
+        assert O.chunk_bytes(d, nb, bundled=False) * 2 == got          # bundling doubles it
+    elif kind == "dram_share":
+        fixed, ffn, frac = inputs.split(";")
+        got = O.dram_share_percent([float(v) for v in fixed.split(",")], float(ffn), float(frac))
+    elif kind == "flash_gb":
+        got = O.flash_to_dram_gb(*map(float, inputs.split(",")))
+    elif kind == "avg_rank":
+        n1, r1, n2, r2 = map(float, inputs.split(","))
+        got = (n1 * r1 + n2 * r2) / (n1 + n2)
+    elif kind == "predictor_fraction":
+        got = O.predictor_weight_fraction(*map(int, inputs.split(",")))
+    elif kind == "kv_fraction":
+        ctx, d, L, params = inputs.split(",")
+        got = O.kv_cache_fraction(int(ctx), int(d), int(L), float(params))
+    else:
+        raise AssertionError(kind)
+    assert got == pytest.approx(value, rel=tol, abs=0), cite
+
+
+def test_bundling_halves_io_latency_as_in_table_1():
+    # same bytes, throughput 1.25 -> 2.25 GB/s: latency ratio 164 / 87 in Table 1
+    a, b = O.io_latency_ms(0.2, 1.25), O.io_latency_ms(0.2, 2.25)
+    assert a / b == pytest.approx(164 / 87, rel=0.05)
