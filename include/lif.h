@@ -1,0 +1,200 @@
+/*
+ * lif.h — C ABI of the sparse-decode FFN path of "LLM in a flash" (arXiv 2312.11514),
+ * implemented as CUDA kernels for sm_100a.
+ *
+ * One `lif_layer` is one FFN layer of a ReLU transformer whose full weights live in a
+ * row-column-bundle store in pinned host memory (standing in for flash) and whose recently
+ * used neurons live in a preallocated cache in device memory (Section 3.3: `matrix`,
+ * `pointers`, `bias`, `num_used`, `last_k_active`).
+ *
+ * Conventions
+ *  - "dev" pointers are device addresses, "host" pointers are host addresses.  The caller
+ *    owns every buffer it passes and keeps it alive until lif_destroy_layer; the library owns
+ *    only the opaque handle (plus two CUDA events inside it).
+ *  - `stream` arguments are `cudaStream_t` values passed as `void*` (NULL = default stream).
+ *  - Calls that take a stream only enqueue work and never synchronise.  Argument errors are
+ *    returned immediately.  Conditions only the device can see (cache overflow, a bounded
+ *    wait that ran out) are written to the layer's device status word, leave the window
+ *    state of that step untouched, and are reported by lif_get_stats.
+ *  - fp16 = IEEE binary16; accumulations are fp32.
+ *  - All counts the kernels need (n_active, n_load, ...) stay in device memory; no call
+ *    needs them on the host to launch the next one.
+ */
+#ifndef LIF_H
+#define LIF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LIF_OK = 0,
+  LIF_ERR_INVALID_ARG = 1,
+  LIF_ERR_ALIGNMENT = 2,
+  LIF_ERR_CAPACITY = 3, /* window union would exceed `capacity` rows */
+  LIF_ERR_STATE = 4,
+  LIF_ERR_CUDA = 5,
+  LIF_ERR_TIMEOUT = 6   /* a bounded device-side wait gave up */
+} lif_status;
+
+const char* lif_status_str(lif_status s);
+
+typedef struct lif_layer lif_layer;
+
+/* Layer description.  Shapes follow Section 3.3: the cache `matrix` is
+ * [capacity][2*d_model]; row s holds up-projection row `pointers[s]` followed by
+ * down-projection column `pointers[s]` (Section 3.2, bundling columns and rows). */
+typedef struct {
+  int32_t d_model;          /* multiple of 8, <= 8192 */
+  int32_t d_ff;             /* multiple of 8 */
+  int32_t rank;             /* predictor rank r, multiple of 8, <= 2048 */
+  int32_t window_k;         /* tokens kept in the window, current one included, >= 1 */
+  int32_t capacity;         /* rows of the cache (the paper's Req_i), 1..d_ff */
+  int32_t n_streams;        /* S: concurrent decode streams sharing the layer, 1..8 */
+  float threshold_logit;    /* theta: neuron active iff score > theta; sigmoid threshold tau
+                               maps to ln(tau/(1-tau)), tau = 0.5 -> 0 (Section 3.1, App. B) */
+  int32_t ffn_mode;         /* 0: FFN over the rows of the currently active neurons;
+                               1: over every cached row [0, num_used) (Section 3.3 item 3) */
+  int32_t activation;       /* 0 = ReLU */
+  const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][2*d_model] */
+  const void* dev_pred_A;   /* fp16 [d_model][rank] */
+  const void* dev_pred_B;   /* fp16 [rank][d_ff] */
+  const float* dev_pred_c;  /* fp32 [d_ff] per-neuron score offset */
+  const void* dev_bias_up;  /* fp16 [d_ff]: up-projection biases, always resident */
+  const void* dev_bias_down;/* fp16 [d_model] or NULL */
+  void* dev_cache;          /* fp16 [capacity][2*d_model], 16-byte aligned */
+  void* dev_workspace;      /* 256-byte aligned, lif_workspace_bytes() bytes; holds the window
+                               state and all lists; initialised by lif_create_layer's reset */
+  size_t workspace_bytes;
+} lif_layer_desc;
+
+/* Indices into the device counts block (int32[LIF_CNT_LEN]). */
+enum {
+  LIF_CNT_N_ACTIVE = 0,     /* neurons predicted active this step */
+  LIF_CNT_N_EVICT = 1,      /* neurons that left the window */
+  LIF_CNT_N_MOVES = 2,      /* rows moved from the tail into freed slots */
+  LIF_CNT_N_LOAD = 3,       /* neurons to bring in */
+  LIF_CNT_N_HITS = 4,       /* active neurons already cached */
+  LIF_CNT_NUM_USED_BEFORE = 5,
+  LIF_CNT_NUM_KEPT = 6,     /* rows left after deleting = first slot of the new rows */
+  LIF_CNT_NUM_USED = 7,     /* rows in use after the step */
+  LIF_CNT_STEP = 8,         /* steps applied so far */
+  LIF_CNT_STATUS = 9,       /* sticky lif_status written by kernels */
+  LIF_CNT_LEN = 64
+};
+
+/* Device addresses of the per-step lists and of the window state, all inside the
+ * workspace.  Lists are int32 and valid after lif_window_update of the same step:
+ *   active_idx[n_active]   ascending neuron ids (as given to lif_window_update)
+ *   evict_ids[n_evict]     deleted neurons in ascending order of the slot they held
+ *   move_src/dst[n_moves]  row move_src[j] was copied to row move_dst[j]
+ *   load_ids[n_load]       neurons to bring in, ascending id; load_slots[j] = num_kept + j
+ *   active_slots[n_active] cache row of active_idx[q] after the update
+ *   hit_slots[n_hits]      rows of the active neurons that were already cached
+ * State: pointers[capacity] (row -> neuron, -1 = free), slot_of[d_ff] (neuron -> row, -1 =
+ * absent), last_active[d_ff] (last step predicted active), bias[capacity] fp16. */
+typedef struct {
+  int32_t* counts;
+  int32_t* active_idx;
+  int32_t* evict_ids;
+  int32_t* move_src;
+  int32_t* move_dst;
+  int32_t* load_ids;
+  int32_t* load_slots;
+  int32_t* active_slots;
+  int32_t* hit_slots;
+  int32_t* pointers;
+  int32_t* slot_of;
+  int32_t* last_active;
+  void* bias;
+} lif_lists;
+
+typedef struct {
+  int32_t counts[16];       /* counts block entries 0..15 of the last step */
+  uint64_t bytes_fetched;   /* cumulative: sum of n_load * bundle bytes */
+  uint64_t rows_moved;      /* cumulative */
+  int32_t status;           /* sticky device status (lif_status) */
+  int32_t reserved;
+} lif_stats;
+
+/* Bytes of device workspace a layer of this description needs (pointer fields ignored). */
+lif_status lif_workspace_bytes(const lif_layer_desc* desc, size_t* out_bytes);
+
+/* Validate `desc` (sizes, NULLs, 16-byte alignment, host_bundles registered as mapped pinned
+ * memory), create the handle and enqueue a cold-cache reset on the default stream.
+ * Allocates no device memory.  Section 3.3: num_used starts at zero. */
+lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out);
+
+/* Frees the handle and its events; never touches caller memory. */
+lif_status lif_destroy_layer(lif_layer* layer);
+
+/* Empty the cache and restart the step counter (cold start). */
+lif_status lif_reset(lif_layer* layer, void* stream);
+
+/* Low-rank predictor (Section 3.1, "Anticipating ReLU Sparsity"): scores = x.A.B + c in fp32,
+ * active iff score > theta for at least one stream.
+ *   dev_x              fp16 [n_streams][d_model]
+ *   dev_logits_or_null fp32 [n_streams][d_ff] scores (optional)
+ *   dev_active_idx     int32 [d_ff]: ascending ids of the active neurons
+ *   dev_n_active       int32 [1] */
+lif_status lif_predict(lif_layer* layer, const void* dev_x, float* dev_logits_or_null,
+                       int32_t* dev_active_idx, int32_t* dev_n_active, void* stream);
+
+/* Sliding-window update (Section 3.1 "The Sliding Window Technique", Section 3.3 items 1-2):
+ * stamps the active neurons, deletes the neurons not active in the last window_k steps by
+ * moving tail rows into their slots (first freed slot <- last surviving row), assigns rows
+ * num_kept.. to the neurons to bring in (ascending id), updates pointers / slot_of / bias /
+ * num_used, writes every list of lif_lists, applies the row moves inside dev_cache, and
+ * advances the step.  On overflow sets LIF_ERR_CAPACITY in the status word and changes
+ * nothing.  dev_active_idx must be ascending and duplicate-free. */
+lif_status lif_window_update(lif_layer* layer, const int32_t* dev_active_idx,
+                             const int32_t* dev_n_active, void* stream);
+
+/* Bring in new neurons (Section 3.3 item 2): copy bundle load_ids[j] from the host store to
+ * cache row load_slots[j], reading host memory directly from the kernel. */
+lif_status lif_fetch_bundles(lif_layer* layer, void* fetch_stream);
+
+/* Inference over cached rows (Section 3.3 item 3):
+ *   y[s] = b_down + sum_q relu(<matrix[slot_q, :d], x[s]> + bias[slot_q]) * matrix[slot_q, d:]
+ *   dev_slots    int32 rows to use, or NULL for rows [0, *dev_n_slots)
+ *   dev_n_slots  int32 [1] (device)
+ *   dev_y        fp32 [n_streams][d_model] */
+lif_status lif_sparse_ffn(lif_layer* layer, const void* dev_x, const int32_t* dev_slots,
+                          const int32_t* dev_n_slots, float* dev_y, void* stream);
+
+/* One token through the layer: predict -> window update -> fetch (on fetch_stream, ordered by
+ * events) -> sparse FFN (ffn_mode selects the rows).  The compute stream ends up ordered
+ * after the fetch, so consecutive calls on the same streams are safe. */
+lif_status lif_decode_step(lif_layer* layer, const void* dev_x, float* dev_y,
+                           void* compute_stream, void* fetch_stream);
+
+/* One token through `n_layers` layers from host buffers: copies host_x (fp16
+ * [n_streams][d_model], pinned) to dev_x, runs lif_decode_step on every layer in order with
+ * layer l writing dev_y + l*n_streams*d_model, copies all outputs to host_y (fp32
+ * [n_layers][n_streams][d_model], pinned) and synchronises compute_stream. */
+lif_status lif_decode_token_host(lif_layer* const* layers, int32_t n_layers, const void* host_x,
+                                 void* dev_x, float* dev_y, float* host_y,
+                                 void* compute_stream, void* fetch_stream);
+
+/* Device addresses of lists and state (valid for the layer's lifetime). */
+lif_status lif_get_lists(lif_layer* layer, lif_lists* host_out);
+
+/* Synchronises the device, then reports counts, cumulative traffic and the status word. */
+lif_status lif_get_stats(lif_layer* layer, lif_stats* host_out);
+
+/* Clears the sticky device status word. */
+lif_status lif_clear_status(lif_layer* layer, void* stream);
+
+/* Bandwidth probe for the host link: a kernel reads `bytes` of mapped pinned host memory
+ * into device memory with the same access pattern as lif_fetch_bundles (chunk_bytes-sized
+ * pieces; chunk_bytes a multiple of 16, bytes a multiple of chunk_bytes).  Enqueue only. */
+lif_status lif_probe_host_read(const void* host_src, void* dev_dst, size_t bytes,
+                               size_t chunk_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LIF_H */

@@ -1,0 +1,330 @@
+// C ABI of liblif.so: argument checking, workspace carve-up and stream/event orchestration.
+// Every step of the path runs in the kernels of predict.cu / window.cu / fetch.cu / ffn.cu.
+#include <new>
+
+#include "lif_internal.cuh"
+
+namespace lif {
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max) {
+  Workspace w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = off;
+    off = align_up(off + bytes, 256);
+    return at;
+  };
+  const size_t F = d.d_ff, cap = d.capacity, S = d.n_streams;
+  const size_t z_ctas = (d.d_model + kZRowsPerCta - 1) / kZRowsPerCta;
+  const size_t n_mask = (F + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
+  w.counts = take(LIF_CNT_LEN * 4);
+  w.pointers = take(cap * 4);
+  w.slot_of = take(F * 4);
+  w.last_active = take(F * 4);
+  w.bias = take(cap * 2);
+  w.active_idx = take(F * 4);
+  w.evict_ids = take(cap * 4);
+  w.evict_slots = take(cap * 4);
+  w.move_src = take(cap * 4);
+  w.move_dst = take(cap * 4);
+  w.load_ids = take(cap * 4);
+  w.load_slots = take(cap * 4);
+  w.active_slots = take(F * 4);
+  w.hit_slots = take(F * 4);
+  w.n_tmp = take(64);
+  w.z_partial = take(z_ctas * S * d.rank * 4);
+  w.mask_words = take(n_mask * 4);
+  w.y_partial = take((size_t)ffn_grid_max * d.d_model * 4);
+  w.total = off;
+  return w;
+}
+
+static int ffn_grid_upper_bound() { return 2 * 256; }   // >= 2 CTAs per SM on any part
+
+static lif_status check_shape(const lif_layer_desc* d) {
+  if (!d) return LIF_ERR_INVALID_ARG;
+  if (d->d_model < 8 || d->d_model % 8 || d->d_model > 8192) return LIF_ERR_INVALID_ARG;
+  if (d->d_ff < 8 || d->d_ff % 8) return LIF_ERR_INVALID_ARG;
+  if (d->rank < 8 || d->rank % 8 || d->rank > 2048) return LIF_ERR_INVALID_ARG;
+  if (d->window_k < 1) return LIF_ERR_INVALID_ARG;
+  if (d->capacity < 1 || d->capacity > d->d_ff) return LIF_ERR_INVALID_ARG;
+  if (d->n_streams < 1 || d->n_streams > kMaxStreams) return LIF_ERR_INVALID_ARG;
+  if (d->ffn_mode != 0 && d->ffn_mode != 1) return LIF_ERR_INVALID_ARG;
+  if (d->activation != 0) return LIF_ERR_INVALID_ARG;
+  if (!(d->threshold_logit == d->threshold_logit)) return LIF_ERR_INVALID_ARG;   // NaN
+  return LIF_OK;
+}
+
+static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+}  // namespace lif
+
+using namespace lif;
+
+extern "C" {
+
+const char* lif_status_str(lif_status s) {
+  switch (s) {
+    case LIF_OK: return "ok";
+    case LIF_ERR_INVALID_ARG: return "invalid argument";
+    case LIF_ERR_ALIGNMENT: return "misaligned pointer";
+    case LIF_ERR_CAPACITY: return "window cache capacity exceeded";
+    case LIF_ERR_STATE: return "invalid state";
+    case LIF_ERR_CUDA: return "CUDA error";
+    case LIF_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown";
+}
+
+lif_status lif_workspace_bytes(const lif_layer_desc* desc, size_t* out_bytes) {
+  if (!out_bytes) return LIF_ERR_INVALID_ARG;
+  lif_status s = check_shape(desc);
+  if (s != LIF_OK) return s;
+  *out_bytes = plan_workspace(*desc, ffn_grid_upper_bound()).total;
+  return LIF_OK;
+}
+
+lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
+  if (!out) return LIF_ERR_INVALID_ARG;
+  *out = nullptr;
+  lif_status s = check_shape(desc);
+  if (s != LIF_OK) return s;
+  if (!desc->host_bundles || !desc->dev_pred_A || !desc->dev_pred_B || !desc->dev_pred_c ||
+      !desc->dev_bias_up || !desc->dev_cache || !desc->dev_workspace)
+    return LIF_ERR_INVALID_ARG;
+  if (!aligned(desc->host_bundles, 16) || !aligned(desc->dev_pred_A, 16) ||
+      !aligned(desc->dev_pred_B, 16) || !aligned(desc->dev_pred_c, 4) ||
+      !aligned(desc->dev_bias_up, 2) || !aligned(desc->dev_cache, 16) ||
+      !aligned(desc->dev_workspace, 256) ||
+      (desc->dev_bias_down && !aligned(desc->dev_bias_down, 8)))
+    return LIF_ERR_ALIGNMENT;
+  Workspace ws = plan_workspace(*desc, ffn_grid_upper_bound());
+  if (desc->workspace_bytes < ws.total) return LIF_ERR_INVALID_ARG;
+
+  void* alias = nullptr;
+  if (cudaHostGetDevicePointer(&alias, const_cast<void*>(desc->host_bundles), 0) != cudaSuccess) {
+    cudaGetLastError();
+    return LIF_ERR_INVALID_ARG;   // not pinned + mapped
+  }
+  lif_layer* L = new (std::nothrow) lif_layer();
+  if (!L) return LIF_ERR_STATE;
+  L->desc = *desc;
+  L->ws = ws;
+  L->dev_bundles = (const __half*)alias;
+  unsigned char* b = (unsigned char*)desc->dev_workspace;
+  L->counts = (int32_t*)(b + ws.counts);
+  L->pointers = (int32_t*)(b + ws.pointers);
+  L->slot_of = (int32_t*)(b + ws.slot_of);
+  L->last_active = (int32_t*)(b + ws.last_active);
+  L->bias = (__half*)(b + ws.bias);
+  L->active_idx = (int32_t*)(b + ws.active_idx);
+  L->evict_ids = (int32_t*)(b + ws.evict_ids);
+  L->evict_slots = (int32_t*)(b + ws.evict_slots);
+  L->move_src = (int32_t*)(b + ws.move_src);
+  L->move_dst = (int32_t*)(b + ws.move_dst);
+  L->load_ids = (int32_t*)(b + ws.load_ids);
+  L->load_slots = (int32_t*)(b + ws.load_slots);
+  L->active_slots = (int32_t*)(b + ws.active_slots);
+  L->hit_slots = (int32_t*)(b + ws.hit_slots);
+  L->n_tmp = (int32_t*)(b + ws.n_tmp);
+  L->z_partial = (float*)(b + ws.z_partial);
+  L->mask_words = (uint32_t*)(b + ws.mask_words);
+  L->y_partial = (float*)(b + ws.y_partial);
+
+  int dev = 0;
+  bool ok = cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&L->n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
+  ok = ok && ffn_configure(L) == cudaSuccess;
+  if (ok) {
+    L->z_ctas = (desc->d_model + kZRowsPerCta - 1) / kZRowsPerCta;
+    L->ffn_grid = L->n_sm < ffn_grid_upper_bound() ? L->n_sm : ffn_grid_upper_bound();
+    L->fetch_grid = L->n_sm;
+    L->move_grid = L->n_sm;
+    ok = cudaEventCreateWithFlags(&L->ev_plan, cudaEventDisableTiming) == cudaSuccess;
+    if (ok && cudaEventCreateWithFlags(&L->ev_fetch, cudaEventDisableTiming) != cudaSuccess) {
+      cudaEventDestroy(L->ev_plan);
+      ok = false;
+    }
+  }
+  if (ok && launch_reset(L, 0) != cudaSuccess) {
+    cudaEventDestroy(L->ev_plan);
+    cudaEventDestroy(L->ev_fetch);
+    ok = false;
+  }
+  if (!ok) {
+    cudaGetLastError();
+    delete L;
+    return LIF_ERR_CUDA;
+  }
+  *out = L;
+  return LIF_OK;
+}
+
+lif_status lif_destroy_layer(lif_layer* L) {
+  if (!L) return LIF_ERR_INVALID_ARG;
+  cudaEventDestroy(L->ev_plan);
+  cudaEventDestroy(L->ev_fetch);
+  delete L;
+  return LIF_OK;
+}
+
+lif_status lif_reset(lif_layer* L, void* stream) {
+  if (!L) return LIF_ERR_INVALID_ARG;
+  return launch_reset(L, (cudaStream_t)stream) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_predict(lif_layer* L, const void* dev_x, float* dev_logits_or_null,
+                       int32_t* dev_active_idx, int32_t* dev_n_active, void* stream) {
+  if (!L || !dev_x || !dev_active_idx || !dev_n_active) return LIF_ERR_INVALID_ARG;
+  if (!aligned(dev_x, 16) || !aligned(dev_active_idx, 4) || !aligned(dev_n_active, 4) ||
+      (dev_logits_or_null && !aligned(dev_logits_or_null, 4)))
+    return LIF_ERR_ALIGNMENT;
+  return launch_predict(L, (const __half*)dev_x, dev_logits_or_null, dev_active_idx,
+                        dev_n_active, (cudaStream_t)stream) == cudaSuccess
+             ? LIF_OK
+             : LIF_ERR_CUDA;
+}
+
+lif_status lif_window_update(lif_layer* L, const int32_t* dev_active_idx,
+                             const int32_t* dev_n_active, void* stream) {
+  if (!L || !dev_active_idx || !dev_n_active) return LIF_ERR_INVALID_ARG;
+  if (!aligned(dev_active_idx, 4) || !aligned(dev_n_active, 4)) return LIF_ERR_ALIGNMENT;
+  return launch_window(L, dev_active_idx, dev_n_active, (cudaStream_t)stream) == cudaSuccess
+             ? LIF_OK
+             : LIF_ERR_CUDA;
+}
+
+lif_status lif_fetch_bundles(lif_layer* L, void* fetch_stream) {
+  if (!L) return LIF_ERR_INVALID_ARG;
+  return launch_fetch(L, (cudaStream_t)fetch_stream) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_sparse_ffn(lif_layer* L, const void* dev_x, const int32_t* dev_slots,
+                          const int32_t* dev_n_slots, float* dev_y, void* stream) {
+  if (!L || !dev_x || !dev_n_slots || !dev_y) return LIF_ERR_INVALID_ARG;
+  if (!aligned(dev_x, 16) || !aligned(dev_y, 16) || !aligned(dev_n_slots, 4) ||
+      (dev_slots && !aligned(dev_slots, 4)))
+    return LIF_ERR_ALIGNMENT;
+  return launch_ffn(L, (const __half*)dev_x, dev_slots, dev_n_slots, nullptr, dev_y, false,
+                    (cudaStream_t)stream) == cudaSuccess
+             ? LIF_OK
+             : LIF_ERR_CUDA;
+}
+
+lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* compute_stream,
+                           void* fetch_stream) {
+  if (!L || !dev_x || !dev_y) return LIF_ERR_INVALID_ARG;
+  if (!aligned(dev_x, 16) || !aligned(dev_y, 16)) return LIF_ERR_ALIGNMENT;
+  cudaStream_t sc = (cudaStream_t)compute_stream, sf = (cudaStream_t)fetch_stream;
+  const __half* x = (const __half*)dev_x;
+  bool ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc) == cudaSuccess;
+  ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc) == cudaSuccess;
+  if (sf != sc) {
+    ok = ok && cudaEventRecord(L->ev_plan, sc) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(sf, L->ev_plan, 0) == cudaSuccess;
+  }
+  ok = ok && launch_fetch(L, sf) == cudaSuccess;
+  if (sf != sc) {
+    ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(sc, L->ev_fetch, 0) == cudaSuccess;
+  }
+  if (L->desc.ffn_mode == 0)
+    ok = ok && launch_ffn(L, x, L->active_slots, L->counts + LIF_CNT_N_ACTIVE, nullptr, dev_y,
+                          false, sc) == cudaSuccess;
+  else
+    ok = ok && launch_ffn(L, x, nullptr, L->counts + LIF_CNT_NUM_USED, nullptr, dev_y, false,
+                          sc) == cudaSuccess;
+  if (!ok) cudaGetLastError();
+  return ok ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_decode_token_host(lif_layer* const* layers, int32_t n_layers, const void* host_x,
+                                 void* dev_x, float* dev_y, float* host_y, void* compute_stream,
+                                 void* fetch_stream) {
+  if (!layers || n_layers < 1 || !host_x || !dev_x || !dev_y || !host_y)
+    return LIF_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!layers[l] || layers[l]->desc.d_model != layers[0]->desc.d_model ||
+        layers[l]->desc.n_streams != layers[0]->desc.n_streams)
+      return LIF_ERR_INVALID_ARG;
+  cudaStream_t sc = (cudaStream_t)compute_stream;
+  const size_t per = (size_t)layers[0]->desc.n_streams * layers[0]->desc.d_model;
+  if (cudaMemcpyAsync(dev_x, host_x, per * 2, cudaMemcpyHostToDevice, sc) != cudaSuccess)
+    return LIF_ERR_CUDA;
+  for (int l = 0; l < n_layers; ++l) {
+    lif_status s = lif_decode_step(layers[l], dev_x, dev_y + (size_t)l * per, compute_stream,
+                                   fetch_stream);
+    if (s != LIF_OK) return s;
+  }
+  if (cudaMemcpyAsync(host_y, dev_y, per * 4 * n_layers, cudaMemcpyDeviceToHost, sc) !=
+      cudaSuccess)
+    return LIF_ERR_CUDA;
+  return cudaStreamSynchronize(sc) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_get_lists(lif_layer* L, lif_lists* o) {
+  if (!L || !o) return LIF_ERR_INVALID_ARG;
+  o->counts = L->counts;
+  o->active_idx = L->active_idx;
+  o->evict_ids = L->evict_ids;
+  o->move_src = L->move_src;
+  o->move_dst = L->move_dst;
+  o->load_ids = L->load_ids;
+  o->load_slots = L->load_slots;
+  o->active_slots = L->active_slots;
+  o->hit_slots = L->hit_slots;
+  o->pointers = L->pointers;
+  o->slot_of = L->slot_of;
+  o->last_active = L->last_active;
+  o->bias = L->bias;
+  return LIF_OK;
+}
+
+lif_status lif_get_stats(lif_layer* L, lif_stats* o) {
+  if (!L || !o) return LIF_ERR_INVALID_ARG;
+  int32_t host[LIF_CNT_LEN];
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(host, L->counts, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return LIF_ERR_CUDA;
+  }
+  for (int i = 0; i < 16; ++i) o->counts[i] = host[i];
+  const uint64_t* totals = reinterpret_cast<const uint64_t*>(host + CNT_TOTALS);
+  o->bytes_fetched = totals[0];
+  o->rows_moved = totals[1];
+  o->status = host[LIF_CNT_STATUS];
+  o->reserved = 0;
+  return LIF_OK;
+}
+
+lif_status lif_clear_status(lif_layer* L, void* stream) {
+  if (!L) return LIF_ERR_INVALID_ARG;
+  return cudaMemsetAsync(L->counts + LIF_CNT_STATUS, 0, 4, (cudaStream_t)stream) == cudaSuccess
+             ? LIF_OK
+             : LIF_ERR_CUDA;
+}
+
+lif_status lif_probe_host_read(const void* host_src, void* dev_dst, size_t bytes,
+                               size_t chunk_bytes, void* stream) {
+  if (!host_src || !dev_dst || !bytes || !chunk_bytes) return LIF_ERR_INVALID_ARG;
+  if (bytes % chunk_bytes || chunk_bytes % 16 || bytes / chunk_bytes > 0x7fffffff)
+    return LIF_ERR_INVALID_ARG;
+  if (!aligned(host_src, 16) || !aligned(dev_dst, 16)) return LIF_ERR_ALIGNMENT;
+  void* alias = nullptr;
+  if (cudaHostGetDevicePointer(&alias, const_cast<void*>(host_src), 0) != cudaSuccess) {
+    cudaGetLastError();
+    return LIF_ERR_INVALID_ARG;
+  }
+  int dev = 0, n_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return LIF_ERR_CUDA;
+  return launch_probe(alias, dev_dst, bytes, chunk_bytes, n_sm, (cudaStream_t)stream) ==
+                 cudaSuccess
+             ? LIF_OK
+             : LIF_ERR_CUDA;
+}
+
+}  // extern "C"

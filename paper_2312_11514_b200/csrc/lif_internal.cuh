@@ -1,0 +1,73 @@
+// Internal declarations shared by the translation units of liblif.so.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lif.h"
+
+namespace lif {
+
+// Private entries of the counts block (public ones: LIF_CNT_* in lif.h).
+enum {
+  CNT_TICKET_PREDICT = 16,  // "last block done" counter of the score kernel
+  CNT_TOTALS = 32           // two uint64: bytes_fetched, rows_moved (8-byte aligned)
+};
+
+constexpr int kNever = -(1 << 30);  // last_active stamp of a neuron never predicted active
+constexpr int kThreads = 256;
+constexpr int kWindowThreads = 1024;
+constexpr int kZRowsPerCta = 256;   // rows of A per CTA in the first predictor stage
+constexpr int kLogitTile = 128;     // neurons per CTA in the second predictor stage
+constexpr int kMaxStreams = 8;
+
+struct Workspace {
+  // offsets in bytes from the workspace base; every block 256-byte aligned
+  size_t counts, pointers, slot_of, last_active, bias, active_idx, evict_ids, evict_slots,
+      move_src, move_dst, load_ids, load_slots, active_slots, hit_slots, n_tmp, z_partial,
+      mask_words, y_partial, total;
+};
+
+Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max);
+
+}  // namespace lif
+
+struct lif_layer {
+  lif_layer_desc desc;
+  lif::Workspace ws;
+  const __half* dev_bundles;  // device alias of desc.host_bundles
+  int32_t* counts;
+  int32_t *pointers, *slot_of, *last_active;
+  __half* bias;
+  int32_t *active_idx, *evict_ids, *evict_slots, *move_src, *move_dst, *load_ids, *load_slots,
+      *active_slots, *hit_slots, *n_tmp;
+  float* z_partial;
+  uint32_t* mask_words;
+  float* y_partial;
+  int n_sm;
+  int z_ctas;         // CTAs of the first predictor stage
+  int ffn_grid;       // CTAs of the sparse-FFN kernel
+  int ffn_stages;     // bundles in flight per CTA
+  size_t ffn_smem;    // dynamic shared memory of the sparse-FFN kernel
+  int fetch_grid;     // CTAs of the fetch kernel
+  int move_grid;
+  cudaEvent_t ev_plan, ev_fetch;
+};
+
+namespace lif {
+
+// kernels' host launchers (each returns the launch's cudaError_t)
+cudaError_t launch_reset(lif_layer* L, cudaStream_t st);
+cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
+                           int32_t* n_active, cudaStream_t st);
+cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st);
+cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
+cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,
+                         int grid, cudaStream_t st);
+// slots == nullptr: rows base[0] .. base[0] + n[0] (base == nullptr: 0)
+cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
+                       const int32_t* base, float* y, bool accumulate, cudaStream_t st);
+cudaError_t ffn_configure(lif_layer* L);
+
+}  // namespace lif

@@ -1,0 +1,236 @@
+// Low-rank sparsity predictor (Section 3.1, "Anticipating ReLU Sparsity"; Appendix B):
+// scores = x.A.B + c, active iff score > theta, compacted to an ascending index list.
+//
+// Both stages are HBM-bound GEMVs over fp16 factors with fp32 accumulation:
+//   stage 1  z_partial[p] = x[rows of p] . A[rows of p]      (A read once, 16-byte loads)
+//   stage 2  score = (sum_p z_partial[p]) . B[:, tile] + c   (B read once, 16-byte loads)
+// Stage 2 also thresholds (warp ballot -> bit mask) and the last CTA to finish turns the bit
+// mask into the sorted list with a block prefix sum, so the list order never depends on
+// scheduling.  Summation orders are fixed: results are bit-reproducible run to run.
+#include "lif_internal.cuh"
+
+namespace lif {
+namespace {
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __half22float2(h[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+
+// ---- stage 1: z_partial[cta][s][j] = sum_{m in rows(cta)} x[s][m] * A[m][j] -------------
+template <int S>
+__global__ void __launch_bounds__(kThreads)
+predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int d, int r,
+                 float* __restrict__ z_partial) {
+  __shared__ float red[2048];
+  const int ncg = r >> 3;            // 8-column groups (16 bytes each)
+  const int nrl = kThreads / ncg;    // row lanes
+  const int tid = threadIdx.x;
+  const int cg = tid % ncg, rl = tid / ncg;
+  const int m0 = blockIdx.x * kZRowsPerCta;
+  const int m1 = min(d, m0 + kZRowsPerCta);
+
+  float acc[S][8];
+#pragma unroll
+  for (int s = 0; s < S; ++s)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[s][e] = 0.f;
+
+  if (rl < nrl) {
+#pragma unroll 4
+    for (int m = m0 + rl; m < m1; m += nrl) {
+      float af[8];
+      unpack8(ldg_stream(A + (size_t)m * r + cg * 8), af);
+#pragma unroll
+      for (int s = 0; s < S; ++s) {
+        const float xs = __half2float(x[(size_t)s * d + m]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[s][e] = fmaf(xs, af[e], acc[s][e]);
+      }
+    }
+  }
+  // fold the row lanes, one stream at a time (8 KB of shared memory)
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+    if (rl < nrl) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) red[rl * r + cg * 8 + e] = acc[s][e];
+    }
+    __syncthreads();
+    for (int j = tid; j < r; j += kThreads) {
+      float v = 0.f;
+      for (int l = 0; l < nrl; ++l) v += red[l * r + j];
+      z_partial[((size_t)blockIdx.x * S + s) * r + j] = v;
+    }
+    __syncthreads();
+  }
+}
+
+__device__ __forceinline__ int block_exclusive_scan_256(int v, int* total, int* warp_sums) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  int base = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) {
+    int ws = warp_sums[w];
+    if (w < warp) base += ws;
+    tot += ws;
+  }
+  *total = tot;
+  __syncthreads();
+  return base + inc - v;
+}
+
+// ---- stage 2: scores, threshold, bit mask; last CTA compacts ------------------------------
+template <int S>
+__global__ void __launch_bounds__(kThreads)
+predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* __restrict__ B,
+                      const float* __restrict__ c, float theta, int r, int F,
+                      float* __restrict__ logits, uint32_t* mask_words, int* ticket,
+                      int* __restrict__ active_idx, int* __restrict__ n_active) {
+  extern __shared__ float zs[];                 // [S][r]
+  __shared__ float red[16][kLogitTile];
+  __shared__ int warp_sums[kThreads / 32];
+  __shared__ int is_last;
+  const int tid = threadIdx.x;
+
+  for (int i = tid; i < S * r; i += kThreads) {
+    float v = 0.f;
+    for (int p = 0; p < P; ++p) v += __ldcg(z_partial + (size_t)p * S * r + i);
+    zs[i] = v;
+  }
+  __syncthreads();
+
+  const int cg = tid & 15, rs = tid >> 4;
+  const int col = blockIdx.x * kLogitTile + cg * 8;
+  float acc[S][8];
+#pragma unroll
+  for (int s = 0; s < S; ++s)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[s][e] = 0.f;
+  if (col < F) {
+#pragma unroll 4
+    for (int j = rs; j < r; j += 16) {
+      float bf[8];
+      unpack8(ldg_stream(B + (size_t)j * F + col), bf);
+#pragma unroll
+      for (int s = 0; s < S; ++s) {
+        const float zz = zs[s * r + j];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[s][e] = fmaf(zz, bf[e], acc[s][e]);
+      }
+    }
+  }
+
+  bool active = false;
+  const int my_col = blockIdx.x * kLogitTile + tid;   // used by threads < kLogitTile
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) red[rs][cg * 8 + e] = acc[s][e];
+    __syncthreads();
+    if (tid < kLogitTile && my_col < F) {
+      float v = 0.f;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) v += red[k][tid];
+      v += c[my_col];
+      if (logits) logits[(size_t)s * F + my_col] = v;
+      active = active || (v > theta);
+    }
+    __syncthreads();
+  }
+  if (tid < kLogitTile) {
+    const unsigned m = __ballot_sync(0xffffffffu, active);
+    if ((tid & 31) == 0) mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = m;
+  }
+
+  // last CTA to arrive compacts the whole mask
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int t = atomicAdd(ticket, 1);
+    is_last = (t == (int)gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+
+  const int nwords = gridDim.x * (kLogitTile / 32);
+  const int wpt = (nwords + kThreads - 1) / kThreads;
+  const int w0 = min(nwords, tid * wpt), w1 = min(nwords, w0 + wpt);
+  int cnt = 0;
+  for (int w = w0; w < w1; ++w) cnt += __popc(__ldcg(mask_words + w));
+  int total;
+  int off = block_exclusive_scan_256(cnt, &total, warp_sums);
+  for (int w = w0; w < w1; ++w) {
+    unsigned m = __ldcg(mask_words + w);
+    while (m) {
+      const int b = __ffs(m) - 1;
+      active_idx[off++] = w * 32 + b;
+      m &= m - 1;
+    }
+  }
+  if (tid == 0) {
+    *n_active = total;
+    *ticket = 0;
+  }
+}
+
+template <int S>
+cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
+                             int32_t* n_active, cudaStream_t st) {
+  const lif_layer_desc& D = L->desc;
+  predict_z_kernel<S><<<L->z_ctas, kThreads, 0, st>>>(
+      x, (const __half*)D.dev_pred_A, D.d_model, D.rank, L->z_partial);
+  const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
+  const size_t smem = (size_t)S * D.rank * sizeof(float);
+  if (smem > 32 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(predict_logits_kernel<S>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  predict_logits_kernel<S><<<grid, kThreads, smem, st>>>(
+      L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit,
+      D.rank, D.d_ff, logits, L->mask_words, L->counts + CNT_TICKET_PREDICT, active_idx,
+      n_active);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
+                           int32_t* n_active, cudaStream_t st) {
+  switch (L->desc.n_streams) {
+    case 1: return launch_predict_s<1>(L, x, logits, active_idx, n_active, st);
+    case 2: return launch_predict_s<2>(L, x, logits, active_idx, n_active, st);
+    case 3: return launch_predict_s<3>(L, x, logits, active_idx, n_active, st);
+    case 4: return launch_predict_s<4>(L, x, logits, active_idx, n_active, st);
+    case 5: return launch_predict_s<5>(L, x, logits, active_idx, n_active, st);
+    case 6: return launch_predict_s<6>(L, x, logits, active_idx, n_active, st);
+    case 7: return launch_predict_s<7>(L, x, logits, active_idx, n_active, st);
+    case 8: return launch_predict_s<8>(L, x, logits, active_idx, n_active, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace lif

@@ -1,0 +1,282 @@
+// Sliding-window neuron cache bookkeeping (Section 3.1 "The Sliding Window Technique" and
+// Section 3.3 "Optimized Data Management in DRAM", items 1 and 2), plus cold-cache reset and
+// the row moves that keep the used rows consecutive.
+//
+// The plan is integer work over n_active + num_used elements, so one 1024-thread CTA does it
+// with ordered block-wide compactions (list order = index order, never atomics order):
+//   A  count what would be deleted / loaded; refuse on overflow before touching anything
+//   B  stamp last_active of the active neurons
+//   C  deleted rows in ascending slot order; surviving tail rows in descending slot order
+//   D  first freed slot <- last surviving row (pointers, slot_of, bias); clear the tail
+//   E  new neurons in ascending id get rows num_kept, num_kept + 1, ...
+//   F  slot lists for the FFN
+// The 4*d_model-byte row copies of step D run in a second, grid-wide kernel.
+#include "lif_internal.cuh"
+
+namespace lif {
+namespace {
+
+struct Scan {
+  int warp_sums[kWindowThreads / 32];
+};
+
+// exclusive prefix of v over the block (thread order); *total = block sum
+__device__ __forceinline__ int block_scan(int v, int* total, Scan& sc) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
+  }
+  if (lane == 31) sc.warp_sums[warp] = inc;
+  __syncthreads();
+  int ws = sc.warp_sums[lane];   // 32 warps
+  int winc = ws;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int n = __shfl_up_sync(0xffffffffu, winc, o);
+    if (lane >= o) winc += n;
+  }
+  const int base = __shfl_sync(0xffffffffu, winc - ws, warp);
+  *total = __shfl_sync(0xffffffffu, winc, 31);
+  __syncthreads();
+  return base + inc - v;
+}
+
+struct WindowArgs {
+  const int32_t* act;
+  const int32_t* n_act;
+  int32_t* counts;
+  int32_t *pointers, *slot_of, *last_active;
+  __half* bias;
+  const __half* bias_up;
+  int32_t *active_idx, *evict_ids, *evict_slots, *move_src, *move_dst, *load_ids, *load_slots,
+      *active_slots, *hit_slots;
+  int F, cap, k;
+  unsigned long long bundle_bytes;
+};
+
+__global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArgs a) {
+  __shared__ Scan sc;
+  const int tid = threadIdx.x;
+  const int n = a.counts[LIF_CNT_NUM_USED];
+  const int t = a.counts[LIF_CNT_STEP];
+  const int na = *a.n_act;
+  const int stale_before = t - a.k;   // last_active <= stale_before: outside the window
+  int tot;
+
+  // ---- A: what would happen ------------------------------------------------------------
+  int bad = 0, c_load = 0, c_back = 0, c_stale = 0;
+  if (na < 0 || na > a.F) bad = 1;
+  if (!bad) {
+    for (int q = tid; q < na; q += kWindowThreads) {
+      const int id = a.act[q];
+      if (id < 0 || id >= a.F) { bad = 1; continue; }
+      if (a.slot_of[id] < 0) ++c_load;
+      else if (a.last_active[id] <= stale_before) ++c_back;   // cached, stale, needed again
+    }
+    for (int s = tid; s < n; s += kWindowThreads)
+      if (a.last_active[a.pointers[s]] <= stale_before) ++c_stale;
+  }
+  block_scan(bad, &tot, sc);
+  const int any_bad = tot;
+  block_scan(c_load, &tot, sc);
+  const int n_load = tot;
+  block_scan(c_back, &tot, sc);
+  const int n_back = tot;
+  block_scan(c_stale, &tot, sc);
+  const int n_evict = tot - n_back;
+  const int n_kept = n - n_evict;
+
+  if (any_bad || n_kept + n_load > a.cap) {
+    if (tid == 0) {
+      if (a.counts[LIF_CNT_STATUS] == LIF_OK)
+        a.counts[LIF_CNT_STATUS] = any_bad ? LIF_ERR_INVALID_ARG : LIF_ERR_CAPACITY;
+      a.counts[LIF_CNT_N_ACTIVE] = 0;
+      a.counts[LIF_CNT_N_EVICT] = 0;
+      a.counts[LIF_CNT_N_MOVES] = 0;
+      a.counts[LIF_CNT_N_LOAD] = 0;
+      a.counts[LIF_CNT_N_HITS] = 0;
+      a.counts[LIF_CNT_NUM_USED_BEFORE] = n;
+      a.counts[LIF_CNT_NUM_KEPT] = n;
+    }
+    return;
+  }
+
+  // ---- B: stamp --------------------------------------------------------------------------
+  for (int q = tid; q < na; q += kWindowThreads) a.last_active[a.act[q]] = t;
+  __syncthreads();
+
+  // ---- C: deleted rows (ascending slot) and surviving tail rows (descending slot) --------
+  int run = 0, holes = 0;
+  for (int b = 0; b < n; b += kWindowThreads) {
+    const int s = b + tid;
+    int id = -1, f = 0;
+    if (s < n) {
+      id = a.pointers[s];
+      f = a.last_active[id] <= stale_before;
+    }
+    const int pos = run + block_scan(f, &tot, sc);
+    if (f) {
+      a.evict_slots[pos] = s;
+      a.evict_ids[pos] = id;
+    }
+    run += tot;
+    block_scan(f && s < n_kept, &tot, sc);
+    holes += tot;
+  }
+  const int n_moves = holes;
+  run = 0;
+  for (int b = 0; b < n - n_kept; b += kWindowThreads) {
+    const int i = b + tid;
+    const int s = n - 1 - i;
+    int f = 0;
+    if (i < n - n_kept) f = a.last_active[a.pointers[s]] > stale_before;
+    const int pos = run + block_scan(f, &tot, sc);
+    if (f) a.move_src[pos] = s;
+    run += tot;
+  }
+  __syncthreads();
+
+  // ---- D: apply deletes to the bookkeeping ------------------------------------------------
+  for (int j = tid; j < n_evict; j += kWindowThreads) a.slot_of[a.evict_ids[j]] = -1;
+  for (int j = tid; j < n_moves; j += kWindowThreads) {
+    const int src = a.move_src[j], dst = a.evict_slots[j];
+    const int id = a.pointers[src];
+    a.move_dst[j] = dst;
+    a.pointers[dst] = id;
+    a.slot_of[id] = dst;
+    a.bias[dst] = a.bias[src];
+  }
+  __syncthreads();
+  for (int s = n_kept + tid; s < n; s += kWindowThreads) a.pointers[s] = -1;
+  __syncthreads();
+
+  // ---- E: rows for the neurons to bring in ------------------------------------------------
+  run = 0;
+  for (int b = 0; b < na; b += kWindowThreads) {
+    const int q = b + tid;
+    int id = -1, f = 0;
+    if (q < na) {
+      id = a.act[q];
+      f = a.slot_of[id] < 0;
+    }
+    const int pos = run + block_scan(f, &tot, sc);
+    if (f) {
+      const int s = n_kept + pos;
+      a.load_ids[pos] = id;
+      a.load_slots[pos] = s;
+      a.slot_of[id] = s;
+      a.pointers[s] = id;
+      a.bias[s] = a.bias_up[id];
+    }
+    run += tot;
+  }
+  __syncthreads();
+
+  // ---- F: slot lists ----------------------------------------------------------------------
+  run = 0;
+  for (int b = 0; b < na; b += kWindowThreads) {
+    const int q = b + tid;
+    int s = -1, f = 0;
+    if (q < na) {
+      const int id = a.act[q];
+      s = a.slot_of[id];
+      a.active_slots[q] = s;
+      if (a.active_idx != a.act) a.active_idx[q] = id;
+      f = s < n_kept;
+    }
+    const int pos = run + block_scan(f, &tot, sc);
+    if (f) a.hit_slots[pos] = s;
+    run += tot;
+  }
+  if (tid == 0) {
+    a.counts[LIF_CNT_N_ACTIVE] = na;
+    a.counts[LIF_CNT_N_EVICT] = n_evict;
+    a.counts[LIF_CNT_N_MOVES] = n_moves;
+    a.counts[LIF_CNT_N_LOAD] = n_load;
+    a.counts[LIF_CNT_N_HITS] = na - n_load;
+    a.counts[LIF_CNT_NUM_USED_BEFORE] = n;
+    a.counts[LIF_CNT_NUM_KEPT] = n_kept;
+    a.counts[LIF_CNT_NUM_USED] = n_kept + n_load;
+    a.counts[LIF_CNT_STEP] = t + 1;
+    unsigned long long* totals = reinterpret_cast<unsigned long long*>(a.counts + CNT_TOTALS);
+    totals[0] += (unsigned long long)n_load * a.bundle_bytes;
+    totals[1] += (unsigned long long)n_moves;
+  }
+}
+
+// Row moves of step D: cache row move_src[j] -> row move_dst[j].  Sources lie at or beyond
+// num_kept, destinations below it, so the copies never overlap.
+__global__ void __launch_bounds__(kThreads)
+move_rows_kernel(uint4* __restrict__ cache, const int32_t* __restrict__ move_src,
+                 const int32_t* __restrict__ move_dst, const int32_t* __restrict__ counts,
+                 int row_vec) {
+  const int n = counts[LIF_CNT_N_MOVES];
+  for (int j = blockIdx.x; j < n; j += gridDim.x) {
+    const uint4* src = cache + (size_t)move_src[j] * row_vec;
+    uint4* dst = cache + (size_t)move_dst[j] * row_vec;
+#pragma unroll 4
+    for (int v = threadIdx.x; v < row_vec; v += kThreads) dst[v] = src[v];
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+reset_kernel(int32_t* counts, int32_t* pointers, int32_t* slot_of, int32_t* last_active,
+             uint32_t* mask_words, int n_mask, int F, int cap) {
+  const int i = blockIdx.x * kThreads + threadIdx.x;
+  const int stride = gridDim.x * kThreads;
+  for (int j = i; j < LIF_CNT_LEN; j += stride) counts[j] = 0;
+  for (int j = i; j < cap; j += stride) pointers[j] = -1;
+  for (int j = i; j < F; j += stride) {
+    slot_of[j] = -1;
+    last_active[j] = kNever;
+  }
+  for (int j = i; j < n_mask; j += stride) mask_words[j] = 0;
+}
+
+}  // namespace
+
+cudaError_t launch_reset(lif_layer* L, cudaStream_t st) {
+  const lif_layer_desc& D = L->desc;
+  const int n_mask = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
+  reset_kernel<<<64, kThreads, 0, st>>>(L->counts, L->pointers, L->slot_of, L->last_active,
+                                        L->mask_words, n_mask, D.d_ff, D.capacity);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act,
+                          cudaStream_t st) {
+  const lif_layer_desc& D = L->desc;
+  WindowArgs a;
+  a.act = act;
+  a.n_act = n_act;
+  a.counts = L->counts;
+  a.pointers = L->pointers;
+  a.slot_of = L->slot_of;
+  a.last_active = L->last_active;
+  a.bias = L->bias;
+  a.bias_up = (const __half*)D.dev_bias_up;
+  a.active_idx = L->active_idx;
+  a.evict_ids = L->evict_ids;
+  a.evict_slots = L->evict_slots;
+  a.move_src = L->move_src;
+  a.move_dst = L->move_dst;
+  a.load_ids = L->load_ids;
+  a.load_slots = L->load_slots;
+  a.active_slots = L->active_slots;
+  a.hit_slots = L->hit_slots;
+  a.F = D.d_ff;
+  a.cap = D.capacity;
+  a.k = D.window_k;
+  a.bundle_bytes = 4ull * D.d_model;
+  window_update_kernel<<<1, kWindowThreads, 0, st>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  move_rows_kernel<<<L->move_grid, kThreads, 0, st>>>((uint4*)D.dev_cache, L->move_src,
+                                                      L->move_dst, L->counts, D.d_model / 4);
+  return cudaGetLastError();
+}
+
+}  // namespace lif
