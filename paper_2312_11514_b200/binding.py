@@ -1,0 +1,200 @@
+"""ctypes binding of liblif.so.  Argument marshalling only: every function forwards to the C
+entry point of the same name (include/lif.h); tensors are passed as raw addresses and
+``torch.cuda.Stream.cuda_stream`` handles.  There is no fallback: if the library is missing
+or cannot be loaded, importing users get an error."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "liblif.so")
+
+LIF_OK, LIF_ERR_INVALID_ARG, LIF_ERR_ALIGNMENT, LIF_ERR_CAPACITY, LIF_ERR_STATE, LIF_ERR_CUDA, \
+    LIF_ERR_TIMEOUT = range(7)
+(CNT_N_ACTIVE, CNT_N_EVICT, CNT_N_MOVES, CNT_N_LOAD, CNT_N_HITS, CNT_NUM_USED_BEFORE,
+ CNT_NUM_KEPT, CNT_NUM_USED, CNT_STEP, CNT_STATUS) = range(10)
+CNT_LEN = 64
+
+EXPORTS = [
+    "lif_status_str", "lif_workspace_bytes", "lif_create_layer", "lif_destroy_layer", "lif_reset",
+    "lif_predict", "lif_window_update", "lif_fetch_bundles", "lif_sparse_ffn", "lif_decode_step",
+    "lif_decode_token_host", "lif_get_lists", "lif_get_stats", "lif_clear_status",
+    "lif_probe_host_read",
+]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [
+        ("d_model", C.c_int32), ("d_ff", C.c_int32), ("rank", C.c_int32), ("window_k", C.c_int32),
+        ("capacity", C.c_int32), ("n_streams", C.c_int32), ("threshold_logit", C.c_float),
+        ("ffn_mode", C.c_int32), ("activation", C.c_int32),
+        ("host_bundles", C.c_void_p), ("dev_pred_A", C.c_void_p), ("dev_pred_B", C.c_void_p),
+        ("dev_pred_c", C.c_void_p), ("dev_bias_up", C.c_void_p), ("dev_bias_down", C.c_void_p),
+        ("dev_cache", C.c_void_p), ("dev_workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+    ]
+
+
+class Lists(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "counts", "active_idx", "evict_ids", "move_src", "move_dst", "load_ids", "load_slots",
+        "active_slots", "hit_slots", "pointers", "slot_of", "last_active", "bias")]
+
+
+class Stats(C.Structure):
+    _fields_ = [("counts", C.c_int32 * 16), ("bytes_fetched", C.c_uint64),
+                ("rows_moved", C.c_uint64), ("status", C.c_int32), ("reserved", C.c_int32)]
+
+
+class LifError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_str(code)} ({code})")
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """Load liblif.so (building it first if the sources are newer).  Raises if unavailable."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    from . import build as _build
+    if _build.needs_build():
+        _build.build()
+    L = C.CDLL(LIB_PATH)
+    vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+    L.lif_status_str.restype = C.c_char_p
+    L.lif_status_str.argtypes = [C.c_int]
+    sigs = {
+        "lif_workspace_bytes": [C.POINTER(LayerDesc), C.POINTER(sz)],
+        "lif_create_layer": [C.POINTER(LayerDesc), C.POINTER(vp)],
+        "lif_destroy_layer": [vp],
+        "lif_reset": [vp, vp],
+        "lif_predict": [vp, vp, vp, vp, vp, vp],
+        "lif_window_update": [vp, vp, vp, vp],
+        "lif_fetch_bundles": [vp, vp],
+        "lif_sparse_ffn": [vp, vp, vp, vp, vp, vp],
+        "lif_decode_step": [vp, vp, vp, vp, vp],
+        "lif_decode_token_host": [C.POINTER(vp), i32, vp, vp, vp, vp, vp, vp],
+        "lif_get_lists": [vp, C.POINTER(Lists)],
+        "lif_get_stats": [vp, C.POINTER(Stats)],
+        "lif_clear_status": [vp, vp],
+        "lif_probe_host_read": [vp, vp, sz, sz, vp],
+    }
+    for name, args in sigs.items():
+        fn = getattr(L, name)
+        fn.restype = C.c_int
+        fn.argtypes = args
+    _lib = L
+    return L
+
+
+def status_str(code: int) -> str:
+    return lib().lif_status_str(code).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != LIF_OK:
+        raise LifError(code, where)
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    return t if isinstance(t, int) else t.data_ptr()
+
+
+def _stream(s) -> Optional[int]:
+    if s is None:
+        return None
+    return s.cuda_stream if hasattr(s, "cuda_stream") else int(s)
+
+
+def make_desc(*, d_model, d_ff, rank, window_k, capacity, n_streams=1, threshold_logit=0.0,
+              ffn_mode=0, activation=0, host_bundles=None, pred_A=None, pred_B=None, pred_c=None,
+              bias_up=None, bias_down=None, cache=None, workspace=None) -> LayerDesc:
+    d = LayerDesc()
+    d.d_model, d.d_ff, d.rank, d.window_k, d.capacity = d_model, d_ff, rank, window_k, capacity
+    d.n_streams, d.threshold_logit, d.ffn_mode, d.activation = n_streams, threshold_logit, ffn_mode, activation
+    d.host_bundles = _ptr(host_bundles)
+    d.dev_pred_A, d.dev_pred_B, d.dev_pred_c = _ptr(pred_A), _ptr(pred_B), _ptr(pred_c)
+    d.dev_bias_up, d.dev_bias_down = _ptr(bias_up), _ptr(bias_down)
+    d.dev_cache, d.dev_workspace = _ptr(cache), _ptr(workspace)
+    d.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    return d
+
+
+def lif_workspace_bytes(desc: LayerDesc) -> int:
+    out = C.c_size_t(0)
+    _check(lib().lif_workspace_bytes(C.byref(desc), C.byref(out)), "lif_workspace_bytes")
+    return out.value
+
+
+def lif_create_layer(desc: LayerDesc) -> int:
+    out = C.c_void_p(None)
+    _check(lib().lif_create_layer(C.byref(desc), C.byref(out)), "lif_create_layer")
+    return out.value
+
+
+def lif_destroy_layer(layer: int) -> None:
+    _check(lib().lif_destroy_layer(layer), "lif_destroy_layer")
+
+
+def lif_reset(layer: int, stream=None) -> None:
+    _check(lib().lif_reset(layer, _stream(stream)), "lif_reset")
+
+
+def lif_predict(layer: int, x, logits, active_idx, n_active, stream=None) -> None:
+    _check(lib().lif_predict(layer, _ptr(x), _ptr(logits), _ptr(active_idx), _ptr(n_active),
+                             _stream(stream)), "lif_predict")
+
+
+def lif_window_update(layer: int, active_idx, n_active, stream=None) -> None:
+    _check(lib().lif_window_update(layer, _ptr(active_idx), _ptr(n_active), _stream(stream)),
+           "lif_window_update")
+
+
+def lif_fetch_bundles(layer: int, stream=None) -> None:
+    _check(lib().lif_fetch_bundles(layer, _stream(stream)), "lif_fetch_bundles")
+
+
+def lif_sparse_ffn(layer: int, x, slots, n_slots, y, stream=None) -> None:
+    _check(lib().lif_sparse_ffn(layer, _ptr(x), _ptr(slots), _ptr(n_slots), _ptr(y),
+                                _stream(stream)), "lif_sparse_ffn")
+
+
+def lif_decode_step(layer: int, x, y, compute_stream=None, fetch_stream=None) -> None:
+    _check(lib().lif_decode_step(layer, _ptr(x), _ptr(y), _stream(compute_stream),
+                                 _stream(fetch_stream)), "lif_decode_step")
+
+
+def lif_decode_token_host(layers, host_x, dev_x, dev_y, host_y, compute_stream=None,
+                          fetch_stream=None) -> None:
+    arr = (C.c_void_p * len(layers))(*layers)
+    _check(lib().lif_decode_token_host(arr, len(layers), _ptr(host_x), _ptr(dev_x), _ptr(dev_y),
+                                       _ptr(host_y), _stream(compute_stream),
+                                       _stream(fetch_stream)), "lif_decode_token_host")
+
+
+def lif_get_lists(layer: int) -> Lists:
+    out = Lists()
+    _check(lib().lif_get_lists(layer, C.byref(out)), "lif_get_lists")
+    return out
+
+
+def lif_get_stats(layer: int) -> Stats:
+    out = Stats()
+    _check(lib().lif_get_stats(layer, C.byref(out)), "lif_get_stats")
+    return out
+
+
+def lif_clear_status(layer: int, stream=None) -> None:
+    _check(lib().lif_clear_status(layer, _stream(stream)), "lif_clear_status")
+
+
+def lif_probe_host_read(host_src, dev_dst, nbytes: int, chunk_bytes: int, stream=None) -> None:
+    _check(lib().lif_probe_host_read(_ptr(host_src), _ptr(dev_dst), nbytes, chunk_bytes,
+                                     _stream(stream)), "lif_probe_host_read")

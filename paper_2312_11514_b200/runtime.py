@@ -1,0 +1,103 @@
+"""Device-memory plumbing around the C ABI: allocates the buffers a layer needs with torch
+(pinned bundle store, window cache, workspace), creates the layer, and exposes the lists
+inside the workspace as tensor views.  No arithmetic of the method lives here."""
+from __future__ import annotations
+
+from typing import Dict, List, Optional
+
+import torch
+
+from . import binding as B
+
+
+class Layer:
+    """One FFN layer: owns its torch buffers and the `lif_layer` handle."""
+
+    def __init__(self, *, d_model: int, d_ff: int, rank: int, window_k: int, capacity: int,
+                 host_bundles: torch.Tensor, pred_A: torch.Tensor, pred_B: torch.Tensor,
+                 pred_c: torch.Tensor, bias_up: torch.Tensor,
+                 bias_down: Optional[torch.Tensor] = None, n_streams: int = 1,
+                 threshold_logit: float = 0.0, ffn_mode: int = 0, device="cuda:0"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_2312_11514_b200 needs a CUDA device; there is no CPU path")
+        self.device = torch.device(device)
+        assert host_bundles.is_pinned() and host_bundles.dtype == torch.float16
+        assert host_bundles.shape == (d_ff, 2 * d_model) and host_bundles.is_contiguous()
+        self.d_model, self.d_ff, self.rank, self.capacity = d_model, d_ff, rank, capacity
+        self.n_streams = n_streams
+        self.keep = dict(host_bundles=host_bundles, pred_A=pred_A, pred_B=pred_B, pred_c=pred_c,
+                         bias_up=bias_up, bias_down=bias_down)
+        self.cache = torch.zeros(capacity, 2 * d_model, dtype=torch.float16, device=self.device)
+        shape = dict(d_model=d_model, d_ff=d_ff, rank=rank, window_k=window_k, capacity=capacity,
+                     n_streams=n_streams, threshold_logit=threshold_logit, ffn_mode=ffn_mode)
+        nbytes = B.lif_workspace_bytes(B.make_desc(**shape))
+        self.workspace = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
+        with torch.cuda.device(self.device):
+            self.handle = B.lif_create_layer(B.make_desc(
+                **shape, host_bundles=host_bundles, pred_A=pred_A, pred_B=pred_B, pred_c=pred_c,
+                bias_up=bias_up, bias_down=bias_down, cache=self.cache, workspace=self.workspace))
+            torch.cuda.synchronize()   # the reset ran on the default stream
+        self._lists = B.lif_get_lists(self.handle)
+        self.counts = self._view("counts", B.CNT_LEN)
+
+    def _view(self, name: str, n: int, dtype=torch.int32) -> torch.Tensor:
+        off = getattr(self._lists, name) - self.workspace.data_ptr()
+        size = n * torch.empty((), dtype=dtype).element_size()
+        return self.workspace[off:off + size].view(dtype)
+
+    def lists(self) -> Dict[str, object]:
+        """Host copies of this step's lists and of the window state (synchronises)."""
+        torch.cuda.synchronize(self.device)
+        c = self.counts.cpu()
+        na, ne, nm, nl, nh = (int(c[i]) for i in (B.CNT_N_ACTIVE, B.CNT_N_EVICT, B.CNT_N_MOVES,
+                                                  B.CNT_N_LOAD, B.CNT_N_HITS))
+        F, cap = self.d_ff, self.capacity
+        out = {
+            "active_idx": self._view("active_idx", F)[:na], "evict_ids": self._view("evict_ids", cap)[:ne],
+            "move_src": self._view("move_src", cap)[:nm], "move_dst": self._view("move_dst", cap)[:nm],
+            "load_ids": self._view("load_ids", cap)[:nl], "load_slots": self._view("load_slots", cap)[:nl],
+            "active_slots": self._view("active_slots", F)[:na], "hit_slots": self._view("hit_slots", F)[:nh],
+            "pointers": self._view("pointers", cap), "slot_of": self._view("slot_of", F),
+            "last_active": self._view("last_active", F),
+            "bias": self._view("bias", cap, torch.float16),
+        }
+        out = {k: v.cpu().numpy() for k, v in out.items()}
+        out.update(num_used_before=int(c[B.CNT_NUM_USED_BEFORE]), num_kept=int(c[B.CNT_NUM_KEPT]),
+                   num_used=int(c[B.CNT_NUM_USED]), step=int(c[B.CNT_STEP]), status=int(c[B.CNT_STATUS]))
+        return out
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            torch.cuda.synchronize(self.device)
+            B.lif_destroy_layer(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def pinned_store(d_ff: int, d_model: int) -> torch.Tensor:
+    """Pinned (and, under unified addressing, device-mapped) host tensor for one layer's
+    bundle store, fp16 [d_ff][2*d_model]."""
+    return torch.empty(d_ff, 2 * d_model, dtype=torch.float16, pin_memory=True)
+
+
+def build_stack(cfg, device="cuda:0", n_layers: Optional[int] = None, capacity_margin: float = 8.0,
+                ffn_mode: int = 0, gen_device=None) -> List[Layer]:
+    """Generate the weights of a named synthetic configuration and create its layers."""
+    from . import workloads as W
+    layers = []
+    gen_device = gen_device or device
+    for l in range(n_layers or cfg.n_layers):
+        store = pinned_store(cfg.d_ff, cfg.d_model)
+        w = W.make_layer(cfg, l, device=gen_device, bundles_out=store)
+        cap = W.window_capacity(cfg, w["p"], capacity_margin)
+        dev = lambda t: t.to(device).contiguous()
+        layers.append(Layer(d_model=cfg.d_model, d_ff=cfg.d_ff, rank=cfg.rank, window_k=cfg.window_k,
+                            capacity=cap, host_bundles=store, pred_A=dev(w["A"]), pred_B=dev(w["B"]),
+                            pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), n_streams=cfg.n_streams,
+                            ffn_mode=ffn_mode, device=device))
+    return layers

@@ -1,0 +1,138 @@
+"""Shared helpers of the GPU parity tests: tolerances and the teacher-forced comparison of the
+CUDA path (through the C ABI) with the CPU oracle, stage by stage."""
+import numpy as np
+import torch
+
+from oracle import lif_oracle as O
+from paper_2312_11514_b200 import binding as B
+from paper_2312_11514_b200 import runtime as R
+from paper_2312_11514_b200 import workloads as W
+
+REL = 2e-3          # max relative error on FFN outputs and predictor scores (fp16 storage, fp32 accumulate)
+BORDER = 1e-3       # mask disagreement is allowed only where |score - theta| < BORDER
+LIST_KEYS = ("evict_ids", "move_src", "move_dst", "load_ids", "load_slots", "active_slots", "hit_slots")
+
+
+def assert_logits_close(got, ref):
+    tol = REL * np.maximum(np.abs(ref), 1.0)
+    bad = np.abs(got - ref) > tol
+    assert not bad.any(), f"{bad.sum()} scores off, worst {np.abs(got - ref).max():.3e}"
+
+
+def assert_mask_borderline(act_gpu, ref_logits, theta):
+    """The GPU's active list may differ from the oracle's only on neurons whose oracle score
+    is within BORDER of the threshold."""
+    ref_act = O.active_set(ref_logits, theta)
+    diff = np.setxor1d(act_gpu, ref_act)
+    if diff.size:
+        margin = np.abs(ref_logits[:, diff] - theta).min(axis=0)
+        assert (margin < BORDER).all(), f"mask differs away from the threshold: {diff[margin >= BORDER]}"
+    assert (np.diff(act_gpu) > 0).all()
+    return diff.size
+
+
+def assert_y_close(got, ref):
+    rms = np.sqrt(np.mean(ref * ref, axis=-1, keepdims=True))
+    tol = REL * np.maximum(np.abs(ref), rms) + 1e-30
+    bad = np.abs(got - ref) > tol
+    assert not bad.any(), f"{bad.sum()} outputs off, worst ratio {(np.abs(got - ref) / tol).max():.3f}"
+
+
+class OracleLayer:
+    """Oracle-side twin of one layer, fed with the same tensors."""
+
+    def __init__(self, w, d_model, d_ff, capacity, window_k, theta=0.0, b_down=None):
+        self.A = w["A"].cpu().numpy().astype(np.float64)
+        self.B = w["B"].cpu().numpy().astype(np.float64)
+        self.c = w["c"].cpu().numpy().astype(np.float64)
+        self.bundles = w["bundles"].cpu().numpy()
+        self.bias_up = w["bias_up"].cpu().numpy()
+        self.b_down = None if b_down is None else b_down.cpu().numpy()
+        self.theta = theta
+        self.cache = O.NeuronCache(d_model, d_ff, capacity, window_k)
+
+
+def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_down=False,
+                    device="cuda:0"):
+    store = R.pinned_store(cfg.d_ff, cfg.d_model)
+    w = W.make_layer(cfg, layer_idx, device=device, bundles_out=store)
+    cap = capacity or W.window_capacity(cfg, w["p"])
+    bd = None
+    if b_down:
+        g = torch.Generator(device="cpu").manual_seed(77 + layer_idx)
+        bd = (torch.randn(cfg.d_model, generator=g) * 0.1).to(torch.float16).to(device)
+    dev = lambda t: t.to(device).contiguous()
+    gpu = R.Layer(d_model=cfg.d_model, d_ff=cfg.d_ff, rank=cfg.rank, window_k=cfg.window_k,
+                  capacity=cap, host_bundles=store, pred_A=dev(w["A"]), pred_B=dev(w["B"]),
+                  pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), bias_down=bd,
+                  n_streams=cfg.n_streams, threshold_logit=theta, ffn_mode=ffn_mode, device=device)
+    ora = OracleLayer(w, cfg.d_model, cfg.d_ff, cap, cfg.window_k, theta, bd)
+    return gpu, ora
+
+
+def compare_lists_and_state(gpu, ora, ref_lists):
+    g = gpu.lists()
+    assert g["status"] == B.LIF_OK
+    for key in LIST_KEYS:
+        np.testing.assert_array_equal(g[key], ref_lists[key], err_msg=key)
+    for key in ("num_used_before", "num_kept", "num_used"):
+        assert g[key] == ref_lists[key], key
+    c = ora.cache
+    assert g["step"] == c.t
+    np.testing.assert_array_equal(g["pointers"], c.pointers)
+    np.testing.assert_array_equal(g["slot_of"], c.slot_of)
+    np.testing.assert_array_equal(g["last_active"], c.last_active)
+    return g
+
+
+def compare_cache_rows(gpu, ora):
+    n = ora.cache.num_used
+    rows = gpu.cache[:n].cpu().numpy()
+    assert np.array_equal(rows.view(np.uint16), ora.cache.matrix[:n].view(np.uint16))
+    bias = gpu.lists()["bias"][:n]
+    assert np.array_equal(bias.view(np.uint16), ora.cache.bias[:n].view(np.uint16))
+
+
+def make_bufs(gpu, device="cuda:0"):
+    S, F, d = gpu.n_streams, gpu.d_ff, gpu.d_model
+    return dict(logits=torch.empty(S, F, dtype=torch.float32, device=device),
+                act=torch.empty(F, dtype=torch.int32, device=device),
+                n_act=torch.zeros(1, dtype=torch.int32, device=device),
+                y=torch.empty(S, d, dtype=torch.float32, device=device))
+
+
+def staged_step(gpu, ora, x_dev, bufs, whole_cache=False):
+    """One token through the four staged entry points, each compared with the oracle run from
+    the GPU's own active list (so borderline predictor decisions do not cascade)."""
+    F = gpu.d_ff
+    logits, act, n_act, y = bufs["logits"], bufs["act"], bufs["n_act"], bufs["y"]
+    B.lif_predict(gpu.handle, x_dev, logits, act, n_act)
+    torch.cuda.synchronize()
+    x_np = x_dev.cpu().numpy()
+    ref_logits = O.predictor_logits(x_np, ora.A, ora.B, ora.c)
+    assert_logits_close(logits.cpu().numpy().astype(np.float64), ref_logits)
+    na = int(n_act.item())
+    act_gpu = act[:na].cpu().numpy()
+    n_border = assert_mask_borderline(act_gpu, ref_logits, ora.theta)
+
+    B.lif_window_update(gpu.handle, act, n_act)
+    ref_lists = ora.cache.window_update(act_gpu)
+    g = compare_lists_and_state(gpu, ora, ref_lists)
+    np.testing.assert_array_equal(g["active_idx"], act_gpu)
+
+    B.lif_fetch_bundles(gpu.handle)
+    ora.cache.insert(ref_lists, ora.bundles, ora.bias_up)
+    compare_cache_rows(gpu, ora)
+
+    if whole_cache:
+        B.lif_sparse_ffn(gpu.handle, x_dev, None, gpu.counts[B.CNT_NUM_USED:], y)
+        slots = np.arange(ora.cache.num_used)
+    else:
+        B.lif_sparse_ffn(gpu.handle, x_dev, gpu._view("active_slots", F),
+                         gpu.counts[B.CNT_N_ACTIVE:], y)
+        slots = ref_lists["active_slots"]
+    torch.cuda.synchronize()
+    ref_y = O.sparse_ffn(ora.cache.matrix, ora.cache.bias, slots, x_np, ora.b_down)
+    assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
+    return dict(n_active=na, n_load=len(ref_lists["load_ids"]), n_evict=len(ref_lists["evict_ids"]),
+                n_border=n_border)

@@ -1,0 +1,191 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs — scores and outputs within 2e-3, index lists and window state bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lif_oracle as O
+from paper_2312_11514_b200 import binding as B
+from paper_2312_11514_b200 import runtime as R
+from paper_2312_11514_b200 import workloads as W
+
+import parity_util as P
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _run_staged(cfg, layer_idx, steps, **kw):
+    whole = kw.get("ffn_mode", 0) == 1
+    gpu, ora = P.make_layer_pair(cfg, layer_idx, **kw)
+    X = W.make_inputs(cfg, device=DEV)
+    bufs = P.make_bufs(gpu)
+    stats = [P.staged_step(gpu, ora, X[t], bufs, whole_cache=whole) for t in range(steps)]
+    st = B.lif_get_stats(gpu.handle)
+    assert st.status == B.LIF_OK
+    assert st.bytes_fetched == ora.cache.bytes_fetched == sum(s["n_load"] for s in stats) * cfg.bundle_bytes
+    assert st.rows_moved == ora.cache.rows_moved
+    gpu.close()
+    return stats
+
+
+@pytest.mark.parametrize("layer_idx", [0, 1])
+def test_tiny_config_every_stage_every_step(layer_idx):
+    cfg = W.CONFIGS["tiny"]
+    stats = _run_staged(cfg, layer_idx, cfg.steps, b_down=(layer_idx == 1))
+    assert stats[0]["n_load"] == stats[0]["n_active"] > 0            # cold start
+    assert sum(s["n_evict"] for s in stats) > 0
+
+
+@pytest.mark.parametrize("d,F,r,k,S", [
+    (264, 1000, 24, 3, 1),      # ragged: nothing a multiple of the tile sizes
+    (328, 2056, 8, 1, 1),       # window of one token, smallest rank
+    (4544, 1280, 128, 2, 1),    # Falcon row length (71 x 64), several rows per CTA round
+    (512, 4096, 40, 4, 3),      # three streams
+    (256, 1536, 16, 2, 8),      # eight streams
+])
+def test_ragged_shapes_and_streams(d, F, r, k, S):
+    cfg = W.LifConfig("ragged", 1, d, F, r, k, S, 12, 0.06, 1.0, 0.8, 0.6, 11)
+    stats = _run_staged(cfg, 0, cfg.steps, b_down=True)
+    assert sum(s["n_evict"] for s in stats) > 0
+
+
+def test_whole_cache_mode_and_more_rows_than_stages():
+    # mode 1 runs the FFN over every cached row (matrix[:num_used]); with ~40% firing the
+    # cache holds far more rows than CTAs x stages of a tiny grid would cover in one round
+    cfg = W.LifConfig("dense", 1, 2048, 8192, 32, 3, 1, 6, 0.40, 0.5, 0.8, 0.6, 12)
+    stats = _run_staged(cfg, 0, cfg.steps, ffn_mode=1, capacity=8192)
+    assert max(s["n_active"] for s in stats) > 148 * 16
+
+
+def test_threshold_extremes():
+    cfg = W.CONFIGS["tiny"]
+    X = W.make_inputs(cfg, device=DEV)
+    # theta = +inf: nothing is active, y = b_down
+    gpu, ora = P.make_layer_pair(cfg, 0, theta=float("inf"), b_down=True)
+    bufs = P.make_bufs(gpu)
+    s = P.staged_step(gpu, ora, X[0], bufs)
+    assert s["n_active"] == 0
+    np.testing.assert_array_equal(bufs["y"].cpu().numpy()[0], ora.b_down.astype(np.float32))
+    gpu.close()
+    # theta = -inf: every neuron is active; the sparse FFN over all rows is the dense FFN
+    gpu, ora = P.make_layer_pair(cfg, 0, theta=float("-inf"), capacity=cfg.d_ff)
+    bufs = P.make_bufs(gpu)
+    s = P.staged_step(gpu, ora, X[0], bufs)
+    assert s["n_active"] == cfg.d_ff == s["n_load"]
+    Wb = ora.bundles.astype(np.float64)
+    x = X[0, 0].cpu().numpy().astype(np.float64)
+    dense = np.maximum(Wb[:, :cfg.d_model] @ x + ora.bias_up.astype(np.float64), 0) @ Wb[:, cfg.d_model:]
+    P.assert_y_close(bufs["y"].cpu().numpy().astype(np.float64), dense[None, :])
+    s = P.staged_step(gpu, ora, X[1], bufs)
+    assert s["n_load"] == 0 and s["n_evict"] == 0
+    gpu.close()
+
+
+def test_capacity_overflow_sets_status_and_leaves_state():
+    cfg = W.CONFIGS["tiny"]
+    X = W.make_inputs(cfg, device=DEV)
+    gpu, ora = P.make_layer_pair(cfg, 0, capacity=64)
+    bufs = P.make_bufs(gpu)
+    act = torch.arange(0, 40, dtype=torch.int32, device=DEV)
+    n = torch.tensor([40], dtype=torch.int32, device=DEV)
+    B.lif_window_update(gpu.handle, act, n)
+    B.lif_fetch_bundles(gpu.handle)
+    before = gpu.lists()
+    assert before["status"] == B.LIF_OK and before["num_used"] == 40
+    act2 = torch.arange(100, 130, dtype=torch.int32, device=DEV)      # 40 kept + 30 new > 64
+    n2 = torch.tensor([30], dtype=torch.int32, device=DEV)
+    B.lif_window_update(gpu.handle, act2, n2)
+    B.lif_fetch_bundles(gpu.handle)
+    B.lif_sparse_ffn(gpu.handle, X[0], gpu._view("active_slots", cfg.d_ff), gpu.counts[B.CNT_N_ACTIVE:], bufs["y"])
+    after = gpu.lists()
+    assert after["status"] == B.LIF_ERR_CAPACITY
+    assert B.lif_get_stats(gpu.handle).status == B.LIF_ERR_CAPACITY
+    for key in ("pointers", "slot_of", "last_active"):
+        np.testing.assert_array_equal(before[key], after[key])
+    assert (after["num_used"], after["step"]) == (before["num_used"], before["step"])
+    assert len(after["load_ids"]) == 0 and len(after["active_slots"]) == 0
+    assert (bufs["y"].cpu().numpy() == 0).all()                       # nothing active, no b_down
+    # out-of-range neuron id: refused the same way
+    B.lif_clear_status(gpu.handle)
+    bad = torch.tensor([5, 5000], dtype=torch.int32, device=DEV)
+    B.lif_window_update(gpu.handle, bad, torch.tensor([2], dtype=torch.int32, device=DEV))
+    assert gpu.lists()["status"] == B.LIF_ERR_INVALID_ARG
+    # after clearing, a fitting step proceeds and matches the oracle
+    B.lif_clear_status(gpu.handle)
+    ora.cache.window_update(np.arange(40, dtype=np.int32))
+    act3 = torch.arange(30, 50, dtype=torch.int32, device=DEV)
+    B.lif_window_update(gpu.handle, act3, torch.tensor([20], dtype=torch.int32, device=DEV))
+    ref = ora.cache.window_update(np.arange(30, 50, dtype=np.int32))
+    P.compare_lists_and_state(gpu, ora, ref)
+    gpu.close()
+
+
+def test_reset_gives_cold_cache_and_runs_are_reproducible():
+    cfg = W.CONFIGS["tiny"]
+    X = W.make_inputs(cfg, device=DEV)
+    gpu, ora = P.make_layer_pair(cfg, 0)
+    y = torch.empty(8, cfg.n_streams, cfg.d_model, dtype=torch.float32, device=DEV)
+    runs = []
+    for _ in range(2):
+        B.lif_reset(gpu.handle)
+        acts = []
+        for t in range(8):
+            B.lif_decode_step(gpu.handle, X[t], y[t])
+            acts.append(gpu.lists()["active_idx"].copy())
+        runs.append((acts, y.cpu().numpy().copy(), gpu.lists()))
+    for a, b in zip(runs[0][0], runs[1][0]):
+        np.testing.assert_array_equal(a, b)
+    assert np.array_equal(runs[0][1].view(np.uint32), runs[1][1].view(np.uint32))     # bitwise
+    np.testing.assert_array_equal(runs[0][2]["pointers"], runs[1][2]["pointers"])
+    assert runs[1][2]["step"] == 8
+    gpu.close()
+
+
+@pytest.mark.parametrize("two_streams", [False, True])
+def test_decode_step_matches_oracle_decode_step(two_streams):
+    cfg = W.CONFIGS["tiny"]
+    X = W.make_inputs(cfg, device=DEV)
+    gpu, ora = P.make_layer_pair(cfg, 1, b_down=True)
+    y = torch.empty(cfg.n_streams, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = (torch.cuda.Stream(), torch.cuda.Stream()) if two_streams else (None, None)
+    if sc is not None:
+        sc.wait_stream(torch.cuda.current_stream())
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        g = gpu.lists()
+        x_np = X[t].cpu().numpy()
+        logits, act, lists, ref_y = O.decode_step(ora.cache, x_np, ora.A, ora.B, ora.c, ora.theta,
+                                                  ora.bundles, ora.bias_up, ora.b_down,
+                                                  act=g["active_idx"])
+        P.assert_mask_borderline(g["active_idx"], logits, ora.theta)
+        P.compare_lists_and_state(gpu, ora, lists)
+        P.compare_cache_rows(gpu, ora)
+        P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
+    gpu.close()
+
+
+def test_decode_token_host_matches_per_layer_decode_steps():
+    cfg = W.CONFIGS["tiny"]
+    X = W.make_inputs(cfg, device=DEV)
+    a = R.build_stack(cfg, DEV)
+    b = R.build_stack(cfg, DEV)
+    L, S, d = cfg.n_layers, cfg.n_streams, cfg.d_model
+    host_x = torch.empty(S, d, dtype=torch.float16, pin_memory=True)
+    host_y = torch.empty(L, S, d, dtype=torch.float32, pin_memory=True)
+    dev_x = torch.empty(S, d, dtype=torch.float16, device=DEV)
+    dev_y = torch.empty(L, S, d, dtype=torch.float32, device=DEV)
+    y_ref = torch.empty(L, S, d, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for t in range(10):
+        host_x.copy_(X[t])
+        B.lif_decode_token_host([l.handle for l in a], host_x, dev_x, dev_y, host_y, sc, sf)
+        for l in range(L):
+            B.lif_decode_step(b[l].handle, X[t], y_ref[l])
+        torch.cuda.synchronize()
+        assert torch.equal(host_y, y_ref.cpu())
+    for l in range(L):
+        assert B.lif_get_stats(a[l].handle).bytes_fetched == B.lif_get_stats(b[l].handle).bytes_fetched > 0
+    for l in a + b:
+        l.close()
