@@ -116,6 +116,8 @@ typedef struct {
   int32_t counts[16];       /* counts block entries 0..15 of the last step */
   uint64_t bytes_fetched;   /* cumulative: sum of n_load * bundle bytes */
   uint64_t rows_moved;      /* cumulative */
+  uint64_t rows_active;     /* cumulative: sum of n_active over steps */
+  uint64_t rows_cached;     /* cumulative: sum of num_used over steps */
   int32_t status;           /* sticky device status (lif_status) */
   int32_t reserved;
 } lif_stats;

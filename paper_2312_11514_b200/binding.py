@@ -44,7 +44,8 @@ class Lists(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [("counts", C.c_int32 * 16), ("bytes_fetched", C.c_uint64),
-                ("rows_moved", C.c_uint64), ("status", C.c_int32), ("reserved", C.c_int32)]
+                ("rows_moved", C.c_uint64), ("rows_active", C.c_uint64),
+                ("rows_cached", C.c_uint64), ("status", C.c_int32), ("reserved", C.c_int32)]
 
 
 class LifError(RuntimeError):

@@ -294,6 +294,8 @@ lif_status lif_get_stats(lif_layer* L, lif_stats* o) {
   const uint64_t* totals = reinterpret_cast<const uint64_t*>(host + CNT_TOTALS);
   o->bytes_fetched = totals[0];
   o->rows_moved = totals[1];
+  o->rows_active = totals[2];
+  o->rows_cached = totals[3];
   o->status = host[LIF_CNT_STATUS];
   o->reserved = 0;
   return LIF_OK;

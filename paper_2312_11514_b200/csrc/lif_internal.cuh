@@ -12,7 +12,7 @@ namespace lif {
 // Private entries of the counts block (public ones: LIF_CNT_* in lif.h).
 enum {
   CNT_TICKET_PREDICT = 16,  // "last block done" counter of the score kernel
-  CNT_TOTALS = 32           // two uint64: bytes_fetched, rows_moved (8-byte aligned)
+  CNT_TOTALS = 32           // four uint64: bytes_fetched, rows_moved, rows_active, rows_cached
 };
 
 constexpr int kNever = -(1 << 30);  // last_active stamp of a neuron never predicted active

@@ -204,6 +204,8 @@ __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArg
     unsigned long long* totals = reinterpret_cast<unsigned long long*>(a.counts + CNT_TOTALS);
     totals[0] += (unsigned long long)n_load * a.bundle_bytes;
     totals[1] += (unsigned long long)n_moves;
+    totals[2] += (unsigned long long)na;
+    totals[3] += (unsigned long long)(n_kept + n_load);
   }
 }
 
