@@ -172,41 +172,49 @@ def run_ours(args):
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1))
 
-    # ---- pass 3: staged entry points with events between them (per-kernel durations) ---------
-    phases = ("predict", "window", "fetch", "ffn")
-    acts = [torch.empty(cfg.d_ff, dtype=torch.int32, device=dev) for _ in range(L)]
-    nact = torch.zeros(L, dtype=torch.int32, device=dev)
-    slots = [l._view("active_slots", cfg.d_ff) for l in layers]
-    evs = [[[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(L)] for _ in range(K)]
+    # ---- pass 3: same loop as pass 1 with the library's per-kernel CUDA events switched on ----
     reset()
-    for t in range(n_tok):
+    for t in range(Wm):
         for l in range(L):
-            h = handles[l]
-            ev = evs[t - Wm][l] if t >= Wm else None
-            if ev: ev[0].record(sc)
-            B.lif_predict(h, X[t], None, acts[l], nact[l:], sc)
-            if ev: ev[1].record(sc)
-            B.lif_window_update(h, acts[l], nact[l:], sc)
-            if ev: ev[2].record(sc)
-            B.lif_fetch_bundles(h, sc)
-            if ev: ev[3].record(sc)
-            B.lif_sparse_ffn(h, X[t], slots[l], layers[l].counts[B.CNT_N_ACTIVE:], Y[l], sc)
-            if ev: ev[4].record(sc)
+            B.lif_decode_step(handles[l], X[t], Y[l], sc, sf)
     barrier()
-    phase_ms = {p: 0.0 for p in phases}
-    for t in range(K):
+    for h in handles:
+        B.lif_timing_enable(h, K)
+    for t in range(Wm, n_tok):
         for l in range(L):
-            for i, p in enumerate(phases):
-                phase_ms[p] += evs[t][l][i].elapsed_time(evs[t][l][i + 1])
+            B.lif_decode_step(handles[l], X[t], Y[l], sc, sf)
+    barrier()
+    phase_us = {p: 0.0 for p in B.PHASES}
+    for h in handles:
+        us, n_rec = B.lif_timing_read(h)
+        assert n_rec == K
+        for p in B.PHASES:
+            phase_us[p] += us[p]
+        B.lif_timing_enable(h, 0)
     n_launch = K * L
+
+    # host-link peak: pinned host -> device cudaMemcpyAsync of 1 GiB, best of 5
+    link_peak = None
+    if rank == 0:
+        nb = 1 << 30
+        hbuf = torch.empty(nb, dtype=torch.uint8, pin_memory=True)
+        dbuf = torch.empty(nb, dtype=torch.uint8, device=dev)
+        best = float("inf")
+        for _ in range(5):
+            e0.record(); dbuf.copy_(hbuf, non_blocking=True); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        link_peak = nb / best / 1e6
+        del hbuf, dbuf
 
     if rank == 0:
         beta = cfg.bundle_bytes
         peak, peak_kind = _peaks()
         ffn_bytes = rows_active * (beta + 2) + n_launch * S * (2 * d + 4 * d)
-        ffn_s = phase_ms["ffn"] / 1e3
-        ffn_gbs = ffn_bytes / ffn_s / 1e9
-        fetch_gbs = fetched / (phase_ms["fetch"] / 1e3) / 1e9
+        ffn_gbs = ffn_bytes / (phase_us["ffn"] * 1e-6) / 1e9
+        fetch_gbs = fetched / (phase_us["fetch"] * 1e-6) / 1e9
+        pred_bytes = n_launch * (2 * cfg.rank * (d + cfg.d_ff) + 4 * cfg.d_ff)
+        pred_gbs = pred_bytes / ((phase_us["predict_z"] + phase_us["predict_scores"]) * 1e-6) / 1e9
         out = {
             "metric": METRIC, "value": world * K / (ms_total / 1e3), "unit": UNIT,
             "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms_total / K,
@@ -222,15 +230,18 @@ def run_ours(args):
                     "h2d_bytes_per_step": S * d * 2, "d2h_bytes_per_step": L * S * d * 4,
                     "host_link_bytes_per_step": fetched / K},
             "gpu_launches": 7 * n_launch,
-            "roofline": {"kernel": "sparse_ffn (gather kernel + partial-sum kernel)", "bound": "hbm",
+            "roofline": {"kernel": "sparse_ffn_kernel", "bound": "hbm",
                          "achieved": ffn_gbs, "peak": peak, "unit": "GB/s", "frac": ffn_gbs / peak,
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": ffn_gbs / NOMINAL_HBM_GBS,
-                         "traffic": None, "us_per_launch": phase_ms["ffn"] * 1e3 / n_launch,
+                         "traffic": None, "us_per_launch": phase_us["ffn"] / n_launch,
                          "bytes_per_launch": ffn_bytes / n_launch},
-            "host_link": {"kernel": "fetch", "achieved": fetch_gbs, "unit": "GB/s",
+            "host_link": {"kernel": "fetch_kernel", "bound": "host_link", "achieved": fetch_gbs,
+                          "peak": link_peak, "unit": "GB/s", "frac": fetch_gbs / link_peak,
+                          "peak_kind": "of measured (1 GiB pinned cudaMemcpyAsync, this run)",
                           "bytes_per_launch": fetched / n_launch,
-                          "us_per_launch": phase_ms["fetch"] * 1e3 / n_launch},
-            "phase_us_per_layer": {p: phase_ms[p] * 1e3 / n_launch for p in phases},
+                          "us_per_launch": phase_us["fetch"] / n_launch},
+            "predictor": {"bound": "hbm", "achieved": pred_gbs, "unit": "GB/s", "frac": pred_gbs / peak},
+            "phase_us_per_layer": {p: phase_us[p] / n_launch for p in B.PHASES},
             "per_token": {"rows_active": rows_active / K, "rows_loaded": fetched / beta / K,
                           "rows_moved": rows_moved / K},
             "clocks": clock_info,

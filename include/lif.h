@@ -49,7 +49,7 @@ typedef struct lif_layer lif_layer;
  * down-projection column `pointers[s]` (Section 3.2, bundling columns and rows). */
 typedef struct {
   int32_t d_model;          /* multiple of 8, <= 8192 */
-  int32_t d_ff;             /* multiple of 8 */
+  int32_t d_ff;             /* multiple of 8, < 2^21 */
   int32_t rank;             /* predictor rank r, multiple of 8, <= 2048 */
   int32_t window_k;         /* tokens kept in the window, current one included, >= 1 */
   int32_t capacity;         /* rows of the cache (the paper's Req_i), 1..d_ff */
@@ -189,6 +189,26 @@ lif_status lif_get_stats(lif_layer* layer, lif_stats* host_out);
 
 /* Clears the sticky device status word. */
 lif_status lif_clear_status(lif_layer* layer, void* stream);
+
+/* Phases timed by lif_timing_* (one CUDA event pair each, inside lif_decode_step). */
+enum {
+  LIF_PHASE_PREDICT_Z = 0,      /* x.A partial sums */
+  LIF_PHASE_PREDICT_SCORES = 1, /* scores, threshold, compaction */
+  LIF_PHASE_WINDOW = 2,         /* window bookkeeping kernel */
+  LIF_PHASE_MOVES = 3,          /* row moves */
+  LIF_PHASE_FETCH = 4,          /* bundle fetch (on the fetch stream) */
+  LIF_PHASE_FFN = 5,            /* sparse FFN gather kernel(s) */
+  LIF_PHASE_FFN_SUM = 6,        /* partial-sum kernel(s) */
+  LIF_PHASE_LEN = 8
+};
+
+/* Profiling aid: with n_steps > 0, the next n_steps calls of lif_decode_step record CUDA
+ * events around every kernel (host-side event objects, no device memory); n_steps = 0 turns
+ * it off and frees the events.  lif_timing_read synchronises the device and returns, per
+ * phase, the summed device time in microseconds over the steps recorded since enabling. */
+lif_status lif_timing_enable(lif_layer* layer, int32_t n_steps);
+lif_status lif_timing_read(lif_layer* layer, float* host_us_sums /* [LIF_PHASE_LEN] */,
+                           int32_t* host_n_steps);
 
 /* Bandwidth probe for the host link: a kernel reads `bytes` of mapped pinned host memory
  * into device memory with the same access pattern as lif_fetch_bundles (chunk_bytes-sized

@@ -21,8 +21,10 @@ EXPORTS = [
     "lif_status_str", "lif_workspace_bytes", "lif_create_layer", "lif_destroy_layer", "lif_reset",
     "lif_predict", "lif_window_update", "lif_fetch_bundles", "lif_sparse_ffn", "lif_decode_step",
     "lif_decode_token_host", "lif_get_lists", "lif_get_stats", "lif_clear_status",
-    "lif_probe_host_read",
+    "lif_probe_host_read", "lif_timing_enable", "lif_timing_read",
 ]
+PHASES = ("predict_z", "predict_scores", "window", "moves", "fetch", "ffn", "ffn_sum")
+PHASE_LEN = 8
 
 
 class LayerDesc(C.Structure):
@@ -84,6 +86,8 @@ def lib() -> C.CDLL:
         "lif_get_stats": [vp, C.POINTER(Stats)],
         "lif_clear_status": [vp, vp],
         "lif_probe_host_read": [vp, vp, sz, sz, vp],
+        "lif_timing_enable": [vp, i32],
+        "lif_timing_read": [vp, C.POINTER(C.c_float), C.POINTER(i32)],
     }
     for name, args in sigs.items():
         fn = getattr(L, name)
@@ -199,3 +203,15 @@ def lif_clear_status(layer: int, stream=None) -> None:
 def lif_probe_host_read(host_src, dev_dst, nbytes: int, chunk_bytes: int, stream=None) -> None:
     _check(lib().lif_probe_host_read(_ptr(host_src), _ptr(dev_dst), nbytes, chunk_bytes,
                                      _stream(stream)), "lif_probe_host_read")
+
+
+def lif_timing_enable(layer: int, n_steps: int) -> None:
+    _check(lib().lif_timing_enable(layer, n_steps), "lif_timing_enable")
+
+
+def lif_timing_read(layer: int):
+    """Returns ({phase: summed microseconds}, steps recorded)."""
+    us = (C.c_float * PHASE_LEN)()
+    n = C.c_int32(0)
+    _check(lib().lif_timing_read(layer, us, C.byref(n)), "lif_timing_read")
+    return {p: float(us[i]) for i, p in enumerate(PHASES)}, n.value

@@ -17,7 +17,7 @@ Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max) {
     return at;
   };
   const size_t F = d.d_ff, cap = d.capacity, S = d.n_streams;
-  const size_t z_ctas = (d.d_model + kZRowsPerCta - 1) / kZRowsPerCta;
+  const size_t z_ctas = z_cta_count(d.d_model);
   const size_t n_mask = (F + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
   w.counts = take(LIF_CNT_LEN * 4);
   w.pointers = take(cap * 4);
@@ -46,7 +46,7 @@ static int ffn_grid_upper_bound() { return 2 * 256; }   // >= 2 CTAs per SM on a
 static lif_status check_shape(const lif_layer_desc* d) {
   if (!d) return LIF_ERR_INVALID_ARG;
   if (d->d_model < 8 || d->d_model % 8 || d->d_model > 8192) return LIF_ERR_INVALID_ARG;
-  if (d->d_ff < 8 || d->d_ff % 8) return LIF_ERR_INVALID_ARG;
+  if (d->d_ff < 8 || d->d_ff % 8 || d->d_ff >= (1 << 21)) return LIF_ERR_INVALID_ARG;
   if (d->rank < 8 || d->rank % 8 || d->rank > 2048) return LIF_ERR_INVALID_ARG;
   if (d->window_k < 1) return LIF_ERR_INVALID_ARG;
   if (d->capacity < 1 || d->capacity > d->d_ff) return LIF_ERR_INVALID_ARG;
@@ -138,7 +138,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
             cudaDeviceGetAttribute(&L->n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
   ok = ok && ffn_configure(L) == cudaSuccess;
   if (ok) {
-    L->z_ctas = (desc->d_model + kZRowsPerCta - 1) / kZRowsPerCta;
+    L->z_ctas = z_cta_count(desc->d_model);
     L->ffn_grid = L->n_sm < ffn_grid_upper_bound() ? L->n_sm : ffn_grid_upper_bound();
     L->fetch_grid = L->n_sm;
     L->move_grid = L->n_sm;
@@ -162,8 +162,61 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
   return LIF_OK;
 }
 
+static void timing_free(lif_layer* L) {
+  if (!L->tm_events) return;
+  for (int i = 0; i < L->tm_steps * kTimingEvents; ++i) cudaEventDestroy(L->tm_events[i]);
+  delete[] L->tm_events;
+  L->tm_events = nullptr;
+  L->tm_steps = L->tm_cursor = 0;
+}
+
+lif_status lif_timing_enable(lif_layer* L, int32_t n_steps) {
+  if (!L || n_steps < 0 || n_steps > (1 << 20)) return LIF_ERR_INVALID_ARG;
+  timing_free(L);
+  if (n_steps == 0) return LIF_OK;
+  const int n = n_steps * kTimingEvents;
+  L->tm_events = new (std::nothrow) cudaEvent_t[n];
+  if (!L->tm_events) return LIF_ERR_STATE;
+  for (int i = 0; i < n; ++i) {
+    if (cudaEventCreate(&L->tm_events[i]) != cudaSuccess) {
+      for (int j = 0; j < i; ++j) cudaEventDestroy(L->tm_events[j]);
+      delete[] L->tm_events;
+      L->tm_events = nullptr;
+      cudaGetLastError();
+      return LIF_ERR_CUDA;
+    }
+  }
+  L->tm_steps = n_steps;
+  L->tm_cursor = 0;
+  return LIF_OK;
+}
+
+lif_status lif_timing_read(lif_layer* L, float* us, int32_t* host_n_steps) {
+  if (!L || !us || !host_n_steps) return LIF_ERR_INVALID_ARG;
+  for (int p = 0; p < LIF_PHASE_LEN; ++p) us[p] = 0.f;
+  *host_n_steps = 0;
+  if (!L->tm_events) return LIF_ERR_STATE;
+  if (cudaDeviceSynchronize() != cudaSuccess) return LIF_ERR_CUDA;
+  // (first event, second event) of each phase within a step's event block
+  static const int pairs[7][2] = {{0, 1}, {1, 2}, {2, 3}, {3, 4}, {5, 6}, {7, 8}, {8, 9}};
+  for (int s = 0; s < L->tm_cursor; ++s) {
+    cudaEvent_t* ev = L->tm_events + (size_t)s * kTimingEvents;
+    for (int p = 0; p < 7; ++p) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, ev[pairs[p][0]], ev[pairs[p][1]]) != cudaSuccess) {
+        cudaGetLastError();
+        return LIF_ERR_CUDA;
+      }
+      us[p] += ms * 1e3f;
+    }
+  }
+  *host_n_steps = L->tm_cursor;
+  return LIF_OK;
+}
+
 lif_status lif_destroy_layer(lif_layer* L) {
   if (!L) return LIF_ERR_INVALID_ARG;
+  timing_free(L);
   cudaEventDestroy(L->ev_plan);
   cudaEventDestroy(L->ev_fetch);
   delete L;
@@ -219,23 +272,29 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   if (!aligned(dev_x, 16) || !aligned(dev_y, 16)) return LIF_ERR_ALIGNMENT;
   cudaStream_t sc = (cudaStream_t)compute_stream, sf = (cudaStream_t)fetch_stream;
   const __half* x = (const __half*)dev_x;
-  bool ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc) == cudaSuccess;
-  ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc) == cudaSuccess;
+  cudaEvent_t* ev = nullptr;
+  if (L->tm_events && L->tm_cursor < L->tm_steps)
+    ev = L->tm_events + (size_t)(L->tm_cursor++) * kTimingEvents;
+  if (ev) cudaEventRecord(ev[0], sc);
+  bool ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
+  ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
   if (sf != sc) {
     ok = ok && cudaEventRecord(L->ev_plan, sc) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(sf, L->ev_plan, 0) == cudaSuccess;
   }
+  if (ev) cudaEventRecord(ev[5], sf);
   ok = ok && launch_fetch(L, sf) == cudaSuccess;
+  if (ev) cudaEventRecord(ev[6], sf);
   if (sf != sc) {
     ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(sc, L->ev_fetch, 0) == cudaSuccess;
   }
   if (L->desc.ffn_mode == 0)
     ok = ok && launch_ffn(L, x, L->active_slots, L->counts + LIF_CNT_N_ACTIVE, nullptr, dev_y,
-                          false, sc) == cudaSuccess;
+                          false, sc, ev) == cudaSuccess;
   else
     ok = ok && launch_ffn(L, x, nullptr, L->counts + LIF_CNT_NUM_USED, nullptr, dev_y, false,
-                          sc) == cudaSuccess;
+                          sc, ev) == cudaSuccess;
   if (!ok) cudaGetLastError();
   return ok ? LIF_OK : LIF_ERR_CUDA;
 }

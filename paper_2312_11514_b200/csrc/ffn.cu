@@ -196,19 +196,23 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
   }
 }
 
-// y[m] = (accumulate ? y[m] : b_down[m]) + sum_{g < min(G, n)} y_partial[g][m], g ascending.
-__global__ void __launch_bounds__(kThreads)
+// y[m] = (accumulate ? y[m] : b_down[m]) + sum_{g < min(G, n)} y_partial[g][m].  1024 threads =
+// 32 float4 columns x 32 slices of g; each slice adds its partials in ascending g, then the
+// slices are added in ascending order: a fixed summation order.
+constexpr int kSumThreads = 1024;
+__global__ void __launch_bounds__(kSumThreads)
 ffn_reduce_kernel(const float* __restrict__ y_partial, int G, const int32_t* __restrict__ n,
                   const __half* __restrict__ b_down, float* __restrict__ y, int d,
                   int accumulate) {
-  __shared__ float4 red[8][32];
+  __shared__ float4 red[32][32];
   const int tid = threadIdx.x;
   const int c4 = tid & 31, gs = tid >> 5;
   const int col4 = blockIdx.x * 32 + c4;       // float4 column
   const int valid = min(G, *n);
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
   if (col4 * 4 < d) {
-    for (int g = gs; g < valid; g += 8) {
+#pragma unroll 4
+    for (int g = gs; g < valid; g += 32) {
       const float4 v = __ldcg(reinterpret_cast<const float4*>(y_partial + (size_t)g * d) + col4);
       s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
     }
@@ -227,7 +231,7 @@ ffn_reduce_kernel(const float* __restrict__ y_partial, int G, const int32_t* __r
       t = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < 32; ++k) {
       t.x += red[k][c4].x; t.y += red[k][c4].y; t.z += red[k][c4].z; t.w += red[k][c4].w;
     }
     reinterpret_cast<float4*>(y)[col4] = t;
@@ -261,9 +265,11 @@ cudaError_t ffn_configure(lif_layer* L) {
 }
 
 cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
-                       const int32_t* base, float* y, bool accumulate, cudaStream_t st) {
+                       const int32_t* base, float* y, bool accumulate, cudaStream_t st,
+                       cudaEvent_t* ev) {
   const lif_layer_desc& D = L->desc;
   const int d = D.d_model;
+  if (ev) cudaEventRecord(ev[7], st);
   for (int s = 0; s < D.n_streams; ++s) {
     FfnArgs a;
     a.cache = (const __half*)D.dev_cache;
@@ -279,12 +285,14 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
     sparse_ffn_kernel<<<L->ffn_grid, kThreads, L->ffn_smem, st>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    ffn_reduce_kernel<<<(d / 4 + 31) / 32, kThreads, 0, st>>>(
+    if (ev && s == D.n_streams - 1) cudaEventRecord(ev[8], st);
+    ffn_reduce_kernel<<<(d / 4 + 31) / 32, kSumThreads, 0, st>>>(
         L->y_partial, L->ffn_grid, n, (const __half*)D.dev_bias_down, y + (size_t)s * d, d,
         accumulate ? 1 : 0);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
+  if (ev) cudaEventRecord(ev[9], st);
   return cudaSuccess;
 }
 

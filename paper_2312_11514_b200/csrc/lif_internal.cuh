@@ -18,9 +18,17 @@ enum {
 constexpr int kNever = -(1 << 30);  // last_active stamp of a neuron never predicted active
 constexpr int kThreads = 256;
 constexpr int kWindowThreads = 1024;
-constexpr int kZRowsPerCta = 256;   // rows of A per CTA in the first predictor stage
+// rows of A per CTA in the first predictor stage: about 32 CTAs, so stage 2 folds few partials
+inline int z_rows_per_cta(int d_model) {
+  const int rows = ((d_model + 31) / 32 + 31) / 32 * 32;
+  return rows < 32 ? 32 : rows;
+}
+inline int z_cta_count(int d_model) {
+  return (d_model + z_rows_per_cta(d_model) - 1) / z_rows_per_cta(d_model);
+}
 constexpr int kLogitTile = 128;     // neurons per CTA in the second predictor stage
 constexpr int kMaxStreams = 8;
+constexpr int kTimingEvents = 10;   // z0 z1 s1 w1 m1 | f0 f1 | g0 g1 r1
 
 struct Workspace {
   // offsets in bytes from the workspace base; every block 256-byte aligned
@@ -53,21 +61,28 @@ struct lif_layer {
   int fetch_grid;     // CTAs of the fetch kernel
   int move_grid;
   cudaEvent_t ev_plan, ev_fetch;
+  // optional per-kernel timing: kTimingEvents events per recorded step
+  cudaEvent_t* tm_events;
+  int tm_steps, tm_cursor;
 };
 
 namespace lif {
 
 // kernels' host launchers (each returns the launch's cudaError_t)
 cudaError_t launch_reset(lif_layer* L, cudaStream_t st);
+// `ev`: optional events of the current timed step (nullptr = no timing); each launcher
+// records the ones between and after its own kernels.
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
-                           int32_t* n_active, cudaStream_t st);
-cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st);
+                           int32_t* n_active, cudaStream_t st, cudaEvent_t* ev = nullptr);
+cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st,
+                          cudaEvent_t* ev = nullptr);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,
                          int grid, cudaStream_t st);
 // slots == nullptr: rows base[0] .. base[0] + n[0] (base == nullptr: 0)
 cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
-                       const int32_t* base, float* y, bool accumulate, cudaStream_t st);
+                       const int32_t* base, float* y, bool accumulate, cudaStream_t st,
+                       cudaEvent_t* ev = nullptr);
 cudaError_t ffn_configure(lif_layer* L);
 
 }  // namespace lif

@@ -34,14 +34,14 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
 template <int S>
 __global__ void __launch_bounds__(kThreads)
 predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int d, int r,
-                 float* __restrict__ z_partial) {
+                 int rows_per_cta, float* __restrict__ z_partial) {
   __shared__ float red[2048];
   const int ncg = r >> 3;            // 8-column groups (16 bytes each)
   const int nrl = kThreads / ncg;    // row lanes
   const int tid = threadIdx.x;
   const int cg = tid % ncg, rl = tid / ncg;
-  const int m0 = blockIdx.x * kZRowsPerCta;
-  const int m1 = min(d, m0 + kZRowsPerCta);
+  const int m0 = blockIdx.x * rows_per_cta;
+  const int m1 = min(d, m0 + rows_per_cta);
 
   float acc[S][8];
 #pragma unroll
@@ -50,7 +50,7 @@ predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int
     for (int e = 0; e < 8; ++e) acc[s][e] = 0.f;
 
   if (rl < nrl) {
-#pragma unroll 4
+#pragma unroll 8
     for (int m = m0 + rl; m < m1; m += nrl) {
       float af[8];
       unpack8(ldg_stream(A + (size_t)m * r + cg * 8), af);
@@ -114,30 +114,49 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
   __shared__ int is_last;
   const int tid = threadIdx.x;
 
+  // B does not depend on stage 1: put the first 128 rows of this CTA's tile in flight before
+  // touching z (8 x 16 bytes per thread), then fold the stage-1 partials while they travel.
+  const int cg = tid & 15, rs = tid >> 4;
+  const int col = blockIdx.x * kLogitTile + cg * 8;
+  uint4 bq[8];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int j = rs + 16 * u;
+    bq[u] = (col < F && j < r) ? ldg_stream(B + (size_t)j * F + col) : make_uint4(0, 0, 0, 0);
+  }
   for (int i = tid; i < S * r; i += kThreads) {
     float v = 0.f;
+#pragma unroll 8
     for (int p = 0; p < P; ++p) v += __ldcg(z_partial + (size_t)p * S * r + i);
     zs[i] = v;
   }
   __syncthreads();
 
-  const int cg = tid & 15, rs = tid >> 4;
-  const int col = blockIdx.x * kLogitTile + cg * 8;
   float acc[S][8];
 #pragma unroll
   for (int s = 0; s < S; ++s)
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[s][e] = 0.f;
-  if (col < F) {
-#pragma unroll 4
-    for (int j = rs; j < r; j += 16) {
-      float bf[8];
-      unpack8(ldg_stream(B + (size_t)j * F + col), bf);
+  for (int j0 = 0; j0 < r; j0 += 128) {
+    if (j0 > 0) {
 #pragma unroll
-      for (int s = 0; s < S; ++s) {
-        const float zz = zs[s * r + j];
+      for (int u = 0; u < 8; ++u) {
+        const int j = j0 + rs + 16 * u;
+        bq[u] = (col < F && j < r) ? ldg_stream(B + (size_t)j * F + col) : make_uint4(0, 0, 0, 0);
+      }
+    }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[s][e] = fmaf(zz, bf[e], acc[s][e]);
+    for (int u = 0; u < 8; ++u) {
+      const int j = j0 + rs + 16 * u;
+      if (j < r) {
+        float bf[8];
+        unpack8(bq[u], bf);
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+          const float zz = zs[s * r + j];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[s][e] = fmaf(zz, bf[e], acc[s][e]);
+        }
       }
     }
   }
@@ -198,10 +217,11 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
 
 template <int S>
 cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
-                             int32_t* n_active, cudaStream_t st) {
+                             int32_t* n_active, cudaStream_t st, cudaEvent_t* ev) {
   const lif_layer_desc& D = L->desc;
   predict_z_kernel<S><<<L->z_ctas, kThreads, 0, st>>>(
-      x, (const __half*)D.dev_pred_A, D.d_model, D.rank, L->z_partial);
+      x, (const __half*)D.dev_pred_A, D.d_model, D.rank, z_rows_per_cta(D.d_model), L->z_partial);
+  if (ev) cudaEventRecord(ev[1], st);
   const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
   const size_t smem = (size_t)S * D.rank * sizeof(float);
   if (smem > 32 * 1024) {
@@ -213,22 +233,23 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
       L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit,
       D.rank, D.d_ff, logits, L->mask_words, L->counts + CNT_TICKET_PREDICT, active_idx,
       n_active);
+  if (ev) cudaEventRecord(ev[2], st);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
-                           int32_t* n_active, cudaStream_t st) {
+                           int32_t* n_active, cudaStream_t st, cudaEvent_t* ev) {
   switch (L->desc.n_streams) {
-    case 1: return launch_predict_s<1>(L, x, logits, active_idx, n_active, st);
-    case 2: return launch_predict_s<2>(L, x, logits, active_idx, n_active, st);
-    case 3: return launch_predict_s<3>(L, x, logits, active_idx, n_active, st);
-    case 4: return launch_predict_s<4>(L, x, logits, active_idx, n_active, st);
-    case 5: return launch_predict_s<5>(L, x, logits, active_idx, n_active, st);
-    case 6: return launch_predict_s<6>(L, x, logits, active_idx, n_active, st);
-    case 7: return launch_predict_s<7>(L, x, logits, active_idx, n_active, st);
-    case 8: return launch_predict_s<8>(L, x, logits, active_idx, n_active, st);
+    case 1: return launch_predict_s<1>(L, x, logits, active_idx, n_active, st, ev);
+    case 2: return launch_predict_s<2>(L, x, logits, active_idx, n_active, st, ev);
+    case 3: return launch_predict_s<3>(L, x, logits, active_idx, n_active, st, ev);
+    case 4: return launch_predict_s<4>(L, x, logits, active_idx, n_active, st, ev);
+    case 5: return launch_predict_s<5>(L, x, logits, active_idx, n_active, st, ev);
+    case 6: return launch_predict_s<6>(L, x, logits, active_idx, n_active, st, ev);
+    case 7: return launch_predict_s<7>(L, x, logits, active_idx, n_active, st, ev);
+    case 8: return launch_predict_s<8>(L, x, logits, active_idx, n_active, st, ev);
   }
   return cudaErrorInvalidValue;
 }

@@ -3,7 +3,8 @@
 // the row moves that keep the used rows consecutive.
 //
 // The plan is integer work over n_active + num_used elements, so one 1024-thread CTA does it
-// with ordered block-wide compactions (list order = index order, never atomics order):
+// with ordered block-wide compactions (one packed prefix scan per pass; list order = index
+// order, never atomics order):
 //   A  count what would be deleted / loaded; refuse on overflow before touching anything
 //   B  stamp last_active of the active neurons
 //   C  deleted rows in ascending slot order; surviving tail rows in descending slot order
@@ -16,29 +17,38 @@
 namespace lif {
 namespace {
 
+// Three counters ride in one 64-bit scan, 21 bits each (d_ff < 2^21 is checked at creation).
+typedef unsigned long long u64;
+constexpr int kField = 21;
+constexpr u64 kFieldMask = (1ull << kField) - 1;
+__device__ __forceinline__ u64 pack3(int a, int b, int c) {
+  return (u64)a | ((u64)b << kField) | ((u64)c << (2 * kField));
+}
+__device__ __forceinline__ int field(u64 v, int i) { return (int)((v >> (i * kField)) & kFieldMask); }
+
 struct Scan {
-  int warp_sums[kWindowThreads / 32];
+  u64 warp_sums[kWindowThreads / 32];
 };
 
 // exclusive prefix of v over the block (thread order); *total = block sum
-__device__ __forceinline__ int block_scan(int v, int* total, Scan& sc) {
+__device__ __forceinline__ u64 block_scan(u64 v, u64* total, Scan& sc) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int inc = v;
+  u64 inc = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    int n = __shfl_up_sync(0xffffffffu, inc, o);
+    u64 n = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= o) inc += n;
   }
   if (lane == 31) sc.warp_sums[warp] = inc;
   __syncthreads();
-  int ws = sc.warp_sums[lane];   // 32 warps
-  int winc = ws;
+  u64 ws = sc.warp_sums[lane];   // 32 warps
+  u64 winc = ws;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    int n = __shfl_up_sync(0xffffffffu, winc, o);
+    u64 n = __shfl_up_sync(0xffffffffu, winc, o);
     if (lane >= o) winc += n;
   }
-  const int base = __shfl_sync(0xffffffffu, winc - ws, warp);
+  const u64 base = __shfl_sync(0xffffffffu, winc - ws, warp);
   *total = __shfl_sync(0xffffffffu, winc, 31);
   __syncthreads();
   return base + inc - v;
@@ -64,11 +74,11 @@ __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArg
   const int t = a.counts[LIF_CNT_STEP];
   const int na = *a.n_act;
   const int stale_before = t - a.k;   // last_active <= stale_before: outside the window
-  int tot;
+  u64 tot;
 
   // ---- A: what would happen ------------------------------------------------------------
-  int bad = 0, c_load = 0, c_back = 0, c_stale = 0;
-  if (na < 0 || na > a.F) bad = 1;
+  int bad = (na < 0 || na > a.F) ? 1 : 0;
+  int c_load = 0, c_back = 0, c_stale = 0;
   if (!bad) {
     for (int q = tid; q < na; q += kWindowThreads) {
       const int id = a.act[q];
@@ -79,14 +89,10 @@ __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArg
     for (int s = tid; s < n; s += kWindowThreads)
       if (a.last_active[a.pointers[s]] <= stale_before) ++c_stale;
   }
-  block_scan(bad, &tot, sc);
-  const int any_bad = tot;
-  block_scan(c_load, &tot, sc);
-  const int n_load = tot;
-  block_scan(c_back, &tot, sc);
-  const int n_back = tot;
-  block_scan(c_stale, &tot, sc);
-  const int n_evict = tot - n_back;
+  const int any_bad = __syncthreads_or(bad);
+  block_scan(pack3(c_load, c_back, c_stale), &tot, sc);
+  const int n_load = field(tot, 0);
+  const int n_evict = field(tot, 2) - field(tot, 1);
   const int n_kept = n - n_evict;
 
   if (any_bad || n_kept + n_load > a.cap) {
@@ -109,33 +115,32 @@ __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArg
   __syncthreads();
 
   // ---- C: deleted rows (ascending slot) and surviving tail rows (descending slot) --------
-  int run = 0, holes = 0;
-  for (int b = 0; b < n; b += kWindowThreads) {
-    const int s = b + tid;
-    int id = -1, f = 0;
-    if (s < n) {
-      id = a.pointers[s];
-      f = a.last_active[id] <= stale_before;
-    }
-    const int pos = run + block_scan(f, &tot, sc);
-    if (f) {
-      a.evict_slots[pos] = s;
-      a.evict_ids[pos] = id;
-    }
-    run += tot;
-    block_scan(f && s < n_kept, &tot, sc);
-    holes += tot;
+  // Each thread owns a contiguous run of slots, so thread order is slot order.
+  const int seg = (n + kWindowThreads - 1) / kWindowThreads;
+  const int s0 = min(n, tid * seg), s1 = min(n, s0 + seg);
+  int c_ev = 0, c_hole = 0, c_surv = 0;
+  for (int s = s0; s < s1; ++s) {
+    const int f = a.last_active[a.pointers[s]] <= stale_before;
+    c_ev += f;
+    c_hole += f && s < n_kept;
+    c_surv += !f && s >= n_kept;
   }
-  const int n_moves = holes;
-  run = 0;
-  for (int b = 0; b < n - n_kept; b += kWindowThreads) {
-    const int i = b + tid;
-    const int s = n - 1 - i;
-    int f = 0;
-    if (i < n - n_kept) f = a.last_active[a.pointers[s]] > stale_before;
-    const int pos = run + block_scan(f, &tot, sc);
-    if (f) a.move_src[pos] = s;
-    run += tot;
+  u64 pre = block_scan(pack3(c_ev, c_hole, c_surv), &tot, sc);
+  const int n_moves = field(tot, 1);          // == surviving tail rows
+  {
+    int p_ev = field(pre, 0), p_surv = field(pre, 2);
+    for (int s = s0; s < s1; ++s) {
+      const int id = a.pointers[s];
+      const int f = a.last_active[id] <= stale_before;
+      if (f) {
+        a.evict_slots[p_ev] = s;
+        a.evict_ids[p_ev] = id;
+        ++p_ev;
+      } else if (s >= n_kept) {
+        a.move_src[n_moves - 1 - p_surv] = s;   // last survivor first
+        ++p_surv;
+      }
+    }
   }
   __syncthreads();
 
@@ -153,43 +158,31 @@ __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArg
   for (int s = n_kept + tid; s < n; s += kWindowThreads) a.pointers[s] = -1;
   __syncthreads();
 
-  // ---- E: rows for the neurons to bring in ------------------------------------------------
-  run = 0;
-  for (int b = 0; b < na; b += kWindowThreads) {
-    const int q = b + tid;
-    int id = -1, f = 0;
-    if (q < na) {
-      id = a.act[q];
-      f = a.slot_of[id] < 0;
-    }
-    const int pos = run + block_scan(f, &tot, sc);
-    if (f) {
-      const int s = n_kept + pos;
-      a.load_ids[pos] = id;
-      a.load_slots[pos] = s;
-      a.slot_of[id] = s;
-      a.pointers[s] = id;
-      a.bias[s] = a.bias_up[id];
-    }
-    run += tot;
-  }
-  __syncthreads();
-
-  // ---- F: slot lists ----------------------------------------------------------------------
-  run = 0;
-  for (int b = 0; b < na; b += kWindowThreads) {
-    const int q = b + tid;
-    int s = -1, f = 0;
-    if (q < na) {
+  // ---- E + F: rows for the neurons to bring in, and the slot lists -----------------------
+  const int qseg = (na + kWindowThreads - 1) / kWindowThreads;
+  const int q0 = min(na, tid * qseg), q1 = min(na, q0 + qseg);
+  int c_l = 0;
+  for (int q = q0; q < q1; ++q) c_l += a.slot_of[a.act[q]] < 0;
+  pre = block_scan(pack3(c_l, (q1 - q0) - c_l, 0), &tot, sc);
+  {
+    int p_l = field(pre, 0), p_h = field(pre, 1);
+    for (int q = q0; q < q1; ++q) {
       const int id = a.act[q];
-      s = a.slot_of[id];
+      int s = a.slot_of[id];
+      if (s < 0) {
+        s = n_kept + p_l;
+        a.load_ids[p_l] = id;
+        a.load_slots[p_l] = s;
+        a.slot_of[id] = s;
+        a.pointers[s] = id;
+        a.bias[s] = a.bias_up[id];
+        ++p_l;
+      } else {
+        a.hit_slots[p_h++] = s;
+      }
       a.active_slots[q] = s;
       if (a.active_idx != a.act) a.active_idx[q] = id;
-      f = s < n_kept;
     }
-    const int pos = run + block_scan(f, &tot, sc);
-    if (f) a.hit_slots[pos] = s;
-    run += tot;
   }
   if (tid == 0) {
     a.counts[LIF_CNT_N_ACTIVE] = na;
@@ -249,7 +242,7 @@ cudaError_t launch_reset(lif_layer* L, cudaStream_t st) {
 }
 
 cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act,
-                          cudaStream_t st) {
+                          cudaStream_t st, cudaEvent_t* ev) {
   const lif_layer_desc& D = L->desc;
   WindowArgs a;
   a.act = act;
@@ -276,8 +269,10 @@ cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act
   window_update_kernel<<<1, kWindowThreads, 0, st>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  if (ev) cudaEventRecord(ev[3], st);
   move_rows_kernel<<<L->move_grid, kThreads, 0, st>>>((uint4*)D.dev_cache, L->move_src,
                                                       L->move_dst, L->counts, D.d_model / 4);
+  if (ev) cudaEventRecord(ev[4], st);
   return cudaGetLastError();
 }
 
