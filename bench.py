@@ -7,8 +7,9 @@ sparse FFN, every layer, one token per step) on seeded synthetic data.
 One step = one decode token through all layers of the configuration.  `value` is tokens/s
 with the decode inputs resident in HBM (the bundle store stays in pinned host memory: reading
 it is part of the method); `e2e` passes pinned HOST inputs/outputs through
-lif_decode_token_host.  Per-kernel durations for the roofline come from a second timed pass
-through the staged entry points with CUDA events between the calls.
+lif_graph_launch_host.  A token is one CUDA graph (lif_graph_capture).  Per-kernel durations
+for the roofline come from a further timed pass over the same tokens with a CUDA event node
+around every kernel of the graph.
 """
 from __future__ import annotations
 
@@ -136,19 +137,27 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    # ---- pass 1: device-resident inputs, whole step through lif_decode_step ------------------
+    # One CUDA graph holds a whole token (every layer's kernels, both streams); the token's
+    # input is copied into dev_x before each launch.
+    dev_x = torch.empty(S, d, dtype=torch.float16, device=dev)
+    graph = B.lif_graph_capture(handles, dev_x, Y, sc, sf)
+
+    def token(t):
+        with torch.cuda.stream(sc):
+            dev_x.copy_(X[t], non_blocking=True)
+        B.lif_graph_launch(graph, sc)
+
+    # ---- pass 1: device-resident inputs ------------------------------------------------------
     reset()
     for t in range(Wm):
-        for l in range(L):
-            B.lif_decode_step(handles[l], X[t], Y[l], sc, sf)
+        token(t)
     barrier()
     s0 = stats_sum()
     clocks = ClockSampler(local) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(sc)
     for t in range(Wm, n_tok):
-        for l in range(L):
-            B.lif_decode_step(handles[l], X[t], Y[l], sc, sf)
+        token(t)
     e1.record(sc)
     barrier()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
@@ -156,40 +165,40 @@ def run_ours(args):
     s1 = stats_sum()
     fetched, rows_active, rows_moved = (s1[i] - s0[i] for i in range(3))
 
-    # ---- pass 2: host buffers through lif_decode_token_host ---------------------------------
+    # ---- pass 2: pinned host inputs and outputs through lif_graph_launch_host ----------------
     host_x = torch.empty(n_tok, S, d, dtype=torch.float16, pin_memory=True)
     host_x.copy_(X)
     host_y = torch.empty(L, S, d, dtype=torch.float32, pin_memory=True)
-    dev_x = torch.empty(S, d, dtype=torch.float16, device=dev)
     reset()
     for t in range(Wm):
-        B.lif_decode_token_host(handles, host_x[t], dev_x, Y, host_y, sc, sf)
+        B.lif_graph_launch_host(graph, host_x[t], host_y, sc)
     barrier()
     e0.record(sc)
     for t in range(Wm, n_tok):
-        B.lif_decode_token_host(handles, host_x[t], dev_x, Y, host_y, sc, sf)
+        B.lif_graph_launch_host(graph, host_x[t], host_y, sc)
     e1.record(sc)
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1))
 
-    # ---- pass 3: same loop as pass 1 with the library's per-kernel CUDA events switched on ----
+    # ---- pass 3: a second graph of the same token with an event-record node around every
+    # kernel; read after each token ------------------------------------------------------------
+    for h in handles:
+        B.lif_timing_enable(h, 1)
+    tgraph = B.lif_graph_capture(handles, dev_x, Y, sc, sf)
     reset()
-    for t in range(Wm):
-        for l in range(L):
-            B.lif_decode_step(handles[l], X[t], Y[l], sc, sf)
-    barrier()
-    for h in handles:
-        B.lif_timing_enable(h, K)
-    for t in range(Wm, n_tok):
-        for l in range(L):
-            B.lif_decode_step(handles[l], X[t], Y[l], sc, sf)
-    barrier()
     phase_us = {p: 0.0 for p in B.PHASES}
+    for t in range(n_tok):
+        with torch.cuda.stream(sc):
+            dev_x.copy_(X[t], non_blocking=True)
+        B.lif_graph_launch(tgraph, sc)
+        if t >= Wm:
+            for h in handles:
+                us, n_rec = B.lif_timing_read(h)
+                for p in B.PHASES:
+                    phase_us[p] += us[p]
+    barrier()
+    B.lif_graph_destroy(tgraph)
     for h in handles:
-        us, n_rec = B.lif_timing_read(h)
-        assert n_rec == K
-        for p in B.PHASES:
-            phase_us[p] += us[p]
         B.lif_timing_enable(h, 0)
     n_launch = K * L
 
@@ -249,6 +258,7 @@ def run_ours(args):
         if args.cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(cfg, layers, X, args.cpu_layers, args.cpu_tokens)
         print(json.dumps(out), flush=True)
+    B.lif_graph_destroy(graph)
     for l in layers:
         l.close()
     if world > 1:

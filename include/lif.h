@@ -181,6 +181,24 @@ lif_status lif_decode_token_host(lif_layer* const* layers, int32_t n_layers, con
                                  void* dev_x, float* dev_y, float* host_y,
                                  void* compute_stream, void* fetch_stream);
 
+/* One token through `n_layers` layers as a CUDA graph.  lif_graph_capture records
+ * lif_decode_step of every layer, in order, reading dev_x (fp16 [n_streams][d_model]) and with
+ * layer l writing dev_y + l*n_streams*d_model, on two distinct non-default streams, and
+ * instantiates the graph; nothing runs during capture.  Every size the kernels need is read
+ * from device memory at run time, so one graph serves every token: put the token's input in
+ * dev_x, then lif_graph_launch.  lif_graph_launch_host does that from pinned host buffers:
+ * copies host_x in, launches, copies all layers' outputs to host_y (fp32
+ * [n_layers][n_streams][d_model]) and synchronises the stream.  The layers must outlive the
+ * graph.  Launch overhead per kernel is several times lower than separate launches. */
+typedef struct lif_graph lif_graph;
+lif_status lif_graph_capture(lif_layer* const* layers, int32_t n_layers, void* dev_x,
+                             float* dev_y, void* compute_stream, void* fetch_stream,
+                             lif_graph** out);
+lif_status lif_graph_launch(lif_graph* graph, void* stream);
+lif_status lif_graph_launch_host(lif_graph* graph, const void* host_x, float* host_y,
+                                 void* stream);
+lif_status lif_graph_destroy(lif_graph* graph);
+
 /* Device addresses of lists and state (valid for the layer's lifetime). */
 lif_status lif_get_lists(lif_layer* layer, lif_lists* host_out);
 

@@ -22,6 +22,7 @@ EXPORTS = [
     "lif_predict", "lif_window_update", "lif_fetch_bundles", "lif_sparse_ffn", "lif_decode_step",
     "lif_decode_token_host", "lif_get_lists", "lif_get_stats", "lif_clear_status",
     "lif_probe_host_read", "lif_timing_enable", "lif_timing_read",
+    "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
 ]
 PHASES = ("predict_z", "predict_scores", "window", "moves", "fetch", "ffn", "ffn_sum")
 PHASE_LEN = 8
@@ -86,6 +87,10 @@ def lib() -> C.CDLL:
         "lif_get_stats": [vp, C.POINTER(Stats)],
         "lif_clear_status": [vp, vp],
         "lif_probe_host_read": [vp, vp, sz, sz, vp],
+        "lif_graph_capture": [C.POINTER(vp), i32, vp, vp, vp, vp, C.POINTER(vp)],
+        "lif_graph_launch": [vp, vp],
+        "lif_graph_launch_host": [vp, vp, vp, vp],
+        "lif_graph_destroy": [vp],
         "lif_timing_enable": [vp, i32],
         "lif_timing_read": [vp, C.POINTER(C.c_float), C.POINTER(i32)],
     }
@@ -215,3 +220,25 @@ def lif_timing_read(layer: int):
     n = C.c_int32(0)
     _check(lib().lif_timing_read(layer, us, C.byref(n)), "lif_timing_read")
     return {p: float(us[i]) for i, p in enumerate(PHASES)}, n.value
+
+
+def lif_graph_capture(layers, dev_x, dev_y, compute_stream, fetch_stream) -> int:
+    arr = (C.c_void_p * len(layers))(*layers)
+    out = C.c_void_p(None)
+    _check(lib().lif_graph_capture(arr, len(layers), _ptr(dev_x), _ptr(dev_y),
+                                   _stream(compute_stream), _stream(fetch_stream), C.byref(out)),
+           "lif_graph_capture")
+    return out.value
+
+
+def lif_graph_launch(graph: int, stream=None) -> None:
+    _check(lib().lif_graph_launch(graph, _stream(stream)), "lif_graph_launch")
+
+
+def lif_graph_launch_host(graph: int, host_x, host_y, stream=None) -> None:
+    _check(lib().lif_graph_launch_host(graph, _ptr(host_x), _ptr(host_y), _stream(stream)),
+           "lif_graph_launch_host")
+
+
+def lif_graph_destroy(graph: int) -> None:
+    _check(lib().lif_graph_destroy(graph), "lif_graph_destroy")

@@ -275,16 +275,16 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   cudaEvent_t* ev = nullptr;
   if (L->tm_events && L->tm_cursor < L->tm_steps)
     ev = L->tm_events + (size_t)(L->tm_cursor++) * kTimingEvents;
-  if (ev) cudaEventRecord(ev[0], sc);
+  if (ev) tm_record(ev[0], sc);
   bool ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
   ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
   if (sf != sc) {
     ok = ok && cudaEventRecord(L->ev_plan, sc) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(sf, L->ev_plan, 0) == cudaSuccess;
   }
-  if (ev) cudaEventRecord(ev[5], sf);
+  if (ev) tm_record(ev[5], sf);
   ok = ok && launch_fetch(L, sf) == cudaSuccess;
-  if (ev) cudaEventRecord(ev[6], sf);
+  if (ev) tm_record(ev[6], sf);
   if (sf != sc) {
     ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(sc, L->ev_fetch, 0) == cudaSuccess;
@@ -321,6 +321,70 @@ lif_status lif_decode_token_host(lif_layer* const* layers, int32_t n_layers, con
       cudaSuccess)
     return LIF_ERR_CUDA;
   return cudaStreamSynchronize(sc) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_graph_capture(lif_layer* const* layers, int32_t n_layers, void* dev_x,
+                             float* dev_y, void* compute_stream, void* fetch_stream,
+                             lif_graph** out) {
+  if (!out) return LIF_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!layers || n_layers < 1 || !dev_x || !dev_y || !compute_stream || !fetch_stream ||
+      compute_stream == fetch_stream)
+    return LIF_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!layers[l] || layers[l]->desc.d_model != layers[0]->desc.d_model ||
+        layers[l]->desc.n_streams != layers[0]->desc.n_streams)
+      return LIF_ERR_INVALID_ARG;
+  if (!aligned(dev_x, 16) || !aligned(dev_y, 16)) return LIF_ERR_ALIGNMENT;
+  cudaStream_t sc = (cudaStream_t)compute_stream;
+  const size_t per = (size_t)layers[0]->desc.n_streams * layers[0]->desc.d_model;
+  lif_graph* g = new (std::nothrow) lif_graph();
+  if (!g) return LIF_ERR_STATE;
+  g->dev_x = dev_x;
+  g->dev_y = dev_y;
+  g->x_bytes = per * 2;
+  g->y_bytes = per * 4 * n_layers;
+  if (cudaStreamBeginCapture(sc, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    delete g;
+    return LIF_ERR_CUDA;
+  }
+  lif_status s = LIF_OK;
+  for (int l = 0; l < n_layers && s == LIF_OK; ++l)
+    s = lif_decode_step(layers[l], dev_x, dev_y + (size_t)l * per, compute_stream, fetch_stream);
+  cudaError_t e = cudaStreamEndCapture(sc, &g->graph);   // always end, also after an error
+  if (s == LIF_OK && e == cudaSuccess && cudaGraphInstantiate(&g->exec, g->graph, 0) == cudaSuccess) {
+    *out = g;
+    return LIF_OK;
+  }
+  if (e == cudaSuccess && g->graph) cudaGraphDestroy(g->graph);
+  cudaGetLastError();
+  delete g;
+  return s != LIF_OK ? s : LIF_ERR_CUDA;
+}
+
+lif_status lif_graph_launch(lif_graph* g, void* stream) {
+  if (!g) return LIF_ERR_INVALID_ARG;
+  return cudaGraphLaunch(g->exec, (cudaStream_t)stream) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_graph_launch_host(lif_graph* g, const void* host_x, float* host_y, void* stream) {
+  if (!g || !host_x || !host_y) return LIF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  bool ok = cudaMemcpyAsync(g->dev_x, host_x, g->x_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaGraphLaunch(g->exec, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(host_y, g->dev_y, g->y_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+  if (!ok) cudaGetLastError();
+  return ok ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_graph_destroy(lif_graph* g) {
+  if (!g) return LIF_ERR_INVALID_ARG;
+  cudaGraphExecDestroy(g->exec);
+  cudaGraphDestroy(g->graph);
+  delete g;
+  return LIF_OK;
 }
 
 lif_status lif_get_lists(lif_layer* L, lif_lists* o) {

@@ -269,7 +269,7 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
                        cudaEvent_t* ev) {
   const lif_layer_desc& D = L->desc;
   const int d = D.d_model;
-  if (ev) cudaEventRecord(ev[7], st);
+  if (ev) tm_record(ev[7], st);
   for (int s = 0; s < D.n_streams; ++s) {
     FfnArgs a;
     a.cache = (const __half*)D.dev_cache;
@@ -285,14 +285,14 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
     sparse_ffn_kernel<<<L->ffn_grid, kThreads, L->ffn_smem, st>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    if (ev && s == D.n_streams - 1) cudaEventRecord(ev[8], st);
+    if (ev && s == D.n_streams - 1) tm_record(ev[8], st);
     ffn_reduce_kernel<<<(d / 4 + 31) / 32, kSumThreads, 0, st>>>(
         L->y_partial, L->ffn_grid, n, (const __half*)D.dev_bias_down, y + (size_t)s * d, d,
         accumulate ? 1 : 0);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  if (ev) cudaEventRecord(ev[9], st);
+  if (ev) tm_record(ev[9], st);
   return cudaSuccess;
 }
 

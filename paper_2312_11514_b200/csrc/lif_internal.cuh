@@ -66,7 +66,23 @@ struct lif_layer {
   int tm_steps, tm_cursor;
 };
 
+struct lif_graph {
+  cudaGraph_t graph;
+  cudaGraphExec_t exec;
+  void* dev_x;
+  float* dev_y;
+  size_t x_bytes, y_bytes;
+};
+
 namespace lif {
+
+// Timing events also work inside stream capture, where they become event-record nodes.
+inline void tm_record(cudaEvent_t e, cudaStream_t st) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  cudaStreamIsCapturing(st, &cs);
+  cudaEventRecordWithFlags(e, st, cs == cudaStreamCaptureStatusActive ? cudaEventRecordExternal
+                                                                      : cudaEventRecordDefault);
+}
 
 // kernels' host launchers (each returns the launch's cudaError_t)
 cudaError_t launch_reset(lif_layer* L, cudaStream_t st);

@@ -221,7 +221,7 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
   const lif_layer_desc& D = L->desc;
   predict_z_kernel<S><<<L->z_ctas, kThreads, 0, st>>>(
       x, (const __half*)D.dev_pred_A, D.d_model, D.rank, z_rows_per_cta(D.d_model), L->z_partial);
-  if (ev) cudaEventRecord(ev[1], st);
+  if (ev) tm_record(ev[1], st);
   const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
   const size_t smem = (size_t)S * D.rank * sizeof(float);
   if (smem > 32 * 1024) {
@@ -233,7 +233,7 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
       L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit,
       D.rank, D.d_ff, logits, L->mask_words, L->counts + CNT_TICKET_PREDICT, active_idx,
       n_active);
-  if (ev) cudaEventRecord(ev[2], st);
+  if (ev) tm_record(ev[2], st);
   return cudaGetLastError();
 }
 

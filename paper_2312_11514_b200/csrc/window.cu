@@ -269,10 +269,10 @@ cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act
   window_update_kernel<<<1, kWindowThreads, 0, st>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (ev) cudaEventRecord(ev[3], st);
+  if (ev) tm_record(ev[3], st);
   move_rows_kernel<<<L->move_grid, kThreads, 0, st>>>((uint4*)D.dev_cache, L->move_src,
                                                       L->move_dst, L->counts, D.d_model / 4);
-  if (ev) cudaEventRecord(ev[4], st);
+  if (ev) tm_record(ev[4], st);
   return cudaGetLastError();
 }
 

@@ -189,3 +189,43 @@ def test_decode_token_host_matches_per_layer_decode_steps():
         assert B.lif_get_stats(a[l].handle).bytes_fetched == B.lif_get_stats(b[l].handle).bytes_fetched > 0
     for l in a + b:
         l.close()
+
+
+def test_graph_replay_matches_direct_decode_steps_bitwise():
+    cfg = W.CONFIGS["tiny"]
+    X = W.make_inputs(cfg, device=DEV)
+    a = R.build_stack(cfg, DEV)
+    b = R.build_stack(cfg, DEV)
+    L, S, d = cfg.n_layers, cfg.n_streams, cfg.d_model
+    dev_x = torch.empty(S, d, dtype=torch.float16, device=DEV)
+    y_g = torch.zeros(L, S, d, dtype=torch.float32, device=DEV)
+    y_d = torch.zeros(L, S, d, dtype=torch.float32, device=DEV)
+    host_x = torch.empty(S, d, dtype=torch.float16, pin_memory=True)
+    host_y = torch.empty(L, S, d, dtype=torch.float32, pin_memory=True)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    g = B.lif_graph_capture([l.handle for l in a], dev_x, y_g, sc, sf)
+    assert all(l.lists()["step"] == 0 for l in a)                     # capture ran nothing
+    for t in range(cfg.steps):
+        if t % 2 == 0:
+            with torch.cuda.stream(sc):
+                dev_x.copy_(X[t])
+            B.lif_graph_launch(g, sc)
+            torch.cuda.synchronize()
+            got = y_g.cpu()
+        else:
+            host_x.copy_(X[t])
+            B.lif_graph_launch_host(g, host_x, host_y, sc)
+            got = host_y.clone()
+        for l in range(L):
+            B.lif_decode_step(b[l].handle, X[t], y_d[l])
+        torch.cuda.synchronize()
+        assert torch.equal(got, y_d.cpu()), t
+    for la, lb in zip(a, b):
+        ga, gb = la.lists(), lb.lists()
+        for key in ("pointers", "slot_of", "last_active", "active_idx", "load_ids"):
+            np.testing.assert_array_equal(ga[key], gb[key])
+        assert ga["step"] == cfg.steps and ga["status"] == B.LIF_OK
+    B.lif_graph_destroy(g)
+    for l in a + b:
+        l.close()
