@@ -167,6 +167,38 @@ lif_status lif_fetch_bundles(lif_layer* layer, void* fetch_stream);
 lif_status lif_sparse_ffn(lif_layer* layer, const void* dev_x, const int32_t* dev_slots,
                           const int32_t* dev_n_slots, float* dev_y, void* stream);
 
+/* Sparse FFN for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this call; it exists for integration.)  lif_sparse_ffn needs a layer, and a layer needs
+ * a caller-allocated workspace for the per-CTA partial sums.  Code that runs where allocation
+ * is off limits — inside another framework's plugin or callback that owns the allocator, in a
+ * process whose device memory was fully handed out at start-up, or in a code path that must
+ * not synchronise the device, which cudaMalloc and cudaFree may do — can call this variant
+ * instead: the partial sums live in a fixed 2 MiB array inside the library's device image
+ * (held on every GPU that loads the library until the process exits), and the call allocates
+ * nothing, on the host or the device.
+ *   dev_matrix     fp16 [rows][2*d_model] cache rows (up half, down half), 16-byte aligned
+ *   dev_bias       fp16 [rows] up-projection bias of each row
+ *   dev_x          fp16 [d_model], one stream
+ *   dev_slots      int32 rows to use, or NULL for rows [0, *dev_n_slots)
+ *   dev_n_slots    int32 [1] on the device
+ *   dev_bias_down  fp16 [d_model] or NULL
+ *   dev_y          fp32 [d_model]
+ * Same arithmetic as lif_sparse_ffn, but the number of CTAs (at most 2 MiB / (4*d_model) and
+ * at most one per SM) and therefore the order of the partial sums can differ, so results
+ * agree to rounding, not bitwise.  d_model above LIF_STATIC_MAX_D_MODEL, or not a multiple of
+ * 8, is refused with LIF_ERR_INVALID_ARG; misaligned pointers with LIF_ERR_ALIGNMENT.
+ * The first call on each device looks up the array's device address and opts the kernel in
+ * to large shared memory; make that first call with the device current and outside any
+ * stream capture.  All calls on a device share the one array and it keeps the previous
+ * call's contents: every call overwrites the part it reads and clears its own status word,
+ * but two calls whose kernels overlap on the GPU (different streams) race on it — keep calls
+ * on one device ordered. */
+#define LIF_STATIC_MAX_D_MODEL 8192
+lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* dev_bias, const void* dev_x,
+                                 const int32_t* dev_slots, const int32_t* dev_n_slots,
+                                 const void* dev_bias_down, float* dev_y, int32_t d_model,
+                                 void* stream);
+
 /* One token through the layer: predict -> window update -> fetch (on fetch_stream, ordered by
  * events) -> sparse FFN (ffn_mode selects the rows).  The compute stream ends up ordered
  * after the fetch, so consecutive calls on the same streams are safe. */

@@ -23,6 +23,7 @@ EXPORTS = [
     "lif_decode_token_host", "lif_get_lists", "lif_get_stats", "lif_clear_status",
     "lif_probe_host_read", "lif_timing_enable", "lif_timing_read",
     "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
+    "lif_sparse_ffn_static",
 ]
 PHASES = ("predict_z", "predict_scores", "window", "moves", "fetch", "ffn", "ffn_sum")
 PHASE_LEN = 8
@@ -91,6 +92,7 @@ def lib() -> C.CDLL:
         "lif_graph_launch": [vp, vp],
         "lif_graph_launch_host": [vp, vp, vp, vp],
         "lif_graph_destroy": [vp],
+        "lif_sparse_ffn_static": [vp, vp, vp, vp, vp, vp, vp, i32, vp],
         "lif_timing_enable": [vp, i32],
         "lif_timing_read": [vp, C.POINTER(C.c_float), C.POINTER(i32)],
     }
@@ -242,3 +244,12 @@ def lif_graph_launch_host(graph: int, host_x, host_y, stream=None) -> None:
 
 def lif_graph_destroy(graph: int) -> None:
     _check(lib().lif_graph_destroy(graph), "lif_graph_destroy")
+
+
+def lif_sparse_ffn_static(matrix, bias, x, slots, n_slots, bias_down, y, d_model: int,
+                          stream=None) -> None:
+    """Sparse FFN without a layer or workspace: the partial sums use the library's built-in
+    2 MiB device array, so nothing is allocated (see include/lif.h for the sharing rules)."""
+    _check(lib().lif_sparse_ffn_static(_ptr(matrix), _ptr(bias), _ptr(x), _ptr(slots),
+                                       _ptr(n_slots), _ptr(bias_down), _ptr(y), d_model,
+                                       _stream(stream)), "lif_sparse_ffn_static")

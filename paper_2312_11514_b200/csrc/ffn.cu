@@ -297,3 +297,97 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
 }
 
 }  // namespace lif
+
+// ---------------------------------------------------------------------------------------------
+// lif_sparse_ffn_static: the same two kernels, for callers that cannot provide a workspace.
+// The CTA partials go to a fixed array in the library's own device image instead of
+// caller-allocated memory.  Nothing here allocates: no cudaMalloc/cudaFree, no events, no
+// library call that allocates.
+// ---------------------------------------------------------------------------------------------
+namespace lif {
+namespace {
+
+constexpr int kStaticFloats = 512 * 1024;   // 2 MiB of partials, resident on every device
+constexpr int kStaticMaxDevices = 64;
+
+struct StaticScratch {
+  int32_t status;                // sink for the kernel's timeout flag; cleared by every call
+  int32_t pad[63];
+  float partial[kStaticFloats];  // [ctas][d_model]
+};
+static __device__ __align__(256) StaticScratch g_static_scratch;
+
+// Per-device set-up, done by the first call on that device: the device address of the
+// scratch array (the symbol's name is only a host-side handle, never a device pointer), the
+// shared-memory opt-in of the kernel on that device, and the launch shape limits.
+struct StaticDevice {
+  bool ready;
+  StaticScratch* scratch;
+  int n_sm, max_smem;
+};
+StaticDevice g_static_dev[kStaticMaxDevices];
+
+}  // namespace
+}  // namespace lif
+
+extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* dev_bias,
+                                            const void* dev_x, const int32_t* dev_slots,
+                                            const int32_t* dev_n_slots, const void* dev_bias_down,
+                                            float* dev_y, int32_t d_model, void* stream) {
+  using namespace lif;
+  if (!dev_matrix || !dev_bias || !dev_x || !dev_n_slots || !dev_y) return LIF_ERR_INVALID_ARG;
+  // the scratch holds at least 64 CTA partials of this width
+  if (d_model < 8 || d_model % 8 || d_model > LIF_STATIC_MAX_D_MODEL) return LIF_ERR_INVALID_ARG;
+  auto mis = [](const void* p, size_t a) { return ((uintptr_t)p % a) != 0; };
+  if (mis(dev_matrix, 16) || mis(dev_x, 16) || mis(dev_y, 16) || mis(dev_bias, 2) ||
+      mis(dev_n_slots, 4) || (dev_slots && mis(dev_slots, 4)) ||
+      (dev_bias_down && mis(dev_bias_down, 8)))
+    return LIF_ERR_ALIGNMENT;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LIF_ERR_CUDA;
+  if (dev < 0 || dev >= kStaticMaxDevices) return LIF_ERR_STATE;
+  StaticDevice& sd = g_static_dev[dev];
+  if (!sd.ready) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sd.n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sd.max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(sparse_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             sd.max_smem) != cudaSuccess) {
+      cudaGetLastError();
+      return LIF_ERR_CUDA;
+    }
+    sd.scratch = static_cast<StaticScratch*>(p);
+    sd.ready = true;
+  }
+
+  int stages = 16;
+  while (stages > 1 && ffn_smem_bytes(d_model, stages) > (size_t)sd.max_smem) --stages;
+  if (ffn_smem_bytes(d_model, stages) > (size_t)sd.max_smem) return LIF_ERR_INVALID_ARG;
+  int grid = kStaticFloats / d_model;
+  if (grid > sd.n_sm) grid = sd.n_sm;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemsetAsync(&sd.scratch->status, 0, sizeof(int32_t), st) != cudaSuccess) {
+    cudaGetLastError();
+    return LIF_ERR_CUDA;
+  }
+  FfnArgs a;
+  a.cache = (const __half*)dev_matrix;
+  a.bias = (const __half*)dev_bias;
+  a.x = (const __half*)dev_x;
+  a.slots = dev_slots;
+  a.n = dev_n_slots;
+  a.base = nullptr;
+  a.y_partial = sd.scratch->partial;
+  a.status = &sd.scratch->status;
+  a.d = d_model;
+  a.stages = stages;
+  sparse_ffn_kernel<<<grid, kThreads, ffn_smem_bytes(d_model, stages), st>>>(a);
+  if (cudaGetLastError() != cudaSuccess) return LIF_ERR_CUDA;
+  ffn_reduce_kernel<<<(d_model / 4 + 31) / 32, kSumThreads, 0, st>>>(
+      sd.scratch->partial, grid, dev_n_slots, (const __half*)dev_bias_down, dev_y, d_model, 0);
+  return cudaGetLastError() == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+}
