@@ -231,6 +231,17 @@ lif_status lif_graph_launch_host(lif_graph* graph, const void* host_x, float* ho
                                  void* stream);
 lif_status lif_graph_destroy(lif_graph* graph);
 
+/* Launch-shape knobs (defaults in parentheses); they change speed, never results beyond the
+ * order of floating-point partial sums.  Set them before capturing a graph. */
+enum {
+  LIF_TUNE_DEPENDENT_LAUNCH = 0, /* (1) programmatic dependent launch along the compute stream */
+  LIF_TUNE_SPLIT_FFN = 1,        /* (1) lif_decode_step runs the FFN of already-cached rows
+                                    while the fetch copies, then the FFN of the new rows */
+  LIF_TUNE_FETCH_CTAS = 2,       /* (SM count) CTAs of the fetch kernel, 1..4096 */
+  LIF_TUNE_FFN_CTAS = 3          /* (SM count) CTAs of the sparse-FFN kernel, 1..256 */
+};
+lif_status lif_set_tuning(lif_layer* layer, int32_t key, int32_t value);
+
 /* Device addresses of lists and state (valid for the layer's lifetime). */
 lif_status lif_get_lists(lif_layer* layer, lif_lists* host_out);
 
@@ -259,6 +270,22 @@ enum {
 lif_status lif_timing_enable(lif_layer* layer, int32_t n_steps);
 lif_status lif_timing_read(lif_layer* layer, float* host_us_sums /* [LIF_PHASE_LEN] */,
                            int32_t* host_n_steps);
+
+/* Profiling aid: enqueue exactly one kernel of the decode step, with the launch shape
+ * lif_decode_step uses, on the layer's current lists (valid after a completed step; these
+ * kernels do not change the window state, so they can be replayed).  dev_x as for
+ * lif_decode_step; dev_y is written only by LIF_KERNEL_FFN_SUM.  n_streams must be 1. */
+enum {
+  LIF_KERNEL_PREDICT_Z = 0,
+  LIF_KERNEL_PREDICT_SCORES = 1,
+  LIF_KERNEL_FETCH = 2,      /* re-copies this step's new bundles */
+  LIF_KERNEL_FFN_ACTIVE = 3, /* sparse FFN kernel over all active rows */
+  LIF_KERNEL_FFN_HITS = 4,   /* ... over the active rows that were already cached */
+  LIF_KERNEL_FFN_NEW = 5,    /* ... over the rows brought in this step */
+  LIF_KERNEL_FFN_SUM = 6     /* partial-sum kernel over the hits + new partials */
+};
+lif_status lif_profile_launch(lif_layer* layer, int32_t kernel, const void* dev_x, float* dev_y,
+                              void* stream);
 
 /* Bandwidth probe for the host link: a kernel reads `bytes` of mapped pinned host memory
  * into device memory with the same access pattern as lif_fetch_bundles (chunk_bytes-sized

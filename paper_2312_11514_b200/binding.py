@@ -23,8 +23,10 @@ EXPORTS = [
     "lif_decode_token_host", "lif_get_lists", "lif_get_stats", "lif_clear_status",
     "lif_probe_host_read", "lif_timing_enable", "lif_timing_read",
     "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
-    "lif_sparse_ffn_static",
+    "lif_sparse_ffn_static", "lif_set_tuning", "lif_profile_launch",
 ]
+KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ffn_new", "ffn_sum")
+TUNE_DEPENDENT_LAUNCH, TUNE_SPLIT_FFN, TUNE_FETCH_CTAS, TUNE_FFN_CTAS = range(4)
 PHASES = ("predict_z", "predict_scores", "window", "moves", "fetch", "ffn", "ffn_sum")
 PHASE_LEN = 8
 
@@ -93,6 +95,8 @@ def lib() -> C.CDLL:
         "lif_graph_launch_host": [vp, vp, vp, vp],
         "lif_graph_destroy": [vp],
         "lif_sparse_ffn_static": [vp, vp, vp, vp, vp, vp, vp, i32, vp],
+        "lif_set_tuning": [vp, i32, i32],
+        "lif_profile_launch": [vp, i32, vp, vp, vp],
         "lif_timing_enable": [vp, i32],
         "lif_timing_read": [vp, C.POINTER(C.c_float), C.POINTER(i32)],
     }
@@ -253,3 +257,12 @@ def lif_sparse_ffn_static(matrix, bias, x, slots, n_slots, bias_down, y, d_model
     _check(lib().lif_sparse_ffn_static(_ptr(matrix), _ptr(bias), _ptr(x), _ptr(slots),
                                        _ptr(n_slots), _ptr(bias_down), _ptr(y), d_model,
                                        _stream(stream)), "lif_sparse_ffn_static")
+
+
+def lif_set_tuning(layer: int, key: int, value: int) -> None:
+    _check(lib().lif_set_tuning(layer, key, value), "lif_set_tuning")
+
+
+def lif_profile_launch(layer: int, kernel: int, x, y, stream=None) -> None:
+    _check(lib().lif_profile_launch(layer, kernel, _ptr(x), _ptr(y), _stream(stream)),
+           "lif_profile_launch")

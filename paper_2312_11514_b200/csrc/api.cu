@@ -142,6 +142,8 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
     L->ffn_grid = L->n_sm < ffn_grid_upper_bound() ? L->n_sm : ffn_grid_upper_bound();
     L->fetch_grid = L->n_sm;
     L->move_grid = L->n_sm;
+    L->use_pdl = 1;
+    L->split_ffn = 1;
     ok = cudaEventCreateWithFlags(&L->ev_plan, cudaEventDisableTiming) == cudaSuccess;
     if (ok && cudaEventCreateWithFlags(&L->ev_fetch, cudaEventDisableTiming) != cudaSuccess) {
       cudaEventDestroy(L->ev_plan);
@@ -285,10 +287,13 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   if (ev) tm_record(ev[5], sf);
   ok = ok && launch_fetch(L, sf) == cudaSuccess;
   if (ev) tm_record(ev[6], sf);
-  if (sf != sc) {
-    ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
-    ok = ok && cudaStreamWaitEvent(sc, L->ev_fetch, 0) == cudaSuccess;
+  if (sf != sc) ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
+  if (L->split_ffn) {
+    ok = ok && launch_ffn_split(L, x, dev_y, sc, sf, ev) == cudaSuccess;
+    if (!ok) cudaGetLastError();
+    return ok ? LIF_OK : LIF_ERR_CUDA;
   }
+  if (sf != sc) ok = ok && cudaStreamWaitEvent(sc, L->ev_fetch, 0) == cudaSuccess;
   if (L->desc.ffn_mode == 0)
     ok = ok && launch_ffn(L, x, L->active_slots, L->counts + LIF_CNT_N_ACTIVE, nullptr, dev_y,
                           false, sc, ev) == cudaSuccess;
@@ -385,6 +390,52 @@ lif_status lif_graph_destroy(lif_graph* g) {
   cudaGraphDestroy(g->graph);
   delete g;
   return LIF_OK;
+}
+
+lif_status lif_profile_launch(lif_layer* L, int32_t kernel, const void* dev_x, float* dev_y,
+                              void* stream) {
+  if (!L || !dev_x || L->desc.n_streams != 1) return LIF_ERR_INVALID_ARG;
+  if (!aligned(dev_x, 16) || (dev_y && !aligned(dev_y, 16))) return LIF_ERR_ALIGNMENT;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e;
+  switch (kernel) {
+    case LIF_KERNEL_PREDICT_Z:
+    case LIF_KERNEL_PREDICT_SCORES:
+      e = launch_predict_one(L, kernel, (const __half*)dev_x, st);
+      break;
+    case LIF_KERNEL_FETCH:
+      e = launch_fetch(L, st);
+      break;
+    case LIF_KERNEL_FFN_SUM:
+      if (!dev_y) return LIF_ERR_INVALID_ARG;
+      /* fall through */
+    case LIF_KERNEL_FFN_ACTIVE:
+    case LIF_KERNEL_FFN_HITS:
+    case LIF_KERNEL_FFN_NEW:
+      e = launch_one(L, kernel, (const __half*)dev_x, dev_y, st);
+      break;
+    default:
+      return LIF_ERR_INVALID_ARG;
+  }
+  if (e != cudaSuccess) cudaGetLastError();
+  return e == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
+  if (!L) return LIF_ERR_INVALID_ARG;
+  switch (key) {
+    case LIF_TUNE_DEPENDENT_LAUNCH: L->use_pdl = value != 0; return LIF_OK;
+    case LIF_TUNE_SPLIT_FFN: L->split_ffn = value != 0; return LIF_OK;
+    case LIF_TUNE_FETCH_CTAS:
+      if (value < 1 || value > 4096) return LIF_ERR_INVALID_ARG;
+      L->fetch_grid = value;
+      return LIF_OK;
+    case LIF_TUNE_FFN_CTAS:
+      if (value < 1 || value > ffn_grid_upper_bound() / 2) return LIF_ERR_INVALID_ARG;
+      L->ffn_grid = value;
+      return LIF_OK;
+  }
+  return LIF_ERR_INVALID_ARG;
 }
 
 lif_status lif_get_lists(lif_layer* L, lif_lists* o) {

@@ -73,6 +73,7 @@ struct FfnArgs {
   int32_t* status;
   int d;
   int stages;
+  int slots_len;          // entries of `slots` that may be read before n is known (0: none)
 };
 
 __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
@@ -81,29 +82,40 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
   const unsigned row_bytes = 4u * d;
   const int stages = a.stages;
   // shared layout: rows[stages][row_bytes] | x[d] fp16 | bars[stages] | part[stages][8] |
-  //                h[stages] | slot[stages]
+  //                h[stages] | bias[stages]
   unsigned char* rows = smem;
   __half* xs = reinterpret_cast<__half*>(rows + (size_t)stages * row_bytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(xs) +
                                                (((size_t)d * 2 + 15) & ~(size_t)15));
   float* part = reinterpret_cast<float*>(bars + stages);
   float* hs = part + stages * 8;
-  int* slot_s = reinterpret_cast<int*>(hs + stages);
+  float* bias_s = hs + stages;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
-  const int n = *a.n;
-  if (cta >= n) return;                       // the reduction only reads min(G, n) partials
-  const int base = a.base ? *a.base : 0;
-  const int my_cnt = (n - cta + G - 1) / G;
   const int nvec = d >> 3;                    // 16-byte chunks per half row
 
+  // nothing below the wait may depend on earlier kernels of the stream
   if (tid == 0) {
     for (int i = 0; i < stages; ++i) mbar_init(bars + i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  __syncthreads();
+  pdl_wait();
+  pdl_trigger();
+
+  // One memory round trip for the row count and this CTA's first slots: thread i reads the
+  // slot of its row before n is known when the list is long enough to make that safe.
+  int my_slot = -1;
+  if (tid < stages && a.slots) {
+    const int q = cta + tid * G;
+    if (q < a.slots_len) my_slot = a.slots[q];
+  }
+  const int n = *a.n;
+  if (cta >= n) return;                       // the reduction only reads min(G, n) partials
+  const int base = a.base ? *a.base : 0;
+  const int my_cnt = (n - cta + G - 1) / G;
+  __syncthreads();                            // barrier init visible
 
   float acc[kMaxChunks][8];
 #pragma unroll
@@ -115,15 +127,17 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
   int timed_out = 0;
   for (int r0 = 0; r0 < my_cnt; r0 += stages) {
     const int rc = min(stages, my_cnt - r0);
-    if (tid == 0) {
-      for (int i = 0; i < rc; ++i) {
-        const int q = cta + (r0 + i) * G;
-        const int slot = a.slots ? a.slots[q] : base + q;
-        slot_s[i] = slot;
-        mbar_expect_tx(bars + i, row_bytes);
-        bulk_g2s(rows + (size_t)i * row_bytes, a.cache + (size_t)slot * 2 * d, row_bytes,
-                 bars + i);
-      }
+    // thread i issues the copy of row i of this round and fetches its bias
+    if (tid < rc) {
+      const int q = cta + (r0 + tid) * G;
+      int slot;
+      if (!a.slots) slot = base + q;
+      else if (r0 == 0 && q < a.slots_len) slot = my_slot;
+      else slot = a.slots[q];
+      mbar_expect_tx(bars + tid, row_bytes);
+      bulk_g2s(rows + (size_t)tid * row_bytes, a.cache + (size_t)slot * 2 * d, row_bytes,
+               bars + tid);
+      bias_s[tid] = __half2float(a.bias[slot]);
     }
     if (r0 == 0) {
       const uint4* xg = reinterpret_cast<const uint4*>(a.x);
@@ -161,8 +175,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
       float v = 0.f;
 #pragma unroll
       for (int w = 0; w < 8; ++w) v += part[tid * 8 + w];
-      v += __half2float(a.bias[slot_s[tid]]);
-      hs[tid] = fmaxf(v, 0.f);
+      hs[tid] = fmaxf(v + bias_s[tid], 0.f);
     }
     __syncthreads();
     // down projection: y += h * down half
@@ -196,40 +209,45 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
   }
 }
 
-// y[m] = (accumulate ? y[m] : b_down[m]) + sum_{g < min(G, n)} y_partial[g][m].  1024 threads =
-// 32 float4 columns x 32 slices of g; each slice adds its partials in ascending g, then the
-// slices are added in ascending order: a fixed summation order.
+// y[m] = (accumulate ? y[m] : b_down[m]) + sum over set 0 then set 1 of the CTA partials
+// (set j holds min(G, *n_j) partials; set 1 is optional).  1024 threads = 32 float4 columns x
+// 32 slices; each slice adds its partials in ascending order, then the slices are added in
+// ascending order: a fixed summation order.
 constexpr int kSumThreads = 1024;
 __global__ void __launch_bounds__(kSumThreads)
-ffn_reduce_kernel(const float* __restrict__ y_partial, int G, const int32_t* __restrict__ n,
+ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
+                  const float* __restrict__ p1, const int32_t* __restrict__ n1, int G,
                   const __half* __restrict__ b_down, float* __restrict__ y, int d,
                   int accumulate) {
   __shared__ float4 red[32][32];
   const int tid = threadIdx.x;
   const int c4 = tid & 31, gs = tid >> 5;
   const int col4 = blockIdx.x * 32 + c4;       // float4 column
-  const int valid = min(G, *n);
+  const bool in = col4 * 4 < d;
+  float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (gs == 0 && in) {                         // independent of earlier kernels' partials
+    if (b_down && !accumulate) {
+      const __half2* b = reinterpret_cast<const __half2*>(b_down) + col4 * 2;
+      const float2 lo = __half22float2(b[0]), hi = __half22float2(b[1]);
+      t = make_float4(lo.x, lo.y, hi.x, hi.y);
+    }
+  }
+  pdl_wait();
+  pdl_trigger();
+  const int v0 = min(G, *n0), v1 = p1 ? min(G, *n1) : 0;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (col4 * 4 < d) {
+  if (in) {
 #pragma unroll 4
-    for (int g = gs; g < valid; g += 32) {
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(y_partial + (size_t)g * d) + col4);
+    for (int g = gs; g < v0 + v1; g += 32) {
+      const float* src = g < v0 ? p0 + (size_t)g * d : p1 + (size_t)(g - v0) * d;
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(src) + col4);
       s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
     }
   }
   red[gs][c4] = s;
   __syncthreads();
-  if (gs == 0 && col4 * 4 < d) {
-    float4 t;
-    if (accumulate) {
-      t = reinterpret_cast<float4*>(y)[col4];
-    } else if (b_down) {
-      const __half2* b = reinterpret_cast<const __half2*>(b_down) + col4 * 2;
-      const float2 lo = __half22float2(b[0]), hi = __half22float2(b[1]);
-      t = make_float4(lo.x, lo.y, hi.x, hi.y);
-    } else {
-      t = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+  if (gs == 0 && in) {
+    if (accumulate) t = reinterpret_cast<float4*>(y)[col4];
 #pragma unroll
     for (int k = 0; k < 32; ++k) {
       t.x += red[k][c4].x; t.y += red[k][c4].y; t.z += red[k][c4].z; t.w += red[k][c4].w;
@@ -264,6 +282,23 @@ cudaError_t ffn_configure(lif_layer* L) {
                               (int)max_smem);
 }
 
+static FfnArgs ffn_args(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
+                        const int32_t* base, float* partial, int slots_len) {
+  FfnArgs a;
+  a.cache = (const __half*)L->desc.dev_cache;
+  a.bias = L->bias;
+  a.x = x;
+  a.slots = slots;
+  a.n = n;
+  a.base = base;
+  a.y_partial = partial;
+  a.status = L->counts + LIF_CNT_STATUS;
+  a.d = L->desc.d_model;
+  a.stages = L->ffn_stages;
+  a.slots_len = slots_len;
+  return a;
+}
+
 cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
                        const int32_t* base, float* y, bool accumulate, cudaStream_t st,
                        cudaEvent_t* ev) {
@@ -271,25 +306,82 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
   const int d = D.d_model;
   if (ev) tm_record(ev[7], st);
   for (int s = 0; s < D.n_streams; ++s) {
-    FfnArgs a;
-    a.cache = (const __half*)D.dev_cache;
-    a.bias = L->bias;
-    a.x = x + (size_t)s * d;
-    a.slots = slots;
-    a.n = n;
-    a.base = base;
-    a.y_partial = L->y_partial;
-    a.status = L->counts + LIF_CNT_STATUS;
-    a.d = d;
-    a.stages = L->ffn_stages;
-    sparse_ffn_kernel<<<L->ffn_grid, kThreads, L->ffn_smem, st>>>(a);
-    cudaError_t e = cudaGetLastError();
+    // a caller's slot list may be shorter than d_ff: never read it before n is known
+    FfnArgs a = ffn_args(L, x + (size_t)s * d, slots, n, base, L->y_partial,
+                         slots && (slots == L->active_slots || slots == L->hit_slots) ? D.d_ff : 0);
+    cudaError_t e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem,
+                             st, L->use_pdl, a);
     if (e != cudaSuccess) return e;
     if (ev && s == D.n_streams - 1) tm_record(ev[8], st);
-    ffn_reduce_kernel<<<(d / 4 + 31) / 32, kSumThreads, 0, st>>>(
-        L->y_partial, L->ffn_grid, n, (const __half*)D.dev_bias_down, y + (size_t)s * d, d,
-        accumulate ? 1 : 0);
-    e = cudaGetLastError();
+    e = launch_k(ffn_reduce_kernel, dim3((d / 4 + 31) / 32), dim3(kSumThreads), 0, st, L->use_pdl,
+                 (const float*)L->y_partial, n, (const float*)nullptr, (const int32_t*)nullptr,
+                 L->ffn_grid, (const __half*)D.dev_bias_down, y + (size_t)s * d, d,
+                 accumulate ? 1 : 0);
+    if (e != cudaSuccess) return e;
+  }
+  if (ev) tm_record(ev[9], st);
+  return cudaSuccess;
+}
+
+cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cudaStream_t st) {
+  const lif_layer_desc& D = L->desc;
+  const int d = D.d_model;
+  const int32_t* cnt = L->counts;
+  float* p0 = L->y_partial;
+  float* p1 = L->y_partial + (size_t)L->ffn_grid * d;
+  FfnArgs a;
+  switch (kernel) {
+    case LIF_KERNEL_FFN_ACTIVE:
+      a = ffn_args(L, x, L->active_slots, cnt + LIF_CNT_N_ACTIVE, nullptr, p0, D.d_ff);
+      break;
+    case LIF_KERNEL_FFN_HITS:
+      a = ffn_args(L, x, L->hit_slots, cnt + LIF_CNT_N_HITS, nullptr, p0, D.d_ff);
+      break;
+    case LIF_KERNEL_FFN_NEW:
+      a = ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
+      break;
+    case LIF_KERNEL_FFN_SUM:
+      return launch_k(ffn_reduce_kernel, dim3((d / 4 + 31) / 32), dim3(kSumThreads), 0, st,
+                      L->use_pdl, (const float*)p0, cnt + LIF_CNT_N_HITS, (const float*)p1,
+                      cnt + LIF_CNT_N_LOAD, L->ffn_grid, (const __half*)D.dev_bias_down, y, d, 0);
+    default:
+      return cudaErrorInvalidValue;
+  }
+  return launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
+                  L->use_pdl, a);
+}
+
+// FFN of a decode step in two parts: the rows that were already cached (they can run while
+// the fetch is still copying), then, after `ev_fetch`, the rows just brought in; one sum.
+cudaError_t launch_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream_t st,
+                             cudaStream_t fetch_st, cudaEvent_t* ev) {
+  const lif_layer_desc& D = L->desc;
+  const int d = D.d_model;
+  const int32_t* cnt = L->counts;
+  float* p0 = L->y_partial;
+  float* p1 = L->y_partial + (size_t)L->ffn_grid * d;
+  if (ev) tm_record(ev[7], st);
+  for (int s = 0; s < D.n_streams; ++s) {
+    const __half* xs = x + (size_t)s * d;
+    const bool last = s == D.n_streams - 1;
+    FfnArgs hit = D.ffn_mode == 0
+                      ? ffn_args(L, xs, L->hit_slots, cnt + LIF_CNT_N_HITS, nullptr, p0, D.d_ff)
+                      : ffn_args(L, xs, nullptr, cnt + LIF_CNT_NUM_KEPT, nullptr, p0, 0);
+    cudaError_t e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem,
+                             st, L->use_pdl, hit);
+    if (e != cudaSuccess) return e;
+    if (s == 0 && fetch_st != st) {
+      e = cudaStreamWaitEvent(st, L->ev_fetch, 0);
+      if (e != cudaSuccess) return e;
+    }
+    FfnArgs miss = ffn_args(L, xs, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
+    e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
+                 L->use_pdl, miss);
+    if (e != cudaSuccess) return e;
+    if (ev && last) tm_record(ev[8], st);
+    e = launch_k(ffn_reduce_kernel, dim3((d / 4 + 31) / 32), dim3(kSumThreads), 0, st, L->use_pdl,
+                 (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,
+                 (const __half*)D.dev_bias_down, y + (size_t)s * d, d, 0);
     if (e != cudaSuccess) return e;
   }
   if (ev) tm_record(ev[9], st);
@@ -385,9 +477,11 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
   a.status = &sd.scratch->status;
   a.d = d_model;
   a.stages = stages;
+  a.slots_len = 0;
   sparse_ffn_kernel<<<grid, kThreads, ffn_smem_bytes(d_model, stages), st>>>(a);
   if (cudaGetLastError() != cudaSuccess) return LIF_ERR_CUDA;
   ffn_reduce_kernel<<<(d_model / 4 + 31) / 32, kSumThreads, 0, st>>>(
-      sd.scratch->partial, grid, dev_n_slots, (const __half*)dev_bias_down, dev_y, d_model, 0);
+      sd.scratch->partial, dev_n_slots, nullptr, nullptr, grid, (const __half*)dev_bias_down,
+      dev_y, d_model, 0);
   return cudaGetLastError() == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
 }

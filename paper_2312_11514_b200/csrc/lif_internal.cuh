@@ -60,6 +60,8 @@ struct lif_layer {
   size_t ffn_smem;    // dynamic shared memory of the sparse-FFN kernel
   int fetch_grid;     // CTAs of the fetch kernel
   int move_grid;
+  int use_pdl;        // programmatic dependent launch along the compute stream
+  int split_ffn;      // decode step: cached rows' FFN overlaps the fetch
   cudaEvent_t ev_plan, ev_fetch;
   // optional per-kernel timing: kTimingEvents events per recorded step
   cudaEvent_t* tm_events;
@@ -99,6 +101,40 @@ cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes,
 cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
                        const int32_t* base, float* y, bool accumulate, cudaStream_t st,
                        cudaEvent_t* ev = nullptr);
+cudaError_t launch_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream_t st,
+                             cudaStream_t fetch_st, cudaEvent_t* ev = nullptr);
+cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cudaStream_t st);
+cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaStream_t st);
 cudaError_t ffn_configure(lif_layer* L);
+
+// Launch with (pdl) or without the programmatic-stream-serialization attribute.  A kernel
+// launched with it may start while the previous kernel of the stream is still running; it
+// must execute pdl_wait() before it touches anything an earlier kernel wrote (every kernel of
+// this library does so on every path, which also keeps the ordering transitive).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                     cudaStream_t st, int pdl, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+#ifdef __CUDACC__
+// Block until every earlier kernel of the stream has completed and its writes are visible
+// (no-op for a kernel launched without the attribute).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Let the next kernel of the stream start its prologue.
+__device__ __forceinline__ void pdl_trigger() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
 
 }  // namespace lif

@@ -49,9 +49,33 @@ predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[s][e] = 0.f;
 
+  // A is a weight: its first 8 rows per thread are put in flight before the dependency wait,
+  // x (possibly written by the previous kernel) only after it.
+  uint4 aq[8];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int m = m0 + rl + u * nrl;
+    aq[u] = (rl < nrl && m < m1) ? ldg_stream(A + (size_t)m * r + cg * 8) : make_uint4(0, 0, 0, 0);
+  }
+  pdl_wait();
+  pdl_trigger();
   if (rl < nrl) {
-#pragma unroll 8
-    for (int m = m0 + rl; m < m1; m += nrl) {
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int m = m0 + rl + u * nrl;
+      if (m < m1) {
+        float af[8];
+        unpack8(aq[u], af);
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+          const float xs = __half2float(x[(size_t)s * d + m]);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[s][e] = fmaf(xs, af[e], acc[s][e]);
+        }
+      }
+    }
+#pragma unroll 4
+    for (int m = m0 + rl + 8 * nrl; m < m1; m += nrl) {
       float af[8];
       unpack8(ldg_stream(A + (size_t)m * r + cg * 8), af);
 #pragma unroll
@@ -124,6 +148,10 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
     const int j = rs + 16 * u;
     bq[u] = (col < F && j < r) ? ldg_stream(B + (size_t)j * F + col) : make_uint4(0, 0, 0, 0);
   }
+  const int my_col = blockIdx.x * kLogitTile + tid;   // used by threads < kLogitTile
+  const float my_c = (tid < kLogitTile && my_col < F) ? c[my_col] : 0.f;
+  pdl_wait();
+  pdl_trigger();
   for (int i = tid; i < S * r; i += kThreads) {
     float v = 0.f;
 #pragma unroll 8
@@ -162,7 +190,6 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
   }
 
   bool active = false;
-  const int my_col = blockIdx.x * kLogitTile + tid;   // used by threads < kLogitTile
 #pragma unroll
   for (int s = 0; s < S; ++s) {
 #pragma unroll
@@ -172,7 +199,7 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
       float v = 0.f;
 #pragma unroll
       for (int k = 0; k < 16; ++k) v += red[k][tid];
-      v += c[my_col];
+      v += my_c;
       if (logits) logits[(size_t)s * F + my_col] = v;
       active = active || (v > theta);
     }
@@ -219,25 +246,42 @@ template <int S>
 cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
                              int32_t* n_active, cudaStream_t st, cudaEvent_t* ev) {
   const lif_layer_desc& D = L->desc;
-  predict_z_kernel<S><<<L->z_ctas, kThreads, 0, st>>>(
-      x, (const __half*)D.dev_pred_A, D.d_model, D.rank, z_rows_per_cta(D.d_model), L->z_partial);
+  cudaError_t e = launch_k(predict_z_kernel<S>, dim3(L->z_ctas), dim3(kThreads), 0, st, L->use_pdl,
+                           x, (const __half*)D.dev_pred_A, D.d_model, D.rank,
+                           z_rows_per_cta(D.d_model), L->z_partial);
+  if (e != cudaSuccess) return e;
   if (ev) tm_record(ev[1], st);
   const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
   const size_t smem = (size_t)S * D.rank * sizeof(float);
   if (smem > 32 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(predict_logits_kernel<S>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(predict_logits_kernel<S>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  predict_logits_kernel<S><<<grid, kThreads, smem, st>>>(
-      L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit,
-      D.rank, D.d_ff, logits, L->mask_words, L->counts + CNT_TICKET_PREDICT, active_idx,
-      n_active);
+  e = launch_k(predict_logits_kernel<S>, dim3(grid), dim3(kThreads), smem, st, L->use_pdl,
+               (const float*)L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c,
+               D.threshold_logit, D.rank, D.d_ff, logits, L->mask_words,
+               (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active);
   if (ev) tm_record(ev[2], st);
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace
+
+cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaStream_t st) {
+  const lif_layer_desc& D = L->desc;
+  if (D.n_streams != 1) return cudaErrorInvalidValue;
+  if (kernel == LIF_KERNEL_PREDICT_Z)
+    return launch_k(predict_z_kernel<1>, dim3(L->z_ctas), dim3(kThreads), 0, st, L->use_pdl, x,
+                    (const __half*)D.dev_pred_A, D.d_model, D.rank, z_rows_per_cta(D.d_model),
+                    L->z_partial);
+  const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
+  return launch_k(predict_logits_kernel<1>, dim3(grid), dim3(kThreads),
+                  (size_t)D.rank * sizeof(float), st, L->use_pdl, (const float*)L->z_partial,
+                  L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit, D.rank,
+                  D.d_ff, (float*)nullptr, L->mask_words, (int*)(L->counts + CNT_TICKET_PREDICT),
+                  (int*)L->active_idx, (int*)L->n_tmp);
+}
 
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
                            int32_t* n_active, cudaStream_t st, cudaEvent_t* ev) {

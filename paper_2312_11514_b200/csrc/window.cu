@@ -70,6 +70,8 @@ struct WindowArgs {
 __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArgs a) {
   __shared__ Scan sc;
   const int tid = threadIdx.x;
+  pdl_wait();
+  pdl_trigger();
   const int n = a.counts[LIF_CNT_NUM_USED];
   const int t = a.counts[LIF_CNT_STEP];
   const int na = *a.n_act;
@@ -208,6 +210,8 @@ __global__ void __launch_bounds__(kThreads)
 move_rows_kernel(uint4* __restrict__ cache, const int32_t* __restrict__ move_src,
                  const int32_t* __restrict__ move_dst, const int32_t* __restrict__ counts,
                  int row_vec) {
+  pdl_wait();
+  pdl_trigger();
   const int n = counts[LIF_CNT_N_MOVES];
   for (int j = blockIdx.x; j < n; j += gridDim.x) {
     const uint4* src = cache + (size_t)move_src[j] * row_vec;
@@ -266,14 +270,14 @@ cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act
   a.cap = D.capacity;
   a.k = D.window_k;
   a.bundle_bytes = 4ull * D.d_model;
-  window_update_kernel<<<1, kWindowThreads, 0, st>>>(a);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_k(window_update_kernel, dim3(1), dim3(kWindowThreads), 0, st, L->use_pdl, a);
   if (e != cudaSuccess) return e;
   if (ev) tm_record(ev[3], st);
-  move_rows_kernel<<<L->move_grid, kThreads, 0, st>>>((uint4*)D.dev_cache, L->move_src,
-                                                      L->move_dst, L->counts, D.d_model / 4);
+  e = launch_k(move_rows_kernel, dim3(L->move_grid), dim3(kThreads), 0, st, L->use_pdl,
+               (uint4*)D.dev_cache, (const int32_t*)L->move_src, (const int32_t*)L->move_dst,
+               (const int32_t*)L->counts, D.d_model / 4);
   if (ev) tm_record(ev[4], st);
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace lif

@@ -142,11 +142,15 @@ def test_reset_gives_cold_cache_and_runs_are_reproducible():
     gpu.close()
 
 
-@pytest.mark.parametrize("two_streams", [False, True])
-def test_decode_step_matches_oracle_decode_step(two_streams):
+@pytest.mark.parametrize("two_streams,pdl,split,ffn_mode", [
+    (False, 1, 1, 0), (True, 1, 1, 0), (True, 0, 1, 0), (True, 1, 0, 0), (True, 0, 0, 0),
+    (True, 1, 1, 1), (False, 1, 0, 1)])
+def test_decode_step_matches_oracle_decode_step(two_streams, pdl, split, ffn_mode):
     cfg = W.CONFIGS["tiny"]
     X = W.make_inputs(cfg, device=DEV)
-    gpu, ora = P.make_layer_pair(cfg, 1, b_down=True)
+    gpu, ora = P.make_layer_pair(cfg, 1, b_down=True, ffn_mode=ffn_mode)
+    B.lif_set_tuning(gpu.handle, B.TUNE_DEPENDENT_LAUNCH, pdl)
+    B.lif_set_tuning(gpu.handle, B.TUNE_SPLIT_FFN, split)
     y = torch.empty(cfg.n_streams, cfg.d_model, dtype=torch.float32, device=DEV)
     sc, sf = (torch.cuda.Stream(), torch.cuda.Stream()) if two_streams else (None, None)
     if sc is not None:
@@ -157,7 +161,7 @@ def test_decode_step_matches_oracle_decode_step(two_streams):
         x_np = X[t].cpu().numpy()
         logits, act, lists, ref_y = O.decode_step(ora.cache, x_np, ora.A, ora.B, ora.c, ora.theta,
                                                   ora.bundles, ora.bias_up, ora.b_down,
-                                                  act=g["active_idx"])
+                                                  whole_cache=(ffn_mode == 1), act=g["active_idx"])
         P.assert_mask_borderline(g["active_idx"], logits, ora.theta)
         P.compare_lists_and_state(gpu, ora, lists)
         P.compare_cache_rows(gpu, ora)
