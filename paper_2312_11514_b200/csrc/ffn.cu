@@ -210,22 +210,23 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
 }
 
 // y[m] = (accumulate ? y[m] : b_down[m]) + sum over set 0 then set 1 of the CTA partials
-// (set j holds min(G, *n_j) partials; set 1 is optional).  1024 threads = 32 float4 columns x
-// 32 slices; each slice adds its partials in ascending order, then the slices are added in
-// ascending order: a fixed summation order.
-constexpr int kSumThreads = 1024;
+// (set j holds min(G, *n_j) partials; set 1 is optional).  A CTA owns 8 float4 columns (one
+// 128-byte line per partial) x 32 slices of the partial index; each slice adds its partials
+// in ascending order, then the slices are added in ascending order: a fixed summation order.
+constexpr int kSumThreads = 256;
+constexpr int kSumCols = 8;                     // float4 columns per CTA
 __global__ void __launch_bounds__(kSumThreads)
 ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
                   const float* __restrict__ p1, const int32_t* __restrict__ n1, int G,
                   const __half* __restrict__ b_down, float* __restrict__ y, int d,
                   int accumulate) {
-  __shared__ float4 red[32][32];
+  __shared__ float4 red[32][kSumCols];
   const int tid = threadIdx.x;
-  const int c4 = tid & 31, gs = tid >> 5;
-  const int col4 = blockIdx.x * 32 + c4;       // float4 column
+  const int c4 = tid & (kSumCols - 1), gs = tid / kSumCols;
+  const int col4 = blockIdx.x * kSumCols + c4;  // float4 column
   const bool in = col4 * 4 < d;
   float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (gs == 0 && in) {                         // independent of earlier kernels' partials
+  if (gs == 0 && in) {                          // independent of earlier kernels' partials
     if (b_down && !accumulate) {
       const __half2* b = reinterpret_cast<const __half2*>(b_down) + col4 * 2;
       const float2 lo = __half22float2(b[0]), hi = __half22float2(b[1]);
@@ -313,7 +314,7 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
                              st, L->use_pdl, a);
     if (e != cudaSuccess) return e;
     if (ev && s == D.n_streams - 1) tm_record(ev[8], st);
-    e = launch_k(ffn_reduce_kernel, dim3((d / 4 + 31) / 32), dim3(kSumThreads), 0, st, L->use_pdl,
+    e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st, L->use_pdl,
                  (const float*)L->y_partial, n, (const float*)nullptr, (const int32_t*)nullptr,
                  L->ffn_grid, (const __half*)D.dev_bias_down, y + (size_t)s * d, d,
                  accumulate ? 1 : 0);
@@ -341,7 +342,7 @@ cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cuda
       a = ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
       break;
     case LIF_KERNEL_FFN_SUM:
-      return launch_k(ffn_reduce_kernel, dim3((d / 4 + 31) / 32), dim3(kSumThreads), 0, st,
+      return launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st,
                       L->use_pdl, (const float*)p0, cnt + LIF_CNT_N_HITS, (const float*)p1,
                       cnt + LIF_CNT_N_LOAD, L->ffn_grid, (const __half*)D.dev_bias_down, y, d, 0);
     default:
@@ -379,7 +380,7 @@ cudaError_t launch_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream
                  L->use_pdl, miss);
     if (e != cudaSuccess) return e;
     if (ev && last) tm_record(ev[8], st);
-    e = launch_k(ffn_reduce_kernel, dim3((d / 4 + 31) / 32), dim3(kSumThreads), 0, st, L->use_pdl,
+    e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st, L->use_pdl,
                  (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,
                  (const __half*)D.dev_bias_down, y + (size_t)s * d, d, 0);
     if (e != cudaSuccess) return e;
@@ -480,7 +481,7 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
   a.slots_len = 0;
   sparse_ffn_kernel<<<grid, kThreads, ffn_smem_bytes(d_model, stages), st>>>(a);
   if (cudaGetLastError() != cudaSuccess) return LIF_ERR_CUDA;
-  ffn_reduce_kernel<<<(d_model / 4 + 31) / 32, kSumThreads, 0, st>>>(
+  ffn_reduce_kernel<<<(d_model / 4 + kSumCols - 1) / kSumCols, kSumThreads, 0, st>>>(
       sd.scratch->partial, dev_n_slots, nullptr, nullptr, grid, (const __half*)dev_bias_down,
       dev_y, d_model, 0);
   return cudaGetLastError() == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
