@@ -238,7 +238,9 @@ enum {
   LIF_TUNE_SPLIT_FFN = 1,        /* (1) lif_decode_step runs the FFN of already-cached rows
                                     while the fetch copies, then the FFN of the new rows */
   LIF_TUNE_FETCH_CTAS = 2,       /* (SM count) CTAs of the fetch kernel, 1..4096 */
-  LIF_TUNE_FFN_CTAS = 3          /* (SM count) CTAs of the sparse-FFN kernel, 1..256 */
+  LIF_TUNE_FFN_CTAS = 3,         /* (SM count) CTAs of the sparse-FFN kernel, 1..256 */
+  LIF_TUNE_FFN_STAGES = 4        /* (as many as fit, at most 16) bundles in flight per CTA;
+                                    fewer stages let several CTAs share an SM */
 };
 lif_status lif_set_tuning(lif_layer* layer, int32_t key, int32_t value);
 

@@ -36,7 +36,11 @@ Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max) {
   w.n_tmp = take(64);
   w.z_partial = take(z_ctas * S * d.rank * 4);
   w.mask_words = take(n_mask * 4);
-  w.y_partial = take((size_t)ffn_grid_max * d.d_model * 4);
+  w.h_rows = take(d.n_streams > 1 ? F * 8 * 4 : 0);
+  size_t partial_rows = (size_t)ffn_grid_max;
+  if (ffn_batched_supported(d) && (size_t)kBatchedMaxPartitions * S > partial_rows)
+    partial_rows = (size_t)kBatchedMaxPartitions * S;
+  w.y_partial = take(partial_rows * d.d_model * 4);
   w.total = off;
   return w;
 }
@@ -132,11 +136,13 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
   L->z_partial = (float*)(b + ws.z_partial);
   L->mask_words = (uint32_t*)(b + ws.mask_words);
   L->y_partial = (float*)(b + ws.y_partial);
+  L->h_rows = (float*)(b + ws.h_rows);
 
   int dev = 0;
   bool ok = cudaGetDevice(&dev) == cudaSuccess &&
             cudaDeviceGetAttribute(&L->n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
   ok = ok && ffn_configure(L) == cudaSuccess;
+  ok = ok && ffn_batched_configure(L) == cudaSuccess;
   if (ok) {
     L->z_ctas = z_cta_count(desc->d_model);
     L->ffn_grid = L->n_sm < ffn_grid_upper_bound() ? L->n_sm : ffn_grid_upper_bound();
@@ -288,7 +294,7 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   ok = ok && launch_fetch(L, sf) == cudaSuccess;
   if (ev) tm_record(ev[6], sf);
   if (sf != sc) ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
-  if (L->split_ffn) {
+  if (L->split_ffn && !L->fb_ok) {
     ok = ok && launch_ffn_split(L, x, dev_y, sc, sf, ev) == cudaSuccess;
     if (!ok) cudaGetLastError();
     return ok ? LIF_OK : LIF_ERR_CUDA;
@@ -433,6 +439,11 @@ lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
     case LIF_TUNE_FFN_CTAS:
       if (value < 1 || value > ffn_grid_upper_bound() / 2) return LIF_ERR_INVALID_ARG;
       L->ffn_grid = value;
+      return LIF_OK;
+    case LIF_TUNE_FFN_STAGES:
+      if (value < 1 || value > L->ffn_stages_max) return LIF_ERR_INVALID_ARG;
+      L->ffn_stages = value;
+      L->ffn_smem = ffn_smem_for(L->desc.d_model, value);
       return LIF_OK;
   }
   return LIF_ERR_INVALID_ARG;

@@ -267,6 +267,8 @@ size_t ffn_smem_bytes(int d, int stages) {
 
 }  // namespace
 
+size_t ffn_smem_for(int d_model, int stages) { return ffn_smem_bytes(d_model, stages); }
+
 cudaError_t ffn_configure(lif_layer* L) {
   const int d = L->desc.d_model;
   int dev = 0, max_smem = 0;
@@ -277,7 +279,7 @@ cudaError_t ffn_configure(lif_layer* L) {
   int stages = 16;
   while (stages > 1 && ffn_smem_bytes(d, stages) > (size_t)max_smem) --stages;
   if (ffn_smem_bytes(d, stages) > (size_t)max_smem) return cudaErrorInvalidValue;
-  L->ffn_stages = stages;
+  L->ffn_stages = L->ffn_stages_max = stages;
   L->ffn_smem = ffn_smem_bytes(d, stages);
   return cudaFuncSetAttribute(sparse_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)max_smem);
@@ -305,6 +307,15 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
                        cudaEvent_t* ev) {
   const lif_layer_desc& D = L->desc;
   const int d = D.d_model;
+  if (L->fb_ok && !accumulate) {   // several streams: tensor-core contraction over the rows
+    if (ev) tm_record(ev[7], st);
+    cudaError_t e = launch_ffn_batched(L, x, slots, n, base, y, st);
+    if (ev) {
+      tm_record(ev[8], st);
+      tm_record(ev[9], st);
+    }
+    return e;
+  }
   if (ev) tm_record(ev[7], st);
   for (int s = 0; s < D.n_streams; ++s) {
     // a caller's slot list may be shorter than d_ff: never read it before n is known

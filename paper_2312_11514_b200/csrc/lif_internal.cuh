@@ -34,7 +34,7 @@ struct Workspace {
   // offsets in bytes from the workspace base; every block 256-byte aligned
   size_t counts, pointers, slot_of, last_active, bias, active_idx, evict_ids, evict_slots,
       move_src, move_dst, load_ids, load_slots, active_slots, hit_slots, n_tmp, z_partial,
-      mask_words, y_partial, total;
+      mask_words, h_rows, y_partial, total;
 };
 
 Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max);
@@ -53,10 +53,15 @@ struct lif_layer {
   float* z_partial;
   uint32_t* mask_words;
   float* y_partial;
+  float* h_rows;      // [d_ff][8] fp32: phase-A output of the multi-stream FFN
+  // multi-stream (tensor-core) FFN configuration; fb_ok = 0: per-stream fallback
+  int fb_ok, fb_up_stages, fb_parts, fb_cols, fb_partitions;
+  size_t fb_up_smem, fb_down_smem;
   int n_sm;
   int z_ctas;         // CTAs of the first predictor stage
   int ffn_grid;       // CTAs of the sparse-FFN kernel
   int ffn_stages;     // bundles in flight per CTA
+  int ffn_stages_max; // what fits the shared memory of one CTA
   size_t ffn_smem;    // dynamic shared memory of the sparse-FFN kernel
   int fetch_grid;     // CTAs of the fetch kernel
   int move_grid;
@@ -106,6 +111,12 @@ cudaError_t launch_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream
 cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cudaStream_t st);
 cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaStream_t st);
 cudaError_t ffn_configure(lif_layer* L);
+constexpr int kBatchedMaxPartitions = 128;
+bool ffn_batched_supported(const lif_layer_desc& D);
+cudaError_t ffn_batched_configure(lif_layer* L);
+cudaError_t launch_ffn_batched(lif_layer* L, const __half* x, const int32_t* slots,
+                               const int32_t* n, const int32_t* base, float* y, cudaStream_t st);
+size_t ffn_smem_for(int d_model, int stages);
 
 // Launch with (pdl) or without the programmatic-stream-serialization attribute.  A kernel
 // launched with it may start while the previous kernel of the stream is still running; it
