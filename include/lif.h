@@ -239,8 +239,10 @@ enum {
                                     while the fetch copies, then the FFN of the new rows */
   LIF_TUNE_FETCH_CTAS = 2,       /* (SM count) CTAs of the fetch kernel, 1..4096 */
   LIF_TUNE_FFN_CTAS = 3,         /* (SM count) CTAs of the sparse-FFN kernel, 1..256 */
-  LIF_TUNE_FFN_STAGES = 4        /* (as many as fit, at most 16) bundles in flight per CTA;
+  LIF_TUNE_FFN_STAGES = 4,       /* (as many as fit, at most 16) bundles in flight per CTA;
                                     fewer stages let several CTAs share an SM */
+  LIF_TUNE_BATCHED_COLUMN_PARTS = 5 /* (fewest that fit) column parts of the multi-stream FFN's
+                                    down-projection kernel, 1..16 */
 };
 lif_status lif_set_tuning(lif_layer* layer, int32_t key, int32_t value);
 

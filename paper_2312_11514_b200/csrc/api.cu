@@ -36,7 +36,7 @@ Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max) {
   w.n_tmp = take(64);
   w.z_partial = take(z_ctas * S * d.rank * 4);
   w.mask_words = take(n_mask * 4);
-  w.h_rows = take(d.n_streams > 1 ? F * 8 * 4 : 0);
+  w.h_rows = take(d.n_streams > 1 ? (size_t)kBatchedMaxKSplit * F * 8 * 4 : 0);
   size_t partial_rows = (size_t)ffn_grid_max;
   if (ffn_batched_supported(d) && (size_t)kBatchedMaxPartitions * S > partial_rows)
     partial_rows = (size_t)kBatchedMaxPartitions * S;
@@ -440,6 +440,10 @@ lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
       if (value < 1 || value > ffn_grid_upper_bound() / 2) return LIF_ERR_INVALID_ARG;
       L->ffn_grid = value;
       return LIF_OK;
+    case LIF_TUNE_BATCHED_COLUMN_PARTS:
+      if (value < 1 || value > 16) return LIF_ERR_INVALID_ARG;
+      L->fb_parts_min = value;
+      return ffn_batched_configure(L) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
     case LIF_TUNE_FFN_STAGES:
       if (value < 1 || value > L->ffn_stages_max) return LIF_ERR_INVALID_ARG;
       L->ffn_stages = value;

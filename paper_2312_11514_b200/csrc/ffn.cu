@@ -218,7 +218,7 @@ constexpr int kSumCols = 8;                     // float4 columns per CTA
 __global__ void __launch_bounds__(kSumThreads)
 ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
                   const float* __restrict__ p1, const int32_t* __restrict__ n1, int G,
-                  const __half* __restrict__ b_down, float* __restrict__ y, int d,
+                  const __half* __restrict__ b_down, int b_period, float* __restrict__ y, int d,
                   int accumulate) {
   __shared__ float4 red[32][kSumCols];
   const int tid = threadIdx.x;
@@ -228,7 +228,7 @@ ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
   float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
   if (gs == 0 && in) {                          // independent of earlier kernels' partials
     if (b_down && !accumulate) {
-      const __half2* b = reinterpret_cast<const __half2*>(b_down) + col4 * 2;
+      const __half2* b = reinterpret_cast<const __half2*>(b_down + (col4 * 4) % b_period);
       const float2 lo = __half22float2(b[0]), hi = __half22float2(b[1]);
       t = make_float4(lo.x, lo.y, hi.x, hi.y);
     }
@@ -327,7 +327,7 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
     if (ev && s == D.n_streams - 1) tm_record(ev[8], st);
     e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st, L->use_pdl,
                  (const float*)L->y_partial, n, (const float*)nullptr, (const int32_t*)nullptr,
-                 L->ffn_grid, (const __half*)D.dev_bias_down, y + (size_t)s * d, d,
+                 L->ffn_grid, (const __half*)D.dev_bias_down, d, y + (size_t)s * d, d,
                  accumulate ? 1 : 0);
     if (e != cudaSuccess) return e;
   }
@@ -355,12 +355,20 @@ cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cuda
     case LIF_KERNEL_FFN_SUM:
       return launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st,
                       L->use_pdl, (const float*)p0, cnt + LIF_CNT_N_HITS, (const float*)p1,
-                      cnt + LIF_CNT_N_LOAD, L->ffn_grid, (const __half*)D.dev_bias_down, y, d, 0);
+                      cnt + LIF_CNT_N_LOAD, L->ffn_grid, (const __half*)D.dev_bias_down, d, y, d, 0);
     default:
       return cudaErrorInvalidValue;
   }
   return launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
                   L->use_pdl, a);
+}
+
+cudaError_t launch_partial_sum(lif_layer* L, const float* partial, const int32_t* n,
+                               int partitions, int width, float* y, cudaStream_t st) {
+  return launch_k(ffn_reduce_kernel, dim3((width / 4 + kSumCols - 1) / kSumCols),
+                  dim3(kSumThreads), 0, st, L->use_pdl, partial, n, (const float*)nullptr,
+                  (const int32_t*)nullptr, partitions, (const __half*)L->desc.dev_bias_down,
+                  L->desc.d_model, y, width, 0);
 }
 
 // FFN of a decode step in two parts: the rows that were already cached (they can run while
@@ -393,7 +401,7 @@ cudaError_t launch_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream
     if (ev && last) tm_record(ev[8], st);
     e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st, L->use_pdl,
                  (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,
-                 (const __half*)D.dev_bias_down, y + (size_t)s * d, d, 0);
+                 (const __half*)D.dev_bias_down, d, y + (size_t)s * d, d, 0);
     if (e != cudaSuccess) return e;
   }
   if (ev) tm_record(ev[9], st);
@@ -494,6 +502,6 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
   if (cudaGetLastError() != cudaSuccess) return LIF_ERR_CUDA;
   ffn_reduce_kernel<<<(d_model / 4 + kSumCols - 1) / kSumCols, kSumThreads, 0, st>>>(
       sd.scratch->partial, dev_n_slots, nullptr, nullptr, grid, (const __half*)dev_bias_down,
-      dev_y, d_model, 0);
+      d_model, dev_y, d_model, 0);
   return cudaGetLastError() == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
 }

@@ -4,13 +4,15 @@
 //   Y[s][m] = b_down[m] + sum_q H[q][s] * M[slot_q, d + m]       (down halves, K = rows)
 // so it runs on tensor cores (mma.sync m16n8k16, fp16 operands, fp32 accumulate) while every
 // bundle half is still read from HBM exactly once:
-//   phase A: CTAs own rows; the up halves stream through a ring of shared-memory stages (one
-//            bulk copy per half row), x (S x d, fp16) stays in shared memory as the A operand,
-//            the rows are the B operand; the 8 warps split K and fold through shared memory.
+//   phase A: CTAs own (row partition, K slice); that slice of the up halves streams through a
+//            ring of shared-memory stages (one bulk copy per row), 16 rows per MMA as the A
+//            operand; the same slice of x (S x d, fp16) stays in shared memory as the B operand;
+//            the 8 warps split the slice and fold through shared memory.  Output: partial
+//            pre-activations per K slice (slice 0 carries the bias).
 //   phase B: CTAs own (row partition, column part); the down halves of the part stream through
-//            the ring, 16 rows per MMA k-step; H (split into fp16 high + low parts, so the
-//            product keeps fp32 accuracy) is the B operand; each warp keeps its column tiles'
-//            accumulators in registers for the whole kernel.
+//            the ring, 16 rows per MMA k-step; H = relu(sum of the K-slice partials), split into
+//            fp16 high + low parts (so the product keeps fp32 accuracy), is the B operand; each
+//            warp keeps its column tiles' accumulators in registers for the whole kernel.
 // Partition partials are added in a fixed order by the partial-sum kernel.  Bound: HBM.
 #include "lif_internal.cuh"
 
@@ -19,7 +21,7 @@ namespace {
 
 constexpr int kPad = 16;                  // bytes added to every shared row: conflict-free ldmatrix
 constexpr unsigned kWaitLimitB = 1u << 22;
-constexpr int kGroupA = 4;                // rows per MMA in phase A (N = 8, half used)
+constexpr int kGroupA = 16;               // rows per MMA in phase A (M = 16)
 constexpr int kMaxTilesPerWarp = 28;      // 16-column tiles per warp in phase B
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -61,6 +63,11 @@ __device__ __forceinline__ void mma16816(float* c, const uint32_t* a, uint32_t b
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t* r, const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(smem_u32(p)));
+}
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, const void* p) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -74,31 +81,35 @@ struct BatchedArgs {
   const int32_t* slots;   // or nullptr: rows base .. base + n
   const int32_t* n;
   const int32_t* base;
-  float* H;               // [n][8] fp32, position-indexed
+  float* H;               // [ksplit][h_stride] fp32; entry [q][8], position-indexed
   float* y_partial;       // [partitions][S][d]
   int32_t* status;
   int d, S, stages, parts, partitions, cols_per_part;
+  int ksplit, k_per_split, up_partitions;   // phase A: K slices (columns, multiple of 16)
+  size_t h_stride;
 };
 
 __device__ __forceinline__ int row_slot(const BatchedArgs& a, int q, int base) {
   return a.slots ? a.slots[q] : base + q;
 }
 
-// ---- phase A: H = relu(Up . X^T + bias) ------------------------------------------------------
+// ---- phase A: partial pre-activations  Hp[slice][q][s] = <Up[q, slice], x[s, slice]> (+ bias) --
 __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int d = a.d;
-  const unsigned half_bytes = 2u * d;
-  const unsigned pitch = half_bytes + kPad;
-  const int stages = a.stages;               // multiple of kGroupA, two groups or more
+  const int ks = blockIdx.x % a.ksplit, prt = blockIdx.x / a.ksplit;
+  const int k0 = ks * a.k_per_split;                    // first column of this K slice
+  const int kcols = min(a.k_per_split, d - k0);
+  const unsigned seg_bytes = 2u * kcols;
+  const unsigned pitch = 2u * a.k_per_split + kPad;
+  const int stages = a.stages;                          // multiple of kGroupA, two groups or more
   unsigned char* xs = smem;                                  // [8][pitch]
   unsigned char* rows = xs + 8 * (size_t)pitch;              // [stages][pitch]
   uint64_t* bars = reinterpret_cast<uint64_t*>(rows + (size_t)stages * pitch);
   float* bias_s = reinterpret_cast<float*>(bars + stages);   // [stages]
-  float* red = bias_s + stages;                              // [8 warps][32 lanes][2]
+  float* red = bias_s + stages;                              // [8 warps][32 lanes][4]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int G = gridDim.x, cta = blockIdx.x;
   if (tid == 0) {
     for (int i = 0; i < stages; ++i) mbar_init(bars + i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -107,34 +118,41 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
   pdl_wait();
   pdl_trigger();
   const int n = *a.n;
-  if (cta >= n) return;
+  if (prt >= n) return;
   const int base = a.base ? *a.base : 0;
-  const int my_cnt = (n - cta + G - 1) / G;   // rows q = cta + i * G
+  const int P = a.up_partitions;
+  const int my_cnt = (n - prt + P - 1) / P;             // rows q = prt + i * P
   __syncthreads();
 
-  // first copies in flight, then x into shared memory (streams beyond S are zero)
+  // first copies in flight, then the x slice into shared memory (streams beyond S are zero)
   if (tid < stages && tid < my_cnt) {
-    const int slot = row_slot(a, cta + tid * G, base);
-    mbar_expect_tx(bars + tid, half_bytes);
-    bulk_g2s(rows + (size_t)tid * pitch, a.cache + (size_t)slot * 2 * d, half_bytes, bars + tid);
-    bias_s[tid] = __half2float(a.bias[slot]);
+    const int slot = row_slot(a, prt + tid * P, base);
+    mbar_expect_tx(bars + tid, seg_bytes);
+    bulk_g2s(rows + (size_t)tid * pitch, a.cache + (size_t)slot * 2 * d + k0, seg_bytes,
+             bars + tid);
+    bias_s[tid] = ks == 0 ? __half2float(a.bias[slot]) : 0.f;
   }
   {
-    const int vec = d >> 3;
+    const int vec = kcols >> 3;
     for (int i = tid; i < 8 * vec; i += kThreads) {
       const int s = i / vec, c = i % vec;
       uint4 v = make_uint4(0, 0, 0, 0);
-      if (s < a.S) v = reinterpret_cast<const uint4*>(a.x + (size_t)s * d)[c];
+      if (s < a.S) v = reinterpret_cast<const uint4*>(a.x + (size_t)s * d + k0)[c];
       *reinterpret_cast<uint4*>(xs + (size_t)s * pitch + (size_t)c * 16) = v;
     }
   }
   __syncthreads();
 
-  const int ksteps = d >> 4;
+  const int ksteps = kcols >> 4;
   const int kper = (ksteps + 7) >> 3;
   const int k_begin = warp * kper, k_end = min(ksteps, k_begin + kper);
-  const int gq = lane >> 2, tq = lane & 3;          // fragment coordinates
-  const unsigned char* xa = xs + (size_t)gq * pitch + tq * 4;           // A: stream gq
+  const int gq = lane >> 2, tq = lane & 3;              // fragment coordinates
+  const unsigned char* xb = xs + (size_t)gq * pitch + tq * 4;            // B: stream gq
+  // A (16 rows x 16 columns): lane supplies row (lane % 8) + 8 * (lane / 8 % 2), columns
+  // 8 * (lane / 16) of the k-step
+  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+  const int a_off = (lane >> 4) * 16;
+  float* Hp = a.H + (size_t)ks * a.h_stride;
   int timed_out = 0;
   const int n_groups = (my_cnt + kGroupA - 1) / kGroupA;
   const int groups_in_ring = stages / kGroupA;
@@ -144,27 +162,19 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
     const int valid = min(kGroupA, my_cnt - g * kGroupA);
     for (int i = 0; i < valid; ++i)
       if (!mbar_wait(bars + st0 + i, parity)) timed_out = 1;
-    // D[stream][row] over this warp's K slice; B column = row gq of the group (gq < 4)
+    // D[row][stream] over this warp's part of the slice
     float c[4] = {0.f, 0.f, 0.f, 0.f};
-    const unsigned char* rb = rows + (size_t)(st0 + (gq & 3)) * pitch + tq * 4;
-    const bool brow = gq < kGroupA;
+    const unsigned char* ab = rows + (size_t)(st0 + a_row) * pitch + a_off;
 #pragma unroll 4
     for (int k = k_begin; k < k_end; ++k) {
       uint32_t af[4];
-      af[0] = *reinterpret_cast<const uint32_t*>(xa + k * 32);
-      af[1] = 0u;
-      af[2] = *reinterpret_cast<const uint32_t*>(xa + k * 32 + 16);
-      af[3] = 0u;
-      uint32_t b0 = 0u, b1 = 0u;
-      if (brow) {
-        b0 = *reinterpret_cast<const uint32_t*>(rb + k * 32);
-        b1 = *reinterpret_cast<const uint32_t*>(rb + k * 32 + 16);
-      }
+      ldmatrix_x4(af, ab + k * 32);
+      const uint32_t b0 = *reinterpret_cast<const uint32_t*>(xb + k * 32);
+      const uint32_t b1 = *reinterpret_cast<const uint32_t*>(xb + k * 32 + 16);
       mma16816(c, af, b0, b1);
     }
-    // c[0], c[1] = (stream gq, rows 2*tq, 2*tq + 1); fold the 8 warps
-    red[(warp * 32 + lane) * 2] = c[0];
-    red[(warp * 32 + lane) * 2 + 1] = c[1];
+    // c[0], c[1] = (row gq, streams 2*tq, 2*tq + 1); c[2], c[3] = row gq + 8; fold the 8 warps
+    *reinterpret_cast<float4*>(red + (warp * 32 + lane) * 4) = make_float4(c[0], c[1], c[2], c[3]);
     if (__syncthreads_or(timed_out)) {
       if (tid == 0) {
         atomicCAS(a.status, LIF_OK, LIF_ERR_TIMEOUT);
@@ -174,27 +184,26 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
       return;
     }
     if (tid < 8 * kGroupA) {
-      const int s = tid >> 2, r = tid & 3;          // stream, row in group
+      const int r = tid >> 3, s = tid & 7;              // row in group, stream
       if (r < valid) {
-        const int src_lane = s * 4 + (r >> 1);
+        const int src = ((r & 7) * 4 + (s >> 1)) * 4 + (r >> 3) * 2 + (s & 1);
         float v = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) v += red[(w * 32 + src_lane) * 2 + (r & 1)];
-        v = fmaxf(v + bias_s[st0 + r], 0.f);
-        const int q = cta + (g * kGroupA + r) * G;
-        a.H[(size_t)q * 8 + s] = v;
+        for (int w = 0; w < 8; ++w) v += red[w * 128 + src];
+        const int q = prt + (g * kGroupA + r) * P;
+        Hp[(size_t)q * 8 + s] = v + bias_s[st0 + r];
       }
     }
-    __syncthreads();                                 // stages st0.. and bias_s are free
+    __syncthreads();                                    // stages st0.. , bias_s and red are free
     // refill with the rows of group g + groups_in_ring
     if (tid < kGroupA) {
       const int i = (g + groups_in_ring) * kGroupA + tid;
       if (i < my_cnt) {
-        const int slot = row_slot(a, cta + i * G, base);
-        mbar_expect_tx(bars + st0 + tid, half_bytes);
-        bulk_g2s(rows + (size_t)(st0 + tid) * pitch, a.cache + (size_t)slot * 2 * d, half_bytes,
-                 bars + st0 + tid);
-        bias_s[st0 + tid] = __half2float(a.bias[slot]);
+        const int slot = row_slot(a, prt + i * P, base);
+        mbar_expect_tx(bars + st0 + tid, seg_bytes);
+        bulk_g2s(rows + (size_t)(st0 + tid) * pitch, a.cache + (size_t)slot * 2 * d + k0,
+                 seg_bytes, bars + st0 + tid);
+        bias_s[st0 + tid] = ks == 0 ? __half2float(a.bias[slot]) : 0.f;
       }
     }
   }
@@ -249,8 +258,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
 
   // H of the next group, prefetched: thread (k = tid / 8, s = tid % 8) for tid < 128
   const int hk = tid >> 3, hs = tid & 7;
+  auto load_h = [&](int i) {                       // relu(sum of the K-slice partials)
+    float v = 0.f;
+    const size_t at = (size_t)(prt + i * P) * 8 + hs;
+    for (int ks = 0; ks < a.ksplit; ++ks) v += a.H[(size_t)ks * a.h_stride + at];
+    return fmaxf(v, 0.f);
+  };
   float h_next = 0.f;
-  if (tid < 128 && hk < my_cnt) h_next = a.H[(size_t)(prt + hk * P) * 8 + hs];
+  if (tid < 128 && hk < my_cnt) h_next = load_h(hk);
 
   int timed_out = 0;
   const int n_groups = (my_cnt + 15) >> 4;
@@ -265,7 +280,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
       h_hi[hs * 16 + hk] = hi;
       h_lo[hs * 16 + hk] = __float2half_rn(h - __half2float(hi));
       const int i = (g + 1) * 16 + hk;
-      h_next = i < my_cnt ? a.H[(size_t)(prt + i * P) * 8 + hs] : 0.f;
+      h_next = i < my_cnt ? load_h(i) : 0.f;
     }
     for (int i = 0; i < valid; ++i)
       if (!mbar_wait(bars + st0 + i, parity)) timed_out = 1;
@@ -322,33 +337,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   }
 }
 
-// y[s][m] = b_down[m] + sum_p y_partial[p][s][m], p ascending
-__global__ void __launch_bounds__(kThreads)
-ffn_batched_sum_kernel(const float* __restrict__ y_partial, int partitions,
-                       const __half* __restrict__ b_down, float* __restrict__ y, int d, int S) {
-  pdl_wait();
-  pdl_trigger();
-  const size_t total4 = (size_t)S * d / 4;
-  const size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x;
-  if (i >= total4) return;
-  const int m = (int)((i * 4) % d);
-  float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (b_down) {
-    const __half2* b = reinterpret_cast<const __half2*>(b_down + m);
-    const float2 lo = __half22float2(b[0]), hi = __half22float2(b[1]);
-    t = make_float4(lo.x, lo.y, hi.x, hi.y);
-  }
-#pragma unroll 8
-  for (int p = 0; p < partitions; ++p) {
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(y_partial + (size_t)p * S * d) + i);
-    t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
-  }
-  reinterpret_cast<float4*>(y)[i] = t;
-}
-
-size_t up_smem(int d, int stages) {
-  const size_t pitch = 2 * (size_t)d + kPad;
-  return (8 + stages) * pitch + stages * 8 + stages * 4 + 8 * 32 * 2 * 4 + 16;
+size_t up_smem(int k_per_split, int stages) {
+  const size_t pitch = 2 * (size_t)k_per_split + kPad;
+  return (8 + stages) * pitch + stages * 8 + stages * 4 + 8 * 32 * 4 * 4 + 16;
 }
 size_t down_smem(int cols_per_part, int stages) {
   return stages * (2 * (size_t)cols_per_part + kPad) + stages * 8 + 2 * 128 * 2 + 16;
@@ -368,16 +359,27 @@ cudaError_t ffn_batched_configure(lif_layer* L) {
   e = cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
   const int d = D.d_model;
-  int st = 16;                                     // phase A: multiple of kGroupA, >= 2 groups
-  while (st > 2 * kGroupA && up_smem(d, st) > (size_t)max_smem) st -= kGroupA;
-  if (up_smem(d, st) > (size_t)max_smem) return cudaSuccess;   // fall back to the per-stream path
   const int tiles = d / 16;
-  int parts = 1;
+  // phase A: split K over 1, 2, 4 or 8 CTAs until three 16-row groups fit beside the x slice
+  int ksplit = 1, kps = d, st = 0;
+  bool found = false;
+  for (int want = 3 * kGroupA; want >= 2 * kGroupA && !found; want -= kGroupA)
+    for (ksplit = 1; ksplit <= kBatchedMaxKSplit && !found; ksplit *= 2) {
+      kps = (tiles + ksplit - 1) / ksplit * 16;
+      st = want;
+      found = up_smem(kps, st) <= (size_t)max_smem;
+      if (found) break;
+    }
+  if (!found) return cudaSuccess;                  // fall back to the per-stream path
+  int parts = L->fb_parts_min > 0 ? L->fb_parts_min : 1;
   while ((tiles + parts - 1) / parts > 8 * kMaxTilesPerWarp ||
          down_smem((tiles + parts - 1) / parts * 16, 32) > (size_t)max_smem)
     ++parts;
+  L->fb_ksplit = ksplit;
+  L->fb_kps = kps;
+  L->fb_up_partitions = L->n_sm / ksplit > 0 ? L->n_sm / ksplit : 1;
   L->fb_up_stages = st;
-  L->fb_up_smem = up_smem(d, st);
+  L->fb_up_smem = up_smem(kps, st);
   L->fb_parts = parts;
   L->fb_cols = (tiles + parts - 1) / parts * 16;
   L->fb_partitions = L->n_sm / parts > 0 ? L->n_sm / parts : 1;
@@ -411,18 +413,19 @@ cudaError_t launch_ffn_batched(lif_layer* L, const __half* x, const int32_t* slo
   a.parts = L->fb_parts;
   a.partitions = L->fb_partitions;
   a.cols_per_part = L->fb_cols;
+  a.ksplit = L->fb_ksplit;
+  a.k_per_split = L->fb_kps;
+  a.up_partitions = L->fb_up_partitions;
+  a.h_stride = (size_t)D.d_ff * 8;
   a.stages = L->fb_up_stages;
-  cudaError_t e = launch_k(ffn_batched_up_kernel, dim3(L->n_sm), dim3(kThreads), L->fb_up_smem, st,
-                           L->use_pdl, a);
+  cudaError_t e = launch_k(ffn_batched_up_kernel, dim3(L->fb_up_partitions * L->fb_ksplit),
+                           dim3(kThreads), L->fb_up_smem, st, L->use_pdl, a);
   if (e != cudaSuccess) return e;
   a.stages = 32;
   e = launch_k(ffn_batched_down_kernel, dim3(L->fb_parts * L->fb_partitions), dim3(kThreads),
                L->fb_down_smem, st, L->use_pdl, a);
   if (e != cudaSuccess) return e;
-  const size_t total4 = (size_t)D.n_streams * D.d_model / 4;
-  return launch_k(ffn_batched_sum_kernel, dim3((unsigned)((total4 + kThreads - 1) / kThreads)),
-                  dim3(kThreads), 0, st, L->use_pdl, (const float*)L->y_partial, L->fb_partitions,
-                  (const __half*)D.dev_bias_down, y, D.d_model, D.n_streams);
+  return launch_partial_sum(L, L->y_partial, n, L->fb_partitions, D.n_streams * D.d_model, y, st);
 }
 
 }  // namespace lif

@@ -53,9 +53,10 @@ struct lif_layer {
   float* z_partial;
   uint32_t* mask_words;
   float* y_partial;
-  float* h_rows;      // [d_ff][8] fp32: phase-A output of the multi-stream FFN
+  float* h_rows;      // [K slices][d_ff][8] fp32: phase-A output of the multi-stream FFN
   // multi-stream (tensor-core) FFN configuration; fb_ok = 0: per-stream fallback
   int fb_ok, fb_up_stages, fb_parts, fb_cols, fb_partitions;
+  int fb_ksplit, fb_kps, fb_up_partitions, fb_parts_min;
   size_t fb_up_smem, fb_down_smem;
   int n_sm;
   int z_ctas;         // CTAs of the first predictor stage
@@ -112,6 +113,10 @@ cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cuda
 cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaStream_t st);
 cudaError_t ffn_configure(lif_layer* L);
 constexpr int kBatchedMaxPartitions = 128;
+constexpr int kBatchedMaxKSplit = 8;
+// y[i] = b_down[i % d_model] + sum_{p < min(partitions, *n)} partial[p][i], i < width
+cudaError_t launch_partial_sum(lif_layer* L, const float* partial, const int32_t* n,
+                               int partitions, int width, float* y, cudaStream_t st);
 bool ffn_batched_supported(const lif_layer_desc& D);
 cudaError_t ffn_batched_configure(lif_layer* L);
 cudaError_t launch_ffn_batched(lif_layer* L, const __half* x, const int32_t* slots,
