@@ -276,6 +276,44 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_kernel_loop(args):
+    """For profilers: W warm-up tokens through the graph, then ONE plain launch of the chosen
+    kernel on every layer's lists (layer 0 first).  Prints the rows each launch processes, so a
+    captured launch can be related to its algorithmic bytes."""
+    import torch
+    from paper_2312_11514_b200 import binding as B
+    from paper_2312_11514_b200 import runtime as R
+    from paper_2312_11514_b200 import workloads as W
+    dev = "cuda:0"
+    cfg = W.CONFIGS[args.config]
+    layers = R.build_stack(cfg, dev, n_layers=args.layers)
+    handles = [l.handle for l in layers]
+    L, S, d = len(layers), cfg.n_streams, cfg.d_model
+    X = _inputs(cfg, args.warmup, dev, W)
+    Y = torch.empty(L, S, d, dtype=torch.float32, device=dev)
+    dev_x = torch.empty(S, d, dtype=torch.float16, device=dev)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    graph = B.lif_graph_capture(handles, dev_x, Y, sc, sf)
+    for t in range(args.warmup):
+        with torch.cuda.stream(sc):
+            dev_x.copy_(X[t], non_blocking=True)
+        B.lif_graph_launch(graph, sc)
+    torch.cuda.synchronize()
+    kind = B.KERNELS.index(args.kernel_loop)
+    cnt = {"ffn_active": B.CNT_N_ACTIVE, "ffn_hits": B.CNT_N_HITS, "ffn_new": B.CNT_N_LOAD,
+           "fetch": B.CNT_N_LOAD}.get(args.kernel_loop)
+    rows = [int(l.counts[cnt]) for l in layers] if cnt is not None else None
+    for l in range(L):
+        B.lif_profile_launch(handles[l], kind, dev_x, Y[l], sc)
+    torch.cuda.synchronize()
+    print(json.dumps({"kernel": args.kernel_loop, "layers": L, "warmup_tokens": args.warmup,
+                      "rows_per_launch": rows, "bundle_bytes": cfg.bundle_bytes}), flush=True)
+    B.lif_graph_destroy(graph)
+    for l in layers:
+        l.close()
+
+
 # ------------------------------------------------------------------------------ CPU oracle
 def _oracle_threads():
     try:
@@ -387,10 +425,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--cpu-layers", type=int, default=2)
     ap.add_argument("--cpu-tokens", type=int, default=30)
+    ap.add_argument("--kernel-loop", default=None,
+                    help="profiling aid: after the warm-up tokens launch this kernel once per layer "
+                         "(predict_z, predict_scores, fetch, ffn_active, ffn_hits, ffn_new, ffn_sum)")
     args = ap.parse_args()
     if args.warmup < 3:
         raise SystemExit("--warmup must be at least 3")
-    if args.impl == "reference":
+    if args.kernel_loop:
+        run_kernel_loop(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         if int(os.environ.get("WORLD_SIZE", 1)) > 1:
