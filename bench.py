@@ -28,6 +28,9 @@ if ROOT not in sys.path:
 METRIC = "ffn_stack_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes of sparse_ffn_kernel, from
+# the ncu capture summarised under profiles/ (set to None when that kernel changes)
+FFN_TRAFFIC_RATIO = 1.005
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -251,7 +254,11 @@ def run_ours(args):
             "roofline": {"kernel": "sparse_ffn_kernel", "bound": "hbm",
                          "achieved": ffn_gbs, "peak": peak, "unit": "GB/s", "frac": ffn_gbs / peak,
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": ffn_gbs / NOMINAL_HBM_GBS,
-                         "traffic": None, "us_per_launch": kernel_us["ffn_active"],
+                         "traffic": FFN_TRAFFIC_RATIO * ffn_bytes if FFN_TRAFFIC_RATIO else None,
+                         "traffic_how": "dram read+write bytes per algorithmic byte from the ncu capture in "
+                                        "profiles/sparse_ffn_kernel_opt6p7b_12layers.md (12 layers, "
+                                        "451-529 rows per launch), scaled by this run's rows per launch",
+                         "us_per_launch": kernel_us["ffn_active"],
                          "bytes_per_launch": ffn_bytes,
                          "how": "graph of this kernel on all layers' active rows of the last token, "
                                 f"{reps} replays, CUDA events",
