@@ -199,9 +199,12 @@ lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* dev_bias, c
                                  const void* dev_bias_down, float* dev_y, int32_t d_model,
                                  void* stream);
 
-/* One token through the layer: predict -> window update -> fetch (on fetch_stream, ordered by
- * events) -> sparse FFN (ffn_mode selects the rows).  The compute stream ends up ordered
- * after the fetch, so consecutive calls on the same streams are safe. */
+/* One token through the layer: predict -> window update -> fetch -> sparse FFN (ffn_mode
+ * selects the rows).  Two streams let the bundle fetch overlap the part of the FFN that does
+ * not need the new rows; which of the two kernels runs on `fetch_stream` is the library's
+ * choice (ordering is by events inside the call).  The compute stream ends up ordered after
+ * everything, so consecutive calls on the same streams are safe.  Passing the same stream
+ * twice runs the step serially. */
 lif_status lif_decode_step(lif_layer* layer, const void* dev_x, float* dev_y,
                            void* compute_stream, void* fetch_stream);
 

@@ -286,6 +286,11 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   if (ev) tm_record(ev[0], sc);
   bool ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
   ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
+  if (L->split_ffn && L->desc.n_streams == 1) {
+    ok = ok && launch_fetch_and_ffn_split(L, x, dev_y, sc, sf, ev) == cudaSuccess;
+    if (!ok) cudaGetLastError();
+    return ok ? LIF_OK : LIF_ERR_CUDA;
+  }
   if (sf != sc) {
     ok = ok && cudaEventRecord(L->ev_plan, sc) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(sf, L->ev_plan, 0) == cudaSuccess;
@@ -293,13 +298,10 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   if (ev) tm_record(ev[5], sf);
   ok = ok && launch_fetch(L, sf) == cudaSuccess;
   if (ev) tm_record(ev[6], sf);
-  if (sf != sc) ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
-  if (L->split_ffn && !L->fb_ok) {
-    ok = ok && launch_ffn_split(L, x, dev_y, sc, sf, ev) == cudaSuccess;
-    if (!ok) cudaGetLastError();
-    return ok ? LIF_OK : LIF_ERR_CUDA;
+  if (sf != sc) {
+    ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(sc, L->ev_fetch, 0) == cudaSuccess;
   }
-  if (sf != sc) ok = ok && cudaStreamWaitEvent(sc, L->ev_fetch, 0) == cudaSuccess;
   if (L->desc.ffn_mode == 0)
     ok = ok && launch_ffn(L, x, L->active_slots, L->counts + LIF_CNT_N_ACTIVE, nullptr, dev_y,
                           false, sc, ev) == cudaSuccess;

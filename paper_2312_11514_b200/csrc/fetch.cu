@@ -53,6 +53,8 @@ __global__ void __launch_bounds__(kThreads)
 fetch_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
              const int32_t* __restrict__ load_ids, const int32_t* __restrict__ load_slots,
              const int32_t* __restrict__ counts, int row_vec) {
+  pdl_wait();
+  pdl_trigger();
   gather_rows(store, cache, load_ids, load_slots, counts[LIF_CNT_N_LOAD], row_vec);
 }
 
@@ -65,10 +67,10 @@ probe_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n_chunk
 }  // namespace
 
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st) {
-  fetch_kernel<<<L->fetch_grid, kThreads, 0, st>>>(
-      (const uint4*)L->dev_bundles, (uint4*)L->desc.dev_cache, L->load_ids, L->load_slots,
-      L->counts, L->desc.d_model / 4);
-  return cudaGetLastError();
+  return launch_k(fetch_kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl,
+                  (const uint4*)L->dev_bundles, (uint4*)L->desc.dev_cache,
+                  (const int32_t*)L->load_ids, (const int32_t*)L->load_slots,
+                  (const int32_t*)L->counts, L->desc.d_model / 4);
 }
 
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,

@@ -371,41 +371,45 @@ cudaError_t launch_partial_sum(lif_layer* L, const float* partial, const int32_t
                   L->desc.d_model, y, width, 0);
 }
 
-// FFN of a decode step in two parts: the rows that were already cached (they can run while
-// the fetch is still copying), then, after `ev_fetch`, the rows just brought in; one sum.
-cudaError_t launch_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream_t st,
-                             cudaStream_t fetch_st, cudaEvent_t* ev) {
+// Fetch + FFN of a single-stream decode step.  The critical chain stays on `st` with dependent
+// launches: fetch -> FFN over the rows just brought in -> sum.  The FFN over the rows that
+// were already cached does not depend on the fetch and runs on `side` meanwhile (forked after
+// the row moves, joined before the sum).
+cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream_t st,
+                                       cudaStream_t side, cudaEvent_t* ev) {
   const lif_layer_desc& D = L->desc;
   const int d = D.d_model;
   const int32_t* cnt = L->counts;
   float* p0 = L->y_partial;
   float* p1 = L->y_partial + (size_t)L->ffn_grid * d;
-  if (ev) tm_record(ev[7], st);
-  for (int s = 0; s < D.n_streams; ++s) {
-    const __half* xs = x + (size_t)s * d;
-    const bool last = s == D.n_streams - 1;
-    FfnArgs hit = D.ffn_mode == 0
-                      ? ffn_args(L, xs, L->hit_slots, cnt + LIF_CNT_N_HITS, nullptr, p0, D.d_ff)
-                      : ffn_args(L, xs, nullptr, cnt + LIF_CNT_NUM_KEPT, nullptr, p0, 0);
-    cudaError_t e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem,
-                             st, L->use_pdl, hit);
-    if (e != cudaSuccess) return e;
-    if (s == 0 && fetch_st != st) {
-      e = cudaStreamWaitEvent(st, L->ev_fetch, 0);
-      if (e != cudaSuccess) return e;
-    }
-    FfnArgs miss = ffn_args(L, xs, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
-    e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
-                 L->use_pdl, miss);
-    if (e != cudaSuccess) return e;
-    if (ev && last) tm_record(ev[8], st);
-    e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st, L->use_pdl,
-                 (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,
-                 (const __half*)D.dev_bias_down, d, y + (size_t)s * d, d, 0);
-    if (e != cudaSuccess) return e;
+  const bool fork = side != st;
+  cudaError_t e;
+  if (fork) {
+    if ((e = cudaEventRecord(L->ev_plan, st)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(side, L->ev_plan, 0)) != cudaSuccess) return e;
   }
+  FfnArgs hit = D.ffn_mode == 0
+                    ? ffn_args(L, x, L->hit_slots, cnt + LIF_CNT_N_HITS, nullptr, p0, D.d_ff)
+                    : ffn_args(L, x, nullptr, cnt + LIF_CNT_NUM_KEPT, nullptr, p0, 0);
+  if (ev) tm_record(ev[7], side);
+  e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, side,
+               fork ? 0 : L->use_pdl, hit);
+  if (e != cudaSuccess) return e;
+  if (ev) tm_record(ev[8], side);
+  if (fork && (e = cudaEventRecord(L->ev_fetch, side)) != cudaSuccess) return e;
+  if (ev) tm_record(ev[5], st);
+  if ((e = launch_fetch(L, st)) != cudaSuccess) return e;
+  if (ev) tm_record(ev[6], st);
+  FfnArgs miss = ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
+  e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st, L->use_pdl,
+               miss);
+  if (e != cudaSuccess) return e;
+  if (fork && (e = cudaStreamWaitEvent(st, L->ev_fetch, 0)) != cudaSuccess) return e;
+  e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0,
+               st, L->use_pdl, (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,
+               (const __half*)D.dev_bias_down, d, y, d, 0);
   if (ev) tm_record(ev[9], st);
-  return cudaSuccess;
+  return e;
 }
 
 }  // namespace lif

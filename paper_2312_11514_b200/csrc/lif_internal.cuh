@@ -107,8 +107,8 @@ cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes,
 cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
                        const int32_t* base, float* y, bool accumulate, cudaStream_t st,
                        cudaEvent_t* ev = nullptr);
-cudaError_t launch_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream_t st,
-                             cudaStream_t fetch_st, cudaEvent_t* ev = nullptr);
+cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream_t st,
+                                       cudaStream_t side, cudaEvent_t* ev = nullptr);
 cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cudaStream_t st);
 cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaStream_t st);
 cudaError_t ffn_configure(lif_layer* L);
