@@ -244,8 +244,10 @@ enum {
   LIF_TUNE_FFN_CTAS = 3,         /* (SM count) CTAs of the sparse-FFN kernel, 1..256 */
   LIF_TUNE_FFN_STAGES = 4,       /* (as many as fit, at most 16) bundles in flight per CTA;
                                     fewer stages let several CTAs share an SM */
-  LIF_TUNE_BATCHED_COLUMN_PARTS = 5 /* (fewest that fit) column parts of the multi-stream FFN's
+  LIF_TUNE_BATCHED_COLUMN_PARTS = 5, /* (fewest that fit) column parts of the multi-stream FFN's
                                     down-projection kernel, 1..16 */
+  LIF_TUNE_FUSED_PLAN = 6        /* (1 when d_ff <= 32768) lif_decode_step: the window update
+                                    reads the predictor's bit mask instead of its index list */
 };
 lif_status lif_set_tuning(lif_layer* layer, int32_t key, int32_t value);
 

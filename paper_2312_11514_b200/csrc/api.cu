@@ -150,6 +150,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
     L->move_grid = L->n_sm;
     L->use_pdl = 1;
     L->split_ffn = 1;
+    L->fused_plan = window_plan_supported(*desc) ? 1 : 0;
     ok = cudaEventCreateWithFlags(&L->ev_plan, cudaEventDisableTiming) == cudaSuccess;
     if (ok && cudaEventCreateWithFlags(&L->ev_fetch, cudaEventDisableTiming) != cudaSuccess) {
       cudaEventDestroy(L->ev_plan);
@@ -284,8 +285,14 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   if (L->tm_events && L->tm_cursor < L->tm_steps)
     ev = L->tm_events + (size_t)(L->tm_cursor++) * kTimingEvents;
   if (ev) tm_record(ev[0], sc);
-  bool ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
-  ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
+  bool ok;
+  if (L->fused_plan) {
+    ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev, 0) == cudaSuccess;
+    ok = ok && launch_window_plan(L, sc, ev) == cudaSuccess;
+  } else {
+    ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
+    ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
+  }
   if (L->split_ffn && L->desc.n_streams == 1) {
     ok = ok && launch_fetch_and_ffn_split(L, x, dev_y, sc, sf, ev) == cudaSuccess;
     if (!ok) cudaGetLastError();
@@ -434,6 +441,9 @@ lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
   switch (key) {
     case LIF_TUNE_DEPENDENT_LAUNCH: L->use_pdl = value != 0; return LIF_OK;
     case LIF_TUNE_SPLIT_FFN: L->split_ffn = value != 0; return LIF_OK;
+    case LIF_TUNE_FUSED_PLAN:
+      L->fused_plan = value != 0 && window_plan_supported(L->desc);
+      return LIF_OK;
     case LIF_TUNE_FETCH_CTAS:
       if (value < 1 || value > 4096) return LIF_ERR_INVALID_ARG;
       L->fetch_grid = value;

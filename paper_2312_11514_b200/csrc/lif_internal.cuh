@@ -68,6 +68,7 @@ struct lif_layer {
   int move_grid;
   int use_pdl;        // programmatic dependent launch along the compute stream
   int split_ffn;      // decode step: cached rows' FFN overlaps the fetch
+  int fused_plan;     // decode step: window update reads the predictor's bit mask directly
   cudaEvent_t ev_plan, ev_fetch;
   // optional per-kernel timing: kTimingEvents events per recorded step
   cudaEvent_t* tm_events;
@@ -97,7 +98,10 @@ cudaError_t launch_reset(lif_layer* L, cudaStream_t st);
 // `ev`: optional events of the current timed step (nullptr = no timing); each launcher
 // records the ones between and after its own kernels.
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
-                           int32_t* n_active, cudaStream_t st, cudaEvent_t* ev = nullptr);
+                           int32_t* n_active, cudaStream_t st, cudaEvent_t* ev = nullptr,
+                           int compact = 1);   // compact = 0: leave only the bit mask
+bool window_plan_supported(const lif_layer_desc& D);
+cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr);
 cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st,
                           cudaEvent_t* ev = nullptr);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);

@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(kThreads)
 predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* __restrict__ B,
                       const float* __restrict__ c, float theta, int r, int F,
                       float* __restrict__ logits, uint32_t* mask_words, int* ticket,
-                      int* __restrict__ active_idx, int* __restrict__ n_active) {
+                      int* __restrict__ active_idx, int* __restrict__ n_active, int compact) {
   extern __shared__ float zs[];                 // [S][r]
   __shared__ float red[16][kLogitTile];
   __shared__ int warp_sums[kThreads / 32];
@@ -210,6 +210,7 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
     if ((tid & 31) == 0) mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = m;
   }
 
+  if (!compact) return;     // the consumer reads the bit mask itself
   // last CTA to arrive compacts the whole mask
   __threadfence();
   __syncthreads();
@@ -244,7 +245,7 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
 
 template <int S>
 cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
-                             int32_t* n_active, cudaStream_t st, cudaEvent_t* ev) {
+                             int32_t* n_active, cudaStream_t st, cudaEvent_t* ev, int compact) {
   const lif_layer_desc& D = L->desc;
   cudaError_t e = launch_k(predict_z_kernel<S>, dim3(L->z_ctas), dim3(kThreads), 0, st, L->use_pdl,
                            x, (const __half*)D.dev_pred_A, D.d_model, D.rank,
@@ -261,7 +262,7 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
   e = launch_k(predict_logits_kernel<S>, dim3(grid), dim3(kThreads), smem, st, L->use_pdl,
                (const float*)L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c,
                D.threshold_logit, D.rank, D.d_ff, logits, L->mask_words,
-               (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active);
+               (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact);
   if (ev) tm_record(ev[2], st);
   return e;
 }
@@ -280,20 +281,20 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
                   (size_t)D.rank * sizeof(float), st, L->use_pdl, (const float*)L->z_partial,
                   L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit, D.rank,
                   D.d_ff, (float*)nullptr, L->mask_words, (int*)(L->counts + CNT_TICKET_PREDICT),
-                  (int*)L->active_idx, (int*)L->n_tmp);
+                  (int*)L->active_idx, (int*)L->n_tmp, 1);
 }
 
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
-                           int32_t* n_active, cudaStream_t st, cudaEvent_t* ev) {
+                           int32_t* n_active, cudaStream_t st, cudaEvent_t* ev, int compact) {
   switch (L->desc.n_streams) {
-    case 1: return launch_predict_s<1>(L, x, logits, active_idx, n_active, st, ev);
-    case 2: return launch_predict_s<2>(L, x, logits, active_idx, n_active, st, ev);
-    case 3: return launch_predict_s<3>(L, x, logits, active_idx, n_active, st, ev);
-    case 4: return launch_predict_s<4>(L, x, logits, active_idx, n_active, st, ev);
-    case 5: return launch_predict_s<5>(L, x, logits, active_idx, n_active, st, ev);
-    case 6: return launch_predict_s<6>(L, x, logits, active_idx, n_active, st, ev);
-    case 7: return launch_predict_s<7>(L, x, logits, active_idx, n_active, st, ev);
-    case 8: return launch_predict_s<8>(L, x, logits, active_idx, n_active, st, ev);
+    case 1: return launch_predict_s<1>(L, x, logits, active_idx, n_active, st, ev, compact);
+    case 2: return launch_predict_s<2>(L, x, logits, active_idx, n_active, st, ev, compact);
+    case 3: return launch_predict_s<3>(L, x, logits, active_idx, n_active, st, ev, compact);
+    case 4: return launch_predict_s<4>(L, x, logits, active_idx, n_active, st, ev, compact);
+    case 5: return launch_predict_s<5>(L, x, logits, active_idx, n_active, st, ev, compact);
+    case 6: return launch_predict_s<6>(L, x, logits, active_idx, n_active, st, ev, compact);
+    case 7: return launch_predict_s<7>(L, x, logits, active_idx, n_active, st, ev, compact);
+    case 8: return launch_predict_s<8>(L, x, logits, active_idx, n_active, st, ev, compact);
   }
   return cudaErrorInvalidValue;
 }

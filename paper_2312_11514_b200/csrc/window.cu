@@ -67,11 +67,9 @@ struct WindowArgs {
   unsigned long long bundle_bytes;
 };
 
-__global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArgs a) {
-  __shared__ Scan sc;
+// General path: any cache size, active list read from memory.
+__device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   const int tid = threadIdx.x;
-  pdl_wait();
-  pdl_trigger();
   const int n = a.counts[LIF_CNT_NUM_USED];
   const int t = a.counts[LIF_CNT_STEP];
   const int na = *a.n_act;
@@ -204,6 +202,206 @@ __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArg
   }
 }
 
+__global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArgs a) {
+  __shared__ Scan sc;
+  pdl_wait();
+  pdl_trigger();
+  window_update_generic(a, sc);
+}
+
+// Fast path of the decode step: consumes the predictor's bit mask directly (the predictor then
+// skips its own compaction) and keeps each thread's few slots and active neurons in registers,
+// so the whole update is three dependent memory round trips (mask + counters; slot_of /
+// pointers / biases; last_active of the cached neurons), three packed scans and the writes.
+// Needs: at most kWindowThreads mask words, num_used <= kPlanSlots * kWindowThreads, at most
+// kPlanBits active neurons per mask word.  Otherwise the CTA compacts the mask into the list
+// and runs the general path.
+constexpr int kPlanSlots = 4;
+constexpr int kPlanBits = 8;
+constexpr int kPlanMaxRows = kPlanSlots * kWindowThreads;
+
+__global__ void __launch_bounds__(kWindowThreads)
+window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nwords,
+                   int32_t* n_act_out) {
+  __shared__ Scan sc;
+  __shared__ uint32_t bits[kWindowThreads];
+  __shared__ int holes[kPlanMaxRows];
+  __shared__ int newslot[kPlanMaxRows];
+  const int tid = threadIdx.x;
+  pdl_wait();
+  pdl_trigger();
+  const int n = a.counts[LIF_CNT_NUM_USED];
+  const int t = a.counts[LIF_CNT_STEP];
+  const uint32_t w = tid < nwords ? mask_words[tid] : 0u;
+  const int cnt = __popc(w);
+  bits[tid] = w;
+  u64 tot;
+  const int q_base = field(block_scan(pack3(cnt, 0, 0), &tot, sc), 0);   // also publishes bits[]
+  const int na = field(tot, 0);
+  const int fast = __syncthreads_and(n <= kPlanMaxRows && cnt <= kPlanBits);
+  if (!fast) {
+    // compact the mask into the ascending list, then take the general path
+    uint32_t m = w;
+    for (int q = q_base; m; ++q, m &= m - 1) a.active_idx[q] = tid * 32 + __ffs(m) - 1;
+    if (tid == 0) *n_act_out = na;
+    __syncthreads();
+    WindowArgs g = a;
+    g.act = a.active_idx;
+    g.n_act = n_act_out;
+    window_update_generic(g, sc);
+    return;
+  }
+  const int stale_before = t - a.k;
+
+  // ---- round trip 2: by neuron id (mine: bits of w) and by slot (mine: a contiguous run) ----
+  int so[kPlanBits];
+  __half bu[kPlanBits];
+  {
+    uint32_t m = w;
+#pragma unroll
+    for (int i = 0; i < kPlanBits; ++i) {
+      so[i] = 0;
+      bu[i] = __half();
+      if (m) {
+        const int id = tid * 32 + __ffs(m) - 1;
+        m &= m - 1;
+        so[i] = a.slot_of[id];
+        bu[i] = a.bias_up[id];
+      }
+    }
+  }
+  const int seg = (n + kWindowThreads - 1) / kWindowThreads;   // <= kPlanSlots
+  const int s0 = min(n, tid * seg);
+  const int my_slots = min(n, s0 + seg) - s0;
+  int pid[kPlanSlots];
+  __half pb[kPlanSlots];
+#pragma unroll
+  for (int j = 0; j < kPlanSlots; ++j) {
+    pid[j] = 0;
+    pb[j] = __half();
+    if (j < my_slots) {
+      pid[j] = a.pointers[s0 + j];
+      pb[j] = a.bias[s0 + j];
+    }
+  }
+  // ---- round trip 3: is each of my cached neurons still inside the window? ------------------
+  unsigned evm = 0;   // bit j: slot s0 + j is deleted
+#pragma unroll
+  for (int j = 0; j < kPlanSlots; ++j)
+    if (j < my_slots) {
+      const int id = pid[j];
+      const bool active_now = (bits[id >> 5] >> (id & 31)) & 1u;
+      if (!active_now && a.last_active[id] <= stale_before) evm |= 1u << j;
+    }
+  int c_load = 0;
+#pragma unroll
+  for (int i = 0; i < kPlanBits; ++i) c_load += (i < cnt && so[i] < 0);
+  u64 pre = block_scan(pack3(c_load, __popc(evm), cnt - c_load), &tot, sc);
+  const int n_load = field(tot, 0), n_evict = field(tot, 1);
+  const int n_kept = n - n_evict;
+  int p_load = field(pre, 0), p_ev = field(pre, 1), p_hit = field(pre, 2);
+
+  if (n_kept + n_load > a.cap) {            // refuse before anything is changed
+    if (tid == 0) {
+      if (a.counts[LIF_CNT_STATUS] == LIF_OK) a.counts[LIF_CNT_STATUS] = LIF_ERR_CAPACITY;
+      a.counts[LIF_CNT_N_ACTIVE] = 0;
+      a.counts[LIF_CNT_N_EVICT] = 0;
+      a.counts[LIF_CNT_N_MOVES] = 0;
+      a.counts[LIF_CNT_N_LOAD] = 0;
+      a.counts[LIF_CNT_N_HITS] = 0;
+      a.counts[LIF_CNT_NUM_USED_BEFORE] = n;
+      a.counts[LIF_CNT_NUM_KEPT] = n;
+    }
+    return;
+  }
+  int c_hole = 0, c_surv = 0;
+#pragma unroll
+  for (int j = 0; j < kPlanSlots; ++j)
+    if (j < my_slots) {
+      const bool e = (evm >> j) & 1u;
+      c_hole += e && (s0 + j) < n_kept;
+      c_surv += !e && (s0 + j) >= n_kept;
+    }
+  pre = block_scan(pack3(c_hole, c_surv, 0), &tot, sc);
+  const int n_moves = field(tot, 0);          // == surviving tail rows
+  int p_hole = field(pre, 0), p_surv = field(pre, 1);
+
+  // ---- writes ---------------------------------------------------------------------------------
+  {
+    uint32_t m = w;
+    for (; m; m &= m - 1) a.last_active[tid * 32 + __ffs(m) - 1] = t;          // stamp
+  }
+#pragma unroll
+  for (int j = 0; j < kPlanSlots; ++j)
+    if (j < my_slots && ((evm >> j) & 1u)) {                                     // deleted rows
+      const int s = s0 + j;
+      a.evict_ids[p_ev++] = pid[j];
+      a.slot_of[pid[j]] = -1;
+      if (s < n_kept) holes[p_hole++] = s;
+    }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < kPlanSlots; ++j)
+    if (j < my_slots) {
+      const int s = s0 + j;
+      if (!((evm >> j) & 1u) && s >= n_kept) {         // surviving tail row: last one first
+        const int jm = n_moves - 1 - p_surv++;
+        const int dst = holes[jm];
+        a.move_src[jm] = s;
+        a.move_dst[jm] = dst;
+        a.pointers[dst] = pid[j];
+        a.slot_of[pid[j]] = dst;
+        a.bias[dst] = pb[j];
+        newslot[s - n_kept] = dst;
+      }
+      if (s >= n_kept + n_load) a.pointers[s] = -1;    // tail beyond the rows to be loaded
+    }
+  __syncthreads();
+  {
+    uint32_t m = w;
+    int q = q_base;
+#pragma unroll
+    for (int i = 0; i < kPlanBits; ++i)
+      if (i < cnt) {
+        const int id = tid * 32 + __ffs(m) - 1;
+        m &= m - 1;
+        int s = so[i];
+        if (s < 0) {                                     // bring in: rows num_kept, num_kept + 1, ...
+          s = n_kept + p_load;
+          a.load_ids[p_load] = id;
+          a.load_slots[p_load] = s;
+          ++p_load;
+          a.slot_of[id] = s;
+          a.pointers[s] = id;
+          a.bias[s] = bu[i];
+        } else {
+          if (s >= n_kept) s = newslot[s - n_kept];      // it was moved into a hole
+          a.hit_slots[p_hit++] = s;
+        }
+        a.active_slots[q] = s;
+        a.active_idx[q] = id;
+        ++q;
+      }
+  }
+  if (tid == 0) {
+    *n_act_out = na;
+    a.counts[LIF_CNT_N_ACTIVE] = na;
+    a.counts[LIF_CNT_N_EVICT] = n_evict;
+    a.counts[LIF_CNT_N_MOVES] = n_moves;
+    a.counts[LIF_CNT_N_LOAD] = n_load;
+    a.counts[LIF_CNT_N_HITS] = na - n_load;
+    a.counts[LIF_CNT_NUM_USED_BEFORE] = n;
+    a.counts[LIF_CNT_NUM_KEPT] = n_kept;
+    a.counts[LIF_CNT_NUM_USED] = n_kept + n_load;
+    a.counts[LIF_CNT_STEP] = t + 1;
+    unsigned long long* totals = reinterpret_cast<unsigned long long*>(a.counts + CNT_TOTALS);
+    totals[0] += (unsigned long long)n_load * a.bundle_bytes;
+    totals[1] += (unsigned long long)n_moves;
+    totals[2] += (unsigned long long)na;
+    totals[3] += (unsigned long long)(n_kept + n_load);
+  }
+}
+
 // Row moves of step D: cache row move_src[j] -> row move_dst[j].  Sources lie at or beyond
 // num_kept, destinations below it, so the copies never overlap.
 __global__ void __launch_bounds__(kThreads)
@@ -245,8 +443,7 @@ cudaError_t launch_reset(lif_layer* L, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act,
-                          cudaStream_t st, cudaEvent_t* ev) {
+static WindowArgs window_args(lif_layer* L, const int32_t* act, const int32_t* n_act) {
   const lif_layer_desc& D = L->desc;
   WindowArgs a;
   a.act = act;
@@ -270,14 +467,39 @@ cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act
   a.cap = D.capacity;
   a.k = D.window_k;
   a.bundle_bytes = 4ull * D.d_model;
-  cudaError_t e = launch_k(window_update_kernel, dim3(1), dim3(kWindowThreads), 0, st, L->use_pdl, a);
-  if (e != cudaSuccess) return e;
+  return a;
+}
+
+static cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev) {
+  const lif_layer_desc& D = L->desc;
+  cudaError_t e;
   if (ev) tm_record(ev[3], st);
   e = launch_k(move_rows_kernel, dim3(L->move_grid), dim3(kThreads), 0, st, L->use_pdl,
                (uint4*)D.dev_cache, (const int32_t*)L->move_src, (const int32_t*)L->move_dst,
                (const int32_t*)L->counts, D.d_model / 4);
   if (ev) tm_record(ev[4], st);
   return e;
+}
+
+cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act,
+                          cudaStream_t st, cudaEvent_t* ev) {
+  cudaError_t e = launch_k(window_update_kernel, dim3(1), dim3(kWindowThreads), 0, st, L->use_pdl,
+                           window_args(L, act, n_act));
+  return e != cudaSuccess ? e : launch_moves(L, st, ev);
+}
+
+bool window_plan_supported(const lif_layer_desc& D) {
+  return (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32) <= kWindowThreads;
+}
+
+// Window update straight from the predictor's bit mask (see window_plan_kernel).
+cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev) {
+  const lif_layer_desc& D = L->desc;
+  const int nwords = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
+  cudaError_t e = launch_k(window_plan_kernel, dim3(1), dim3(kWindowThreads), 0, st, L->use_pdl,
+                           window_args(L, L->active_idx, L->n_tmp), (const uint32_t*)L->mask_words,
+                           nwords, (int32_t*)L->n_tmp);
+  return e != cudaSuccess ? e : launch_moves(L, st, ev);
 }
 
 }  // namespace lif

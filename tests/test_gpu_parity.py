@@ -142,15 +142,16 @@ def test_reset_gives_cold_cache_and_runs_are_reproducible():
     gpu.close()
 
 
-@pytest.mark.parametrize("two_streams,pdl,split,ffn_mode", [
-    (False, 1, 1, 0), (True, 1, 1, 0), (True, 0, 1, 0), (True, 1, 0, 0), (True, 0, 0, 0),
-    (True, 1, 1, 1), (False, 1, 0, 1)])
-def test_decode_step_matches_oracle_decode_step(two_streams, pdl, split, ffn_mode):
+@pytest.mark.parametrize("two_streams,pdl,split,ffn_mode,fused", [
+    (False, 1, 1, 0, 1), (True, 1, 1, 0, 1), (True, 0, 1, 0, 1), (True, 1, 0, 0, 1), (True, 0, 0, 0, 0),
+    (True, 1, 1, 1, 1), (False, 1, 0, 1, 0), (True, 1, 1, 0, 0)])
+def test_decode_step_matches_oracle_decode_step(two_streams, pdl, split, ffn_mode, fused):
     cfg = W.CONFIGS["tiny"]
     X = W.make_inputs(cfg, device=DEV)
     gpu, ora = P.make_layer_pair(cfg, 1, b_down=True, ffn_mode=ffn_mode)
     B.lif_set_tuning(gpu.handle, B.TUNE_DEPENDENT_LAUNCH, pdl)
     B.lif_set_tuning(gpu.handle, B.TUNE_SPLIT_FFN, split)
+    B.lif_set_tuning(gpu.handle, B.TUNE_FUSED_PLAN, fused)
     y = torch.empty(cfg.n_streams, cfg.d_model, dtype=torch.float32, device=DEV)
     sc, sf = (torch.cuda.Stream(), torch.cuda.Stream()) if two_streams else (None, None)
     if sc is not None:
@@ -233,3 +234,26 @@ def test_graph_replay_matches_direct_decode_steps_bitwise():
     B.lif_graph_destroy(g)
     for l in a + b:
         l.close()
+
+
+def test_decode_step_with_dense_mask_and_large_cache():
+    # ~40 % of the neurons fire: mask words hold more active neurons than the fused window
+    # update keeps in registers, and the cache outgrows its per-thread slots, so the kernel
+    # must hand over to its general path inside the same launch
+    cfg = W.LifConfig("dense", 1, 512, 16384, 32, 2, 1, 5, 0.40, 0.5, 0.8, 0.6, 13)
+    X = W.make_inputs(cfg, device=DEV)
+    gpu, ora = P.make_layer_pair(cfg, 0, capacity=cfg.d_ff)
+    y = torch.empty(1, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        g = gpu.lists()
+        logits, act, lists, ref_y = O.decode_step(ora.cache, X[t].cpu().numpy(), ora.A, ora.B, ora.c,
+                                                  0.0, ora.bundles, ora.bias_up, act=g["active_idx"])
+        P.assert_mask_borderline(g["active_idx"], logits, 0.0)
+        P.compare_lists_and_state(gpu, ora, lists)
+        P.compare_cache_rows(gpu, ora)
+        P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
+    assert g["num_used"] > 4096
+    gpu.close()
