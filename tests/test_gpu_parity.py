@@ -181,13 +181,13 @@ def test_decode_token_host_matches_per_layer_decode_steps():
     dev_x = torch.empty(S, d, dtype=torch.float16, device=DEV)
     dev_y = torch.empty(L, S, d, dtype=torch.float32, device=DEV)
     y_ref = torch.empty(L, S, d, dtype=torch.float32, device=DEV)
-    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    sc, sf, sc2, sf2 = (torch.cuda.Stream() for _ in range(4))
     torch.cuda.synchronize()
     for t in range(10):
         host_x.copy_(X[t])
         B.lif_decode_token_host([l.handle for l in a], host_x, dev_x, dev_y, host_y, sc, sf)
         for l in range(L):
-            B.lif_decode_step(b[l].handle, X[t], y_ref[l])
+            B.lif_decode_step(b[l].handle, X[t], y_ref[l], sc2, sf2)
         torch.cuda.synchronize()
         assert torch.equal(host_y, y_ref.cpu())
     for l in range(L):
@@ -207,7 +207,7 @@ def test_graph_replay_matches_direct_decode_steps_bitwise():
     y_d = torch.zeros(L, S, d, dtype=torch.float32, device=DEV)
     host_x = torch.empty(S, d, dtype=torch.float16, pin_memory=True)
     host_y = torch.empty(L, S, d, dtype=torch.float32, pin_memory=True)
-    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    sc, sf, sc2, sf2 = (torch.cuda.Stream() for _ in range(4))
     torch.cuda.synchronize()
     g = B.lif_graph_capture([l.handle for l in a], dev_x, y_g, sc, sf)
     assert all(l.lists()["step"] == 0 for l in a)                     # capture ran nothing
@@ -223,7 +223,7 @@ def test_graph_replay_matches_direct_decode_steps_bitwise():
             B.lif_graph_launch_host(g, host_x, host_y, sc)
             got = host_y.clone()
         for l in range(L):
-            B.lif_decode_step(b[l].handle, X[t], y_d[l])
+            B.lif_decode_step(b[l].handle, X[t], y_d[l], sc2, sf2)
         torch.cuda.synchronize()
         assert torch.equal(got, y_d.cpu()), t
     for la, lb in zip(a, b):
