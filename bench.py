@@ -211,11 +211,26 @@ def run_ours(args):
     n_act_l, n_load_l, n_hit_l = (cnts[:, i].sum().item() for i in (B.CNT_N_ACTIVE, B.CNT_N_LOAD, B.CNT_N_HITS))
     kernel_us = {}
     reps = 20
-    for kind, name in enumerate(B.KERNELS):
+    if S == 1:
+        launchers = {name: (lambda l, kind=kind: B.lif_profile_launch(handles[l], kind, dev_x, Y[l], sc))
+                     for kind, name in enumerate(B.KERNELS)}
+    else:
+        # several streams: the staged entry points (predictor = 2 kernels; FFN = the tensor-core
+        # up, down and partial-sum kernels over all active rows)
+        acts = torch.empty(cfg.d_ff, dtype=torch.int32, device=dev)
+        nact = torch.zeros(1, dtype=torch.int32, device=dev)
+        slot_views = [l._view("active_slots", cfg.d_ff) for l in layers]
+        launchers = {
+            "predict": lambda l: B.lif_predict(handles[l], dev_x, None, acts, nact, sc),
+            "fetch": lambda l: B.lif_fetch_bundles(handles[l], sc),
+            "ffn_active": lambda l: B.lif_sparse_ffn(handles[l], dev_x, slot_views[l],
+                                                     layers[l].counts[B.CNT_N_ACTIVE:], Y[l], sc),
+        }
+    for name, launch in launchers.items():
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=sc):
             for l in range(L):
-                B.lif_profile_launch(handles[l], kind, dev_x, Y[l], sc)
+                launch(l)
         with torch.cuda.stream(sc):
             for _ in range(3):
                 g.replay()
@@ -246,14 +261,17 @@ def run_ours(args):
         beta = cfg.bundle_bytes
         peak, peak_kind = _peaks()
         # algorithmic bytes of one launch: bundle + bias per row, x in, partials out
-        ffn_bytes = (n_act_l * (beta + 2) + L * 6 * d) / L
+        ffn_bytes = (n_act_l * (beta + 2) + L * S * 6 * d) / L
         ffn_gbs = ffn_bytes / (kernel_us["ffn_active"] * 1e-6) / 1e9
         fetch_bytes = n_load_l * beta / L
         fetch_gbs = fetch_bytes / (kernel_us["fetch"] * 1e-6) / 1e9
         pred_bytes = 2 * cfg.rank * (d + cfg.d_ff) + 4 * cfg.d_ff
-        pred_gbs = pred_bytes / ((kernel_us["predict_z"] + kernel_us["predict_scores"]) * 1e-6) / 1e9
-        hits_gbs = (n_hit_l * (beta + 2) / L + 6 * d) / (kernel_us["ffn_hits"] * 1e-6) / 1e9
-        new_gbs = (n_load_l * (beta + 2) / L + 6 * d) / (kernel_us["ffn_new"] * 1e-6) / 1e9
+        pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_z"] + kernel_us["predict_scores"]
+        pred_gbs = pred_bytes / (pred_us * 1e-6) / 1e9
+        split = None
+        if S == 1:
+            split = {"already_cached_rows_GBs": (n_hit_l * (beta + 2) / L + 6 * d) / (kernel_us["ffn_hits"] * 1e-6) / 1e9,
+                     "new_rows_GBs": (n_load_l * (beta + 2) / L + 6 * d) / (kernel_us["ffn_new"] * 1e-6) / 1e9}
         out = {
             "metric": METRIC, "value": whole_job_tokens_per_s(K, world, ms_total), "unit": UNIT,
             "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms_total / K,
@@ -269,10 +287,12 @@ def run_ours(args):
                     "h2d_bytes_per_step": S * d * 2, "d2h_bytes_per_step": L * S * d * 4,
                     "host_link_bytes_per_step": fetched / K},
             "gpu_launches": 7 * n_launch,
-            "roofline": {"kernel": "sparse_ffn_kernel", "bound": "hbm",
+            "roofline": {"kernel": "sparse_ffn_kernel" if S == 1 else
+                                   "ffn_batched_up_kernel + ffn_batched_down_kernel + ffn_reduce_kernel",
+                         "bound": "hbm",
                          "achieved": ffn_gbs, "peak": peak, "unit": "GB/s", "frac": ffn_gbs / peak,
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": ffn_gbs / NOMINAL_HBM_GBS,
-                         "traffic": FFN_TRAFFIC_RATIO * ffn_bytes if FFN_TRAFFIC_RATIO else None,
+                         "traffic": FFN_TRAFFIC_RATIO * ffn_bytes if FFN_TRAFFIC_RATIO and S == 1 else None,
                          "traffic_how": "dram read+write bytes per algorithmic byte from the ncu capture in "
                                         "profiles/sparse_ffn_kernel_opt6p7b_12layers.md (12 layers, "
                                         "451-529 rows per launch), scaled by this run's rows per launch",
@@ -280,7 +300,7 @@ def run_ours(args):
                          "bytes_per_launch": ffn_bytes,
                          "how": "graph of this kernel on all layers' active rows of the last token, "
                                 f"{reps} replays, CUDA events",
-                         "split_launches": {"already_cached_rows_GBs": hits_gbs, "new_rows_GBs": new_gbs}},
+                         "split_launches": split},
             "host_link": {"kernel": "fetch_kernel", "bound": "host_link", "achieved": fetch_gbs,
                           "peak": link_peak, "unit": "GB/s", "frac": fetch_gbs / link_peak,
                           "peak_kind": "of measured (1 GiB pinned cudaMemcpyAsync, this run)",
@@ -325,12 +345,15 @@ def run_kernel_loop(args):
             dev_x.copy_(X[t], non_blocking=True)
         B.lif_graph_launch(graph, sc)
     torch.cuda.synchronize()
-    kind = B.KERNELS.index(args.kernel_loop)
     cnt = {"ffn_active": B.CNT_N_ACTIVE, "ffn_hits": B.CNT_N_HITS, "ffn_new": B.CNT_N_LOAD,
-           "fetch": B.CNT_N_LOAD}.get(args.kernel_loop)
+           "fetch": B.CNT_N_LOAD, "ffn_api": B.CNT_N_ACTIVE}.get(args.kernel_loop)
     rows = [int(l.counts[cnt]) for l in layers] if cnt is not None else None
     for l in range(L):
-        B.lif_profile_launch(handles[l], kind, dev_x, Y[l], sc)
+        if args.kernel_loop == "ffn_api":     # lif_sparse_ffn over the active rows, any stream count
+            B.lif_sparse_ffn(handles[l], dev_x, layers[l]._view("active_slots", cfg.d_ff),
+                             layers[l].counts[B.CNT_N_ACTIVE:], Y[l], sc)
+        else:
+            B.lif_profile_launch(handles[l], B.KERNELS.index(args.kernel_loop), dev_x, Y[l], sc)
     torch.cuda.synchronize()
     print(json.dumps({"kernel": args.kernel_loop, "layers": L, "warmup_tokens": args.warmup,
                       "rows_per_launch": rows, "bundle_bytes": cfg.bundle_bytes}), flush=True)
@@ -452,7 +475,8 @@ def main():
     ap.add_argument("--cpu-tokens", type=int, default=30)
     ap.add_argument("--kernel-loop", default=None,
                     help="profiling aid: after the warm-up tokens launch this kernel once per layer "
-                         "(predict_z, predict_scores, fetch, ffn_active, ffn_hits, ffn_new, ffn_sum)")
+                         "(predict_z, predict_scores, fetch, ffn_active, ffn_hits, ffn_new, ffn_sum; "
+                         "ffn_api = lif_sparse_ffn over the active rows, for any number of streams)")
     args = ap.parse_args()
     if args.warmup < 3:
         raise SystemExit("--warmup must be at least 3")
