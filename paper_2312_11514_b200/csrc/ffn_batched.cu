@@ -23,6 +23,8 @@ constexpr int kPad = 16;                  // bytes added to every shared row: co
 constexpr unsigned kWaitLimitB = 1u << 22;
 constexpr int kGroupA = 16;               // rows per MMA in phase A (M = 16)
 constexpr int kMaxTilesPerWarp = 28;      // 16-column tiles per warp in phase B
+constexpr int kRowCacheA = 512;           // rows per CTA whose slot and bias are preloaded (phase A)
+constexpr int kRowCacheB = 256;           // rows per CTA whose slot is preloaded (phase B)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -108,6 +110,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
   uint64_t* bars = reinterpret_cast<uint64_t*>(rows + (size_t)stages * pitch);
   float* bias_s = reinterpret_cast<float*>(bars + stages);   // [stages]
   float* red = bias_s + stages;                              // [8 warps][32 lanes][4]
+  int* slot_all = reinterpret_cast<int*>(red + 8 * 32 * 4);  // [kRowCacheA]
+  float* bias_all = reinterpret_cast<float*>(slot_all + kRowCacheA);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
@@ -124,13 +128,19 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
   const int my_cnt = (n - prt + P - 1) / P;             // rows q = prt + i * P
   __syncthreads();
 
-  // first copies in flight, then the x slice into shared memory (streams beyond S are zero)
-  if (tid < stages && tid < my_cnt) {
-    const int slot = row_slot(a, prt + tid * P, base);
-    mbar_expect_tx(bars + tid, seg_bytes);
-    bulk_g2s(rows + (size_t)tid * pitch, a.cache + (size_t)slot * 2 * d + k0, seg_bytes,
-             bars + tid);
-    bias_s[tid] = ks == 0 ? __half2float(a.bias[slot]) : 0.f;
+  // Slots and biases of this CTA's rows go to shared memory once, so the group loop below has
+  // no dependent global loads; the first copies are issued on the way.  Then the x slice
+  // (streams beyond S are zero).
+  for (int i = tid; i < min(my_cnt, kRowCacheA); i += kThreads) {
+    const int slot = row_slot(a, prt + i * P, base);
+    slot_all[i] = slot;
+    if (i < stages) {
+      mbar_expect_tx(bars + i, seg_bytes);
+      bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * 2 * d + k0, seg_bytes, bars + i);
+    }
+    const float b = ks == 0 ? __half2float(a.bias[slot]) : 0.f;
+    bias_all[i] = b;
+    if (i < stages) bias_s[i] = b;
   }
   {
     const int vec = kcols >> 3;
@@ -199,11 +209,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
     if (tid < kGroupA) {
       const int i = (g + groups_in_ring) * kGroupA + tid;
       if (i < my_cnt) {
-        const int slot = row_slot(a, prt + i * P, base);
+        const bool cached = i < kRowCacheA;
+        const int slot = cached ? slot_all[i] : row_slot(a, prt + i * P, base);
         mbar_expect_tx(bars + st0 + tid, seg_bytes);
         bulk_g2s(rows + (size_t)(st0 + tid) * pitch, a.cache + (size_t)slot * 2 * d + k0,
                  seg_bytes, bars + st0 + tid);
-        bias_s[st0 + tid] = ks == 0 ? __half2float(a.bias[slot]) : 0.f;
+        bias_s[st0 + tid] = cached ? bias_all[i] : (ks == 0 ? __half2float(a.bias[slot]) : 0.f);
       }
     }
   }
@@ -223,6 +234,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   uint64_t* bars = reinterpret_cast<uint64_t*>(rows + (size_t)stages * pitch);
   __half* h_hi = reinterpret_cast<__half*>(bars + stages);             // [8][16]
   __half* h_lo = h_hi + 128;
+  int* slot_all = reinterpret_cast<int*>(h_lo + 128);                  // [kRowCacheB]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // zero the row buffers once: padded k-steps multiply by H = 0 and need finite operands
@@ -242,11 +254,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   const int my_cnt = prt < n ? (n - prt + P - 1) / P : 0;       // rows q = prt + i * P
   const size_t col_off = (size_t)d + col0;
 
-  if (tid < stages && tid < my_cnt) {
-    const int slot = row_slot(a, prt + tid * P, base);
-    mbar_expect_tx(bars + tid, seg_bytes);
-    bulk_g2s(rows + (size_t)tid * pitch, a.cache + (size_t)slot * 2 * d + col_off, seg_bytes,
-             bars + tid);
+  for (int i = tid; i < min(my_cnt, kRowCacheB); i += kThreads) {   // slots once, first copies
+    const int slot = row_slot(a, prt + i * P, base);
+    slot_all[i] = slot;
+    if (i < stages) {
+      mbar_expect_tx(bars + i, seg_bytes);
+      bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * 2 * d + col_off, seg_bytes,
+               bars + i);
+    }
   }
 
   const int tiles = (ncols + 15) >> 4;
@@ -314,7 +329,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     if (tid < 16) {
       const int i = (g + 2) * 16 + tid;
       if (i < my_cnt) {
-        const int slot = row_slot(a, prt + i * P, base);
+        const int slot = i < kRowCacheB ? slot_all[i] : row_slot(a, prt + i * P, base);
         mbar_expect_tx(bars + st0 + tid, seg_bytes);
         bulk_g2s(rows + (size_t)(st0 + tid) * pitch, a.cache + (size_t)slot * 2 * d + col_off,
                  seg_bytes, bars + st0 + tid);
@@ -339,10 +354,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
 
 size_t up_smem(int k_per_split, int stages) {
   const size_t pitch = 2 * (size_t)k_per_split + kPad;
-  return (8 + stages) * pitch + stages * 8 + stages * 4 + 8 * 32 * 4 * 4 + 16;
+  return (8 + stages) * pitch + stages * 8 + stages * 4 + 8 * 32 * 4 * 4 + kRowCacheA * 8 + 16;
 }
 size_t down_smem(int cols_per_part, int stages) {
-  return stages * (2 * (size_t)cols_per_part + kPad) + stages * 8 + 2 * 128 * 2 + 16;
+  return stages * (2 * (size_t)cols_per_part + kPad) + stages * 8 + 2 * 128 * 2 + kRowCacheB * 4 +
+         16;
 }
 
 }  // namespace
