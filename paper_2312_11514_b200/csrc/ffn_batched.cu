@@ -22,6 +22,12 @@ namespace {
 constexpr int kPad = 16;                  // bytes added to every shared row: conflict-free ldmatrix
 constexpr unsigned kWaitLimitB = 1u << 22;
 constexpr int kGroupA = 16;               // rows per MMA in phase A (M = 16)
+// One mbarrier per group of 16 ring stages (the first stage's): arrival count 16, one arrival
+// per stage — with the stage's byte count where a row is copied, plain where the list has ended.
+constexpr int kGroup = 16;
+__device__ __forceinline__ uint64_t* group_bar(uint64_t* bars, int stage) {
+  return bars + (stage / kGroup) * kGroup;
+}
 constexpr int kMaxTilesPerWarp = 28;      // 16-column tiles per warp in phase B
 constexpr int kRowCacheA = 512;           // rows per CTA whose slot and bias are preloaded (phase A)
 constexpr int kRowCacheB = 256;           // rows per CTA whose slot is preloaded (phase B)
@@ -36,6 +42,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
                "r"(bytes)
                : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
   for (unsigned i = 0; i < kWaitLimitB; ++i) {
@@ -115,7 +124,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
-    for (int i = 0; i < stages; ++i) mbar_init(bars + i, 1);
+    for (int i = 0; i < stages; ++i) mbar_init(bars + i, kGroup);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -135,13 +144,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
     const int slot = row_slot(a, prt + i * P, base);
     slot_all[i] = slot;
     if (i < stages) {
-      mbar_expect_tx(bars + i, seg_bytes);
-      bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * 2 * d + k0, seg_bytes, bars + i);
+      mbar_expect_tx(group_bar(bars, i), seg_bytes);
+      bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * 2 * d + k0, seg_bytes,
+               group_bar(bars, i));
     }
     const float b = ks == 0 ? __half2float(a.bias[slot]) : 0.f;
     bias_all[i] = b;
     if (i < stages) bias_s[i] = b;
   }
+  for (int i = my_cnt + tid; i < stages; i += kThreads) mbar_arrive(group_bar(bars, i));
   {
     const int vec = kcols >> 3;
     for (int i = tid; i < 8 * vec; i += kThreads) {
@@ -170,8 +181,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
     const int st0 = (g % groups_in_ring) * kGroupA;
     const unsigned parity = (unsigned)(g / groups_in_ring) & 1u;
     const int valid = min(kGroupA, my_cnt - g * kGroupA);
-    for (int i = 0; i < valid; ++i)
-      if (!mbar_wait(bars + st0 + i, parity)) timed_out = 1;
+    if (!mbar_wait(bars + st0, parity)) timed_out = 1;
     // D[row][stream] over this warp's part of the slice
     float c[4] = {0.f, 0.f, 0.f, 0.f};
     const unsigned char* ab = rows + (size_t)(st0 + a_row) * pitch + a_off;
@@ -188,7 +198,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
     if (__syncthreads_or(timed_out)) {
       if (tid == 0) {
         atomicCAS(a.status, LIF_OK, LIF_ERR_TIMEOUT);
-        for (int i = 0; i < valid; ++i) mbar_wait(bars + st0 + i, parity);
+        mbar_wait(bars + st0, parity);
       }
       __syncthreads();
       return;
@@ -211,10 +221,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
       if (i < my_cnt) {
         const bool cached = i < kRowCacheA;
         const int slot = cached ? slot_all[i] : row_slot(a, prt + i * P, base);
-        mbar_expect_tx(bars + st0 + tid, seg_bytes);
+        mbar_expect_tx(bars + st0, seg_bytes);
         bulk_g2s(rows + (size_t)(st0 + tid) * pitch, a.cache + (size_t)slot * 2 * d + k0,
-                 seg_bytes, bars + st0 + tid);
+                 seg_bytes, bars + st0);
         bias_s[st0 + tid] = cached ? bias_all[i] : (ks == 0 ? __half2float(a.bias[slot]) : 0.f);
+      } else {
+        mbar_arrive(bars + st0);
       }
     }
   }
@@ -241,7 +253,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   for (size_t i = (size_t)tid * 16; i < (size_t)stages * pitch; i += kThreads * 16)
     *reinterpret_cast<uint4*>(rows + i) = make_uint4(0, 0, 0, 0);
   if (tid == 0) {
-    for (int i = 0; i < stages; ++i) mbar_init(bars + i, 1);
+    for (int i = 0; i < stages; ++i) mbar_init(bars + i, kGroup);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -258,11 +270,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     const int slot = row_slot(a, prt + i * P, base);
     slot_all[i] = slot;
     if (i < stages) {
-      mbar_expect_tx(bars + i, seg_bytes);
+      mbar_expect_tx(group_bar(bars, i), seg_bytes);
       bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * 2 * d + col_off, seg_bytes,
-               bars + i);
+               group_bar(bars, i));
     }
   }
+  for (int i = my_cnt + tid; i < stages; i += kThreads) mbar_arrive(group_bar(bars, i));
 
   const int tiles = (ncols + 15) >> 4;
   float acc[kMaxTilesPerWarp][4];
@@ -297,12 +310,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
       const int i = (g + 1) * 16 + hk;
       h_next = i < my_cnt ? load_h(i) : 0.f;
     }
-    for (int i = 0; i < valid; ++i)
-      if (!mbar_wait(bars + st0 + i, parity)) timed_out = 1;
+    if (!mbar_wait(bars + st0, parity)) timed_out = 1;
     if (__syncthreads_or(timed_out)) {
       if (tid == 0) {
         atomicCAS(a.status, LIF_OK, LIF_ERR_TIMEOUT);
-        for (int i = 0; i < valid; ++i) mbar_wait(bars + st0 + i, parity);
+        mbar_wait(bars + st0, parity);
       }
       __syncthreads();
       return;
@@ -330,9 +342,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
       const int i = (g + 2) * 16 + tid;
       if (i < my_cnt) {
         const int slot = i < kRowCacheB ? slot_all[i] : row_slot(a, prt + i * P, base);
-        mbar_expect_tx(bars + st0 + tid, seg_bytes);
+        mbar_expect_tx(bars + st0, seg_bytes);
         bulk_g2s(rows + (size_t)(st0 + tid) * pitch, a.cache + (size_t)slot * 2 * d + col_off,
-                 seg_bytes, bars + st0 + tid);
+                 seg_bytes, bars + st0);
+      } else {
+        mbar_arrive(bars + st0);
       }
     }
   }
