@@ -166,15 +166,32 @@ class NeuronCache:
 # --------------------------------------------------------------------------------------
 # Step 5: sparse FFN over the cached bundles (Section 3.3 item 3)
 # --------------------------------------------------------------------------------------
-def sparse_ffn(matrix, bias, slots, x, b_down=None):
-    """y[s] = b_down + sum_q relu(<matrix[slots[q], :d], x[s]> + bias[slots[q]]) * matrix[slots[q], d:]
+RELU, RELU_SQUARED, FATRELU = 0, 1, 2
+
+
+def activation_fn(pre, activation=RELU, threshold=0.0):
+    """The FFN non-linearities the paper runs: ReLU (OPT, relufied Falcon and Phi-2), squared
+    ReLU (Appendix C, Persimmon 8B) and FATReLU (Appendix C, Llama 2: a neuron passes its
+    pre-activation only when it exceeds a threshold)."""
+    if activation == RELU:
+        return np.maximum(pre, 0.0)
+    if activation == RELU_SQUARED:
+        return np.maximum(pre, 0.0) ** 2
+    if activation == FATRELU:
+        return np.where(pre > threshold, pre, 0.0)
+    raise ValueError(activation)
+
+
+def sparse_ffn(matrix, bias, slots, x, b_down=None, activation=RELU, threshold=0.0):
+    """y[s] = b_down + sum_q act(<matrix[slots[q], :d], x[s]> + bias[slots[q]]) * matrix[slots[q], d:]
 
     matrix: [cap][2d] (fp16 values), bias: [cap], slots: row indices, x: [S][d].  float64."""
     x = np.asarray(x, dtype=np.float64)
     d = x.shape[1]
     rows = np.asarray(matrix)[np.asarray(slots, dtype=np.int64)].astype(np.float64)
     up, down = rows[:, :d], rows[:, d:]
-    h = np.maximum(x @ up.T + np.asarray(bias, dtype=np.float64)[slots][None, :], 0.0)
+    h = activation_fn(x @ up.T + np.asarray(bias, dtype=np.float64)[slots][None, :], activation,
+                      threshold)
     y = h @ down
     if b_down is not None:
         y = y + np.asarray(b_down, dtype=np.float64)[None, :]
@@ -182,7 +199,7 @@ def sparse_ffn(matrix, bias, slots, x, b_down=None):
 
 
 def decode_step(cache, x, A, B, c, theta, bundles, bias_up, b_down=None, whole_cache=False,
-                act=None):
+                act=None, activation=RELU, threshold=0.0):
     """One layer, one token: predict -> window update -> insert -> FFN.  ``act`` overrides the
     predicted active list (used to follow another implementation's borderline decisions).
     ``whole_cache`` runs the FFN over every cached row (matrix[:num_used]) instead of only the
@@ -193,7 +210,7 @@ def decode_step(cache, x, A, B, c, theta, bundles, bias_up, b_down=None, whole_c
     lists = cache.window_update(act)
     cache.insert(lists, bundles, bias_up)
     slots = np.arange(cache.num_used) if whole_cache else lists["active_slots"]
-    y = sparse_ffn(cache.matrix, cache.bias, slots, x, b_down)
+    y = sparse_ffn(cache.matrix, cache.bias, slots, x, b_down, activation, threshold)
     return logits, act, lists, y
 
 

@@ -249,21 +249,24 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   int* slot_all = reinterpret_cast<int*>(h_lo + 128);                  // [kRowCacheB]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // zero the row buffers once: padded k-steps multiply by H = 0 and need finite operands
-  for (size_t i = (size_t)tid * 16; i < (size_t)stages * pitch; i += kThreads * 16)
-    *reinterpret_cast<uint4*>(rows + i) = make_uint4(0, 0, 0, 0);
   if (tid == 0) {
     for (int i = 0; i < stages; ++i) mbar_init(bars + i, kGroup);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  __syncthreads();
   pdl_wait();
   pdl_trigger();
   const int n = *a.n;
   const int base = a.base ? *a.base : 0;
   const int P = a.partitions;
   const int my_cnt = prt < n ? (n - prt + P - 1) / P : 0;       // rows q = prt + i * P
+  // Padded k-steps (rows past the end of the list) multiply by H = 0 and need finite operands.
+  // Once the ring has been filled they hold earlier rows' weights; a list shorter than the
+  // ring leaves stages never written, so those are zeroed first.
+  if (my_cnt < stages)
+    for (size_t i = (size_t)tid * 16; i < (size_t)stages * pitch; i += kThreads * 16)
+      *reinterpret_cast<uint4*>(rows + i) = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
   const size_t col_off = (size_t)d + col0;
 
   for (int i = tid; i < min(my_cnt, kRowCacheB); i += kThreads) {   // slots once, first copies

@@ -350,3 +350,36 @@ def test_bundling_halves_io_latency_as_in_table_1():
     # same bytes, throughput 1.25 -> 2.25 GB/s: latency ratio 164 / 87 in Table 1
     a, b = O.io_latency_ms(0.2, 1.25), O.io_latency_ms(0.2, 2.25)
     assert a / b == pytest.approx(164 / 87, rel=0.05)
+
+
+# ------------------------------------------------------------------ activation variants
+@pytest.mark.parametrize("activation,threshold", [(O.RELU_SQUARED, 0.0), (O.FATRELU, 0.7), (O.FATRELU, 0.0)])
+def test_activation_variants_match_scalar_loops(activation, threshold):
+    r = _rng(20 + activation)
+    F, d = 17, 5
+    W_up, W_down = r.normal(size=(F, d)), r.normal(size=(d, F))
+    b_up, b_down, x = r.normal(size=F), r.normal(size=d), r.normal(size=d)
+    want = b_down.copy()
+    n_pass = 0
+    for i in range(F):
+        pre = b_up[i] + sum(W_up[i, m] * x[m] for m in range(d))
+        if activation == O.RELU_SQUARED:
+            h = pre * pre if pre > 0 else 0.0            # Appendix C, Persimmon: squared ReLU
+        else:
+            h = pre if pre > threshold else 0.0          # Appendix C, Llama 2: FATReLU
+        n_pass += h != 0.0
+        for m in range(d):
+            want[m] += h * W_down[m, i]
+    assert 0 < n_pass < F
+    M, bias = _cache_from_dense(W_up, b_up, W_down, list(range(F)))
+    got = O.sparse_ffn(M, bias, np.arange(F), x[None, :], b_down, activation, threshold)[0]
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    if activation == O.FATRELU and threshold == 0.0:     # threshold 0 is plain ReLU
+        np.testing.assert_allclose(got, O.sparse_ffn(M, bias, np.arange(F), x[None, :], b_down)[0], rtol=1e-12)
+
+
+def test_fatrelu_threshold_only_removes_neurons():
+    pre = np.array([-1.0, 0.2, 0.7, 0.70001, 3.0])
+    np.testing.assert_array_equal(O.activation_fn(pre, O.FATRELU, 0.7), [0, 0, 0, 0.70001, 3.0])
+    np.testing.assert_array_equal(O.activation_fn(pre, O.RELU_SQUARED), [0, 0.2 ** 2, 0.7 ** 2, 0.70001 ** 2, 9.0])
+    np.testing.assert_array_equal(O.activation_fn(pre), [0, 0.2, 0.7, 0.70001, 3.0])
