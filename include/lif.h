@@ -42,6 +42,11 @@ typedef enum {
 
 const char* lif_status_str(lif_status s);
 
+/* FFN non-linearities the paper runs (Appendix C): ReLU for OPT and the relufied Falcon and
+ * Phi-2; squared ReLU for Persimmon 8B; FATReLU for the sparsified Llama 2 — a neuron passes
+ * its pre-activation v only when v > activation_threshold (threshold 0 is ReLU). */
+enum { LIF_ACT_RELU = 0, LIF_ACT_RELU_SQUARED = 1, LIF_ACT_FATRELU = 2 };
+
 typedef struct lif_layer lif_layer;
 
 /* Layer description.  Shapes follow Section 3.3: the cache `matrix` is
@@ -58,7 +63,8 @@ typedef struct {
                                maps to ln(tau/(1-tau)), tau = 0.5 -> 0 (Section 3.1, App. B) */
   int32_t ffn_mode;         /* 0: FFN over the rows of the currently active neurons;
                                1: over every cached row [0, num_used) (Section 3.3 item 3) */
-  int32_t activation;       /* 0 = ReLU */
+  int32_t activation;       /* LIF_ACT_*: the FFN non-linearity applied to <up row, x> + bias */
+  float activation_threshold; /* FATReLU threshold (LIF_ACT_FATRELU only; >= 0) */
   const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][2*d_model] */
   const void* dev_pred_A;   /* fp16 [d_model][rank] */
   const void* dev_pred_B;   /* fp16 [rank][d_ff] */

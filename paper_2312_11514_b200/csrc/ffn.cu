@@ -74,6 +74,8 @@ struct FfnArgs {
   int d;
   int stages;
   int slots_len;          // entries of `slots` that may be read before n is known (0: none)
+  int act;                // LIF_ACT_*
+  float act_thr;
 };
 
 __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
@@ -175,7 +177,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
       float v = 0.f;
 #pragma unroll
       for (int w = 0; w < 8; ++w) v += part[tid * 8 + w];
-      hs[tid] = fmaxf(v + bias_s[tid], 0.f);
+      hs[tid] = apply_activation(v + bias_s[tid], a.act, a.act_thr);
     }
     __syncthreads();
     // down projection: y += h * down half
@@ -299,6 +301,8 @@ static FfnArgs ffn_args(lif_layer* L, const __half* x, const int32_t* slots, con
   a.d = L->desc.d_model;
   a.stages = L->ffn_stages;
   a.slots_len = slots_len;
+  a.act = L->desc.activation;
+  a.act_thr = L->desc.activation_threshold;
   return a;
 }
 
@@ -502,6 +506,8 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
   a.d = d_model;
   a.stages = stages;
   a.slots_len = 0;
+  a.act = LIF_ACT_RELU;
+  a.act_thr = 0.f;
   sparse_ffn_kernel<<<grid, kThreads, ffn_smem_bytes(d_model, stages), st>>>(a);
   if (cudaGetLastError() != cudaSuccess) return LIF_ERR_CUDA;
   ffn_reduce_kernel<<<(d_model / 4 + kSumCols - 1) / kSumCols, kSumThreads, 0, st>>>(

@@ -98,6 +98,8 @@ struct BatchedArgs {
   int d, S, stages, parts, partitions, cols_per_part;
   int ksplit, k_per_split, up_partitions;   // phase A: K slices (columns, multiple of 16)
   size_t h_stride;
+  int act;                // LIF_ACT_*
+  float act_thr;
 };
 
 __device__ __forceinline__ int row_slot(const BatchedArgs& a, int q, int base) {
@@ -293,7 +295,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     float v = 0.f;
     const size_t at = (size_t)(prt + i * P) * 8 + hs;
     for (int ks = 0; ks < a.ksplit; ++ks) v += a.H[(size_t)ks * a.h_stride + at];
-    return fmaxf(v, 0.f);
+    return apply_activation(v, a.act, a.act_thr);
   };
   float h_next = 0.f;
   if (tid < 128 && hk < my_cnt) h_next = load_h(hk);
@@ -450,6 +452,8 @@ cudaError_t launch_ffn_batched(lif_layer* L, const __half* x, const int32_t* slo
   a.k_per_split = L->fb_kps;
   a.up_partitions = L->fb_up_partitions;
   a.h_stride = (size_t)D.d_ff * 8;
+  a.act = D.activation;
+  a.act_thr = D.activation_threshold;
   a.stages = L->fb_up_stages;
   cudaError_t e = launch_k(ffn_batched_up_kernel, dim3(L->fb_up_partitions * L->fb_ksplit),
                            dim3(kThreads), L->fb_up_smem, st, L->use_pdl, a);

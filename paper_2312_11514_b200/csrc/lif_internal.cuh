@@ -151,6 +151,14 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
 // Block until every earlier kernel of the stream has completed and its writes are visible
 // (no-op for a kernel launched without the attribute).
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ float apply_activation(float v, int act, float thr) {
+  if (act == LIF_ACT_RELU_SQUARED) {
+    v = fmaxf(v, 0.f);
+    return v * v;
+  }
+  if (act == LIF_ACT_FATRELU) return v > thr ? v : 0.f;
+  return fmaxf(v, 0.f);
+}
 // Let the next kernel of the stream start its prologue.
 __device__ __forceinline__ void pdl_trigger() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

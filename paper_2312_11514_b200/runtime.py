@@ -17,7 +17,8 @@ class Layer:
                  host_bundles: torch.Tensor, pred_A: torch.Tensor, pred_B: torch.Tensor,
                  pred_c: torch.Tensor, bias_up: torch.Tensor,
                  bias_down: Optional[torch.Tensor] = None, n_streams: int = 1,
-                 threshold_logit: float = 0.0, ffn_mode: int = 0, device="cuda:0"):
+                 threshold_logit: float = 0.0, ffn_mode: int = 0, activation: int = 0,
+                 activation_threshold: float = 0.0, device="cuda:0"):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2312_11514_b200 needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
@@ -29,7 +30,8 @@ class Layer:
                          bias_up=bias_up, bias_down=bias_down)
         self.cache = torch.zeros(capacity, 2 * d_model, dtype=torch.float16, device=self.device)
         shape = dict(d_model=d_model, d_ff=d_ff, rank=rank, window_k=window_k, capacity=capacity,
-                     n_streams=n_streams, threshold_logit=threshold_logit, ffn_mode=ffn_mode)
+                     n_streams=n_streams, threshold_logit=threshold_logit, ffn_mode=ffn_mode,
+                     activation=activation, activation_threshold=activation_threshold)
         nbytes = B.lif_workspace_bytes(B.make_desc(**shape))
         self.workspace = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
         with torch.cuda.device(self.device):

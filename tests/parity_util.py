@@ -41,7 +41,9 @@ def assert_y_close(got, ref):
 class OracleLayer:
     """Oracle-side twin of one layer, fed with the same tensors."""
 
-    def __init__(self, w, d_model, d_ff, capacity, window_k, theta=0.0, b_down=None):
+    def __init__(self, w, d_model, d_ff, capacity, window_k, theta=0.0, b_down=None,
+                 activation=0, act_threshold=0.0):
+        self.activation, self.act_threshold = activation, act_threshold
         self.A = w["A"].cpu().numpy().astype(np.float64)
         self.B = w["B"].cpu().numpy().astype(np.float64)
         self.c = w["c"].cpu().numpy().astype(np.float64)
@@ -53,7 +55,7 @@ class OracleLayer:
 
 
 def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_down=False,
-                    device="cuda:0"):
+                    activation=0, act_threshold=0.0, device="cuda:0"):
     store = R.pinned_store(cfg.d_ff, cfg.d_model)
     w = W.make_layer(cfg, layer_idx, device=device, bundles_out=store)
     cap = capacity or W.window_capacity(cfg, w["p"])
@@ -65,8 +67,9 @@ def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_d
     gpu = R.Layer(d_model=cfg.d_model, d_ff=cfg.d_ff, rank=cfg.rank, window_k=cfg.window_k,
                   capacity=cap, host_bundles=store, pred_A=dev(w["A"]), pred_B=dev(w["B"]),
                   pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), bias_down=bd,
-                  n_streams=cfg.n_streams, threshold_logit=theta, ffn_mode=ffn_mode, device=device)
-    ora = OracleLayer(w, cfg.d_model, cfg.d_ff, cap, cfg.window_k, theta, bd)
+                  n_streams=cfg.n_streams, threshold_logit=theta, ffn_mode=ffn_mode,
+                  activation=activation, activation_threshold=act_threshold, device=device)
+    ora = OracleLayer(w, cfg.d_model, cfg.d_ff, cap, cfg.window_k, theta, bd, activation, act_threshold)
     return gpu, ora
 
 
@@ -132,7 +135,8 @@ def staged_step(gpu, ora, x_dev, bufs, whole_cache=False):
                          gpu.counts[B.CNT_N_ACTIVE:], y)
         slots = ref_lists["active_slots"]
     torch.cuda.synchronize()
-    ref_y = O.sparse_ffn(ora.cache.matrix, ora.cache.bias, slots, x_np, ora.b_down)
+    ref_y = O.sparse_ffn(ora.cache.matrix, ora.cache.bias, slots, x_np, ora.b_down, ora.activation,
+                         ora.act_threshold)
     assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
     return dict(n_active=na, n_load=len(ref_lists["load_ids"]), n_evict=len(ref_lists["evict_ids"]),
                 n_border=n_border)

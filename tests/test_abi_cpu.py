@@ -44,7 +44,8 @@ def test_workspace_bytes_and_shape_validation():
     assert B.lif_workspace_bytes(_shape(d_ff=2048, capacity=512)) > n
     for bad in (dict(d_model=260), dict(d_model=0), dict(d_model=16384), dict(d_ff=1001), dict(rank=12),
                 dict(rank=4096), dict(window_k=0), dict(capacity=0), dict(capacity=2048),
-                dict(n_streams=0), dict(n_streams=9), dict(ffn_mode=2), dict(activation=3),
+                dict(n_streams=0), dict(n_streams=9), dict(ffn_mode=2), dict(activation=3), dict(activation=-1),
+                dict(activation=2, activation_threshold=-0.5), dict(activation=2, activation_threshold=float("nan")),
                 dict(threshold_logit=float("nan"))):
         with pytest.raises(B.LifError) as e:
             B.lif_workspace_bytes(_shape(**bad))

@@ -257,3 +257,14 @@ def test_decode_step_with_dense_mask_and_large_cache():
         P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
     assert g["num_used"] > 4096
     gpu.close()
+
+
+@pytest.mark.parametrize("activation,thr,S", [(B.ACT_RELU_SQUARED, 0.0, 1), (B.ACT_FATRELU, 0.15, 1),
+                                              (B.ACT_RELU_SQUARED, 0.0, 3), (B.ACT_FATRELU, 0.15, 8)])
+def test_activation_variants(activation, thr, S):
+    # squared ReLU and FATReLU (Appendix C: Persimmon 8B, Llama 2) through the staged entry
+    # points; a high firing rate so that many neurons pass the non-linearity
+    cfg = W.LifConfig("act", 1, 512, 2048, 16, 3, S, 6, 0.30, 0.5, 0.8, 0.6, 14)
+    stats = _run_staged(cfg, 0, cfg.steps, b_down=True, activation=activation, act_threshold=thr,
+                        capacity=2048)
+    assert min(s["n_active"] for s in stats) > 100
