@@ -65,6 +65,10 @@ typedef struct {
                                1: over every cached row [0, num_used) (Section 3.3 item 3) */
   int32_t activation;       /* LIF_ACT_*: the FFN non-linearity applied to <up row, x> + bias */
   float activation_threshold; /* FATReLU threshold (LIF_ACT_FATRELU only; >= 0) */
+  int32_t budget_rows;      /* 0 = off.  Memory budget (Appendix C, Persimmon 8B / Phi-2): rows
+                               the cache may hold, <= capacity.  When a step would pass it, that
+                               step deletes with the widest window k' <= window_k (at least 1)
+                               that fits; LIF_CNT_K_EFF reports k'.  Needs window_k <= 32. */
   const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][2*d_model] */
   const void* dev_pred_A;   /* fp16 [d_model][rank] */
   const void* dev_pred_B;   /* fp16 [rank][d_ff] */
@@ -89,6 +93,7 @@ enum {
   LIF_CNT_NUM_USED = 7,     /* rows in use after the step */
   LIF_CNT_STEP = 8,         /* steps applied so far */
   LIF_CNT_STATUS = 9,       /* sticky lif_status written by kernels */
+  LIF_CNT_K_EFF = 10,       /* window actually applied this step (= window_k without a budget) */
   LIF_CNT_LEN = 64
 };
 

@@ -72,8 +72,12 @@ class NeuronCache:
     ``last_k_active`` is kept as ``last_active[i]`` = the last step at which neuron i was
     predicted active, so "still inside the window of k tokens" is last_active[i] > t - k."""
 
-    def __init__(self, d_model, d_ff, capacity, window_k):
+    def __init__(self, d_model, d_ff, capacity, window_k, budget_rows=0):
+        """``budget_rows`` > 0 turns on the memory budget of Appendix C (Persimmon 8B, Phi-2):
+        whenever the cache would pass the budget, the window is shrunk for that step."""
         self.d_model, self.d_ff, self.capacity, self.k = d_model, d_ff, capacity, window_k
+        self.budget_rows = budget_rows
+        self.k_eff = window_k
         self.matrix = np.zeros((capacity, 2 * d_model), dtype=np.float16)
         self.pointers = np.full(capacity, -1, dtype=np.int32)
         self.bias = np.zeros(capacity, dtype=np.float16)
@@ -95,13 +99,26 @@ class NeuronCache:
         in_act[act] = True
 
         # what would be deleted / loaded, before anything is changed
-        evict_slots = [s for s in range(n)
-                       if not in_act[self.pointers[s]]
-                       and self.last_active[self.pointers[s]] <= t - k]
         load_ids = [int(i) for i in act if self.slot_of[i] < 0]
+
+        def would_evict(kk):
+            return [s for s in range(n)
+                    if not in_act[self.pointers[s]]
+                    and self.last_active[self.pointers[s]] <= t - kk]
+
+        evict_slots = would_evict(k)
+        limit = self.capacity
+        if self.budget_rows > 0:
+            # Memory budget: keep the widest window k' <= k whose rows, with the rows to
+            # bring in, fit the budget; the choice is made anew at every step.
+            limit = min(limit, self.budget_rows)
+            while k > 1 and n - len(evict_slots) + len(load_ids) > limit:
+                k -= 1
+                evict_slots = would_evict(k)
         n_new = n - len(evict_slots)
-        if n_new + len(load_ids) > self.capacity:
-            raise CapacityError(f"need {n_new + len(load_ids)} rows, have {self.capacity}")
+        if n_new + len(load_ids) > limit:
+            raise CapacityError(f"need {n_new + len(load_ids)} rows, have {limit}")
+        self.k_eff = k
 
         self.last_active[act] = t
         evict_ids = [int(self.pointers[s]) for s in evict_slots]
@@ -148,6 +165,7 @@ class NeuronCache:
             "load_ids": i32(load_ids), "load_slots": i32(load_slots),
             "active_slots": active_slots, "hit_slots": i32(hit_slots),
             "num_used_before": n, "num_kept": n_new, "num_used": self.num_used,
+            "k_eff": self.k_eff,
         }
 
     # -- insert -------------------------------------------------------------------------

@@ -56,6 +56,8 @@ static lif_status check_shape(const lif_layer_desc* d) {
   if (d->capacity < 1 || d->capacity > d->d_ff) return LIF_ERR_INVALID_ARG;
   if (d->n_streams < 1 || d->n_streams > kMaxStreams) return LIF_ERR_INVALID_ARG;
   if (d->ffn_mode != 0 && d->ffn_mode != 1) return LIF_ERR_INVALID_ARG;
+  if (d->budget_rows < 0 || d->budget_rows > d->capacity) return LIF_ERR_INVALID_ARG;
+  if (d->budget_rows > 0 && d->window_k > 32) return LIF_ERR_INVALID_ARG;
   if (d->activation < LIF_ACT_RELU || d->activation > LIF_ACT_FATRELU) return LIF_ERR_INVALID_ARG;
   if (d->activation == LIF_ACT_FATRELU && !(d->activation_threshold >= 0.f)) return LIF_ERR_INVALID_ARG;
   if (!(d->threshold_logit == d->threshold_logit)) return LIF_ERR_INVALID_ARG;   // NaN

@@ -64,8 +64,24 @@ struct WindowArgs {
   int32_t *active_idx, *evict_ids, *evict_slots, *move_src, *move_dst, *load_ids, *load_slots,
       *active_slots, *hit_slots;
   int F, cap, k;
+  int budget;             // 0 = off; else rows the cache may hold (Appendix C memory budget)
   unsigned long long bundle_bytes;
 };
+
+// Memory-budgeted window (Appendix C, Persimmon 8B / Phi-2): hist[a] = cached rows that are not
+// active now and were last active a steps ago (a = 1 .. k, older ones in bin k).  Returns the
+// widest window k' <= k for which the rows kept plus the rows to load fit `limit`, at least 1.
+constexpr int kMaxBudgetWindow = 32;
+__device__ __forceinline__ int widest_window_that_fits(const int* hist, int k, int n, int n_load,
+                                                       int limit) {
+  int evicted = 0;          // rows deleted under window kk = sum of hist[a], a >= kk
+  int kk = k;
+  for (; kk >= 1; --kk) {
+    evicted += hist[kk];
+    if (n - evicted + n_load <= limit) break;
+  }
+  return kk < 1 ? 1 : kk;
+}
 
 // General path: any cache size, active list read from memory.
 __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
@@ -73,11 +89,36 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   const int n = a.counts[LIF_CNT_NUM_USED];
   const int t = a.counts[LIF_CNT_STEP];
   const int na = *a.n_act;
-  const int stale_before = t - a.k;   // last_active <= stale_before: outside the window
   u64 tot;
+  int bad = (na < 0 || na > a.F) ? 1 : 0;
+  int k_eff = a.k;
+  if (a.budget > 0) {
+    // age histogram of the cached rows, minus those that are active again now
+    __shared__ int hist[kMaxBudgetWindow + 1];
+    __shared__ int loads;
+    if (tid <= kMaxBudgetWindow) hist[tid] = 0;
+    if (tid == 0) loads = 0;
+    __syncthreads();
+    if (!bad) {
+      int c = 0;
+      for (int q = tid; q < na; q += kWindowThreads) {
+        const int id = a.act[q];
+        if (id < 0 || id >= a.F) continue;
+        if (a.slot_of[id] < 0) ++c;
+        else atomicSub(&hist[min(a.k, max(1, t - a.last_active[id]))], 1);
+      }
+      if (c) atomicAdd(&loads, c);
+      for (int s = tid; s < n; s += kWindowThreads)
+        atomicAdd(&hist[min(a.k, max(1, t - a.last_active[a.pointers[s]]))], 1);
+    }
+    __syncthreads();
+    k_eff = widest_window_that_fits(hist, a.k, n, loads, min(a.cap, a.budget));
+    __syncthreads();
+  }
+  const int limit = a.budget > 0 ? min(a.cap, a.budget) : a.cap;
+  const int stale_before = t - k_eff;   // last_active <= stale_before: outside the window
 
   // ---- A: what would happen ------------------------------------------------------------
-  int bad = (na < 0 || na > a.F) ? 1 : 0;
   int c_load = 0, c_back = 0, c_stale = 0;
   if (!bad) {
     for (int q = tid; q < na; q += kWindowThreads) {
@@ -95,7 +136,7 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   const int n_evict = field(tot, 2) - field(tot, 1);
   const int n_kept = n - n_evict;
 
-  if (any_bad || n_kept + n_load > a.cap) {
+  if (any_bad || n_kept + n_load > limit) {
     if (tid == 0) {
       if (a.counts[LIF_CNT_STATUS] == LIF_OK)
         a.counts[LIF_CNT_STATUS] = any_bad ? LIF_ERR_INVALID_ARG : LIF_ERR_CAPACITY;
@@ -194,6 +235,7 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
     a.counts[LIF_CNT_NUM_KEPT] = n_kept;
     a.counts[LIF_CNT_NUM_USED] = n_kept + n_load;
     a.counts[LIF_CNT_STEP] = t + 1;
+    a.counts[LIF_CNT_K_EFF] = k_eff;
     unsigned long long* totals = reinterpret_cast<unsigned long long*>(a.counts + CNT_TOTALS);
     totals[0] += (unsigned long long)n_load * a.bundle_bytes;
     totals[1] += (unsigned long long)n_moves;
@@ -251,7 +293,6 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
     window_update_generic(g, sc);
     return;
   }
-  const int stale_before = t - a.k;
 
   // ---- round trip 2: by neuron id (mine: bits of w) and by slot (mine: a contiguous run) ----
   int so[kPlanBits];
@@ -285,23 +326,44 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
     }
   }
   // ---- round trip 3: is each of my cached neurons still inside the window? ------------------
-  unsigned evm = 0;   // bit j: slot s0 + j is deleted
+  int age[kPlanSlots];          // steps since last active; 0 = active now
 #pragma unroll
-  for (int j = 0; j < kPlanSlots; ++j)
+  for (int j = 0; j < kPlanSlots; ++j) {
+    age[j] = 0;
     if (j < my_slots) {
       const int id = pid[j];
       const bool active_now = (bits[id >> 5] >> (id & 31)) & 1u;
-      if (!active_now && a.last_active[id] <= stale_before) evm |= 1u << j;
+      if (!active_now) age[j] = max(1, t - a.last_active[id]);
     }
+  }
   int c_load = 0;
 #pragma unroll
   for (int i = 0; i < kPlanBits; ++i) c_load += (i < cnt && so[i] < 0);
+  int k_eff = a.k;
+  if (a.budget > 0) {           // memory budget: shrink the window for this step if needed
+    __shared__ int hist[kMaxBudgetWindow + 1];
+    __shared__ int loads;
+    if (tid <= kMaxBudgetWindow) hist[tid] = 0;
+    if (tid == 0) loads = 0;
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < kPlanSlots; ++j)
+      if (age[j] > 0) atomicAdd(&hist[min(a.k, age[j])], 1);
+    if (c_load) atomicAdd(&loads, c_load);
+    __syncthreads();
+    k_eff = widest_window_that_fits(hist, a.k, n, loads, min(a.cap, a.budget));
+  }
+  const int limit = a.budget > 0 ? min(a.cap, a.budget) : a.cap;
+  unsigned evm = 0;             // bit j: slot s0 + j is deleted
+#pragma unroll
+  for (int j = 0; j < kPlanSlots; ++j)
+    if (age[j] >= k_eff) evm |= 1u << j;
   u64 pre = block_scan(pack3(c_load, __popc(evm), cnt - c_load), &tot, sc);
   const int n_load = field(tot, 0), n_evict = field(tot, 1);
   const int n_kept = n - n_evict;
   int p_load = field(pre, 0), p_ev = field(pre, 1), p_hit = field(pre, 2);
 
-  if (n_kept + n_load > a.cap) {            // refuse before anything is changed
+  if (n_kept + n_load > limit) {            // refuse before anything is changed
     if (tid == 0) {
       if (a.counts[LIF_CNT_STATUS] == LIF_OK) a.counts[LIF_CNT_STATUS] = LIF_ERR_CAPACITY;
       a.counts[LIF_CNT_N_ACTIVE] = 0;
@@ -394,6 +456,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
     a.counts[LIF_CNT_NUM_KEPT] = n_kept;
     a.counts[LIF_CNT_NUM_USED] = n_kept + n_load;
     a.counts[LIF_CNT_STEP] = t + 1;
+    a.counts[LIF_CNT_K_EFF] = k_eff;
     unsigned long long* totals = reinterpret_cast<unsigned long long*>(a.counts + CNT_TOTALS);
     totals[0] += (unsigned long long)n_load * a.bundle_bytes;
     totals[1] += (unsigned long long)n_moves;
@@ -466,6 +529,7 @@ static WindowArgs window_args(lif_layer* L, const int32_t* act, const int32_t* n
   a.F = D.d_ff;
   a.cap = D.capacity;
   a.k = D.window_k;
+  a.budget = D.budget_rows;
   a.bundle_bytes = 4ull * D.d_model;
   return a;
 }

@@ -42,7 +42,7 @@ class OracleLayer:
     """Oracle-side twin of one layer, fed with the same tensors."""
 
     def __init__(self, w, d_model, d_ff, capacity, window_k, theta=0.0, b_down=None,
-                 activation=0, act_threshold=0.0):
+                 activation=0, act_threshold=0.0, budget_rows=0):
         self.activation, self.act_threshold = activation, act_threshold
         self.A = w["A"].cpu().numpy().astype(np.float64)
         self.B = w["B"].cpu().numpy().astype(np.float64)
@@ -51,11 +51,11 @@ class OracleLayer:
         self.bias_up = w["bias_up"].cpu().numpy()
         self.b_down = None if b_down is None else b_down.cpu().numpy()
         self.theta = theta
-        self.cache = O.NeuronCache(d_model, d_ff, capacity, window_k)
+        self.cache = O.NeuronCache(d_model, d_ff, capacity, window_k, budget_rows)
 
 
 def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_down=False,
-                    activation=0, act_threshold=0.0, device="cuda:0"):
+                    activation=0, act_threshold=0.0, budget_rows=0, device="cuda:0"):
     store = R.pinned_store(cfg.d_ff, cfg.d_model)
     w = W.make_layer(cfg, layer_idx, device=device, bundles_out=store)
     cap = capacity or W.window_capacity(cfg, w["p"])
@@ -68,8 +68,10 @@ def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_d
                   capacity=cap, host_bundles=store, pred_A=dev(w["A"]), pred_B=dev(w["B"]),
                   pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), bias_down=bd,
                   n_streams=cfg.n_streams, threshold_logit=theta, ffn_mode=ffn_mode,
-                  activation=activation, activation_threshold=act_threshold, device=device)
-    ora = OracleLayer(w, cfg.d_model, cfg.d_ff, cap, cfg.window_k, theta, bd, activation, act_threshold)
+                  activation=activation, activation_threshold=act_threshold, budget_rows=budget_rows,
+                  device=device)
+    ora = OracleLayer(w, cfg.d_model, cfg.d_ff, cap, cfg.window_k, theta, bd, activation, act_threshold,
+                      budget_rows)
     return gpu, ora
 
 
@@ -78,7 +80,7 @@ def compare_lists_and_state(gpu, ora, ref_lists):
     assert g["status"] == B.LIF_OK
     for key in LIST_KEYS:
         np.testing.assert_array_equal(g[key], ref_lists[key], err_msg=key)
-    for key in ("num_used_before", "num_kept", "num_used"):
+    for key in ("num_used_before", "num_kept", "num_used", "k_eff"):
         assert g[key] == ref_lists[key], key
     c = ora.cache
     assert g["step"] == c.t
@@ -139,4 +141,4 @@ def staged_step(gpu, ora, x_dev, bufs, whole_cache=False):
                          ora.act_threshold)
     assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
     return dict(n_active=na, n_load=len(ref_lists["load_ids"]), n_evict=len(ref_lists["evict_ids"]),
-                n_border=n_border)
+                n_border=n_border, k_eff=ref_lists["k_eff"], num_used=ref_lists["num_used"])

@@ -268,3 +268,35 @@ def test_activation_variants(activation, thr, S):
     stats = _run_staged(cfg, 0, cfg.steps, b_down=True, activation=activation, act_threshold=thr,
                         capacity=2048)
     assert min(s["n_active"] for s in stats) > 100
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+def test_memory_budget_shrinks_the_window(fused):
+    # Appendix C (Persimmon 8B, Phi-2): a row budget below the natural window union forces
+    # the window to shrink on some steps.  fused = 0: staged entry points (general window
+    # kernel); fused = 1: lif_decode_step (mask-fed kernel).
+    cfg = W.LifConfig("budget", 1, 256, 4096, 16, 5, 1, 24, 0.05, 1.0, 0.5, 0.87, 15)
+    budget = 600
+    if not fused:
+        stats = _run_staged(cfg, 0, cfg.steps, budget_rows=budget, capacity=1024)
+        ks = [s["k_eff"] for s in stats]
+        assert max(s["num_used"] for s in stats) <= budget
+    else:
+        gpu, ora = P.make_layer_pair(cfg, 0, budget_rows=budget, capacity=1024)
+        X = W.make_inputs(cfg, device=DEV)
+        y = torch.empty(1, cfg.d_model, dtype=torch.float32, device=DEV)
+        sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+        ks = []
+        for t in range(cfg.steps):
+            B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+            g = gpu.lists()
+            _, _, lists, ref_y = O.decode_step(ora.cache, X[t].cpu().numpy(), ora.A, ora.B, ora.c, 0.0,
+                                               ora.bundles, ora.bias_up, act=g["active_idx"])
+            P.compare_lists_and_state(gpu, ora, lists)
+            P.compare_cache_rows(gpu, ora)
+            P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
+            assert g["num_used"] <= budget
+            ks.append(g["k_eff"])
+        gpu.close()
+    assert min(ks) < cfg.window_k and max(ks) == cfg.window_k, ks     # shrinks on some steps only

@@ -383,3 +383,51 @@ def test_fatrelu_threshold_only_removes_neurons():
     np.testing.assert_array_equal(O.activation_fn(pre, O.FATRELU, 0.7), [0, 0, 0, 0.70001, 3.0])
     np.testing.assert_array_equal(O.activation_fn(pre, O.RELU_SQUARED), [0, 0.2 ** 2, 0.7 ** 2, 0.70001 ** 2, 9.0])
     np.testing.assert_array_equal(O.activation_fn(pre), [0, 0.2, 0.7, 0.70001, 3.0])
+
+
+# ------------------------------------------------------------------ memory-budgeted window
+def test_budgeted_window_brute_force():
+    # Appendix C (Persimmon 8B, Phi-2): the window shrinks whenever the cache would pass the
+    # budget.  Brute force from the stored history of active sets and of what was cached.
+    F, T, k, budget = 300, 60, 5, 70
+    sets = _random_active_sets(F, T, 0.07, seed=31, sticky=0.3)
+    cache = O.NeuronCache(2, F, capacity=F, window_k=k, budget_rows=budget)
+    free = O.NeuronCache(2, F, capacity=F, window_k=k)
+    last_seen = {}
+    shrunk = 0
+    for t, act in enumerate(sets):
+        before = cache.cached_ids()
+        lists = cache.window_update(act)
+        free.window_update(act)
+        for i in act.tolist():
+            last_seen[i] = t
+        ke = lists["k_eff"]
+        assert 1 <= ke <= k
+        kept_expected = lambda kk: {i for i in before | set(act.tolist()) if last_seen[i] > t - kk}
+        assert cache.cached_ids() == kept_expected(ke)                  # exactly the k'-window
+        assert cache.num_used <= budget
+        if ke < k:                                                      # widest that fits
+            shrunk += 1
+            assert len(kept_expected(ke + 1)) > budget
+        assert set(act.tolist()) <= cache.cached_ids() <= free.cached_ids()
+        _check_structure(cache)
+    assert 5 < shrunk < T                                               # the budget really binds
+    # a budget nothing ever reaches changes nothing
+    a, b = O.NeuronCache(2, F, F, k, budget_rows=F), O.NeuronCache(2, F, F, k)
+    for act in sets[:20]:
+        la, lb = a.window_update(act), b.window_update(act)
+        assert la["k_eff"] == k
+        for key in ("evict_ids", "move_src", "load_ids", "active_slots"):
+            np.testing.assert_array_equal(la[key], lb[key])
+
+
+def test_budget_smaller_than_active_set_is_refused_unchanged():
+    cache = O.NeuronCache(2, 64, capacity=64, window_k=3, budget_rows=8)
+    cache.window_update(np.arange(6, dtype=np.int32))
+    snap = (cache.pointers.copy(), cache.last_active.copy(), cache.num_used, cache.t)
+    with pytest.raises(O.CapacityError):
+        cache.window_update(np.arange(20, 30, dtype=np.int32))           # 10 active > budget 8
+    assert (cache.pointers == snap[0]).all() and (cache.last_active == snap[1]).all()
+    assert (cache.num_used, cache.t) == snap[2:]
+    ls = cache.window_update(np.arange(20, 27, dtype=np.int32))          # 7 fit once the window is 1
+    assert ls["k_eff"] == 1 and cache.num_used == 7
