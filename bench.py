@@ -362,6 +362,57 @@ def run_kernel_loop(args):
         l.close()
 
 
+def run_sweep_k(args):
+    """Memory-latency trade-off (the paper's Section 4 figure of latency against the share of
+    the model kept in memory): one JSON line per window size k with tokens/s, the share of
+    the FFN resident in HBM and the bytes fetched per token."""
+    import torch
+    from paper_2312_11514_b200 import binding as B
+    from paper_2312_11514_b200 import runtime as R
+    from paper_2312_11514_b200 import workloads as W
+    dev = "cuda:0"
+    base = W.CONFIGS[args.config]
+    K, Wm = args.steps, args.warmup
+    for k in [int(v) for v in args.sweep_k.split(",")]:
+        cfg = base.scaled(window_k=k)
+        # small windows see the step-to-step swings of the active set undamped: wide margin
+        layers = R.build_stack(cfg, dev, n_layers=args.layers, capacity_margin=40.0)
+        handles = [l.handle for l in layers]
+        L, S, d = len(layers), cfg.n_streams, cfg.d_model
+        X = _inputs(cfg, Wm + K, dev, W)
+        Y = torch.empty(L, S, d, dtype=torch.float32, device=dev)
+        dev_x = torch.empty(S, d, dtype=torch.float16, device=dev)
+        sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+        graph = B.lif_graph_capture(handles, dev_x, Y, sc, sf)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for t in range(Wm + K):
+            if t == Wm:
+                torch.cuda.synchronize()
+                s0 = [B.lif_get_stats(h) for h in handles]
+                e0.record(sc)
+            with torch.cuda.stream(sc):
+                dev_x.copy_(X[t], non_blocking=True)
+            B.lif_graph_launch(graph, sc)
+        e1.record(sc)
+        torch.cuda.synchronize()
+        s1 = [B.lif_get_stats(h) for h in handles]
+        assert all(s.status == B.LIF_OK for s in s1), [B.status_str(s.status) for s in s1]
+        ms = e0.elapsed_time(e1)
+        fetched = sum(b.bytes_fetched - a.bytes_fetched for a, b in zip(s0, s1))
+        cached = sum(b.rows_cached - a.rows_cached for a, b in zip(s0, s1)) / (K * L)
+        print(json.dumps({"window_k": k, "tokens_per_s": K / (ms / 1e3), "ms_per_token": ms / K,
+                          "ffn_share_resident": cached / cfg.d_ff,
+                          "new_share_per_token": fetched / K / L / cfg.bundle_bytes / cfg.d_ff,
+                          "host_link_MB_per_token": fetched / K / 1e6, "layers": L,
+                          "config": cfg.name}), flush=True)
+        B.lif_graph_destroy(graph)
+        for l in layers:
+            l.close()
+        del layers, graph
+        torch.cuda.empty_cache()
+
+
 # ------------------------------------------------------------------------------ CPU oracle
 def _oracle_threads():
     try:
@@ -477,10 +528,14 @@ def main():
                     help="profiling aid: after the warm-up tokens launch this kernel once per layer "
                          "(predict_z, predict_scores, fetch, ffn_active, ffn_hits, ffn_new, ffn_sum; "
                          "ffn_api = lif_sparse_ffn over the active rows, for any number of streams)")
+    ap.add_argument("--sweep-k", default=None,
+                    help="comma-separated window sizes: memory-latency trade-off, one line per k")
     args = ap.parse_args()
     if args.warmup < 3:
         raise SystemExit("--warmup must be at least 3")
-    if args.kernel_loop:
+    if args.sweep_k:
+        run_sweep_k(args)
+    elif args.kernel_loop:
         run_kernel_loop(args)
     elif args.impl == "reference":
         run_reference(args)
