@@ -54,6 +54,14 @@ def active_set(logits, theta):
     return np.nonzero(mask)[0].astype(np.int32)
 
 
+def keep_tokens(logits, theta, act, keep):
+    """For a pass of consecutive tokens (rows of ``logits``): the last token j < keep in which
+    each neuron of ``act`` is active, -1 if none."""
+    m = np.asarray(logits)[:keep, :][:, act] > theta          # [keep][n_act]
+    last = np.where(m.any(axis=0), keep - 1 - np.argmax(m[::-1], axis=0), -1)
+    return last.astype(np.int64)
+
+
 def sigmoid_threshold_to_logit(tau):
     """theta = ln(tau / (1 - tau)); tau = 0.5 is the "positive output" rule."""
     return float(np.log(tau / (1.0 - tau)))
@@ -89,12 +97,27 @@ class NeuronCache:
         self.rows_moved = 0
 
     # -- delete + plan ------------------------------------------------------------------
-    def window_update(self, act):
+    def window_update(self, act, keep_token=None, keep=1):
         """One window step for the ascending active list ``act``.  Deletes the neurons that
         left the window (Section 3.3 item 1), and assigns rows to the ones to bring in
-        (item 2).  Returns the lists; the new rows' weights arrive with ``insert``."""
+        (item 2).  Returns the lists; the new rows' weights arrive with ``insert``.
+
+        Speculative decoding (Section 4, "Speculative Decoding"): the pass holds several
+        consecutive tokens and the window is updated with all of them at once, keeping the
+        last k tokens that end with token ``keep`` of the pass.  ``act`` is then the union
+        over the pass and ``keep_token[q]`` the last token j < keep in which neuron act[q] is
+        active, or -1 if it is active only in later tokens: such a neuron is needed for this
+        pass but does not enter the kept window, so it gets the oldest stamp still inside it.
+        Time advances by ``keep`` tokens."""
         act = np.asarray(act, dtype=np.int32)
-        t, k, n = self.t, self.k, self.num_used
+        k, n = self.k, self.num_used
+        if keep_token is None:
+            keep_token = np.zeros(len(act), dtype=np.int64)
+        keep_token = np.asarray(keep_token, dtype=np.int64)
+        assert keep >= 1 and len(keep_token) == len(act) and (keep_token < keep).all()
+        assert keep == 1 or self.budget_rows == 0
+        t0 = self.t
+        t = t0 + keep - 1                       # the kept window ends at this token
         in_act = np.zeros(self.d_ff, dtype=bool)
         in_act[act] = True
 
@@ -120,7 +143,9 @@ class NeuronCache:
             raise CapacityError(f"need {n_new + len(load_ids)} rows, have {limit}")
         self.k_eff = k
 
-        self.last_active[act] = t
+        stamps = np.where(keep_token >= 0, t0 + keep_token,
+                          np.maximum(self.last_active[act], t - k + 1))
+        self.last_active[act] = stamps
         evict_ids = [int(self.pointers[s]) for s in evict_slots]
 
         # Deleting: walk the freed rows in ascending order; the current last row replaces
@@ -155,7 +180,7 @@ class NeuronCache:
             self.pointers[s] = i
             self.slot_of[i] = s
         self.num_used = n_new + len(load_ids)
-        self.t = t + 1
+        self.t = t0 + keep
 
         active_slots = self.slot_of[act].astype(np.int32)
         hit_slots = active_slots[active_slots < n_new]
@@ -217,7 +242,7 @@ def sparse_ffn(matrix, bias, slots, x, b_down=None, activation=RELU, threshold=0
 
 
 def decode_step(cache, x, A, B, c, theta, bundles, bias_up, b_down=None, whole_cache=False,
-                act=None, activation=RELU, threshold=0.0):
+                act=None, activation=RELU, threshold=0.0, keep_token=None, keep=1):
     """One layer, one token: predict -> window update -> insert -> FFN.  ``act`` overrides the
     predicted active list (used to follow another implementation's borderline decisions).
     ``whole_cache`` runs the FFN over every cached row (matrix[:num_used]) instead of only the
@@ -225,7 +250,9 @@ def decode_step(cache, x, A, B, c, theta, bundles, bias_up, b_down=None, whole_c
     logits = predictor_logits(x, A, B, c)
     if act is None:
         act = active_set(logits, theta)
-    lists = cache.window_update(act)
+    if keep > 1 and keep_token is None:
+        keep_token = keep_tokens(logits, theta, act, keep)
+    lists = cache.window_update(act, keep_token, keep)
     cache.insert(lists, bundles, bias_up)
     slots = np.arange(cache.num_used) if whole_cache else lists["active_slots"]
     y = sparse_ffn(cache.matrix, cache.bias, slots, x, b_down, activation, threshold)

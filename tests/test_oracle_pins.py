@@ -431,3 +431,73 @@ def test_budget_smaller_than_active_set_is_refused_unchanged():
     assert (cache.num_used, cache.t) == snap[2:]
     ls = cache.window_update(np.arange(20, 27, dtype=np.int32))          # 7 fit once the window is 1
     assert ls["k_eff"] == 1 and cache.num_used == 7
+
+
+# ------------------------------------------------------------------ multi-token window update
+def _pass_info(sets, F, keep):
+    """Union and keep_token of a pass given its per-token active sets."""
+    union = sorted(set().union(*[set(a.tolist()) for a in sets]))
+    kt = [max([j for j in range(keep) if i in set(sets[j].tolist())], default=-1) for i in union]
+    return np.array(union, dtype=np.int32), np.array(kt)
+
+
+def test_multi_token_update_equals_sequential_updates_when_everything_is_kept():
+    # a pass of S <= k consecutive tokens, all kept: same cached set and same stamps as S
+    # single-token updates (Section 4, speculative decoding: the window is updated with
+    # several tokens at once)
+    F, k = 200, 5
+    sets = _random_active_sets(F, 24, 0.06, seed=41)
+    for S in (1, 2, 4):
+        multi, single = O.NeuronCache(2, F, F, k), O.NeuronCache(2, F, F, k)
+        for p in range(0, 24, S):
+            chunk = sets[p:p + S]
+            act, kt = _pass_info(chunk, F, S)
+            ls = multi.window_update(act, kt, keep=S)
+            for a in chunk:
+                single.window_update(a)
+            assert multi.t == single.t == p + S
+            assert multi.cached_ids() == single.cached_ids()
+            np.testing.assert_array_equal(multi.last_active, single.last_active)
+            assert [int(multi.pointers[s]) for s in ls["active_slots"]] == act.tolist()
+            _check_structure(multi)
+
+
+def test_multi_token_update_keeps_the_window_ending_at_the_kept_token():
+    # 5 tokens per pass (lambda = 4), keep the window ending with token m of the pass:
+    # brute force from the history of kept tokens
+    F, k, S, m = 300, 3, 5, 2
+    sets = _random_active_sets(F, 40, 0.05, seed=43)
+    cache = O.NeuronCache(2, F, F, k)
+    kept_history = []                                    # active sets of the kept tokens, in time order
+    for p in range(0, 40, S):
+        chunk = sets[p:p + S]
+        act, kt = _pass_info(chunk, F, m)
+        before = cache.cached_ids()
+        ls = cache.window_update(act, kt, keep=m)
+        kept_history += [set(a.tolist()) for a in chunk[:m]]
+        window = set().union(*kept_history[-k:])
+        needed_now = set(act.tolist())
+        assert cache.cached_ids() == (before & window) | needed_now | (window & needed_now)
+        assert cache.cached_ids() == ((before | needed_now) & window) | needed_now
+        assert cache.t == len(kept_history)
+        assert ls["load_ids"].tolist() == sorted(needed_now - before)
+        # a neuron active only beyond the kept token is dropped by the next pass unless needed again
+        late_only = needed_now - set().union(*[set(a.tolist()) for a in chunk[:m]]) - (before & window)
+        if p + S < 40:
+            nxt = sets[p + S:p + 2 * S]
+            act2, kt2 = _pass_info(nxt, F, m)
+            probe = O.NeuronCache(2, F, F, k)
+            probe.__dict__.update({k_: (v.copy() if isinstance(v, np.ndarray) else v)
+                                   for k_, v in cache.__dict__.items()})
+            probe.window_update(act2, kt2, keep=m)
+            assert not (late_only - set(act2.tolist())) & probe.cached_ids()
+        _check_structure(cache)
+
+
+def test_keep_tokens_helper():
+    logits = np.array([[1.0, -1, -1, 1], [-1, 1.0, -1, 1], [-1, -1, 1.0, -1]])
+    act = O.active_set(logits, 0.0)
+    assert act.tolist() == [0, 1, 2, 3]
+    assert O.keep_tokens(logits, 0.0, act, 3).tolist() == [0, 1, 2, 1]
+    assert O.keep_tokens(logits, 0.0, act, 2).tolist() == [0, 1, -1, 1]
+    assert O.keep_tokens(logits, 0.0, act, 1).tolist() == [0, -1, -1, 0]
