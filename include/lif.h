@@ -69,6 +69,13 @@ typedef struct {
                                the cache may hold, <= capacity.  When a step would pass it, that
                                step deletes with the widest window k' <= window_k (at least 1)
                                that fits; LIF_CNT_K_EFF reports k'.  Needs window_k <= 32. */
+  int32_t spec_keep;        /* 0 = off.  Speculative decoding (Section 4): the n_streams inputs of
+                               a step are consecutive tokens of one sequence and the window is
+                               updated with all of them at once, keeping the last window_k
+                               tokens that end with token spec_keep (1..n_streams) of the
+                               step; a neuron active only in later tokens is used by this
+                               step but gets the oldest stamp still inside the window.  The
+                               step counter advances by spec_keep.  Not with budget_rows. */
   const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][2*d_model] */
   const void* dev_pred_A;   /* fp16 [d_model][rank] */
   const void* dev_pred_B;   /* fp16 [rank][d_ff] */
@@ -121,6 +128,9 @@ typedef struct {
   int32_t* slot_of;
   int32_t* last_active;
   void* bias;
+  int8_t* keep_token;       /* [d_ff], spec_keep > 0 only: per neuron, the last token j <
+                               spec_keep of the step in which it is active, -1 if none; written
+                               by lif_predict, read by lif_window_update for the active ones */
 } lif_lists;
 
 typedef struct {

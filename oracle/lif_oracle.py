@@ -107,7 +107,8 @@ class NeuronCache:
         last k tokens that end with token ``keep`` of the pass.  ``act`` is then the union
         over the pass and ``keep_token[q]`` the last token j < keep in which neuron act[q] is
         active, or -1 if it is active only in later tokens: such a neuron is needed for this
-        pass but does not enter the kept window, so it gets the oldest stamp still inside it.
+        pass but does not enter the kept window, so it gets the oldest stamp still inside it
+        (as does a neuron whose kept token is already older than the window).
         Time advances by ``keep`` tokens."""
         act = np.asarray(act, dtype=np.int32)
         k, n = self.k, self.num_used
@@ -143,8 +144,10 @@ class NeuronCache:
             raise CapacityError(f"need {n_new + len(load_ids)} rows, have {limit}")
         self.k_eff = k
 
-        stamps = np.where(keep_token >= 0, t0 + keep_token,
-                          np.maximum(self.last_active[act], t - k + 1))
+        # no neuron used by this pass is deleted by it: stamps never fall below the oldest
+        # one still inside the kept window (only matters when the pass is longer than k)
+        stamps = np.maximum(np.where(keep_token >= 0, t0 + keep_token, self.last_active[act]),
+                            t - self.k + 1)
         self.last_active[act] = stamps
         evict_ids = [int(self.pointers[s]) for s in evict_slots]
 

@@ -36,6 +36,7 @@ Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max) {
   w.n_tmp = take(64);
   w.z_partial = take(z_ctas * S * d.rank * 4);
   w.mask_words = take(n_mask * 4);
+  w.keep_tok = take(d.spec_keep > 0 ? F : 0);
   w.h_rows = take(d.n_streams > 1 ? (size_t)kBatchedMaxKSplit * F * 8 * 4 : 0);
   size_t partial_rows = (size_t)ffn_grid_max;
   if (ffn_batched_supported(d) && (size_t)kBatchedMaxPartitions * S > partial_rows)
@@ -57,6 +58,8 @@ static lif_status check_shape(const lif_layer_desc* d) {
   if (d->n_streams < 1 || d->n_streams > kMaxStreams) return LIF_ERR_INVALID_ARG;
   if (d->ffn_mode != 0 && d->ffn_mode != 1) return LIF_ERR_INVALID_ARG;
   if (d->budget_rows < 0 || d->budget_rows > d->capacity) return LIF_ERR_INVALID_ARG;
+  if (d->spec_keep < 0 || d->spec_keep > d->n_streams) return LIF_ERR_INVALID_ARG;
+  if (d->spec_keep > 0 && d->budget_rows > 0) return LIF_ERR_INVALID_ARG;
   if (d->budget_rows > 0 && d->window_k > 32) return LIF_ERR_INVALID_ARG;
   if (d->activation < LIF_ACT_RELU || d->activation > LIF_ACT_FATRELU) return LIF_ERR_INVALID_ARG;
   if (d->activation == LIF_ACT_FATRELU && !(d->activation_threshold >= 0.f)) return LIF_ERR_INVALID_ARG;
@@ -138,6 +141,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
   L->n_tmp = (int32_t*)(b + ws.n_tmp);
   L->z_partial = (float*)(b + ws.z_partial);
   L->mask_words = (uint32_t*)(b + ws.mask_words);
+  L->keep_tok = desc->spec_keep > 0 ? (int8_t*)(b + ws.keep_tok) : nullptr;
   L->y_partial = (float*)(b + ws.y_partial);
   L->h_rows = (float*)(b + ws.h_rows);
 
@@ -483,6 +487,7 @@ lif_status lif_get_lists(lif_layer* L, lif_lists* o) {
   o->slot_of = L->slot_of;
   o->last_active = L->last_active;
   o->bias = L->bias;
+  o->keep_token = L->keep_tok;
   return LIF_OK;
 }
 

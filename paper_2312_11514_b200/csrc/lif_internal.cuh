@@ -34,7 +34,7 @@ struct Workspace {
   // offsets in bytes from the workspace base; every block 256-byte aligned
   size_t counts, pointers, slot_of, last_active, bias, active_idx, evict_ids, evict_slots,
       move_src, move_dst, load_ids, load_slots, active_slots, hit_slots, n_tmp, z_partial,
-      mask_words, h_rows, y_partial, total;
+      mask_words, keep_tok, h_rows, y_partial, total;
 };
 
 Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max);
@@ -52,6 +52,7 @@ struct lif_layer {
       *active_slots, *hit_slots, *n_tmp;
   float* z_partial;
   uint32_t* mask_words;
+  int8_t* keep_tok;   // [d_ff] last kept token per neuron (speculative mode)
   float* y_partial;
   float* h_rows;      // [K slices][d_ff][8] fp32: phase-A output of the multi-stream FFN
   // multi-stream (tensor-core) FFN configuration; fb_ok = 0: per-stream fallback

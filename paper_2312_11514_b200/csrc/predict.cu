@@ -131,7 +131,8 @@ __global__ void __launch_bounds__(kThreads)
 predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* __restrict__ B,
                       const float* __restrict__ c, float theta, int r, int F,
                       float* __restrict__ logits, uint32_t* mask_words, int* ticket,
-                      int* __restrict__ active_idx, int* __restrict__ n_active, int compact) {
+                      int* __restrict__ active_idx, int* __restrict__ n_active, int compact,
+                      int8_t* __restrict__ keep_tok, int keep) {
   extern __shared__ float zs[];                 // [S][r]
   __shared__ float red[16][kLogitTile];
   __shared__ int warp_sums[kThreads / 32];
@@ -190,6 +191,7 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
   }
 
   bool active = false;
+  int last_kept = -1;        // speculative mode: last token < keep in which the neuron is active
 #pragma unroll
   for (int s = 0; s < S; ++s) {
 #pragma unroll
@@ -202,9 +204,11 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
       v += my_c;
       if (logits) logits[(size_t)s * F + my_col] = v;
       active = active || (v > theta);
+      if (v > theta && s < keep) last_kept = s;
     }
     __syncthreads();
   }
+  if (keep_tok && tid < kLogitTile && my_col < F) keep_tok[my_col] = (int8_t)last_kept;
   if (tid < kLogitTile) {
     const unsigned m = __ballot_sync(0xffffffffu, active);
     if ((tid & 31) == 0) mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = m;
@@ -262,7 +266,8 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
   e = launch_k(predict_logits_kernel<S>, dim3(grid), dim3(kThreads), smem, st, L->use_pdl,
                (const float*)L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c,
                D.threshold_logit, D.rank, D.d_ff, logits, L->mask_words,
-               (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact);
+               (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
+               L->keep_tok, D.spec_keep);
   if (ev) tm_record(ev[2], st);
   return e;
 }
@@ -281,7 +286,7 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
                   (size_t)D.rank * sizeof(float), st, L->use_pdl, (const float*)L->z_partial,
                   L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit, D.rank,
                   D.d_ff, (float*)nullptr, L->mask_words, (int*)(L->counts + CNT_TICKET_PREDICT),
-                  (int*)L->active_idx, (int*)L->n_tmp, 1);
+                  (int*)L->active_idx, (int*)L->n_tmp, 1, L->keep_tok, D.spec_keep);
 }
 
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,

@@ -65,12 +65,25 @@ struct WindowArgs {
       *active_slots, *hit_slots;
   int F, cap, k;
   int budget;             // 0 = off; else rows the cache may hold (Appendix C memory budget)
+  // Speculative decoding (Section 4): the step holds consecutive tokens; the kept window ends
+  // with token `keep` of the step (keep = 1, keep_tok = nullptr: ordinary single-token update).
+  const int8_t* keep_tok; // [F] last kept token per neuron, -1 if active only in later tokens
+  int keep;
   unsigned long long bundle_bytes;
 };
 
 // Memory-budgeted window (Appendix C, Persimmon 8B / Phi-2): hist[a] = cached rows that are not
 // active now and were last active a steps ago (a = 1 .. k, older ones in bin k).  Returns the
 // widest window k' <= k for which the rows kept plus the rows to load fit `limit`, at least 1.
+// Stamp of an active neuron: the time of the last kept token in which it is active (its old
+// stamp if it is active only beyond the kept token), but never below the oldest stamp still
+// inside the window that ends at t_end: this step does not delete it, the next one may.
+__device__ __forceinline__ int active_stamp(const WindowArgs& a, int id, int t, int t_end) {
+  if (!a.keep_tok) return t;
+  const int j = a.keep_tok[id];
+  return max(j >= 0 ? t + j : a.last_active[id], t_end - a.k + 1);
+}
+
 constexpr int kMaxBudgetWindow = 32;
 __device__ __forceinline__ int widest_window_that_fits(const int* hist, int k, int n, int n_load,
                                                        int limit) {
@@ -89,6 +102,7 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   const int n = a.counts[LIF_CNT_NUM_USED];
   const int t = a.counts[LIF_CNT_STEP];
   const int na = *a.n_act;
+  const int t_end = t + a.keep - 1;   // the kept window ends at this token
   u64 tot;
   int bad = (na < 0 || na > a.F) ? 1 : 0;
   int k_eff = a.k;
@@ -105,18 +119,18 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
         const int id = a.act[q];
         if (id < 0 || id >= a.F) continue;
         if (a.slot_of[id] < 0) ++c;
-        else atomicSub(&hist[min(a.k, max(1, t - a.last_active[id]))], 1);
+        else atomicSub(&hist[min(a.k, max(1, t_end - a.last_active[id]))], 1);
       }
       if (c) atomicAdd(&loads, c);
       for (int s = tid; s < n; s += kWindowThreads)
-        atomicAdd(&hist[min(a.k, max(1, t - a.last_active[a.pointers[s]]))], 1);
+        atomicAdd(&hist[min(a.k, max(1, t_end - a.last_active[a.pointers[s]]))], 1);
     }
     __syncthreads();
     k_eff = widest_window_that_fits(hist, a.k, n, loads, min(a.cap, a.budget));
     __syncthreads();
   }
   const int limit = a.budget > 0 ? min(a.cap, a.budget) : a.cap;
-  const int stale_before = t - k_eff;   // last_active <= stale_before: outside the window
+  const int stale_before = t_end - k_eff;   // last_active <= stale_before: outside the window
 
   // ---- A: what would happen ------------------------------------------------------------
   int c_load = 0, c_back = 0, c_stale = 0;
@@ -152,7 +166,10 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   }
 
   // ---- B: stamp --------------------------------------------------------------------------
-  for (int q = tid; q < na; q += kWindowThreads) a.last_active[a.act[q]] = t;
+  for (int q = tid; q < na; q += kWindowThreads) {
+    const int id = a.act[q];
+    a.last_active[id] = active_stamp(a, id, t, t_end);
+  }
   __syncthreads();
 
   // ---- C: deleted rows (ascending slot) and surviving tail rows (descending slot) --------
@@ -234,7 +251,7 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
     a.counts[LIF_CNT_NUM_USED_BEFORE] = n;
     a.counts[LIF_CNT_NUM_KEPT] = n_kept;
     a.counts[LIF_CNT_NUM_USED] = n_kept + n_load;
-    a.counts[LIF_CNT_STEP] = t + 1;
+    a.counts[LIF_CNT_STEP] = t + a.keep;
     a.counts[LIF_CNT_K_EFF] = k_eff;
     unsigned long long* totals = reinterpret_cast<unsigned long long*>(a.counts + CNT_TOTALS);
     totals[0] += (unsigned long long)n_load * a.bundle_bytes;
@@ -274,6 +291,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
   pdl_trigger();
   const int n = a.counts[LIF_CNT_NUM_USED];
   const int t = a.counts[LIF_CNT_STEP];
+  const int t_end = t + a.keep - 1;   // the kept window ends at this token
   const uint32_t w = tid < nwords ? mask_words[tid] : 0u;
   const int cnt = __popc(w);
   bits[tid] = w;
@@ -333,7 +351,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
     if (j < my_slots) {
       const int id = pid[j];
       const bool active_now = (bits[id >> 5] >> (id & 31)) & 1u;
-      if (!active_now) age[j] = max(1, t - a.last_active[id]);
+      if (!active_now) age[j] = max(1, t_end - a.last_active[id]);
     }
   }
   int c_load = 0;
@@ -391,7 +409,10 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
   // ---- writes ---------------------------------------------------------------------------------
   {
     uint32_t m = w;
-    for (; m; m &= m - 1) a.last_active[tid * 32 + __ffs(m) - 1] = t;          // stamp
+    for (; m; m &= m - 1) {                                                    // stamp
+      const int id = tid * 32 + __ffs(m) - 1;
+      a.last_active[id] = active_stamp(a, id, t, t_end);
+    }
   }
 #pragma unroll
   for (int j = 0; j < kPlanSlots; ++j)
@@ -455,7 +476,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
     a.counts[LIF_CNT_NUM_USED_BEFORE] = n;
     a.counts[LIF_CNT_NUM_KEPT] = n_kept;
     a.counts[LIF_CNT_NUM_USED] = n_kept + n_load;
-    a.counts[LIF_CNT_STEP] = t + 1;
+    a.counts[LIF_CNT_STEP] = t + a.keep;
     a.counts[LIF_CNT_K_EFF] = k_eff;
     unsigned long long* totals = reinterpret_cast<unsigned long long*>(a.counts + CNT_TOTALS);
     totals[0] += (unsigned long long)n_load * a.bundle_bytes;
@@ -530,6 +551,8 @@ static WindowArgs window_args(lif_layer* L, const int32_t* act, const int32_t* n
   a.cap = D.capacity;
   a.k = D.window_k;
   a.budget = D.budget_rows;
+  a.keep_tok = D.spec_keep > 0 ? L->keep_tok : nullptr;
+  a.keep = D.spec_keep > 0 ? D.spec_keep : 1;
   a.bundle_bytes = 4ull * D.d_model;
   return a;
 }

@@ -18,7 +18,8 @@ class Layer:
                  pred_c: torch.Tensor, bias_up: torch.Tensor,
                  bias_down: Optional[torch.Tensor] = None, n_streams: int = 1,
                  threshold_logit: float = 0.0, ffn_mode: int = 0, activation: int = 0,
-                 activation_threshold: float = 0.0, budget_rows: int = 0, device="cuda:0"):
+                 activation_threshold: float = 0.0, budget_rows: int = 0, spec_keep: int = 0,
+                 device="cuda:0"):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2312_11514_b200 needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
@@ -32,7 +33,8 @@ class Layer:
         shape = dict(d_model=d_model, d_ff=d_ff, rank=rank, window_k=window_k, capacity=capacity,
                      n_streams=n_streams, threshold_logit=threshold_logit, ffn_mode=ffn_mode,
                      activation=activation, activation_threshold=activation_threshold,
-                     budget_rows=budget_rows)
+                     budget_rows=budget_rows, spec_keep=spec_keep)
+        self.spec_keep = spec_keep
         nbytes = B.lif_workspace_bytes(B.make_desc(**shape))
         self.workspace = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
         with torch.cuda.device(self.device):
@@ -64,6 +66,8 @@ class Layer:
             "last_active": self._view("last_active", F),
             "bias": self._view("bias", cap, torch.float16),
         }
+        if self.spec_keep > 0:
+            out["keep_token"] = self._view("keep_token", F, torch.int8)
         out = {k: v.cpu().numpy() for k, v in out.items()}
         out.update(num_used_before=int(c[B.CNT_NUM_USED_BEFORE]), num_kept=int(c[B.CNT_NUM_KEPT]),
                    num_used=int(c[B.CNT_NUM_USED]), step=int(c[B.CNT_STEP]), status=int(c[B.CNT_STATUS]),

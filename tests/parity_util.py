@@ -55,7 +55,7 @@ class OracleLayer:
 
 
 def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_down=False,
-                    activation=0, act_threshold=0.0, budget_rows=0, device="cuda:0"):
+                    activation=0, act_threshold=0.0, budget_rows=0, spec_keep=0, device="cuda:0"):
     store = R.pinned_store(cfg.d_ff, cfg.d_model)
     w = W.make_layer(cfg, layer_idx, device=device, bundles_out=store)
     cap = capacity or W.window_capacity(cfg, w["p"])
@@ -69,7 +69,7 @@ def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_d
                   pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), bias_down=bd,
                   n_streams=cfg.n_streams, threshold_logit=theta, ffn_mode=ffn_mode,
                   activation=activation, activation_threshold=act_threshold, budget_rows=budget_rows,
-                  device=device)
+                  spec_keep=spec_keep, device=device)
     ora = OracleLayer(w, cfg.d_model, cfg.d_ff, cap, cfg.window_k, theta, bd, activation, act_threshold,
                       budget_rows)
     return gpu, ora
@@ -98,6 +98,22 @@ def compare_cache_rows(gpu, ora):
     assert np.array_equal(bias.view(np.uint16), ora.cache.bias[:n].view(np.uint16))
 
 
+def keep_tokens_checked(gpu, act_gpu, ref_logits, theta):
+    """Speculative mode: the GPU's per-neuron last kept token, checked against the oracle's
+    scores (it may differ only where a score of a kept token is within BORDER of the
+    threshold); the oracle then continues from the GPU's values."""
+    keep = gpu.spec_keep
+    torch.cuda.synchronize()
+    kt_gpu = gpu._view("keep_token", gpu.d_ff, torch.int8).cpu().numpy().astype(np.int64)[act_gpu]
+    kt_ref = O.keep_tokens(ref_logits, theta, act_gpu, keep)
+    diff = np.nonzero(kt_gpu != kt_ref)[0]
+    if diff.size:
+        margin = np.abs(ref_logits[:keep][:, act_gpu[diff]] - theta).min(axis=0)
+        assert (margin < BORDER).all(), "kept-token index differs away from the threshold"
+    assert ((kt_gpu >= -1) & (kt_gpu < keep)).all()
+    return kt_gpu
+
+
 def make_bufs(gpu, device="cuda:0"):
     S, F, d = gpu.n_streams, gpu.d_ff, gpu.d_model
     return dict(logits=torch.empty(S, F, dtype=torch.float32, device=device),
@@ -120,8 +136,11 @@ def staged_step(gpu, ora, x_dev, bufs, whole_cache=False):
     act_gpu = act[:na].cpu().numpy()
     n_border = assert_mask_borderline(act_gpu, ref_logits, ora.theta)
 
+    kt, keep = None, 1
+    if gpu.spec_keep > 0:
+        kt, keep = keep_tokens_checked(gpu, act_gpu, ref_logits, ora.theta), gpu.spec_keep
     B.lif_window_update(gpu.handle, act, n_act)
-    ref_lists = ora.cache.window_update(act_gpu)
+    ref_lists = ora.cache.window_update(act_gpu, kt, keep)
     g = compare_lists_and_state(gpu, ora, ref_lists)
     np.testing.assert_array_equal(g["active_idx"], act_gpu)
 

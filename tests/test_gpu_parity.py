@@ -300,3 +300,36 @@ def test_memory_budget_shrinks_the_window(fused):
             ks.append(g["k_eff"])
         gpu.close()
     assert min(ks) < cfg.window_k and max(ks) == cfg.window_k, ks     # shrinks on some steps only
+
+
+@pytest.mark.parametrize("keep,fused", [(5, 0), (2, 0), (2, 1), (1, 1)])
+def test_speculative_multi_token_window(keep, fused):
+    # Section 4, speculative decoding: a step verifies lambda + 1 = 5 consecutive tokens; the
+    # window keeps the last k tokens ending with token `keep` of the step
+    S = 5
+    cfg = W.LifConfig("spec", 1, 256, 4096, 16, 3, S, 10, 0.03, 1.0, 0.8, 0.6, 16)
+    gpu, ora = P.make_layer_pair(cfg, 0, spec_keep=keep, capacity=2048)
+    Xs = W.make_inputs(cfg.scaled(n_streams=1, steps=cfg.steps * S), device=DEV)   # one sequence
+    X = Xs.reshape(cfg.steps, S, cfg.d_model).contiguous()                          # S tokens per step
+    if not fused:
+        bufs = P.make_bufs(gpu)
+        stats = [P.staged_step(gpu, ora, X[t], bufs) for t in range(cfg.steps)]
+        assert sum(s["n_evict"] for s in stats) > 0
+    else:
+        y = torch.empty(S, cfg.d_model, dtype=torch.float32, device=DEV)
+        sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+        for t in range(cfg.steps):
+            B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+            g = gpu.lists()
+            x_np = X[t].cpu().numpy()
+            logits = O.predictor_logits(x_np, ora.A, ora.B, ora.c)
+            P.assert_mask_borderline(g["active_idx"], logits, 0.0)
+            kt = P.keep_tokens_checked(gpu, g["active_idx"], logits, 0.0)
+            _, _, lists, ref_y = O.decode_step(ora.cache, x_np, ora.A, ora.B, ora.c, 0.0, ora.bundles,
+                                               ora.bias_up, act=g["active_idx"], keep_token=kt, keep=keep)
+            P.compare_lists_and_state(gpu, ora, lists)
+            P.compare_cache_rows(gpu, ora)
+            P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
+    assert gpu.lists()["step"] == cfg.steps * keep == ora.cache.t
+    gpu.close()
