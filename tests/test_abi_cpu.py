@@ -75,3 +75,29 @@ def test_create_layer_rejects_null_and_misaligned_pointers_on_the_host():
     assert B.lib().lif_destroy_layer(None) == B.LIF_ERR_INVALID_ARG
     assert B.lib().lif_decode_step(None, None, None, None, None) == B.LIF_ERR_INVALID_ARG
     assert B.lib().lif_probe_host_read(None, None, 0, 0, None) == B.LIF_ERR_INVALID_ARG
+
+
+def test_new_fields_are_validated_on_the_host():
+    ok = dict(n_streams=5, spec_keep=2)
+    assert B.lif_workspace_bytes(_shape(**ok)) > B.lif_workspace_bytes(_shape(n_streams=5))   # keep_token array
+    assert B.lif_workspace_bytes(_shape(budget_rows=128)) > 0
+    for bad in (dict(n_streams=4, spec_keep=5), dict(spec_keep=-1), dict(budget_rows=-3),
+                dict(budget_rows=512), dict(n_streams=4, spec_keep=2, budget_rows=100),
+                dict(window_k=40, budget_rows=100)):
+        with pytest.raises(B.LifError) as e:
+            B.lif_workspace_bytes(_shape(**bad))
+        assert e.value.code == B.LIF_ERR_INVALID_ARG, bad
+
+
+def test_graph_and_profiling_calls_reject_null_handles():
+    lib = B.lib()
+    out = C.c_void_p(None)
+    assert lib.lif_graph_capture(None, 0, None, None, None, None, C.byref(out)) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_graph_capture(None, 0, None, None, None, None, None) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_graph_launch(None, None) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_graph_launch_host(None, None, None, None) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_graph_destroy(None) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_profile_launch(None, 0, None, None, None) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_set_tuning(None, 0, 0) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_timing_enable(None, 1) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_sparse_ffn_static(None, None, None, None, None, None, None, 256, None) == B.LIF_ERR_INVALID_ARG
