@@ -278,6 +278,22 @@ lif_status lif_get_lists(lif_layer* layer, lif_lists* host_out);
 /* Synchronises the device, then reports counts, cumulative traffic and the status word. */
 lif_status lif_get_stats(lif_layer* layer, lif_stats* host_out);
 
+/* Host copies of the window state (any pointer may be NULL): pointers[capacity],
+ * slot_of[d_ff], last_active[d_ff], num_used[1].  Synchronises the device. */
+lif_status lif_read_state(lif_layer* layer, int32_t* host_pointers, int32_t* host_slot_of,
+                          int32_t* host_last_active, int32_t* host_num_used);
+
+/* Checkpoint / resume of one layer's window.  A snapshot holds the bookkeeping of Section 3.3
+ * (counters including the step, pointers, slot_of, last_active, bias), not the cached rows:
+ * lif_restore copies it back and re-reads rows 0..num_used-1 from the host bundle store, so a
+ * restored layer continues exactly as the snapshotted one would have.  Both synchronise the
+ * device; the buffer is plain host memory of at least lif_snapshot_bytes() bytes and is only
+ * valid for a layer of the same description.  LIF_ERR_STATE: the buffer's counters do not fit
+ * this layer. */
+lif_status lif_snapshot_bytes(lif_layer* layer, size_t* out_bytes);
+lif_status lif_snapshot(lif_layer* layer, void* host_buf, size_t bytes);
+lif_status lif_restore(lif_layer* layer, const void* host_buf, size_t bytes);
+
 /* Clears the sticky device status word. */
 lif_status lif_clear_status(lif_layer* layer, void* stream);
 

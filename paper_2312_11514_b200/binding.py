@@ -25,6 +25,7 @@ EXPORTS = [
     "lif_probe_host_read", "lif_timing_enable", "lif_timing_read",
     "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
     "lif_sparse_ffn_static", "lif_set_tuning", "lif_profile_launch",
+    "lif_read_state", "lif_snapshot_bytes", "lif_snapshot", "lif_restore",
 ]
 KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ffn_new", "ffn_sum")
 (TUNE_DEPENDENT_LAUNCH, TUNE_SPLIT_FFN, TUNE_FETCH_CTAS, TUNE_FFN_CTAS, TUNE_FFN_STAGES,
@@ -99,6 +100,10 @@ def lib() -> C.CDLL:
         "lif_graph_destroy": [vp],
         "lif_sparse_ffn_static": [vp, vp, vp, vp, vp, vp, vp, i32, vp],
         "lif_set_tuning": [vp, i32, i32],
+        "lif_read_state": [vp, vp, vp, vp, vp],
+        "lif_snapshot_bytes": [vp, C.POINTER(sz)],
+        "lif_snapshot": [vp, vp, sz],
+        "lif_restore": [vp, vp, sz],
         "lif_profile_launch": [vp, i32, vp, vp, vp],
         "lif_timing_enable": [vp, i32],
         "lif_timing_read": [vp, C.POINTER(C.c_float), C.POINTER(i32)],
@@ -272,3 +277,23 @@ def lif_set_tuning(layer: int, key: int, value: int) -> None:
 def lif_profile_launch(layer: int, kernel: int, x, y, stream=None) -> None:
     _check(lib().lif_profile_launch(layer, kernel, _ptr(x), _ptr(y), _stream(stream)),
            "lif_profile_launch")
+
+
+def lif_read_state(layer: int, pointers=None, slot_of=None, last_active=None, num_used=None) -> None:
+    """Arguments are host int32 numpy arrays (or None)."""
+    ptr = lambda a: None if a is None else a.ctypes.data
+    _check(lib().lif_read_state(layer, ptr(pointers), ptr(slot_of), ptr(last_active), ptr(num_used)),
+           "lif_read_state")
+
+
+def lif_snapshot(layer: int) -> bytes:
+    n = C.c_size_t(0)
+    _check(lib().lif_snapshot_bytes(layer, C.byref(n)), "lif_snapshot_bytes")
+    buf = C.create_string_buffer(n.value)
+    _check(lib().lif_snapshot(layer, C.cast(buf, C.c_void_p), n.value), "lif_snapshot")
+    return buf.raw
+
+
+def lif_restore(layer: int, snapshot: bytes) -> None:
+    buf = C.create_string_buffer(snapshot, len(snapshot))
+    _check(lib().lif_restore(layer, C.cast(buf, C.c_void_p), len(snapshot)), "lif_restore")

@@ -491,6 +491,95 @@ lif_status lif_get_lists(lif_layer* L, lif_lists* o) {
   return LIF_OK;
 }
 
+// Window state that a snapshot holds, in this order: counts block, pointers, slot_of,
+// last_active, bias.  The cache rows are not part of it: they are re-read from the host store.
+namespace {
+struct StatePart {
+  void* dev;
+  size_t bytes;
+};
+int state_parts(lif_layer* L, StatePart* p) {
+  const size_t F = L->desc.d_ff, cap = L->desc.capacity;
+  p[0] = {L->counts, LIF_CNT_LEN * 4};
+  p[1] = {L->pointers, cap * 4};
+  p[2] = {L->slot_of, F * 4};
+  p[3] = {L->last_active, F * 4};
+  p[4] = {L->bias, cap * 2};
+  return 5;
+}
+}  // namespace
+
+lif_status lif_read_state(lif_layer* L, int32_t* host_pointers, int32_t* host_slot_of,
+                          int32_t* host_last_active, int32_t* host_num_used) {
+  if (!L) return LIF_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return LIF_ERR_CUDA;
+  const size_t F = L->desc.d_ff, cap = L->desc.capacity;
+  bool ok = true;
+  if (host_pointers)
+    ok = ok && cudaMemcpy(host_pointers, L->pointers, cap * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (host_slot_of)
+    ok = ok && cudaMemcpy(host_slot_of, L->slot_of, F * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (host_last_active)
+    ok = ok && cudaMemcpy(host_last_active, L->last_active, F * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (host_num_used)
+    ok = ok && cudaMemcpy(host_num_used, L->counts + LIF_CNT_NUM_USED, 4, cudaMemcpyDeviceToHost) ==
+                   cudaSuccess;
+  if (!ok) cudaGetLastError();
+  return ok ? LIF_OK : LIF_ERR_CUDA;
+}
+
+lif_status lif_snapshot_bytes(lif_layer* L, size_t* out_bytes) {
+  if (!L || !out_bytes) return LIF_ERR_INVALID_ARG;
+  StatePart p[5];
+  size_t total = 0;
+  for (int i = 0, n = state_parts(L, p); i < n; ++i) total += p[i].bytes;
+  *out_bytes = total;
+  return LIF_OK;
+}
+
+lif_status lif_snapshot(lif_layer* L, void* host_buf, size_t bytes) {
+  size_t need = 0;
+  if (!L || !host_buf || lif_snapshot_bytes(L, &need) != LIF_OK || bytes < need)
+    return LIF_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return LIF_ERR_CUDA;
+  StatePart p[5];
+  unsigned char* out = (unsigned char*)host_buf;
+  for (int i = 0, n = state_parts(L, p); i < n; ++i) {
+    if (cudaMemcpy(out, p[i].dev, p[i].bytes, cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaGetLastError();
+      return LIF_ERR_CUDA;
+    }
+    out += p[i].bytes;
+  }
+  return LIF_OK;
+}
+
+lif_status lif_restore(lif_layer* L, const void* host_buf, size_t bytes) {
+  size_t need = 0;
+  if (!L || !host_buf || lif_snapshot_bytes(L, &need) != LIF_OK || bytes < need)
+    return LIF_ERR_INVALID_ARG;
+  // a snapshot of another shape or a damaged one: check the counters it carries
+  const int32_t* cnt = (const int32_t*)host_buf;
+  if (cnt[LIF_CNT_NUM_USED] < 0 || cnt[LIF_CNT_NUM_USED] > L->desc.capacity ||
+      cnt[LIF_CNT_STEP] < 0)
+    return LIF_ERR_STATE;
+  if (cudaDeviceSynchronize() != cudaSuccess) return LIF_ERR_CUDA;
+  StatePart p[5];
+  const unsigned char* in = (const unsigned char*)host_buf;
+  for (int i = 0, n = state_parts(L, p); i < n; ++i) {
+    if (cudaMemcpy(p[i].dev, in, p[i].bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaGetLastError();
+      return LIF_ERR_CUDA;
+    }
+    in += p[i].bytes;
+  }
+  if (launch_refill(L, 0) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+    cudaGetLastError();
+    return LIF_ERR_CUDA;
+  }
+  return LIF_OK;
+}
+
 lif_status lif_get_stats(lif_layer* L, lif_stats* o) {
   if (!L || !o) return LIF_ERR_INVALID_ARG;
   int32_t host[LIF_CNT_LEN];

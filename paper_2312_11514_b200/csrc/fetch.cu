@@ -64,7 +64,22 @@ probe_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n_chunk
   gather_rows(src, dst, nullptr, nullptr, n_chunks, chunk_vec);
 }
 
+// Refill after a restore: cache row s <- bundle pointers[s] for s < num_used.
+__global__ void __launch_bounds__(kThreads)
+refill_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
+              const int32_t* __restrict__ pointers, const int32_t* __restrict__ counts,
+              int row_vec) {
+  gather_rows(store, cache, pointers, nullptr, counts[LIF_CNT_NUM_USED], row_vec);
+}
+
 }  // namespace
+
+cudaError_t launch_refill(lif_layer* L, cudaStream_t st) {
+  refill_kernel<<<L->fetch_grid, kThreads, 0, st>>>((const uint4*)L->dev_bundles,
+                                                    (uint4*)L->desc.dev_cache, L->pointers,
+                                                    L->counts, L->desc.d_model / 4);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st) {
   return launch_k(fetch_kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl,

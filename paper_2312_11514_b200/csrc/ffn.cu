@@ -8,6 +8,8 @@
 // axpy the down half into fp32 register accumulators.  Rows whose ReLU is zero skip the axpy.
 // CTA partials go to a [G][d] fp32 scratch; a second kernel adds them in CTA order, so the
 // result does not depend on scheduling.  Bound: HBM bandwidth, 4*d_model bytes per row.
+#include <mutex>
+
 #include "lif_internal.cuh"
 
 namespace lif {
@@ -446,6 +448,7 @@ struct StaticDevice {
   int n_sm, max_smem;
 };
 StaticDevice g_static_dev[kStaticMaxDevices];
+std::mutex g_static_mutex;
 
 }  // namespace
 }  // namespace lif
@@ -468,6 +471,7 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
   if (cudaGetDevice(&dev) != cudaSuccess) return LIF_ERR_CUDA;
   if (dev < 0 || dev >= kStaticMaxDevices) return LIF_ERR_STATE;
   StaticDevice& sd = g_static_dev[dev];
+  std::lock_guard<std::mutex> setup_lock(g_static_mutex);   // first calls from several threads
   if (!sd.ready) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess ||

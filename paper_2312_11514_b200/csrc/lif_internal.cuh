@@ -106,6 +106,7 @@ cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = 
 cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st,
                           cudaEvent_t* ev = nullptr);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
+cudaError_t launch_refill(lif_layer* L, cudaStream_t st);
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,
                          int grid, cudaStream_t st);
 // slots == nullptr: rows base[0] .. base[0] + n[0] (base == nullptr: 0)

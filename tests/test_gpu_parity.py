@@ -333,3 +333,45 @@ def test_speculative_multi_token_window(keep, fused):
             P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
     assert gpu.lists()["step"] == cfg.steps * keep == ora.cache.t
     gpu.close()
+
+
+def test_snapshot_restore_resumes_bit_identically():
+    cfg = W.CONFIGS["tiny"]
+    X = W.make_inputs(cfg, device=DEV)
+    gpu, ora = P.make_layer_pair(cfg, 0)
+    y = torch.empty(cfg.steps, 1, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    def run(t0, t1):
+        out = []
+        for t in range(t0, t1):
+            B.lif_decode_step(gpu.handle, X[t], y[t], sc, sf)
+            out.append(gpu.lists())
+        return out, y[t0:t1].cpu().numpy().copy()
+    run(0, 10)
+    snap = B.lif_snapshot(gpu.handle)
+    # read_state agrees with the device views
+    ptr = np.empty(gpu.capacity, dtype=np.int32); so = np.empty(cfg.d_ff, dtype=np.int32)
+    la = np.empty(cfg.d_ff, dtype=np.int32); nu = np.empty(1, dtype=np.int32)
+    B.lif_read_state(gpu.handle, ptr, so, la, nu)
+    g = gpu.lists()
+    np.testing.assert_array_equal(ptr, g["pointers"]); np.testing.assert_array_equal(so, g["slot_of"])
+    np.testing.assert_array_equal(la, g["last_active"]); assert nu[0] == g["num_used"]
+    first_lists, first_y = run(10, 20)
+    # wreck the device state and cache, then restore and replay
+    B.lif_reset(gpu.handle)
+    gpu.cache.zero_()
+    torch.cuda.synchronize()
+    B.lif_restore(gpu.handle, snap)
+    assert gpu.lists()["step"] == 10
+    again_lists, again_y = run(10, 20)
+    assert np.array_equal(first_y.view(np.uint32), again_y.view(np.uint32))
+    for a, b in zip(first_lists, again_lists):
+        for key in ("active_idx", "load_ids", "evict_ids", "move_src", "active_slots", "pointers", "last_active"):
+            np.testing.assert_array_equal(a[key], b[key], err_msg=key)
+    # a snapshot whose counters do not fit is refused
+    bad = bytearray(snap); bad[B.CNT_NUM_USED * 4:B.CNT_NUM_USED * 4 + 4] = (10 ** 6).to_bytes(4, "little")
+    with pytest.raises(B.LifError) as e:
+        B.lif_restore(gpu.handle, bytes(bad))
+    assert e.value.code == B.LIF_ERR_STATE
+    gpu.close()
