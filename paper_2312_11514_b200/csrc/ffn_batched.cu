@@ -255,8 +255,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     for (int i = 0; i < stages; ++i) mbar_init(bars + i, kGroup);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  pdl_wait();
-  pdl_trigger();
+  // This kernel always follows ffn_batched_up_kernel on its stream and depends on it only
+  // through H.  Rows, slots and counters were final before that kernel passed its own
+  // dependency wait (it signals its dependents only afterwards), so they are read, and the
+  // first copies issued, before the wait below: the prologue overlaps the up kernel's tail.
   const int n = *a.n;
   const int base = a.base ? *a.base : 0;
   const int P = a.partitions;
@@ -297,6 +299,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     for (int ks = 0; ks < a.ksplit; ++ks) v += a.H[(size_t)ks * a.h_stride + at];
     return apply_activation(v, a.act, a.act_thr);
   };
+  pdl_wait();                                      // H is complete from here on
+  pdl_trigger();
   float h_next = 0.f;
   if (tid < 128 && hk < my_cnt) h_next = load_h(hk);
 
