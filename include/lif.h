@@ -267,6 +267,8 @@ enum {
                                     fewer stages let several CTAs share an SM */
   LIF_TUNE_BATCHED_COLUMN_PARTS = 5, /* (fewest that fit) column parts of the multi-stream FFN's
                                     down-projection kernel, 1..16 */
+  LIF_TUNE_BATCHED_UP_TWO_CTAS = 7, /* (0) multi-stream FFN, up-projection kernel: two light CTAs
+                                    per SM instead of one with a deep ring */
   LIF_TUNE_FUSED_PLAN = 6        /* (1 when d_ff <= 32768) lif_decode_step: the window update
                                     reads the predictor's bit mask instead of its index list */
 };

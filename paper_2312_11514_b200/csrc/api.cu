@@ -149,6 +149,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
   bool ok = cudaGetDevice(&dev) == cudaSuccess &&
             cudaDeviceGetAttribute(&L->n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
   ok = ok && ffn_configure(L) == cudaSuccess;
+  L->fb_up_two_ctas = 0;
   ok = ok && ffn_batched_configure(L) == cudaSuccess;
   if (ok) {
     L->z_ctas = z_cta_count(desc->d_model);
@@ -462,6 +463,9 @@ lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
     case LIF_TUNE_BATCHED_COLUMN_PARTS:
       if (value < 1 || value > 16) return LIF_ERR_INVALID_ARG;
       L->fb_parts_min = value;
+      return ffn_batched_configure(L) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+    case LIF_TUNE_BATCHED_UP_TWO_CTAS:
+      L->fb_up_two_ctas = value != 0;
       return ffn_batched_configure(L) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
     case LIF_TUNE_FFN_STAGES:
       if (value < 1 || value > L->ffn_stages_max) return LIF_ERR_INVALID_ARG;

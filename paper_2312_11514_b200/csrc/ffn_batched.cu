@@ -25,8 +25,8 @@ constexpr int kGroupA = 16;               // rows per MMA in phase A (M = 16)
 // One mbarrier per group of 16 ring stages (the first stage's): arrival count 16, one arrival
 // per stage — with the stage's byte count where a row is copied, plain where the list has ended.
 constexpr int kGroup = 16;
-__device__ __forceinline__ uint64_t* group_bar(uint64_t* bars, int stage) {
-  return bars + (stage / kGroup) * kGroup;
+__device__ __forceinline__ uint64_t* group_bar(uint64_t* bars, int stage, int group = kGroup) {
+  return bars + (stage / group) * group;
 }
 constexpr int kMaxTilesPerWarp = 28;      // 16-column tiles per warp in phase B
 constexpr int kRowCacheA = 512;           // rows per CTA whose slot and bias are preloaded (phase A)
@@ -97,6 +97,7 @@ struct BatchedArgs {
   int32_t* status;
   int d, S, stages, parts, partitions, cols_per_part;
   int ksplit, k_per_split, up_partitions;   // phase A: K slices (columns, multiple of 16)
+  int up_group;                             // phase A: rows per group (8 or 16; MMA M is 16)
   size_t h_stride;
   int act;                // LIF_ACT_*
   float act_thr;
@@ -107,7 +108,7 @@ __device__ __forceinline__ int row_slot(const BatchedArgs& a, int q, int base) {
 }
 
 // ---- phase A: partial pre-activations  Hp[slice][q][s] = <Up[q, slice], x[s, slice]> (+ bias) --
-__global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int d = a.d;
   const int ks = blockIdx.x % a.ksplit, prt = blockIdx.x / a.ksplit;
@@ -115,7 +116,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
   const int kcols = min(a.k_per_split, d - k0);
   const unsigned seg_bytes = 2u * kcols;
   const unsigned pitch = 2u * a.k_per_split + kPad;
-  const int stages = a.stages;                          // multiple of kGroupA, two groups or more
+  const int stages = a.stages;                          // multiple of the group size
+  const int G = a.up_group;                             // rows per group: 8 or 16
   unsigned char* xs = smem;                                  // [8][pitch]
   unsigned char* rows = xs + 8 * (size_t)pitch;              // [stages][pitch]
   uint64_t* bars = reinterpret_cast<uint64_t*>(rows + (size_t)stages * pitch);
@@ -126,7 +128,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
-    for (int i = 0; i < stages; ++i) mbar_init(bars + i, kGroup);
+    for (int i = 0; i < stages; ++i) mbar_init(bars + i, G);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -146,15 +148,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
     const int slot = row_slot(a, prt + i * P, base);
     slot_all[i] = slot;
     if (i < stages) {
-      mbar_expect_tx(group_bar(bars, i), seg_bytes);
+      mbar_expect_tx(group_bar(bars, i, G), seg_bytes);
       bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * 2 * d + k0, seg_bytes,
-               group_bar(bars, i));
+               group_bar(bars, i, G));
     }
     const float b = ks == 0 ? __half2float(a.bias[slot]) : 0.f;
     bias_all[i] = b;
     if (i < stages) bias_s[i] = b;
   }
-  for (int i = my_cnt + tid; i < stages; i += kThreads) mbar_arrive(group_bar(bars, i));
+  for (int i = my_cnt + tid; i < stages; i += kThreads) mbar_arrive(group_bar(bars, i, G));
   {
     const int vec = kcols >> 3;
     for (int i = tid; i < 8 * vec; i += kThreads) {
@@ -173,16 +175,17 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
   const unsigned char* xb = xs + (size_t)gq * pitch + tq * 4;            // B: stream gq
   // A (16 rows x 16 columns): lane supplies row (lane % 8) + 8 * (lane / 8 % 2), columns
   // 8 * (lane / 16) of the k-step
-  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+  // (with 8-row groups the upper half of the tile repeats the lower one; its results are unused)
+  const int a_row = (lane & 7) + (G == 16 ? ((lane >> 3) & 1) * 8 : 0);
   const int a_off = (lane >> 4) * 16;
   float* Hp = a.H + (size_t)ks * a.h_stride;
   int timed_out = 0;
-  const int n_groups = (my_cnt + kGroupA - 1) / kGroupA;
-  const int groups_in_ring = stages / kGroupA;
+  const int n_groups = (my_cnt + G - 1) / G;
+  const int groups_in_ring = stages / G;
   for (int g = 0; g < n_groups; ++g) {
-    const int st0 = (g % groups_in_ring) * kGroupA;
+    const int st0 = (g % groups_in_ring) * G;
     const unsigned parity = (unsigned)(g / groups_in_ring) & 1u;
-    const int valid = min(kGroupA, my_cnt - g * kGroupA);
+    const int valid = min(G, my_cnt - g * G);
     if (!mbar_wait(bars + st0, parity)) timed_out = 1;
     // D[row][stream] over this warp's part of the slice
     float c[4] = {0.f, 0.f, 0.f, 0.f};
@@ -205,21 +208,21 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_up_kernel(BatchedArgs
       __syncthreads();
       return;
     }
-    if (tid < 8 * kGroupA) {
+    if (tid < 8 * G) {
       const int r = tid >> 3, s = tid & 7;              // row in group, stream
       if (r < valid) {
         const int src = ((r & 7) * 4 + (s >> 1)) * 4 + (r >> 3) * 2 + (s & 1);
         float v = 0.f;
 #pragma unroll
         for (int w = 0; w < 8; ++w) v += red[w * 128 + src];
-        const int q = prt + (g * kGroupA + r) * P;
+        const int q = prt + (g * G + r) * P;
         Hp[(size_t)q * 8 + s] = v + bias_s[st0 + r];
       }
     }
     __syncthreads();                                    // stages st0.. , bias_s and red are free
     // refill with the rows of group g + groups_in_ring
-    if (tid < kGroupA) {
-      const int i = (g + groups_in_ring) * kGroupA + tid;
+    if (tid < G) {
+      const int i = (g + groups_in_ring) * G + tid;
       if (i < my_cnt) {
         const bool cached = i < kRowCacheA;
         const int slot = cached ? slot_all[i] : row_slot(a, prt + i * P, base);
@@ -410,13 +413,22 @@ cudaError_t ffn_batched_configure(lif_layer* L) {
       if (found) break;
     }
   if (!found) return cudaSuccess;                  // fall back to the per-stream path
+  // A CTA keeps only about 6-8 bulk copies in flight, so with short row slices two lighter
+  // CTAs per SM (ring of two 8-row groups) move more bytes than one CTA with a deep ring.
+  int up_group = kGroupA, up_ctas = 1;
+  if (L->fb_up_two_ctas && ksplit > 1 && 2 * (up_smem(kps, 16) + 1024) <= (size_t)max_smem) {
+    up_group = 8;
+    up_ctas = 2;
+    st = 16;
+  }
   int parts = L->fb_parts_min > 0 ? L->fb_parts_min : 1;
   while ((tiles + parts - 1) / parts > 8 * kMaxTilesPerWarp ||
          down_smem((tiles + parts - 1) / parts * 16, 32) > (size_t)max_smem)
     ++parts;
   L->fb_ksplit = ksplit;
   L->fb_kps = kps;
-  L->fb_up_partitions = L->n_sm / ksplit > 0 ? L->n_sm / ksplit : 1;
+  L->fb_up_group = up_group;
+  L->fb_up_partitions = L->n_sm * up_ctas / ksplit > 0 ? L->n_sm * up_ctas / ksplit : 1;
   L->fb_up_stages = st;
   L->fb_up_smem = up_smem(kps, st);
   L->fb_parts = parts;
@@ -455,6 +467,7 @@ cudaError_t launch_ffn_batched(lif_layer* L, const __half* x, const int32_t* slo
   a.ksplit = L->fb_ksplit;
   a.k_per_split = L->fb_kps;
   a.up_partitions = L->fb_up_partitions;
+  a.up_group = L->fb_up_group;
   a.h_stride = (size_t)D.d_ff * 8;
   a.act = D.activation;
   a.act_thr = D.activation_threshold;

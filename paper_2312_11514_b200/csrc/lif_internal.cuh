@@ -57,7 +57,7 @@ struct lif_layer {
   float* h_rows;      // [K slices][d_ff][8] fp32: phase-A output of the multi-stream FFN
   // multi-stream (tensor-core) FFN configuration; fb_ok = 0: per-stream fallback
   int fb_ok, fb_up_stages, fb_parts, fb_cols, fb_partitions;
-  int fb_ksplit, fb_kps, fb_up_partitions, fb_parts_min;
+  int fb_ksplit, fb_kps, fb_up_partitions, fb_parts_min, fb_up_group, fb_up_two_ctas;
   size_t fb_up_smem, fb_down_smem;
   int n_sm;
   int z_ctas;         // CTAs of the first predictor stage
