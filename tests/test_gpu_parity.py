@@ -375,3 +375,15 @@ def test_snapshot_restore_resumes_bit_identically():
         B.lif_restore(gpu.handle, bytes(bad))
     assert e.value.code == B.LIF_ERR_STATE
     gpu.close()
+
+
+def test_window_longer_than_the_sequence_never_evicts():
+    cfg = W.LifConfig("longwin", 1, 256, 2048, 16, 64, 1, 10, 0.04, 1.0, 0.8, 0.6, 17)
+    gpu, ora = P.make_layer_pair(cfg, 0, capacity=2048)
+    X = W.make_inputs(cfg, device=DEV)
+    bufs = P.make_bufs(gpu)
+    stats = [P.staged_step(gpu, ora, X[t], bufs) for t in range(cfg.steps)]
+    assert sum(s["n_evict"] for s in stats) == 0 and B.lif_get_stats(gpu.handle).rows_moved == 0
+    used = [s["num_used"] for s in stats]
+    assert used == sorted(used) and used[-1] > used[0]                # the cache only grows
+    gpu.close()
