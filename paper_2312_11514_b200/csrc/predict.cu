@@ -126,7 +126,8 @@ __device__ __forceinline__ int block_exclusive_scan_256(int v, int* total, int* 
 }
 
 // ---- stage 2: scores, threshold, bit mask; last CTA compacts ------------------------------
-template <int S>
+// kSpec: also record per neuron the last token < keep in which it is active (speculative mode).
+template <int S, bool kSpec>
 __global__ void __launch_bounds__(kThreads)
 predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* __restrict__ B,
                       const float* __restrict__ c, float theta, int r, int F,
@@ -204,11 +205,11 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
       v += my_c;
       if (logits) logits[(size_t)s * F + my_col] = v;
       active = active || (v > theta);
-      if (v > theta && s < keep) last_kept = s;
+      if (kSpec && v > theta && s < keep) last_kept = s;
     }
     __syncthreads();
   }
-  if (keep_tok && tid < kLogitTile && my_col < F) keep_tok[my_col] = (int8_t)last_kept;
+  if (kSpec && tid < kLogitTile && my_col < F) keep_tok[my_col] = (int8_t)last_kept;
   if (tid < kLogitTile) {
     const unsigned m = __ballot_sync(0xffffffffu, active);
     if ((tid & 31) == 0) mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = m;
@@ -259,11 +260,15 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
   const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
   const size_t smem = (size_t)S * D.rank * sizeof(float);
   if (smem > 32 * 1024) {
-    e = cudaFuncSetAttribute(predict_logits_kernel<S>,
+    e = cudaFuncSetAttribute(predict_logits_kernel<S, false>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(predict_logits_kernel<S, true>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  e = launch_k(predict_logits_kernel<S>, dim3(grid), dim3(kThreads), smem, st, L->use_pdl,
+  auto kernel = L->keep_tok ? predict_logits_kernel<S, true> : predict_logits_kernel<S, false>;
+  e = launch_k(kernel, dim3(grid), dim3(kThreads), smem, st, L->use_pdl,
                (const float*)L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c,
                D.threshold_logit, D.rank, D.d_ff, logits, L->mask_words,
                (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
@@ -282,7 +287,8 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
                     (const __half*)D.dev_pred_A, D.d_model, D.rank, z_rows_per_cta(D.d_model),
                     L->z_partial);
   const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
-  return launch_k(predict_logits_kernel<1>, dim3(grid), dim3(kThreads),
+  return launch_k(L->keep_tok ? predict_logits_kernel<1, true> : predict_logits_kernel<1, false>,
+                  dim3(grid), dim3(kThreads),
                   (size_t)D.rank * sizeof(float), st, L->use_pdl, (const float*)L->z_partial,
                   L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit, D.rank,
                   D.d_ff, (float*)nullptr, L->mask_words, (int*)(L->counts + CNT_TICKET_PREDICT),
