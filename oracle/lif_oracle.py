@@ -80,13 +80,16 @@ class NeuronCache:
     ``last_k_active`` is kept as ``last_active[i]`` = the last step at which neuron i was
     predicted active, so "still inside the window of k tokens" is last_active[i] > t - k."""
 
-    def __init__(self, d_model, d_ff, capacity, window_k, budget_rows=0):
+    def __init__(self, d_model, d_ff, capacity, window_k, budget_rows=0, n_vec=2):
         """``budget_rows`` > 0 turns on the memory budget of Appendix C (Persimmon 8B, Phi-2):
-        whenever the cache would pass the budget, the window is shrunk for that step."""
+        whenever the cache would pass the budget, the window is shrunk for that step.
+        ``n_vec`` = vectors of d_model values per bundle: 2 (up row, down column; Section 3.2)
+        or 3 for a gated FFN (gate row, up row, down column; Appendix C, Llama 2)."""
         self.d_model, self.d_ff, self.capacity, self.k = d_model, d_ff, capacity, window_k
         self.budget_rows = budget_rows
+        self.n_vec = n_vec
         self.k_eff = window_k
-        self.matrix = np.zeros((capacity, 2 * d_model), dtype=np.float16)
+        self.matrix = np.zeros((capacity, n_vec * d_model), dtype=np.float16)
         self.pointers = np.full(capacity, -1, dtype=np.int32)
         self.bias = np.zeros(capacity, dtype=np.float16)
         self.slot_of = np.full(d_ff, -1, dtype=np.int32)
@@ -203,7 +206,7 @@ class NeuronCache:
         for i, s in zip(lists["load_ids"], lists["load_slots"]):
             self.matrix[s] = bundles[i]
             self.bias[s] = bias_up[i]
-        self.bytes_fetched += len(lists["load_ids"]) * 2 * self.d_model * self.matrix.itemsize
+        self.bytes_fetched += len(lists["load_ids"]) * self.n_vec * self.d_model * self.matrix.itemsize
 
     def cached_ids(self):
         return set(int(i) for i in self.pointers[: self.num_used])
@@ -228,24 +231,50 @@ def activation_fn(pre, activation=RELU, threshold=0.0):
     raise ValueError(activation)
 
 
-def sparse_ffn(matrix, bias, slots, x, b_down=None, activation=RELU, threshold=0.0):
+def sparse_ffn(matrix, bias, slots, x, b_down=None, activation=RELU, threshold=0.0,
+               gated=False, gate_pre=None):
     """y[s] = b_down + sum_q act(<matrix[slots[q], :d], x[s]> + bias[slots[q]]) * matrix[slots[q], d:]
 
-    matrix: [cap][2d] (fp16 values), bias: [cap], slots: row indices, x: [S][d].  float64."""
+    matrix: [cap][2d] (fp16 values), bias: [cap], slots: row indices, x: [S][d].  float64.
+
+    ``gated`` (Appendix C, Llama 2: a gated linear unit, an up and a down projection, the
+    activation applied to the gate value): rows are [cap][3d] = gate | up | down and
+    y[s] = b_down + sum_q act(<gate_q, x[s]> + bias_q) * <up_q, x[s]> * down_q.
+
+    ``gate_pre`` [S][len(slots)] (Appendix C, Llama 2, "alternative approaches": the gate
+    projection stays resident and doubles as the predictor): the gate pre-activations of the
+    rows are given, rows are [cap][2d] = up | down, ``bias`` is not used:
+    y[s] = b_down + sum_q act(gate_pre[s][q]) * <up_q, x[s]> * down_q."""
     x = np.asarray(x, dtype=np.float64)
     d = x.shape[1]
     rows = np.asarray(matrix)[np.asarray(slots, dtype=np.int64)].astype(np.float64)
-    up, down = rows[:, :d], rows[:, d:]
-    h = activation_fn(x @ up.T + np.asarray(bias, dtype=np.float64)[slots][None, :], activation,
-                      threshold)
+    assert rows.shape[1] == (3 if gated else 2) * d and not (gated and gate_pre is not None)
+    first, down = rows[:, :d], rows[:, -d:]
+    if gate_pre is not None:
+        h = activation_fn(np.asarray(gate_pre, dtype=np.float64), activation, threshold) * (x @ first.T)
+    else:
+        h = activation_fn(x @ first.T + np.asarray(bias, dtype=np.float64)[slots][None, :],
+                          activation, threshold)
+        if gated:
+            h = h * (x @ rows[:, d:2 * d].T)
     y = h @ down
     if b_down is not None:
         y = y + np.asarray(b_down, dtype=np.float64)[None, :]
     return y
 
 
+def gate_scores(x, gate_matrix, gate_bias=None):
+    """Gate pre-activations of every neuron, g[s][i] = <gate_matrix[i], x[s]> + gate_bias[i]:
+    with the gate projection resident they are the predictor's scores, and a neuron is active
+    iff its gate value passes the activation's threshold (Appendix C, Llama 2)."""
+    g = np.asarray(x, dtype=np.float64) @ np.asarray(gate_matrix, dtype=np.float64).T
+    if gate_bias is not None:
+        g = g + np.asarray(gate_bias, dtype=np.float64)[None, :]
+    return g
+
+
 def decode_step(cache, x, A, B, c, theta, bundles, bias_up, b_down=None, whole_cache=False,
-                act=None, activation=RELU, threshold=0.0, keep_token=None, keep=1):
+                act=None, activation=RELU, threshold=0.0, keep_token=None, keep=1, gated=False):
     """One layer, one token: predict -> window update -> insert -> FFN.  ``act`` overrides the
     predicted active list (used to follow another implementation's borderline decisions).
     ``whole_cache`` runs the FFN over every cached row (matrix[:num_used]) instead of only the
@@ -258,8 +287,27 @@ def decode_step(cache, x, A, B, c, theta, bundles, bias_up, b_down=None, whole_c
     lists = cache.window_update(act, keep_token, keep)
     cache.insert(lists, bundles, bias_up)
     slots = np.arange(cache.num_used) if whole_cache else lists["active_slots"]
-    y = sparse_ffn(cache.matrix, cache.bias, slots, x, b_down, activation, threshold)
+    y = sparse_ffn(cache.matrix, cache.bias, slots, x, b_down, activation, threshold, gated)
     return logits, act, lists, y
+
+
+def decode_step_gate_predictor(cache, x, gate_matrix, gate_bias, bundles, b_down=None,
+                               whole_cache=False, act=None, activation=FATRELU, threshold=0.0):
+    """One layer, one token with the resident gate projection as the predictor (Appendix C,
+    Llama 2, "alternative approaches"): scores = gate pre-activations, active iff a score
+    exceeds the activation's threshold (0 for ReLU), bundles = up | down, and the FFN reuses
+    the scores as gate values.  Rows cached but not active now contribute act(gate) = 0."""
+    g = gate_scores(x, gate_matrix, gate_bias)
+    theta = threshold if activation == FATRELU else 0.0
+    if act is None:
+        act = active_set(g, theta)
+    lists = cache.window_update(act)
+    cache.insert(lists, bundles, np.zeros(cache.d_ff, dtype=np.float16))
+    slots = np.arange(cache.num_used) if whole_cache else lists["active_slots"]
+    ids = cache.pointers[np.asarray(slots, dtype=np.int64)]
+    y = sparse_ffn(cache.matrix, cache.bias, slots, x, b_down, activation, threshold,
+                   gate_pre=g[:, ids])
+    return g, act, lists, y
 
 
 # --------------------------------------------------------------------------------------

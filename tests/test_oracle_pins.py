@@ -501,3 +501,146 @@ def test_keep_tokens_helper():
     assert O.keep_tokens(logits, 0.0, act, 3).tolist() == [0, 1, 2, 1]
     assert O.keep_tokens(logits, 0.0, act, 2).tolist() == [0, 1, -1, 1]
     assert O.keep_tokens(logits, 0.0, act, 1).tolist() == [0, -1, -1, 0]
+
+
+# ------------------------------------------------------------------ gated FFN (Appendix C, Llama 2)
+def _gated_loops(W_gate, b_gate, W_up, W_down, x, b_down, activation, threshold):
+    """Textbook gated FFN, scalar loops: y = W_down (act(W_gate x + b) * (W_up x)) + b_down."""
+    F, d = W_gate.shape
+    y = [b_down[m] for m in range(d)]
+    n_pass = 0
+    for i in range(F):
+        g = b_gate[i] + sum(W_gate[i, m] * x[m] for m in range(d))
+        u = sum(W_up[i, m] * x[m] for m in range(d))
+        if activation == O.FATRELU:
+            a = g if g > threshold else 0.0
+        elif activation == O.RELU_SQUARED:
+            a = g * g if g > 0 else 0.0
+        else:
+            a = g if g > 0 else 0.0
+        n_pass += a != 0.0
+        for m in range(d):
+            y[m] += a * u * W_down[m, i]
+    return np.array(y), n_pass
+
+
+def _gated_cache(W_gate, b_gate, W_up, W_down, ids):
+    F, d = W_gate.shape
+    M = np.zeros((len(ids), 3 * d)); bias = np.zeros(len(ids))
+    for s, i in enumerate(ids):
+        M[s, :d] = W_gate[i]; M[s, d:2 * d] = W_up[i]; M[s, 2 * d:] = W_down[:, i]; bias[s] = b_gate[i]
+    return M, bias
+
+
+@pytest.mark.parametrize("activation,threshold", [(O.FATRELU, 0.4), (O.RELU, 0.0), (O.RELU_SQUARED, 0.0)])
+def test_gated_ffn_matches_scalar_loops_and_library_form(activation, threshold):
+    r = _rng(40 + activation)
+    F, d, S = 19, 6, 2
+    W_gate, W_up, W_down = r.normal(size=(F, d)), r.normal(size=(F, d)), r.normal(size=(d, F))
+    b_gate, b_down, X = r.normal(size=F) * 0.3, r.normal(size=d), r.normal(size=(S, d))
+    order = r.permutation(F)                                  # rows in any order
+    M, bias = _gated_cache(W_gate, b_gate, W_up, W_down, order)
+    got = O.sparse_ffn(M, bias, np.arange(F), X, b_down, activation, threshold, gated=True)
+    for s in range(S):
+        want, n_pass = _gated_loops(W_gate, b_gate, W_up, W_down, X[s], b_down, activation, threshold)
+        assert 0 < n_pass < F
+        np.testing.assert_allclose(got[s], want, rtol=1e-12, atol=1e-12)
+    lib = (O.activation_fn(X @ W_gate.T + b_gate, activation, threshold) * (X @ W_up.T)) @ W_down.T + b_down
+    np.testing.assert_allclose(got, lib, rtol=1e-12, atol=1e-12)
+    # only the neurons whose gate passes matter: dropping the others changes nothing
+    passing = [q for q in range(F)
+               if (O.activation_fn(X @ M[q, :d] + bias[q], activation, threshold) != 0).any()]
+    np.testing.assert_allclose(O.sparse_ffn(M, bias, np.array(passing), X, b_down, activation, threshold,
+                                            gated=True), got, rtol=1e-12, atol=1e-12)
+
+
+def test_gated_ffn_special_cases_reduce_to_the_plain_ffn():
+    r = _rng(44)
+    F, d = 15, 5
+    W_gate, W_down = r.normal(size=(F, d)), r.normal(size=(d, F))
+    b_down, x = r.normal(size=d), r.normal(size=d)
+    zero = np.zeros(F)
+    # up row == gate row, no bias, ReLU: relu(g) * g is the squared ReLU of the plain FFN
+    M3, bias3 = _gated_cache(W_gate, zero, W_gate, W_down, list(range(F)))
+    M2, bias2 = _cache_from_dense(W_gate, zero, W_down, list(range(F)))
+    np.testing.assert_allclose(O.sparse_ffn(M3, bias3, np.arange(F), x[None], b_down, O.RELU, gated=True),
+                               O.sparse_ffn(M2, bias2, np.arange(F), x[None], b_down, O.RELU_SQUARED),
+                               rtol=1e-12, atol=1e-12)
+    # up rows with <up_i, x> = 1: the gate value passes through, i.e. the plain FFN (with its bias)
+    b_gate = r.normal(size=F)
+    W_one = np.tile(x / (x @ x), (F, 1))
+    M3, bias3 = _gated_cache(W_gate, b_gate, W_one, W_down, list(range(F)))
+    M2, bias2 = _cache_from_dense(W_gate, b_gate, W_down, list(range(F)))
+    np.testing.assert_allclose(O.sparse_ffn(M3, bias3, np.arange(F), x[None], b_down, O.FATRELU, 0.3, gated=True),
+                               O.sparse_ffn(M2, bias2, np.arange(F), x[None], b_down, O.FATRELU, 0.3),
+                               rtol=1e-11, atol=1e-12)
+    # the activation acts on the gate only: exchanging gate and up rows changes the result
+    W_up = r.normal(size=(F, d))
+    Ma, ba = _gated_cache(W_gate, zero, W_up, W_down, list(range(F)))
+    Mb, bb = _gated_cache(W_up, zero, W_gate, W_down, list(range(F)))
+    ya = O.sparse_ffn(Ma, ba, np.arange(F), x[None], None, O.RELU, gated=True)
+    yb = O.sparse_ffn(Mb, bb, np.arange(F), x[None], None, O.RELU, gated=True)
+    assert np.abs(ya - yb).max() > 1e-3
+    # empty list
+    np.testing.assert_array_equal(O.sparse_ffn(Ma, ba, np.array([], dtype=np.int64), x[None], b_down, gated=True)[0], b_down)
+
+
+def test_gate_projection_as_predictor_reproduces_the_dense_gated_ffn_at_every_step():
+    """With the resident gate as predictor the active set is exactly the set of neurons with a
+    non-zero activation, so every step's output is the dense gated FFN, whatever the window."""
+    r = _rng(45)
+    F, d, S, k, thr = 40, 6, 2, 3, 0.5
+    W_gate, W_up, W_down = r.normal(size=(F, d)), r.normal(size=(F, d)), r.normal(size=(d, F))
+    b_gate, b_down = r.normal(size=F) * 0.2 - 0.8, r.normal(size=d)
+    bundles = np.concatenate([W_up, W_down.T], axis=1).astype(np.float16)     # up | down
+    Wg16, bg16 = W_gate.astype(np.float16), b_gate.astype(np.float16)
+    cache = O.NeuronCache(d, F, F, k)
+    history, n_loaded = [], 0
+    for t in range(10):
+        X = r.normal(size=(S, d)).astype(np.float16)
+        g, act, lists, y = O.decode_step_gate_predictor(cache, X, Wg16, bg16, bundles, b_down,
+                                                        activation=O.FATRELU, threshold=thr)
+        for s in range(S):
+            want, _ = _gated_loops(Wg16.astype(float), bg16.astype(float), bundles[:, :d].astype(float),
+                                   bundles[:, d:].astype(float).T, X[s].astype(float), b_down, O.FATRELU, thr)
+            np.testing.assert_allclose(y[s], want, rtol=1e-11, atol=1e-12)
+        # score = gate pre-activation (scalar loop on a few entries); active = passes for some stream
+        for i in (0, 7, F - 1):
+            assert abs(g[1, i] - (float(bg16[i]) + sum(float(Wg16[i, m]) * float(X[1, m]) for m in range(d)))) < 1e-12
+        assert act.tolist() == [i for i in range(F) if (g[:, i] > thr).any()]
+        history.append(set(act.tolist()))
+        n_loaded += len(lists["load_ids"])
+        assert cache.cached_ids() == set().union(*history[-k:])
+        assert 0 < len(act) < F
+        # whole-cache FFN gives the same result: cached, inactive rows have a zero activation
+        ids = cache.pointers[:cache.num_used]
+        yw = O.sparse_ffn(cache.matrix, cache.bias, np.arange(cache.num_used), X, b_down, O.FATRELU, thr,
+                          gate_pre=g[:, ids])
+        np.testing.assert_allclose(yw, y, rtol=1e-11, atol=1e-12)
+    assert cache.bytes_fetched == n_loaded * 2 * d * 2          # two vectors per bundle: the gate stays resident
+    assert cache.matrix.shape[1] == 2 * d
+
+
+def test_gated_decode_step_three_vector_bundles():
+    """Low-rank predictor + three-vector bundles: with a predictor that is exact for the gate
+    (rank d: A = I, B = W_gate^T, c = b_gate, theta = threshold) a step equals the dense gated
+    FFN, and the traffic is 6*d bytes per new neuron."""
+    r = _rng(46)
+    F, d, k, thr = 30, 5, 2, 0.3
+    W_gate, W_up, W_down = (r.normal(size=(F, d)).astype(np.float16), r.normal(size=(F, d)).astype(np.float16),
+                            r.normal(size=(d, F)).astype(np.float16))
+    b_gate = (r.normal(size=F) * 0.2 - 0.5).astype(np.float16)
+    bundles = np.concatenate([W_gate, W_up, W_down.T], axis=1)
+    cache = O.NeuronCache(d, F, F, k, n_vec=3)
+    n_loaded = 0
+    for t in range(8):
+        x = r.normal(size=(1, d)).astype(np.float16)
+        logits, act, lists, y = O.decode_step(cache, x, np.eye(d), W_gate.astype(float).T, b_gate.astype(float),
+                                              thr, bundles, b_gate, activation=O.FATRELU, threshold=thr, gated=True)
+        want, n_pass = _gated_loops(W_gate.astype(float), b_gate.astype(float), W_up.astype(float),
+                                    W_down.astype(float), x[0].astype(float), np.zeros(d), O.FATRELU, thr)
+        assert n_pass == len(act)
+        np.testing.assert_allclose(y[0], want, rtol=1e-11, atol=1e-12)
+        n_loaded += len(lists["load_ids"])
+    assert cache.bytes_fetched == n_loaded * 3 * d * 2 and n_loaded > 0
+    assert cache.matrix.shape == (F, 3 * d)
