@@ -47,11 +47,27 @@ const char* lif_status_str(lif_status s);
  * its pre-activation v only when v > activation_threshold (threshold 0 is ReLU). */
 enum { LIF_ACT_RELU = 0, LIF_ACT_RELU_SQUARED = 1, LIF_ACT_FATRELU = 2 };
 
+/* Gated FFN (Appendix C, Llama 2: a gated linear unit, an up and a down projection; the
+ * activation is applied to the gate value):
+ *   y = b_down + sum_i act(<gate_i, x> + bias_i) * <up_i, x> * down_i.
+ * LIF_GATE_NONE      plain FFN, bundle = up row | down column (Section 3.2).
+ * LIF_GATE_BUNDLED   the gate row travels with the neuron: bundle and cache row are
+ *                    gate | up | down, 6*d_model bytes; the low-rank predictor decides what to
+ *                    load; bias_up is the gate's bias.
+ * LIF_GATE_RESIDENT  the gate projection stays in device memory and is the predictor
+ *                    (Appendix C, Llama 2, "alternative approaches"): score_i = <gate_i, x> +
+ *                    bias_i exactly, a neuron is active iff its score exceeds the activation's
+ *                    threshold (activation_threshold for FATReLU, 0 otherwise) for at least one
+ *                    stream, bundles are up | down, and the FFN reuses the scores as gate
+ *                    values.  dev_pred_A/B/c, rank and threshold_logit are ignored. */
+enum { LIF_GATE_NONE = 0, LIF_GATE_BUNDLED = 1, LIF_GATE_RESIDENT = 2 };
+
 typedef struct lif_layer lif_layer;
 
 /* Layer description.  Shapes follow Section 3.3: the cache `matrix` is
- * [capacity][2*d_model]; row s holds up-projection row `pointers[s]` followed by
- * down-projection column `pointers[s]` (Section 3.2, bundling columns and rows). */
+ * [capacity][V*d_model]; row s holds up-projection row `pointers[s]` followed by
+ * down-projection column `pointers[s]` (Section 3.2, bundling columns and rows), preceded by
+ * the gate row when gate_mode is LIF_GATE_BUNDLED.  V = 3 in that mode, 2 otherwise. */
 typedef struct {
   int32_t d_model;          /* multiple of 8, <= 8192 */
   int32_t d_ff;             /* multiple of 8, < 2^21 */
@@ -76,13 +92,16 @@ typedef struct {
                                step; a neuron active only in later tokens is used by this
                                step but gets the oldest stamp still inside the window.  The
                                step counter advances by spec_keep.  Not with budget_rows. */
-  const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][2*d_model] */
+  int32_t gate_mode;        /* LIF_GATE_*.  LIF_GATE_RESIDENT: not with spec_keep */
+  const void* dev_gate;     /* LIF_GATE_RESIDENT: fp16 [d_ff][d_model] gate projection, 16-byte
+                               aligned; otherwise ignored */
+  const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][V*d_model] */
   const void* dev_pred_A;   /* fp16 [d_model][rank] */
   const void* dev_pred_B;   /* fp16 [rank][d_ff] */
   const float* dev_pred_c;  /* fp32 [d_ff] per-neuron score offset */
-  const void* dev_bias_up;  /* fp16 [d_ff]: up-projection biases, always resident */
+  const void* dev_bias_up;  /* fp16 [d_ff]: up-projection (gated: gate) biases, always resident */
   const void* dev_bias_down;/* fp16 [d_model] or NULL */
-  void* dev_cache;          /* fp16 [capacity][2*d_model], 16-byte aligned */
+  void* dev_cache;          /* fp16 [capacity][V*d_model], 16-byte aligned */
   void* dev_workspace;      /* 256-byte aligned, lif_workspace_bytes() bytes; holds the window
                                state and all lists; initialised by lif_create_layer's reset */
   size_t workspace_bytes;
@@ -158,7 +177,8 @@ lif_status lif_destroy_layer(lif_layer* layer);
 lif_status lif_reset(lif_layer* layer, void* stream);
 
 /* Low-rank predictor (Section 3.1, "Anticipating ReLU Sparsity"): scores = x.A.B + c in fp32,
- * active iff score > theta for at least one stream.
+ * active iff score > theta for at least one stream.  With LIF_GATE_RESIDENT the scores are the
+ * gate pre-activations <gate_i, x> + bias_i and theta is the activation's threshold.
  *   dev_x              fp16 [n_streams][d_model]
  *   dev_logits_or_null fp32 [n_streams][d_ff] scores (optional)
  *   dev_active_idx     int32 [d_ff]: ascending ids of the active neurons
@@ -181,7 +201,9 @@ lif_status lif_window_update(lif_layer* layer, const int32_t* dev_active_idx,
 lif_status lif_fetch_bundles(lif_layer* layer, void* fetch_stream);
 
 /* Inference over cached rows (Section 3.3 item 3):
- *   y[s] = b_down + sum_q relu(<matrix[slot_q, :d], x[s]> + bias[slot_q]) * matrix[slot_q, d:]
+ *   y[s] = b_down + sum_q act(<matrix[slot_q, :d], x[s]> + bias[slot_q]) * matrix[slot_q, d:]
+ * (gated layers: see LIF_GATE_*; with LIF_GATE_RESIDENT the gate values are those of the last
+ * lif_predict / lif_decode_step of the layer, which must have been given the same x)
  *   dev_slots    int32 rows to use, or NULL for rows [0, *dev_n_slots)
  *   dev_n_slots  int32 [1] (device)
  *   dev_y        fp32 [n_streams][d_model] */
@@ -324,8 +346,8 @@ lif_status lif_timing_read(lif_layer* layer, float* host_us_sums /* [LIF_PHASE_L
  * kernels do not change the window state, so they can be replayed).  dev_x as for
  * lif_decode_step; dev_y is written only by LIF_KERNEL_FFN_SUM.  n_streams must be 1. */
 enum {
-  LIF_KERNEL_PREDICT_Z = 0,
-  LIF_KERNEL_PREDICT_SCORES = 1,
+  LIF_KERNEL_PREDICT_Z = 0,  /* not with LIF_GATE_RESIDENT */
+  LIF_KERNEL_PREDICT_SCORES = 1, /* LIF_GATE_RESIDENT: the gate-projection kernel */
   LIF_KERNEL_FETCH = 2,      /* re-copies this step's new bundles */
   LIF_KERNEL_FFN_ACTIVE = 3, /* sparse FFN kernel over all active rows */
   LIF_KERNEL_FFN_HITS = 4,   /* ... over the active rows that were already cached */

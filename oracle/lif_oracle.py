@@ -302,7 +302,9 @@ def decode_step_gate_predictor(cache, x, gate_matrix, gate_bias, bundles, b_down
     if act is None:
         act = active_set(g, theta)
     lists = cache.window_update(act)
-    cache.insert(lists, bundles, np.zeros(cache.d_ff, dtype=np.float16))
+    # the per-row scalars still follow the neurons (Section 3.3), though this FFN does not use them
+    cache.insert(lists, bundles, gate_bias if gate_bias is not None
+                 else np.zeros(cache.d_ff, dtype=np.float16))
     slots = np.arange(cache.num_used) if whole_cache else lists["active_slots"]
     ids = cache.pointers[np.asarray(slots, dtype=np.int64)]
     y = sparse_ffn(cache.matrix, cache.bias, slots, x, b_down, activation, threshold,

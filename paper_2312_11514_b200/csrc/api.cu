@@ -37,7 +37,10 @@ Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max) {
   w.z_partial = take(z_ctas * S * d.rank * 4);
   w.mask_words = take(n_mask * 4);
   w.keep_tok = take(d.spec_keep > 0 ? F : 0);
-  w.h_rows = take(d.n_streams > 1 ? (size_t)kBatchedMaxKSplit * F * 8 * 4 : 0);
+  w.h_rows = take(d.n_streams > 1 ? (size_t)kBatchedMaxKSplit * F * 8 * 4 *
+                                        (d.gate_mode == LIF_GATE_BUNDLED ? 2 : 1)
+                                  : 0);
+  w.gate_val = take(d.gate_mode == LIF_GATE_RESIDENT ? S * F * 4 : 0);
   size_t partial_rows = (size_t)ffn_grid_max;
   if (ffn_batched_supported(d) && (size_t)kBatchedMaxPartitions * S > partial_rows)
     partial_rows = (size_t)kBatchedMaxPartitions * S;
@@ -64,6 +67,8 @@ static lif_status check_shape(const lif_layer_desc* d) {
   if (d->activation < LIF_ACT_RELU || d->activation > LIF_ACT_FATRELU) return LIF_ERR_INVALID_ARG;
   if (d->activation == LIF_ACT_FATRELU && !(d->activation_threshold >= 0.f)) return LIF_ERR_INVALID_ARG;
   if (!(d->threshold_logit == d->threshold_logit)) return LIF_ERR_INVALID_ARG;   // NaN
+  if (d->gate_mode < LIF_GATE_NONE || d->gate_mode > LIF_GATE_RESIDENT) return LIF_ERR_INVALID_ARG;
+  if (d->gate_mode == LIF_GATE_RESIDENT && d->spec_keep > 0) return LIF_ERR_INVALID_ARG;
   return LIF_OK;
 }
 
@@ -101,11 +106,15 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
   *out = nullptr;
   lif_status s = check_shape(desc);
   if (s != LIF_OK) return s;
-  if (!desc->host_bundles || !desc->dev_pred_A || !desc->dev_pred_B || !desc->dev_pred_c ||
-      !desc->dev_bias_up || !desc->dev_cache || !desc->dev_workspace)
+  const bool resident = desc->gate_mode == LIF_GATE_RESIDENT;
+  if (!desc->host_bundles || !desc->dev_bias_up || !desc->dev_cache || !desc->dev_workspace)
     return LIF_ERR_INVALID_ARG;
-  if (!aligned(desc->host_bundles, 16) || !aligned(desc->dev_pred_A, 16) ||
-      !aligned(desc->dev_pred_B, 16) || !aligned(desc->dev_pred_c, 4) ||
+  if (resident ? !desc->dev_gate
+               : (!desc->dev_pred_A || !desc->dev_pred_B || !desc->dev_pred_c))
+    return LIF_ERR_INVALID_ARG;
+  if (!aligned(desc->host_bundles, 16) || (resident && !aligned(desc->dev_gate, 16)) ||
+      (!resident && (!aligned(desc->dev_pred_A, 16) || !aligned(desc->dev_pred_B, 16) ||
+                     !aligned(desc->dev_pred_c, 4))) ||
       !aligned(desc->dev_bias_up, 2) || !aligned(desc->dev_cache, 16) ||
       !aligned(desc->dev_workspace, 256) ||
       (desc->dev_bias_down && !aligned(desc->dev_bias_down, 8)))
@@ -144,6 +153,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
   L->keep_tok = desc->spec_keep > 0 ? (int8_t*)(b + ws.keep_tok) : nullptr;
   L->y_partial = (float*)(b + ws.y_partial);
   L->h_rows = (float*)(b + ws.h_rows);
+  L->gate_val = resident ? (float*)(b + ws.gate_val) : nullptr;
 
   int dev = 0;
   bool ok = cudaGetDevice(&dev) == cudaSuccess &&
@@ -470,7 +480,7 @@ lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
     case LIF_TUNE_FFN_STAGES:
       if (value < 1 || value > L->ffn_stages_max) return LIF_ERR_INVALID_ARG;
       L->ffn_stages = value;
-      L->ffn_smem = ffn_smem_for(L->desc.d_model, value);
+      L->ffn_smem = ffn_smem_for(L, value);
       return LIF_OK;
   }
   return LIF_ERR_INVALID_ARG;

@@ -77,7 +77,7 @@ refill_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
 cudaError_t launch_refill(lif_layer* L, cudaStream_t st) {
   refill_kernel<<<L->fetch_grid, kThreads, 0, st>>>((const uint4*)L->dev_bundles,
                                                     (uint4*)L->desc.dev_cache, L->pointers,
-                                                    L->counts, L->desc.d_model / 4);
+                                                    L->counts, row_elems(L->desc) / 8);
   return cudaGetLastError();
 }
 
@@ -85,7 +85,7 @@ cudaError_t launch_fetch(lif_layer* L, cudaStream_t st) {
   return launch_k(fetch_kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl,
                   (const uint4*)L->dev_bundles, (uint4*)L->desc.dev_cache,
                   (const int32_t*)L->load_ids, (const int32_t*)L->load_slots,
-                  (const int32_t*)L->counts, L->desc.d_model / 4);
+                  (const int32_t*)L->counts, row_elems(L->desc) / 8);
 }
 
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,

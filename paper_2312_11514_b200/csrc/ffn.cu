@@ -1,5 +1,8 @@
 // Sparse FFN over cached row-column bundles (Section 3.3 item 3):
 //   y = b_down + sum_q relu(<M[slot_q, :d], x> + bias[slot_q]) * M[slot_q, d:]
+// Gated layers (Appendix C, Llama 2): rows are gate | up | down and the row's weight is
+// act(<gate, x> + bias) * <up, x>; or, with the gate projection resident, rows are up | down and
+// the gate value of the row's neuron comes from the predictor's score array.
 // A bundle is one contiguous 4*d_model-byte row (Section 3.2), so the unit of HBM traffic is
 // one bulk asynchronous copy (TMA, cp.async.bulk) of a whole row into shared memory.  Each
 // CTA owns rows q = cta, cta + G, ...; it issues the copies for all its rows up front (up to
@@ -78,21 +81,28 @@ struct FfnArgs {
   int slots_len;          // entries of `slots` that may be read before n is known (0: none)
   int act;                // LIF_ACT_*
   float act_thr;
+  const float* gate_val;  // resident gate: this stream's gate pre-activations, by neuron id
+  const int32_t* pointers;  // resident gate: row -> neuron id
 };
 
+// kGate = LIF_GATE_*: none (row = up | down), bundled (gate | up | down), resident (up | down,
+// gate value looked up by neuron id).
+template <int kGate>
 __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int d = a.d;
-  const unsigned row_bytes = 4u * d;
+  constexpr int kVec = kGate == LIF_GATE_BUNDLED ? 3 : 2;       // d-vectors per row
+  constexpr int kParts = kGate == LIF_GATE_BUNDLED ? 16 : 8;    // warp partials per row
+  const unsigned row_bytes = 2u * kVec * d;
   const int stages = a.stages;
-  // shared layout: rows[stages][row_bytes] | x[d] fp16 | bars[stages] | part[stages][8] |
+  // shared layout: rows[stages][row_bytes] | x[d] fp16 | bars[stages] | part[stages][kParts] |
   //                h[stages] | bias[stages]
   unsigned char* rows = smem;
   __half* xs = reinterpret_cast<__half*>(rows + (size_t)stages * row_bytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(xs) +
                                                (((size_t)d * 2 + 15) & ~(size_t)15));
   float* part = reinterpret_cast<float*>(bars + stages);
-  float* hs = part + stages * 8;
+  float* hs = part + stages * kParts;
   float* bias_s = hs + stages;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -139,9 +149,10 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
       else if (r0 == 0 && q < a.slots_len) slot = my_slot;
       else slot = a.slots[q];
       mbar_expect_tx(bars + tid, row_bytes);
-      bulk_g2s(rows + (size_t)tid * row_bytes, a.cache + (size_t)slot * 2 * d, row_bytes,
+      bulk_g2s(rows + (size_t)tid * row_bytes, a.cache + (size_t)slot * kVec * d, row_bytes,
                bars + tid);
-      bias_s[tid] = __half2float(a.bias[slot]);
+      bias_s[tid] = kGate == LIF_GATE_RESIDENT ? a.gate_val[a.pointers[slot]]
+                                               : __half2float(a.bias[slot]);
     }
     if (r0 == 0) {
       const uint4* xg = reinterpret_cast<const uint4*>(a.x);
@@ -152,17 +163,29 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
     for (int i = 0; i < rc; ++i) {
       if (!mbar_wait(bars + i, parity)) timed_out = 1;
       const uint4* up = reinterpret_cast<const uint4*>(rows + (size_t)i * row_bytes);
-      float p = 0.f;
+      float p = 0.f, p2 = 0.f;
       for (int c = tid; c < nvec; c += kThreads) {
         float uf[8], xf[8];
         unpack8(up[c], uf);
         unpack8(reinterpret_cast<const uint4*>(xs)[c], xf);
 #pragma unroll
         for (int e = 0; e < 8; ++e) p = fmaf(uf[e], xf[e], p);
+        if (kGate == LIF_GATE_BUNDLED) {       // first vector = gate row, second = up row
+          unpack8(up[nvec + c], uf);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) p2 = fmaf(uf[e], xf[e], p2);
+        }
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
-      if (lane == 0) part[i * 8 + warp] = p;
+      if (kGate == LIF_GATE_BUNDLED) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) p2 += __shfl_xor_sync(0xffffffffu, p2, o);
+      }
+      if (lane == 0) {
+        part[i * kParts + warp] = p;
+        if (kGate == LIF_GATE_BUNDLED) part[i * kParts + 8 + warp] = p2;
+      }
     }
     if (__syncthreads_or(timed_out)) {
       // A copy did not arrive in time: flag it, give the copies still in flight one more
@@ -178,15 +201,25 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
     if (tid < rc) {
       float v = 0.f;
 #pragma unroll
-      for (int w = 0; w < 8; ++w) v += part[tid * 8 + w];
-      hs[tid] = apply_activation(v + bias_s[tid], a.act, a.act_thr);
+      for (int w = 0; w < 8; ++w) v += part[tid * kParts + w];
+      if (kGate == LIF_GATE_NONE) {
+        hs[tid] = apply_activation(v + bias_s[tid], a.act, a.act_thr);
+      } else if (kGate == LIF_GATE_BUNDLED) {
+        float u = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) u += part[tid * kParts + 8 + w];
+        hs[tid] = apply_activation(v + bias_s[tid], a.act, a.act_thr) * u;
+      } else {
+        hs[tid] = apply_activation(bias_s[tid], a.act, a.act_thr) * v;
+      }
     }
     __syncthreads();
     // down projection: y += h * down half
     for (int i = 0; i < rc; ++i) {
       const float h = hs[i];
       if (h == 0.f) continue;
-      const uint4* down = reinterpret_cast<const uint4*>(rows + (size_t)i * row_bytes) + nvec;
+      const uint4* down =
+          reinterpret_cast<const uint4*>(rows + (size_t)i * row_bytes) + (kVec - 1) * nvec;
 #pragma unroll
       for (int k = 0; k < kMaxChunks; ++k) {
         const int c = tid + k * kThreads;
@@ -261,17 +294,27 @@ ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
   }
 }
 
-size_t ffn_smem_bytes(int d, int stages) {
-  size_t b = (size_t)stages * 4 * d;              // rows
+size_t ffn_smem_bytes(int d, int stages, int gate_mode = LIF_GATE_NONE) {
+  const bool bundled = gate_mode == LIF_GATE_BUNDLED;
+  size_t b = (size_t)stages * (bundled ? 6 : 4) * d;   // rows
   b += ((size_t)d * 2 + 15) & ~(size_t)15;        // x
   b += (size_t)stages * 8;                        // barriers
-  b += (size_t)stages * 8 * 4 + (size_t)stages * 4 + (size_t)stages * 4;
+  b += (size_t)stages * (bundled ? 16 : 8) * 4 + (size_t)stages * 4 + (size_t)stages * 4;
   return b + 16;
+}
+
+using FfnKernel = void (*)(FfnArgs);
+FfnKernel ffn_kernel_for(int gate_mode) {
+  if (gate_mode == LIF_GATE_BUNDLED) return sparse_ffn_kernel<LIF_GATE_BUNDLED>;
+  if (gate_mode == LIF_GATE_RESIDENT) return sparse_ffn_kernel<LIF_GATE_RESIDENT>;
+  return sparse_ffn_kernel<LIF_GATE_NONE>;
 }
 
 }  // namespace
 
-size_t ffn_smem_for(int d_model, int stages) { return ffn_smem_bytes(d_model, stages); }
+size_t ffn_smem_for(const lif_layer* L, int stages) {
+  return ffn_smem_bytes(L->desc.d_model, stages, L->desc.gate_mode);
+}
 
 cudaError_t ffn_configure(lif_layer* L) {
   const int d = L->desc.d_model;
@@ -280,12 +323,13 @@ cudaError_t ffn_configure(lif_layer* L) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
+  const int gm = L->desc.gate_mode;
   int stages = 16;
-  while (stages > 1 && ffn_smem_bytes(d, stages) > (size_t)max_smem) --stages;
-  if (ffn_smem_bytes(d, stages) > (size_t)max_smem) return cudaErrorInvalidValue;
+  while (stages > 1 && ffn_smem_bytes(d, stages, gm) > (size_t)max_smem) --stages;
+  if (ffn_smem_bytes(d, stages, gm) > (size_t)max_smem) return cudaErrorInvalidValue;
   L->ffn_stages = L->ffn_stages_max = stages;
-  L->ffn_smem = ffn_smem_bytes(d, stages);
-  return cudaFuncSetAttribute(sparse_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  L->ffn_smem = ffn_smem_bytes(d, stages, gm);
+  return cudaFuncSetAttribute(ffn_kernel_for(gm), cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)max_smem);
 }
 
@@ -305,6 +349,8 @@ static FfnArgs ffn_args(lif_layer* L, const __half* x, const int32_t* slots, con
   a.slots_len = slots_len;
   a.act = L->desc.activation;
   a.act_thr = L->desc.activation_threshold;
+  a.gate_val = L->gate_val;
+  a.pointers = L->pointers;
   return a;
 }
 
@@ -327,8 +373,9 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
     // a caller's slot list may be shorter than d_ff: never read it before n is known
     FfnArgs a = ffn_args(L, x + (size_t)s * d, slots, n, base, L->y_partial,
                          slots && (slots == L->active_slots || slots == L->hit_slots) ? D.d_ff : 0);
-    cudaError_t e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem,
-                             st, L->use_pdl, a);
+    if (a.gate_val) a.gate_val += (size_t)s * D.d_ff;
+    cudaError_t e = launch_k(ffn_kernel_for(D.gate_mode), dim3(L->ffn_grid), dim3(kThreads),
+                             L->ffn_smem, st, L->use_pdl, a);
     if (e != cudaSuccess) return e;
     if (ev && s == D.n_streams - 1) tm_record(ev[8], st);
     e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st, L->use_pdl,
@@ -365,7 +412,7 @@ cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cuda
     default:
       return cudaErrorInvalidValue;
   }
-  return launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
+  return launch_k(ffn_kernel_for(D.gate_mode), dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
                   L->use_pdl, a);
 }
 
@@ -398,7 +445,7 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
                     ? ffn_args(L, x, L->hit_slots, cnt + LIF_CNT_N_HITS, nullptr, p0, D.d_ff)
                     : ffn_args(L, x, nullptr, cnt + LIF_CNT_NUM_KEPT, nullptr, p0, 0);
   if (ev) tm_record(ev[7], side);
-  e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, side,
+  e = launch_k(ffn_kernel_for(D.gate_mode), dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, side,
                fork ? 0 : L->use_pdl, hit);
   if (e != cudaSuccess) return e;
   if (ev) tm_record(ev[8], side);
@@ -407,8 +454,8 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
   if ((e = launch_fetch(L, st)) != cudaSuccess) return e;
   if (ev) tm_record(ev[6], st);
   FfnArgs miss = ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
-  e = launch_k(sparse_ffn_kernel, dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st, L->use_pdl,
-               miss);
+  e = launch_k(ffn_kernel_for(D.gate_mode), dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
+               L->use_pdl, miss);
   if (e != cudaSuccess) return e;
   if (fork && (e = cudaStreamWaitEvent(st, L->ev_fetch, 0)) != cudaSuccess) return e;
   e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0,
@@ -478,7 +525,8 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
         cudaDeviceGetAttribute(&sd.n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sd.max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) !=
             cudaSuccess ||
-        cudaFuncSetAttribute(sparse_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(sparse_ffn_kernel<LIF_GATE_NONE>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                              sd.max_smem) != cudaSuccess) {
       cudaGetLastError();
       return LIF_ERR_CUDA;
@@ -512,7 +560,9 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
   a.slots_len = 0;
   a.act = LIF_ACT_RELU;
   a.act_thr = 0.f;
-  sparse_ffn_kernel<<<grid, kThreads, ffn_smem_bytes(d_model, stages), st>>>(a);
+  a.gate_val = nullptr;
+  a.pointers = nullptr;
+  sparse_ffn_kernel<LIF_GATE_NONE><<<grid, kThreads, ffn_smem_bytes(d_model, stages), st>>>(a);
   if (cudaGetLastError() != cudaSuccess) return LIF_ERR_CUDA;
   ffn_reduce_kernel<<<(d_model / 4 + kSumCols - 1) / kSumCols, kSumThreads, 0, st>>>(
       sd.scratch->partial, dev_n_slots, nullptr, nullptr, grid, (const __half*)dev_bias_down,

@@ -14,6 +14,10 @@
 //            fp16 high + low parts (so the product keeps fp32 accuracy), is the B operand; each
 //            warp keeps its column tiles' accumulators in registers for the whole kernel.
 // Partition partials are added in a fixed order by the partial-sum kernel.  Bound: HBM.
+// Gated layers (Appendix C, Llama 2): with the gate row in the bundle, phase A runs twice (gate
+// rows with the bias, then up rows) and phase B uses H = act(gate) * up; with the gate
+// projection resident, phase A contracts the up rows and phase B takes the gate value of each
+// row's neuron from the predictor's score array.
 #include "lif_internal.cuh"
 
 namespace lif {
@@ -101,6 +105,15 @@ struct BatchedArgs {
   size_t h_stride;
   int act;                // LIF_ACT_*
   float act_thr;
+  int row_elems;          // fp16 elements per cache row
+  int vec_off;            // phase A: first element of the vector it contracts (gate or up row)
+  int down_off;           // phase B: first element of the down column
+  int add_bias;           // phase A: K slice 0 adds the row's bias
+  int gate_mode;          // LIF_GATE_*
+  int F;
+  const float* H2;        // bundled gate: phase-A output of the up rows (H holds the gate rows)
+  const float* gate_val;  // resident gate: [S][F] gate pre-activations by neuron id
+  const int32_t* pointers;  // resident gate: row -> neuron id
 };
 
 __device__ __forceinline__ int row_slot(const BatchedArgs& a, int q, int base) {
@@ -149,10 +162,10 @@ __global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs
     slot_all[i] = slot;
     if (i < stages) {
       mbar_expect_tx(group_bar(bars, i, G), seg_bytes);
-      bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * 2 * d + k0, seg_bytes,
-               group_bar(bars, i, G));
+      bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * a.row_elems + a.vec_off + k0,
+               seg_bytes, group_bar(bars, i, G));
     }
-    const float b = ks == 0 ? __half2float(a.bias[slot]) : 0.f;
+    const float b = (ks == 0 && a.add_bias) ? __half2float(a.bias[slot]) : 0.f;
     bias_all[i] = b;
     if (i < stages) bias_s[i] = b;
   }
@@ -227,9 +240,10 @@ __global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs
         const bool cached = i < kRowCacheA;
         const int slot = cached ? slot_all[i] : row_slot(a, prt + i * P, base);
         mbar_expect_tx(bars + st0, seg_bytes);
-        bulk_g2s(rows + (size_t)(st0 + tid) * pitch, a.cache + (size_t)slot * 2 * d + k0,
-                 seg_bytes, bars + st0);
-        bias_s[st0 + tid] = cached ? bias_all[i] : (ks == 0 ? __half2float(a.bias[slot]) : 0.f);
+        bulk_g2s(rows + (size_t)(st0 + tid) * pitch,
+                 a.cache + (size_t)slot * a.row_elems + a.vec_off + k0, seg_bytes, bars + st0);
+        bias_s[st0 + tid] =
+            cached ? bias_all[i] : ((ks == 0 && a.add_bias) ? __half2float(a.bias[slot]) : 0.f);
       } else {
         mbar_arrive(bars + st0);
       }
@@ -274,15 +288,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
       *reinterpret_cast<uint4*>(rows + i) = make_uint4(0, 0, 0, 0);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
-  const size_t col_off = (size_t)d + col0;
+  const size_t col_off = (size_t)a.down_off + col0;
 
   for (int i = tid; i < min(my_cnt, kRowCacheB); i += kThreads) {   // slots once, first copies
     const int slot = row_slot(a, prt + i * P, base);
     slot_all[i] = slot;
     if (i < stages) {
       mbar_expect_tx(group_bar(bars, i), seg_bytes);
-      bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * 2 * d + col_off, seg_bytes,
-               group_bar(bars, i));
+      bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * a.row_elems + col_off,
+               seg_bytes, group_bar(bars, i));
     }
   }
   for (int i = my_cnt + tid; i < stages; i += kThreads) mbar_arrive(group_bar(bars, i));
@@ -300,6 +314,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     float v = 0.f;
     const size_t at = (size_t)(prt + i * P) * 8 + hs;
     for (int ks = 0; ks < a.ksplit; ++ks) v += a.H[(size_t)ks * a.h_stride + at];
+    if (a.gate_mode == LIF_GATE_BUNDLED) {       // H = gate pre-activation, H2 = up value
+      float u = 0.f;
+      for (int ks = 0; ks < a.ksplit; ++ks) u += a.H2[(size_t)ks * a.h_stride + at];
+      return apply_activation(v, a.act, a.act_thr) * u;
+    }
+    if (a.gate_mode == LIF_GATE_RESIDENT) {      // H = up value, gate from the score array
+      if (hs >= a.S) return 0.f;
+      const int id = a.pointers[row_slot(a, prt + i * P, base)];
+      return apply_activation(a.gate_val[(size_t)hs * a.F + id], a.act, a.act_thr) * v;
+    }
     return apply_activation(v, a.act, a.act_thr);
   };
   pdl_wait();                                      // H is complete from here on
@@ -355,8 +379,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
       if (i < my_cnt) {
         const int slot = i < kRowCacheB ? slot_all[i] : row_slot(a, prt + i * P, base);
         mbar_expect_tx(bars + st0, seg_bytes);
-        bulk_g2s(rows + (size_t)(st0 + tid) * pitch, a.cache + (size_t)slot * 2 * d + col_off,
-                 seg_bytes, bars + st0);
+        bulk_g2s(rows + (size_t)(st0 + tid) * pitch,
+                 a.cache + (size_t)slot * a.row_elems + col_off, seg_bytes, bars + st0);
       } else {
         mbar_arrive(bars + st0);
       }
@@ -471,10 +495,30 @@ cudaError_t launch_ffn_batched(lif_layer* L, const __half* x, const int32_t* slo
   a.h_stride = (size_t)D.d_ff * 8;
   a.act = D.activation;
   a.act_thr = D.activation_threshold;
+  a.row_elems = row_elems(D);
+  a.gate_mode = D.gate_mode;
+  a.vec_off = 0;
+  a.down_off = a.row_elems - D.d_model;
+  a.add_bias = D.gate_mode != LIF_GATE_RESIDENT;   // resident gate: the bias is in the gate values
+  a.F = D.d_ff;
+  a.H2 = nullptr;
+  a.gate_val = L->gate_val;
+  a.pointers = L->pointers;
   a.stages = L->fb_up_stages;
   cudaError_t e = launch_k(ffn_batched_up_kernel, dim3(L->fb_up_partitions * L->fb_ksplit),
                            dim3(kThreads), L->fb_up_smem, st, L->use_pdl, a);
   if (e != cudaSuccess) return e;
+  if (D.gate_mode == LIF_GATE_BUNDLED) {           // second pass of phase A: the up rows
+    float* h2 = L->h_rows + (size_t)kBatchedMaxKSplit * D.d_ff * 8;
+    a.H = h2;
+    a.vec_off = D.d_model;
+    a.add_bias = 0;
+    e = launch_k(ffn_batched_up_kernel, dim3(L->fb_up_partitions * L->fb_ksplit), dim3(kThreads),
+                 L->fb_up_smem, st, L->use_pdl, a);
+    if (e != cudaSuccess) return e;
+    a.H = L->h_rows;
+    a.H2 = h2;
+  }
   a.stages = 32;
   e = launch_k(ffn_batched_down_kernel, dim3(L->fb_parts * L->fb_partitions), dim3(kThreads),
                L->fb_down_smem, st, L->use_pdl, a);

@@ -1,0 +1,171 @@
+// The resident gate projection as the predictor (Appendix C, Llama 2, "alternative
+// approaches"): with a gated FFN whose activation makes the gate values sparse, the gate
+// projection kept in device memory gives the exact gate pre-activation of every neuron,
+//   g[s][i] = <gate_i, x[s]> + bias_i,
+// a neuron is active iff g exceeds the activation's threshold for at least one stream, and the
+// FFN reuses g instead of recomputing it.  A dense fp16 GEMV over [d_ff][d_model] with fp32
+// accumulation: every gate row is read once with 16-byte loads.  A CTA owns 32 consecutive
+// neurons (one word of the bit mask), a warp four of them, so a thread keeps four independent
+// rows in flight.  Bound: HBM bandwidth, 2*d_model bytes per neuron.
+#include "lif_internal.cuh"
+#include "mask_compact.cuh"
+
+namespace lif {
+namespace {
+
+constexpr int kGateTile = 32;          // neurons per CTA = one mask word
+constexpr int kRowsPerWarp = 4;
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __half22float2(h[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+
+template <int S>
+__global__ void __launch_bounds__(kThreads)
+gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate,
+                   const __half* __restrict__ bias, float theta, int d, int F,
+                   float* __restrict__ gate_val, float* __restrict__ logits,
+                   uint32_t* mask_words, int* ticket, int* __restrict__ active_idx,
+                   int* __restrict__ n_active, int compact, int nwords) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4* xs = reinterpret_cast<uint4*>(smem_raw);          // [S][d / 8]
+  __shared__ int act_flag[kGateTile];
+  __shared__ int warp_sums[kThreads / 32];
+  __shared__ int is_last;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = d >> 3;
+  const int i0 = blockIdx.x * kGateTile + warp * kRowsPerWarp;   // this warp's first neuron
+
+  // The gate rows are weights: the first 16-byte piece of each of the four rows is in flight
+  // before the dependency wait; x (possibly written by the previous kernel) comes after it.
+  uint4 w[kRowsPerWarp];
+#pragma unroll
+  for (int q = 0; q < kRowsPerWarp; ++q)
+    w[q] = (i0 + q < F && lane < nvec) ? ldg_stream(gate + (size_t)(i0 + q) * d + lane * 8)
+                                       : make_uint4(0, 0, 0, 0);
+  pdl_wait();
+  pdl_trigger();
+  for (int c = tid; c < S * nvec; c += kThreads) xs[c] = reinterpret_cast<const uint4*>(x)[c];
+  __syncthreads();
+
+  float acc[kRowsPerWarp][S];
+#pragma unroll
+  for (int q = 0; q < kRowsPerWarp; ++q)
+#pragma unroll
+    for (int s = 0; s < S; ++s) acc[q][s] = 0.f;
+
+  for (int c = lane; c < nvec; c += 32) {
+    uint4 nxt[kRowsPerWarp];
+    const int cn = c + 32;
+#pragma unroll
+    for (int q = 0; q < kRowsPerWarp; ++q)
+      nxt[q] = (i0 + q < F && cn < nvec) ? ldg_stream(gate + (size_t)(i0 + q) * d + cn * 8)
+                                         : make_uint4(0, 0, 0, 0);
+    float wf[kRowsPerWarp][8];
+#pragma unroll
+    for (int q = 0; q < kRowsPerWarp; ++q) unpack8(w[q], wf[q]);
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+      float xf[8];
+      unpack8(xs[s * nvec + c], xf);
+#pragma unroll
+      for (int q = 0; q < kRowsPerWarp; ++q)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[q][s] = fmaf(wf[q][e], xf[e], acc[q][s]);
+    }
+#pragma unroll
+    for (int q = 0; q < kRowsPerWarp; ++q) w[q] = nxt[q];
+  }
+
+  // warp sums in a fixed order; lane q finishes neuron i0 + q
+#pragma unroll
+  for (int q = 0; q < kRowsPerWarp; ++q)
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+      float v = acc[q][s];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      acc[q][s] = v;
+    }
+  if (lane < kRowsPerWarp) {
+    const int i = i0 + lane;
+    bool active = false;
+    if (i < F) {
+      const float b = __half2float(bias[i]);
+#pragma unroll
+      for (int s = 0; s < S; ++s) {
+        float v = 0.f;
+#pragma unroll
+        for (int q = 0; q < kRowsPerWarp; ++q)
+          if (q == lane) v = acc[q][s];
+        v += b;
+        gate_val[(size_t)s * F + i] = v;
+        if (logits) logits[(size_t)s * F + i] = v;
+        active = active || (v > theta);
+      }
+    }
+    act_flag[warp * kRowsPerWarp + lane] = active ? 1 : 0;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const unsigned m = __ballot_sync(0xffffffffu, act_flag[lane] != 0);
+    if (lane == 0) mask_words[blockIdx.x] = m;
+  }
+  if (!compact) return;     // the consumer reads the bit mask itself
+  compact_mask_last_cta(mask_words, nwords, ticket, active_idx, n_active, warp_sums, &is_last);
+}
+
+template <int S>
+cudaError_t launch_gate_s(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
+                          int32_t* n_active, cudaStream_t st, int compact) {
+  const lif_layer_desc& D = L->desc;
+  const int grid = (D.d_ff + kGateTile - 1) / kGateTile;
+  const size_t smem = (size_t)S * D.d_model * 2;
+  if (smem > 32 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(gate_scores_kernel<S>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  const float theta = D.activation == LIF_ACT_FATRELU ? D.activation_threshold : 0.f;
+  return launch_k(gate_scores_kernel<S>, dim3(grid), dim3(kThreads), smem, st, L->use_pdl, x,
+                  (const __half*)D.dev_gate, (const __half*)D.dev_bias_up, theta, D.d_model,
+                  D.d_ff, L->gate_val, logits, L->mask_words,
+                  (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
+                  grid);
+}
+
+}  // namespace
+
+cudaError_t launch_gate_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
+                                int32_t* n_active, cudaStream_t st, cudaEvent_t* ev, int compact) {
+  if (ev) tm_record(ev[1], st);     // no first stage in this mode
+  cudaError_t e = cudaErrorInvalidValue;
+  switch (L->desc.n_streams) {
+    case 1: e = launch_gate_s<1>(L, x, logits, active_idx, n_active, st, compact); break;
+    case 2: e = launch_gate_s<2>(L, x, logits, active_idx, n_active, st, compact); break;
+    case 3: e = launch_gate_s<3>(L, x, logits, active_idx, n_active, st, compact); break;
+    case 4: e = launch_gate_s<4>(L, x, logits, active_idx, n_active, st, compact); break;
+    case 5: e = launch_gate_s<5>(L, x, logits, active_idx, n_active, st, compact); break;
+    case 6: e = launch_gate_s<6>(L, x, logits, active_idx, n_active, st, compact); break;
+    case 7: e = launch_gate_s<7>(L, x, logits, active_idx, n_active, st, compact); break;
+    case 8: e = launch_gate_s<8>(L, x, logits, active_idx, n_active, st, compact); break;
+  }
+  if (ev) tm_record(ev[2], st);
+  return e;
+}
+
+}  // namespace lif

@@ -34,8 +34,13 @@ struct Workspace {
   // offsets in bytes from the workspace base; every block 256-byte aligned
   size_t counts, pointers, slot_of, last_active, bias, active_idx, evict_ids, evict_slots,
       move_src, move_dst, load_ids, load_slots, active_slots, hit_slots, n_tmp, z_partial,
-      mask_words, keep_tok, h_rows, y_partial, total;
+      mask_words, keep_tok, h_rows, gate_val, y_partial, total;
 };
+
+// fp16 elements per bundle / cache row: up | down, preceded by the gate row when it is bundled
+inline int row_elems(const lif_layer_desc& d) {
+  return (d.gate_mode == LIF_GATE_BUNDLED ? 3 : 2) * d.d_model;
+}
 
 Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max);
 
@@ -55,6 +60,8 @@ struct lif_layer {
   int8_t* keep_tok;   // [d_ff] last kept token per neuron (speculative mode)
   float* y_partial;
   float* h_rows;      // [K slices][d_ff][8] fp32: phase-A output of the multi-stream FFN
+                      // (bundled gate: a second block of the same size for the up values)
+  float* gate_val;    // [S][d_ff] fp32 gate pre-activations (resident gate only)
   // multi-stream (tensor-core) FFN configuration; fb_ok = 0: per-stream fallback
   int fb_ok, fb_up_stages, fb_parts, fb_cols, fb_partitions;
   int fb_ksplit, fb_kps, fb_up_partitions, fb_parts_min, fb_up_group, fb_up_two_ctas;
@@ -101,6 +108,9 @@ cudaError_t launch_reset(lif_layer* L, cudaStream_t st);
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
                            int32_t* n_active, cudaStream_t st, cudaEvent_t* ev = nullptr,
                            int compact = 1);   // compact = 0: leave only the bit mask
+// Resident gate projection as the predictor: scores, threshold, bit mask, optional compaction.
+cudaError_t launch_gate_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
+                                int32_t* n_active, cudaStream_t st, cudaEvent_t* ev, int compact);
 bool window_plan_supported(const lif_layer_desc& D);
 cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr);
 cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st,
@@ -127,7 +137,7 @@ bool ffn_batched_supported(const lif_layer_desc& D);
 cudaError_t ffn_batched_configure(lif_layer* L);
 cudaError_t launch_ffn_batched(lif_layer* L, const __half* x, const int32_t* slots,
                                const int32_t* n, const int32_t* base, float* y, cudaStream_t st);
-size_t ffn_smem_for(int d_model, int stages);
+size_t ffn_smem_for(const lif_layer* L, int stages);
 
 // Launch with (pdl) or without the programmatic-stream-serialization attribute.  A kernel
 // launched with it may start while the previous kernel of the stream is still running; it

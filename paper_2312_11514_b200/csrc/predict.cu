@@ -8,6 +8,7 @@
 // mask into the sorted list with a block prefix sum, so the list order never depends on
 // scheduling.  Summation orders are fixed: results are bit-reproducible run to run.
 #include "lif_internal.cuh"
+#include "mask_compact.cuh"
 
 namespace lif {
 namespace {
@@ -103,28 +104,6 @@ predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int
   }
 }
 
-__device__ __forceinline__ int block_exclusive_scan_256(int v, int* total, int* warp_sums) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int n = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += n;
-  }
-  if (lane == 31) warp_sums[warp] = inc;
-  __syncthreads();
-  int base = 0, tot = 0;
-#pragma unroll
-  for (int w = 0; w < kThreads / 32; ++w) {
-    int ws = warp_sums[w];
-    if (w < warp) base += ws;
-    tot += ws;
-  }
-  *total = tot;
-  __syncthreads();
-  return base + inc - v;
-}
-
 // ---- stage 2: scores, threshold, bit mask; last CTA compacts ------------------------------
 // kSpec: also record per neuron the last token < keep in which it is active (speculative mode).
 template <int S, bool kSpec>
@@ -216,36 +195,8 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
   }
 
   if (!compact) return;     // the consumer reads the bit mask itself
-  // last CTA to arrive compacts the whole mask
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int t = atomicAdd(ticket, 1);
-    is_last = (t == (int)gridDim.x - 1);
-  }
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-
-  const int nwords = gridDim.x * (kLogitTile / 32);
-  const int wpt = (nwords + kThreads - 1) / kThreads;
-  const int w0 = min(nwords, tid * wpt), w1 = min(nwords, w0 + wpt);
-  int cnt = 0;
-  for (int w = w0; w < w1; ++w) cnt += __popc(__ldcg(mask_words + w));
-  int total;
-  int off = block_exclusive_scan_256(cnt, &total, warp_sums);
-  for (int w = w0; w < w1; ++w) {
-    unsigned m = __ldcg(mask_words + w);
-    while (m) {
-      const int b = __ffs(m) - 1;
-      active_idx[off++] = w * 32 + b;
-      m &= m - 1;
-    }
-  }
-  if (tid == 0) {
-    *n_active = total;
-    *ticket = 0;
-  }
+  compact_mask_last_cta(mask_words, gridDim.x * (kLogitTile / 32), ticket, active_idx, n_active,
+                        warp_sums, &is_last);
 }
 
 template <int S>
@@ -282,6 +233,10 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
 cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaStream_t st) {
   const lif_layer_desc& D = L->desc;
   if (D.n_streams != 1) return cudaErrorInvalidValue;
+  if (D.gate_mode == LIF_GATE_RESIDENT)
+    return kernel == LIF_KERNEL_PREDICT_SCORES
+               ? launch_gate_predict(L, x, nullptr, L->active_idx, L->n_tmp, st, nullptr, 1)
+               : cudaErrorInvalidValue;
   if (kernel == LIF_KERNEL_PREDICT_Z)
     return launch_k(predict_z_kernel<1>, dim3(L->z_ctas), dim3(kThreads), 0, st, L->use_pdl, x,
                     (const __half*)D.dev_pred_A, D.d_model, D.rank, z_rows_per_cta(D.d_model),
@@ -297,6 +252,8 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
 
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
                            int32_t* n_active, cudaStream_t st, cudaEvent_t* ev, int compact) {
+  if (L->desc.gate_mode == LIF_GATE_RESIDENT)
+    return launch_gate_predict(L, x, logits, active_idx, n_active, st, ev, compact);
   switch (L->desc.n_streams) {
     case 1: return launch_predict_s<1>(L, x, logits, active_idx, n_active, st, ev, compact);
     case 2: return launch_predict_s<2>(L, x, logits, active_idx, n_active, st, ev, compact);

@@ -553,7 +553,7 @@ static WindowArgs window_args(lif_layer* L, const int32_t* act, const int32_t* n
   a.budget = D.budget_rows;
   a.keep_tok = D.spec_keep > 0 ? L->keep_tok : nullptr;
   a.keep = D.spec_keep > 0 ? D.spec_keep : 1;
-  a.bundle_bytes = 4ull * D.d_model;
+  a.bundle_bytes = 2ull * row_elems(D);
   return a;
 }
 
@@ -563,7 +563,7 @@ static cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev) 
   if (ev) tm_record(ev[3], st);
   e = launch_k(move_rows_kernel, dim3(L->move_grid), dim3(kThreads), 0, st, L->use_pdl,
                (uint4*)D.dev_cache, (const int32_t*)L->move_src, (const int32_t*)L->move_dst,
-               (const int32_t*)L->counts, D.d_model / 4);
+               (const int32_t*)L->counts, row_elems(D) / 8);
   if (ev) tm_record(ev[4], st);
   return e;
 }

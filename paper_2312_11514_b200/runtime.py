@@ -14,33 +14,38 @@ class Layer:
     """One FFN layer: owns its torch buffers and the `lif_layer` handle."""
 
     def __init__(self, *, d_model: int, d_ff: int, rank: int, window_k: int, capacity: int,
-                 host_bundles: torch.Tensor, pred_A: torch.Tensor, pred_B: torch.Tensor,
-                 pred_c: torch.Tensor, bias_up: torch.Tensor,
+                 host_bundles: torch.Tensor, bias_up: torch.Tensor,
+                 pred_A: Optional[torch.Tensor] = None, pred_B: Optional[torch.Tensor] = None,
+                 pred_c: Optional[torch.Tensor] = None,
                  bias_down: Optional[torch.Tensor] = None, n_streams: int = 1,
                  threshold_logit: float = 0.0, ffn_mode: int = 0, activation: int = 0,
                  activation_threshold: float = 0.0, budget_rows: int = 0, spec_keep: int = 0,
-                 device="cuda:0"):
+                 gate_mode: int = 0, gate: Optional[torch.Tensor] = None, device="cuda:0"):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2312_11514_b200 needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
         assert host_bundles.is_pinned() and host_bundles.dtype == torch.float16
-        assert host_bundles.shape == (d_ff, 2 * d_model) and host_bundles.is_contiguous()
+        n_vec = 3 if gate_mode == B.GATE_BUNDLED else 2      # d_model-vectors per bundle
+        assert host_bundles.shape == (d_ff, n_vec * d_model) and host_bundles.is_contiguous()
+        assert gate is None or (gate.shape == (d_ff, d_model) and gate.dtype == torch.float16
+                                and gate.is_contiguous())
         self.d_model, self.d_ff, self.rank, self.capacity = d_model, d_ff, rank, capacity
         self.n_streams = n_streams
         self.keep = dict(host_bundles=host_bundles, pred_A=pred_A, pred_B=pred_B, pred_c=pred_c,
-                         bias_up=bias_up, bias_down=bias_down)
-        self.cache = torch.zeros(capacity, 2 * d_model, dtype=torch.float16, device=self.device)
+                         bias_up=bias_up, bias_down=bias_down, gate=gate)
+        self.cache = torch.zeros(capacity, n_vec * d_model, dtype=torch.float16, device=self.device)
         shape = dict(d_model=d_model, d_ff=d_ff, rank=rank, window_k=window_k, capacity=capacity,
                      n_streams=n_streams, threshold_logit=threshold_logit, ffn_mode=ffn_mode,
                      activation=activation, activation_threshold=activation_threshold,
-                     budget_rows=budget_rows, spec_keep=spec_keep)
-        self.spec_keep = spec_keep
+                     budget_rows=budget_rows, spec_keep=spec_keep, gate_mode=gate_mode)
+        self.spec_keep, self.gate_mode = spec_keep, gate_mode
         nbytes = B.lif_workspace_bytes(B.make_desc(**shape))
         self.workspace = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
         with torch.cuda.device(self.device):
             self.handle = B.lif_create_layer(B.make_desc(
                 **shape, host_bundles=host_bundles, pred_A=pred_A, pred_B=pred_B, pred_c=pred_c,
-                bias_up=bias_up, bias_down=bias_down, cache=self.cache, workspace=self.workspace))
+                bias_up=bias_up, bias_down=bias_down, gate=gate, cache=self.cache,
+                workspace=self.workspace))
             torch.cuda.synchronize()   # the reset ran on the default stream
         self._lists = B.lif_get_lists(self.handle)
         self.counts = self._view("counts", B.CNT_LEN)
@@ -87,25 +92,29 @@ class Layer:
             pass
 
 
-def pinned_store(d_ff: int, d_model: int) -> torch.Tensor:
+def pinned_store(d_ff: int, d_model: int, n_vec: int = 2) -> torch.Tensor:
     """Pinned (and, under unified addressing, device-mapped) host tensor for one layer's
-    bundle store, fp16 [d_ff][2*d_model]."""
-    return torch.empty(d_ff, 2 * d_model, dtype=torch.float16, pin_memory=True)
+    bundle store, fp16 [d_ff][n_vec*d_model] (n_vec = 3 when the gate row is bundled)."""
+    return torch.empty(d_ff, n_vec * d_model, dtype=torch.float16, pin_memory=True)
 
 
 def build_stack(cfg, device="cuda:0", n_layers: Optional[int] = None, capacity_margin: float = 8.0,
-                ffn_mode: int = 0, gen_device=None) -> List[Layer]:
+                ffn_mode: int = 0, gen_device=None, gate_mode: int = 0, activation: int = 0,
+                activation_threshold: float = 0.0) -> List[Layer]:
     """Generate the weights of a named synthetic configuration and create its layers."""
     from . import workloads as W
     layers = []
     gen_device = gen_device or device
     for l in range(n_layers or cfg.n_layers):
-        store = pinned_store(cfg.d_ff, cfg.d_model)
-        w = W.make_layer(cfg, l, device=gen_device, bundles_out=store)
+        store = pinned_store(cfg.d_ff, cfg.d_model, 3 if gate_mode == B.GATE_BUNDLED else 2)
+        w = W.make_layer(cfg, l, device=gen_device, bundles_out=store, gate_mode=gate_mode,
+                         act_threshold=activation_threshold)
         cap = W.window_capacity(cfg, w["p"], capacity_margin)
-        dev = lambda t: t.to(device).contiguous()
+        dev = lambda t: None if t is None else t.to(device).contiguous()
         layers.append(Layer(d_model=cfg.d_model, d_ff=cfg.d_ff, rank=cfg.rank, window_k=cfg.window_k,
                             capacity=cap, host_bundles=store, pred_A=dev(w["A"]), pred_B=dev(w["B"]),
                             pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), n_streams=cfg.n_streams,
-                            ffn_mode=ffn_mode, device=device))
+                            ffn_mode=ffn_mode, gate_mode=gate_mode, gate=dev(w.get("gate")),
+                            activation=activation, activation_threshold=activation_threshold,
+                            device=device))
     return layers

@@ -16,7 +16,11 @@ The five named configurations stand in for trained ReLU models decoding a text c
   probability ``p_i``;
 * low-rank predictor factors ``A[d][r]``, ``B[r][F]`` ~ N(0, 1) with unit-norm columns, so a
   N(0, I) input gives N(0, 1) scores; per-neuron offset ``c_i = Phi^-1(p_i)``, threshold 0;
-* decode inputs ``x_t = rho * x_{t-1} + noise * eps_t``, ``x_0, eps_t ~ N(0, I)``, fp16.
+* decode inputs ``x_t = rho * x_{t-1} + noise * eps_t``, ``x_0, eps_t ~ N(0, I)``, fp16;
+* gated layers (Appendix C, Llama 2): a gate row per neuron drawn like the up row; the bias
+  ``b_i = threshold + ||gate_i|| * Phi^-1(p_i)`` makes the gate value pass the activation's
+  threshold with probability ``p_i``; bundle = gate | up | down, or up | down with the gate
+  rows returned apart as the resident gate projection.
 """
 from __future__ import annotations
 
@@ -65,6 +69,9 @@ CONFIGS: Dict[str, LifConfig] = {
                       _ar_noise(0.7), 3),
     "batched8": LifConfig("batched8", 48, 7168, 28672, 256, 5, 8, 64, 0.03, 1.0, 0.9,
                           _ar_noise(0.9), 4),
+    # gated FFN of Appendix C (Llama 2 7B shapes: sparsity above 90 %, window of 2, rank 256)
+    "llama2_7b": LifConfig("llama2_7b", 32, 4096, 11008, 256, 2, 1, 64, 0.08, 1.0, 0.9,
+                           _ar_noise(0.9), 5),
 }
 
 
@@ -90,28 +97,42 @@ def popularity(cfg: LifConfig, layer: int) -> torch.Tensor:
     return torch.clamp(0.5 * (lo + hi) * e, max=0.95)
 
 
+GATE_NONE, GATE_BUNDLED, GATE_RESIDENT = range(3)
+
+
 def make_layer(cfg: LifConfig, layer: int, device: Optional[torch.device] = None,
-               bundles_out: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+               bundles_out: Optional[torch.Tensor] = None, gate_mode: int = GATE_NONE,
+               act_threshold: float = 0.0) -> Dict[str, torch.Tensor]:
     """Generate one layer.  Random draws run on ``device`` (Philox on CUDA, MT on CPU; a run
     feeds the same tensors to every consumer, so the two never need to agree).  ``bundles_out``
     (fp16 ``[F][2d]``, typically a pinned host tensor) receives the bundle store; otherwise
-    the bundles stay on ``device``."""
+    the bundles stay on ``device``.  ``gate_mode``: GATE_BUNDLED gives ``[F][3d]`` bundles
+    (gate | up | down), GATE_RESIDENT ``[F][2d]`` bundles (up | down) plus ``gate`` ``[F][d]``;
+    in both ``bias_up`` is the gate's bias, placed so that the gate value passes
+    ``act_threshold`` with probability p_i."""
     device = torch.device(device or "cpu")
     d, F, r = cfg.d_model, cfg.d_ff, cfg.rank
     g = _generator(device, cfg.seed * 1000 + layer + 500)
     p = popularity(cfg, layer)
     q = torch.special.ndtri(p)                                        # Phi^-1(p_i), float64
 
-    bundles = torch.empty(F, 2 * d, dtype=torch.float16, device=device)
+    drawn = 2 if gate_mode == GATE_NONE else 3                        # vectors drawn per neuron
+    stored = 2 if gate_mode != GATE_BUNDLED else 3                    # vectors per bundle
+    bundles = torch.empty(F, stored * d, dtype=torch.float16, device=device)
+    gate = torch.empty(F, d, dtype=torch.float16, device=device) if gate_mode == GATE_RESIDENT else None
     norms = torch.empty(F, dtype=torch.float64, device=device)
-    rows = max(1, min(F, (64 << 20) // (2 * d)))                      # ~256 MB fp32 scratch
+    rows = max(1, min(F, (64 << 20) // (drawn * d)))                  # ~256 MB fp32 scratch
     for i0 in range(0, F, rows):
         i1 = min(F, i0 + rows)
-        blk = (torch.randn(i1 - i0, 2 * d, generator=g, device=device, dtype=torch.float32)
+        blk = (torch.randn(i1 - i0, drawn * d, generator=g, device=device, dtype=torch.float32)
                * 0.02).to(torch.float16)
-        bundles[i0:i1] = blk
+        if gate is None:
+            bundles[i0:i1] = blk
+        else:
+            gate[i0:i1] = blk[:, :d]
+            bundles[i0:i1] = blk[:, d:]
         norms[i0:i1] = blk[:, :d].double().square().sum(dim=1).sqrt()
-    bias_up = (norms * q.to(device)).to(torch.float16)
+    bias_up = (norms * q.to(device) + act_threshold).to(torch.float16)
 
     A = torch.randn(d, r, generator=g, device=device, dtype=torch.float32)
     A = (A / A.norm(dim=0, keepdim=True)).to(torch.float16)
@@ -120,6 +141,8 @@ def make_layer(cfg: LifConfig, layer: int, device: Optional[torch.device] = None
     c = q.to(torch.float32).to(device)
 
     out = {"bias_up": bias_up, "A": A.contiguous(), "B": B.contiguous(), "c": c, "p": p}
+    if gate is not None:
+        out["gate"] = gate
     if bundles_out is not None:
         bundles_out.copy_(bundles)
         out["bundles"] = bundles_out
