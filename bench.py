@@ -103,6 +103,16 @@ def whole_job_tokens_per_s(steps, world, ms_slowest):
     return world * steps / (ms_slowest / 1e3)
 
 
+GATE_MODES = {"none": 0, "bundled": 1, "resident": 2}
+
+
+def _gate_setup(args):
+    """(gate_mode, activation, threshold): gated runs use FATReLU on the gate value (Appendix C,
+    Llama 2); ungated runs use ReLU."""
+    gm = GATE_MODES[args.gate]
+    return (gm, 2, args.act_threshold) if gm else (0, 0, 0.0)
+
+
 def _inputs(cfg, n_tokens, device, W):
     return W.make_inputs(cfg.scaled(steps=max(cfg.steps, n_tokens)), device=device)[:n_tokens]
 
@@ -131,7 +141,9 @@ def run_ours(args):
     cfg = rank_config(cfg, rank)
     K, Wm = args.steps, args.warmup
     n_tok = Wm + K
-    layers = R.build_stack(cfg, dev, n_layers=args.layers)
+    gate_mode, activation, act_thr = _gate_setup(args)
+    layers = R.build_stack(cfg, dev, n_layers=args.layers, gate_mode=gate_mode, activation=activation,
+                           activation_threshold=act_thr)
     handles = [l.handle for l in layers]
     L, S, d = len(layers), cfg.n_streams, cfg.d_model
     X = _inputs(cfg, n_tok, dev, W)
@@ -219,7 +231,8 @@ def run_ours(args):
     reps = 20
     if S == 1:
         launchers = {name: (lambda l, kind=kind: B.lif_profile_launch(handles[l], kind, dev_x, Y[l], sc))
-                     for kind, name in enumerate(B.KERNELS)}
+                     for kind, name in enumerate(B.KERNELS)
+                     if not (gate_mode == B.GATE_RESIDENT and name == "predict_z")}
     else:
         # several streams: the staged entry points (predictor = 2 kernels; FFN = the tensor-core
         # up, down and partial-sum kernels over all active rows)
@@ -264,27 +277,33 @@ def run_ours(args):
         del hbuf, dbuf
 
     if rank == 0:
-        beta = cfg.bundle_bytes
+        beta = (3 if gate_mode == B.GATE_BUNDLED else 2) * d * 2
+        row_extra = 8 if gate_mode == B.GATE_RESIDENT else 2    # bias, or neuron id + gate value
         peak, peak_kind = _peaks()
         # algorithmic bytes of one launch: bundle + bias per row, x in, partials out
-        ffn_bytes = (n_act_l * (beta + 2) + L * S * 6 * d) / L
+        ffn_bytes = (n_act_l * (beta + row_extra) + L * S * 6 * d) / L
         ffn_gbs = ffn_bytes / (kernel_us["ffn_active"] * 1e-6) / 1e9
         fetch_bytes = n_load_l * beta / L
         fetch_gbs = fetch_bytes / (kernel_us["fetch"] * 1e-6) / 1e9
-        pred_bytes = 2 * cfg.rank * (d + cfg.d_ff) + 4 * cfg.d_ff
-        pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_z"] + kernel_us["predict_scores"]
+        if gate_mode == B.GATE_RESIDENT:       # gate matrix + bias in, gate values out
+            pred_bytes = 2 * cfg.d_ff * d + 2 * cfg.d_ff + 4 * S * cfg.d_ff
+            pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_scores"]
+        else:
+            pred_bytes = 2 * cfg.rank * (d + cfg.d_ff) + 4 * cfg.d_ff
+            pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_z"] + kernel_us["predict_scores"]
         pred_gbs = pred_bytes / (pred_us * 1e-6) / 1e9
         split = None
         if S == 1:
-            split = {"already_cached_rows_GBs": (n_hit_l * (beta + 2) / L + 6 * d) / (kernel_us["ffn_hits"] * 1e-6) / 1e9,
-                     "new_rows_GBs": (n_load_l * (beta + 2) / L + 6 * d) / (kernel_us["ffn_new"] * 1e-6) / 1e9}
+            split = {"already_cached_rows_GBs": (n_hit_l * (beta + row_extra) / L + 6 * d) / (kernel_us["ffn_hits"] * 1e-6) / 1e9,
+                     "new_rows_GBs": (n_load_l * (beta + row_extra) / L + 6 * d) / (kernel_us["ffn_new"] * 1e-6) / 1e9}
         out = {
             "metric": METRIC, "value": whole_job_tokens_per_s(K, world, ms_total), "unit": UNIT,
             "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms_total / K,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
             "config": {"workload": f"{cfg.name}: {L} layers d_model={d} d_ff={cfg.d_ff} rank={cfg.rank} "
-                                   f"window_k={cfg.window_k} streams={S}, AR(1) decode inputs",
+                                   f"window_k={cfg.window_k} streams={S}, AR(1) decode inputs"
+                                   + (f", gated FFN ({args.gate} gate, FATReLU {act_thr})" if gate_mode else ""),
                        "l2": "per-token working set (all layers' window caches, "
                              f"{s1[3] / n_tok * beta / 2**20:.0f} MiB) exceeds the 126 MB L2",
                        "bundle_store": "pinned host memory, read by the fetch kernel",
@@ -298,7 +317,8 @@ def run_ours(args):
                          "bound": "hbm",
                          "achieved": ffn_gbs, "peak": peak, "unit": "GB/s", "frac": ffn_gbs / peak,
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": ffn_gbs / NOMINAL_HBM_GBS,
-                         "traffic": FFN_TRAFFIC_RATIO * ffn_bytes if FFN_TRAFFIC_RATIO and S == 1 else None,
+                         "traffic": FFN_TRAFFIC_RATIO * ffn_bytes
+                                    if FFN_TRAFFIC_RATIO and S == 1 and not gate_mode else None,
                          "traffic_how": "dram read+write bytes per algorithmic byte from the ncu capture in "
                                         "profiles/sparse_ffn_kernel_opt6p7b_12layers.md (12 layers, "
                                         "451-529 rows per launch), scaled by this run's rows per launch",
@@ -311,7 +331,8 @@ def run_ours(args):
                           "peak": link_peak, "unit": "GB/s", "frac": fetch_gbs / link_peak,
                           "peak_kind": "of measured (1 GiB pinned cudaMemcpyAsync, this run)",
                           "bytes_per_launch": fetch_bytes, "us_per_launch": kernel_us["fetch"]},
-            "predictor": {"bound": "hbm", "achieved": pred_gbs, "unit": "GB/s", "frac": pred_gbs / peak},
+            "predictor": {"bound": "hbm", "achieved": pred_gbs, "unit": "GB/s", "frac": pred_gbs / peak,
+                          "bytes_per_launch": pred_bytes, "us_per_launch": pred_us},
             "kernel_us_per_launch": kernel_us,
             "per_token": {"rows_active": rows_active / K, "rows_loaded": fetched / beta / K,
                           "rows_moved": rows_moved / K},
@@ -322,7 +343,8 @@ def run_ours(args):
             "clocks": clock_info,
         }
         if args.cpu_baseline:
-            out["cpu_baseline"] = cpu_baseline(cfg, layers, X, args.cpu_layers, args.cpu_tokens)
+            out["cpu_baseline"] = cpu_baseline(cfg, layers, X, args.cpu_layers, args.cpu_tokens,
+                                               _gate_setup(args))
         print(json.dumps(out), flush=True)
     B.lif_graph_destroy(graph)
     for l in layers:
@@ -341,7 +363,9 @@ def run_kernel_loop(args):
     from paper_2312_11514_b200 import workloads as W
     dev = "cuda:0"
     cfg = W.CONFIGS[args.config]
-    layers = R.build_stack(cfg, dev, n_layers=args.layers)
+    gate_mode, activation, act_thr = _gate_setup(args)
+    layers = R.build_stack(cfg, dev, n_layers=args.layers, gate_mode=gate_mode, activation=activation,
+                           activation_threshold=act_thr)
     handles = [l.handle for l in layers]
     L, S, d = len(layers), cfg.n_streams, cfg.d_model
     X = _inputs(cfg, args.warmup, dev, W)
@@ -366,7 +390,8 @@ def run_kernel_loop(args):
             B.lif_profile_launch(handles[l], B.KERNELS.index(args.kernel_loop), dev_x, Y[l], sc)
     torch.cuda.synchronize()
     print(json.dumps({"kernel": args.kernel_loop, "layers": L, "warmup_tokens": args.warmup,
-                      "rows_per_launch": rows, "bundle_bytes": cfg.bundle_bytes}), flush=True)
+                      "rows_per_launch": rows,
+                      "bundle_bytes": (3 if gate_mode == 1 else 2) * d * 2}), flush=True)
     B.lif_graph_destroy(graph)
     for l in layers:
         l.close()
@@ -435,38 +460,47 @@ def _oracle_threads():
     return len(os.sched_getaffinity(0))
 
 
-def _oracle_layers(cfg, tensors, O):
+def _oracle_layers(cfg, tensors, O, gate=(0, 0, 0.0)):
     import numpy as np
     out = []
     for w, cap in tensors:
         out.append(dict(A=w["A"].cpu().numpy().astype(np.float64), B=w["B"].cpu().numpy().astype(np.float64),
                         c=w["c"].cpu().numpy().astype(np.float64), bundles=w["bundles"].cpu().numpy(),
                         bias_up=w["bias_up"].cpu().numpy(),
-                        cache=O.NeuronCache(cfg.d_model, cfg.d_ff, cap, cfg.window_k)))
+                        gate=w["gate"].cpu().numpy() if gate[0] == 2 else None,
+                        cache=O.NeuronCache(cfg.d_model, cfg.d_ff, cap, cfg.window_k,
+                                            n_vec=3 if gate[0] == 1 else 2)))
     return out
 
 
-def _oracle_token(ol, x_np, O):
+def _oracle_token(ol, x_np, O, gate=(0, 0, 0.0)):
+    gm, act, thr = gate
     for w in ol:
-        O.decode_step(w["cache"], x_np, w["A"], w["B"], w["c"], 0.0, w["bundles"], w["bias_up"])
+        if gm == 2:
+            O.decode_step_gate_predictor(w["cache"], x_np, w["gate"], w["bias_up"], w["bundles"],
+                                         activation=act, threshold=thr)
+        else:
+            O.decode_step(w["cache"], x_np, w["A"], w["B"], w["c"], 0.0, w["bundles"], w["bias_up"],
+                          activation=act, threshold=thr, gated=gm == 1)
 
 
-def cpu_baseline(cfg, layers, X, n_layers, n_tokens):
+def cpu_baseline(cfg, layers, X, n_layers, n_tokens, gate=(0, 0, 0.0)):
     """The oracle, as it stands, on a bounded sample: the first n_layers layers over the first
     n_tokens tokens; tokens/s scaled to the full stack by layers."""
     from oracle import lif_oracle as O
     n_layers = min(n_layers, len(layers))
     tensors = [({"A": l.keep["pred_A"], "B": l.keep["pred_B"], "c": l.keep["pred_c"],
-                 "bundles": l.keep["host_bundles"], "bias_up": l.keep["bias_up"]}, l.capacity)
+                 "bundles": l.keep["host_bundles"], "bias_up": l.keep["bias_up"],
+                 "gate": l.keep["gate"]}, l.capacity)
                for l in layers[:n_layers]]
-    ol = _oracle_layers(cfg, tensors, O)
+    ol = _oracle_layers(cfg, tensors, O, gate)
     xs = X[:n_tokens].cpu().numpy()
     warm = min(cfg.window_k + 1, n_tokens - 1)
     for t in range(warm):
-        _oracle_token(ol, xs[t], O)
+        _oracle_token(ol, xs[t], O, gate)
     t0 = time.perf_counter()
     for t in range(warm, n_tokens):
-        _oracle_token(ol, xs[t], O)
+        _oracle_token(ol, xs[t], O, gate)
     dt = time.perf_counter() - t0
     per_layer_step = dt / ((n_tokens - warm) * n_layers)
     return {"value": 1.0 / (per_layer_step * cfg.n_layers), "unit": UNIT, "cores": _oracle_threads(),
@@ -483,32 +517,33 @@ def run_reference(args):
     from oracle import lif_oracle as O
     from paper_2312_11514_b200 import workloads as W
     cfg = W.CONFIGS[args.config]
+    gate = _gate_setup(args)
     gen = "cuda:0" if torch.cuda.is_available() else "cpu"
+    mk = lambda l: W.make_layer(cfg, l, device=gen, gate_mode=gate[0], act_threshold=gate[2])
     L = args.layers or cfg.n_layers
     if not args.layers:
         # bound the run: time one layer-step, then keep as many layers as fit ~2 minutes
-        w0 = {k: v.cpu() for k, v in W.make_layer(cfg, 0, device=gen).items()}
-        probe = _oracle_layers(cfg, [(w0, W.window_capacity(cfg, w0["p"]))], O)
+        w0 = {k: v.cpu() for k, v in mk(0).items()}
+        probe = _oracle_layers(cfg, [(w0, W.window_capacity(cfg, w0["p"]))], O, gate)
         x0 = _inputs(cfg, 2, gen, W).cpu().numpy()
-        _oracle_token(probe, x0[0], O)
+        _oracle_token(probe, x0[0], O, gate)
         t0 = time.perf_counter()
-        _oracle_token(probe, x0[1], O)
+        _oracle_token(probe, x0[1], O, gate)
         per = max(time.perf_counter() - t0, 1e-4)
         L = max(1, min(cfg.n_layers, int(120.0 / ((args.steps + args.warmup) * per))))
         del probe, w0
     tensors = []
     for l in range(L):
-        w = W.make_layer(cfg, l, device=gen)
-        w = {k: v.cpu() for k, v in w.items()}
+        w = {k: v.cpu() for k, v in mk(l).items()}
         tensors.append((w, W.window_capacity(cfg, w["p"])))
-    ol = _oracle_layers(cfg, tensors, O)
+    ol = _oracle_layers(cfg, tensors, O, gate)
     K, Wm = args.steps, args.warmup
     xs = _inputs(cfg, Wm + K, gen, W).cpu().numpy()
     for t in range(Wm):
-        _oracle_token(ol, xs[t], O)
+        _oracle_token(ol, xs[t], O, gate)
     t0 = time.perf_counter()
     for t in range(Wm, Wm + K):
-        _oracle_token(ol, xs[t], O)
+        _oracle_token(ol, xs[t], O, gate)
     dt = time.perf_counter() - t0
     v = K / dt * (cfg.n_layers / L)
     cores = _oracle_threads()
@@ -531,6 +566,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="opt6p7b")
     ap.add_argument("--layers", type=int, default=None, help="use only the first N layers")
+    ap.add_argument("--gate", default="none", choices=sorted(GATE_MODES),
+                    help="gated FFN: gate row inside the bundle, or resident gate projection as the "
+                         "predictor (use with --config llama2_7b)")
+    ap.add_argument("--act-threshold", type=float, default=0.05, help="FATReLU threshold of gated runs")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--cpu-layers", type=int, default=2)
     ap.add_argument("--cpu-tokens", type=int, default=30)

@@ -212,3 +212,20 @@ def staged_step(gpu, ora, x_dev, bufs, whole_cache=False):
     assert_y_close(y.cpu().numpy().astype(np.float64), ref_y, flips)
     return dict(n_active=na, n_load=len(ref_lists["load_ids"]), n_evict=len(ref_lists["evict_ids"]),
                 n_border=n_border, k_eff=ref_lists["k_eff"], num_used=ref_lists["num_used"])
+
+
+def check_decode_step(gpu, ora, x_np, y_np):
+    """After one lif_decode_step of ``gpu`` on ``x_np``: the active list may differ from the
+    oracle's only at borderline scores; from that list on, the oracle reproduces lists, window
+    state and (within tolerance) the output ``y_np`` [S][d].  Returns the step's lists."""
+    g = gpu.lists()
+    scores = ora.scores(x_np)
+    assert_mask_borderline(g["active_idx"], scores, ora.theta)
+    lists = ora.cache.window_update(g["active_idx"])
+    ora.cache.insert(lists, ora.bundles, ora.bias_up)
+    compare_lists_and_state(gpu, ora, lists)
+    slots = lists["active_slots"]
+    gate_pre = scores[:, g["active_idx"]] if ora.gate_mode == 2 else None
+    ref_y, flips = ffn_reference(ora, slots, x_np, gate_pre)
+    assert_y_close(y_np, ref_y, flips)
+    return lists

@@ -8,7 +8,6 @@ import psutil
 import pytest
 import torch
 
-from oracle import lif_oracle as O
 from paper_2312_11514_b200 import binding as B
 from paper_2312_11514_b200 import runtime as R
 from paper_2312_11514_b200 import workloads as W
@@ -19,9 +18,11 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _run_config(name, n_tokens, sample_layers, oracle_tokens=None):
+def _run_config(name, n_tokens, sample_layers, oracle_tokens=None, gate_mode=0, activation=0, thr=0.0):
     cfg = W.CONFIGS[name]
-    store_gib = cfg.n_layers * cfg.d_ff * cfg.bundle_bytes / 2**30
+    n_vec = 3 if gate_mode == B.GATE_BUNDLED else 2
+    bundle_bytes = n_vec * cfg.d_model * 2
+    store_gib = cfg.n_layers * cfg.d_ff * bundle_bytes / 2**30
     if psutil.virtual_memory().available / 2**30 < store_gib * 1.3 + 8:
         pytest.skip(f"host memory too small for the {store_gib:.0f} GiB bundle store")
     n_tokens = min(n_tokens, cfg.steps)
@@ -29,14 +30,16 @@ def _run_config(name, n_tokens, sample_layers, oracle_tokens=None):
     L, S, d, F = cfg.n_layers, cfg.n_streams, cfg.d_model, cfg.d_ff
     layers, oras = [], {}
     for l in range(L):
-        store = R.pinned_store(F, d)
-        w = W.make_layer(cfg, l, device=DEV, bundles_out=store)
+        store = R.pinned_store(F, d, n_vec)
+        w = W.make_layer(cfg, l, device=DEV, bundles_out=store, gate_mode=gate_mode, act_threshold=thr)
         cap = W.window_capacity(cfg, w["p"])
         layers.append(R.Layer(d_model=d, d_ff=F, rank=cfg.rank, window_k=cfg.window_k, capacity=cap,
                               host_bundles=store, pred_A=w["A"], pred_B=w["B"], pred_c=w["c"],
-                              bias_up=w["bias_up"], n_streams=S, device=DEV))
+                              bias_up=w["bias_up"], n_streams=S, gate_mode=gate_mode, gate=w.get("gate"),
+                              activation=activation, activation_threshold=thr, device=DEV))
         if l in sample_layers:
-            oras[l] = P.OracleLayer(w, d, F, cap, cfg.window_k)
+            oras[l] = P.OracleLayer(w, d, F, cap, cfg.window_k, activation=activation,
+                                    act_threshold=thr, gate_mode=gate_mode)
         del w
     X = W.make_inputs(cfg, device=DEV)
     dev_x = torch.empty(S, d, dtype=torch.float16, device=DEV)
@@ -44,7 +47,7 @@ def _run_config(name, n_tokens, sample_layers, oracle_tokens=None):
     sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
     torch.cuda.synchronize()
     graph = B.lif_graph_capture([l.handle for l in layers], dev_x, Y, sc, sf)
-    n_border = n_loaded = 0
+    n_loaded = 0
     for t in range(n_tokens):
         with torch.cuda.stream(sc):
             dev_x.copy_(X[t])
@@ -55,12 +58,7 @@ def _run_config(name, n_tokens, sample_layers, oracle_tokens=None):
         x_np = X[t].cpu().numpy()
         y_np = Y.cpu().numpy().astype(np.float64)
         for l, ora in oras.items():
-            g = layers[l].lists()
-            logits, _, lists, ref_y = O.decode_step(ora.cache, x_np, ora.A, ora.B, ora.c, 0.0,
-                                                    ora.bundles, ora.bias_up, act=g["active_idx"])
-            n_border += P.assert_mask_borderline(g["active_idx"], logits, 0.0)
-            P.compare_lists_and_state(layers[l], ora, lists)
-            P.assert_y_close(y_np[l], ref_y)
+            lists = P.check_decode_step(layers[l], ora, x_np, y_np[l])
             n_loaded += len(lists["load_ids"])
     # every layer: properties that hold at any size
     for l, lay in enumerate(layers):
@@ -69,7 +67,7 @@ def _run_config(name, n_tokens, sample_layers, oracle_tokens=None):
         assert st.status == B.LIF_OK, (l, st.status)
         n = g["num_used"]
         assert g["step"] == n_tokens and 0 < n <= lay.capacity
-        assert st.bytes_fetched % cfg.bundle_bytes == 0 and st.bytes_fetched >= n * cfg.bundle_bytes
+        assert st.bytes_fetched % bundle_bytes == 0 and st.bytes_fetched >= n * bundle_bytes
         ptr = g["pointers"][:n]
         assert len(np.unique(ptr)) == n and ptr.min() >= 0
         assert (g["slot_of"][ptr] == np.arange(n)).all() and (g["slot_of"] >= 0).sum() == n
@@ -87,7 +85,6 @@ def _run_config(name, n_tokens, sample_layers, oracle_tokens=None):
     B.lif_graph_destroy(graph)
     for lay in layers:
         lay.close()
-    return n_border
 
 
 def test_opt6p7b_full_stack_all_tokens():
@@ -104,3 +101,11 @@ def test_phi2_full_stack():
 
 def test_batched8_full_stack_eight_streams():
     _run_config("batched8", 8, sample_layers=(1, 46), oracle_tokens=6)
+
+
+@pytest.mark.parametrize("gate_mode", [B.GATE_BUNDLED, B.GATE_RESIDENT])
+def test_llama2_7b_gated_full_stack(gate_mode):
+    # Appendix C, Llama 2: gated FFN with FATReLU, window of 2; the gate row either travels in
+    # the bundle (low-rank predictor) or stays resident and is the predictor
+    _run_config("llama2_7b", 32, sample_layers=(0, 20), oracle_tokens=24, gate_mode=gate_mode,
+                activation=B.ACT_FATRELU, thr=0.05)

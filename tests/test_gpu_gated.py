@@ -67,18 +67,8 @@ def test_gated_decode_step(gate_mode, S, two_streams, fused):
     n_evict = 0
     for t in range(cfg.steps):
         B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
-        g = gpu.lists()
-        x_np = X[t].cpu().numpy()
-        scores = ora.scores(x_np)
-        P.assert_mask_borderline(g["active_idx"], scores, ora.theta)
-        lists = ora.cache.window_update(g["active_idx"])
-        ora.cache.insert(lists, ora.bundles, ora.bias_up)
-        P.compare_lists_and_state(gpu, ora, lists)
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
         P.compare_cache_rows(gpu, ora)
-        slots = lists["active_slots"]
-        gate_pre = scores[:, g["active_idx"]] if gate_mode == B.GATE_RESIDENT else None
-        ref_y, flips = P.ffn_reference(ora, slots, x_np, gate_pre)
-        P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y, flips)
         n_evict += len(lists["evict_ids"])
     assert n_evict > 0
     gpu.close()
