@@ -15,6 +15,10 @@ namespace {
 
 constexpr int kGateTile = 32;          // neurons per CTA = one mask word
 constexpr int kRowsPerWarp = 4;
+#ifndef LIF_GATE_DEPTH
+#define LIF_GATE_DEPTH 2
+#endif
+constexpr int kDepth = LIF_GATE_DEPTH;   // load groups in flight per lane (4 x 16 bytes each)
 
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   uint4 v;
@@ -50,13 +54,20 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
   const int nvec = d >> 3;
   const int i0 = blockIdx.x * kGateTile + warp * kRowsPerWarp;   // this warp's first neuron
 
-  // The gate rows are weights: the first 16-byte piece of each of the four rows is in flight
-  // before the dependency wait; x (possibly written by the previous kernel) comes after it.
-  uint4 w[kRowsPerWarp];
+  // Each lane keeps kDepth groups of loads in flight, a group being one 16-byte piece of each of
+  // its four rows.  The gate rows are weights: the first groups are issued before the
+  // dependency wait; x (possibly written by the previous kernel) comes after it.
+  const int ngroups = (nvec + 31) >> 5;
+  auto load_group = [&](uint4* dst, int g) {
+    const int c = lane + 32 * g;
 #pragma unroll
-  for (int q = 0; q < kRowsPerWarp; ++q)
-    w[q] = (i0 + q < F && lane < nvec) ? ldg_stream(gate + (size_t)(i0 + q) * d + lane * 8)
-                                       : make_uint4(0, 0, 0, 0);
+    for (int q = 0; q < kRowsPerWarp; ++q)
+      dst[q] = (i0 + q < F && c < nvec) ? ldg_stream(gate + (size_t)(i0 + q) * d + c * 8)
+                                        : make_uint4(0, 0, 0, 0);
+  };
+  uint4 w[kDepth][kRowsPerWarp];
+#pragma unroll
+  for (int j = 0; j < kDepth; ++j) load_group(w[j], j);
   pdl_wait();
   pdl_trigger();
   for (int c = tid; c < S * nvec; c += kThreads) xs[c] = reinterpret_cast<const uint4*>(x)[c];
@@ -68,27 +79,26 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
 #pragma unroll
     for (int s = 0; s < S; ++s) acc[q][s] = 0.f;
 
-  for (int c = lane; c < nvec; c += 32) {
-    uint4 nxt[kRowsPerWarp];
-    const int cn = c + 32;
+  for (int g0 = 0; g0 < ngroups; g0 += kDepth) {
 #pragma unroll
-    for (int q = 0; q < kRowsPerWarp; ++q)
-      nxt[q] = (i0 + q < F && cn < nvec) ? ldg_stream(gate + (size_t)(i0 + q) * d + cn * 8)
-                                         : make_uint4(0, 0, 0, 0);
-    float wf[kRowsPerWarp][8];
+    for (int j = 0; j < kDepth; ++j) {
+      const int c = lane + 32 * (g0 + j);
+      if (c < nvec) {
+        float wf[kRowsPerWarp][8];
 #pragma unroll
-    for (int q = 0; q < kRowsPerWarp; ++q) unpack8(w[q], wf[q]);
+        for (int q = 0; q < kRowsPerWarp; ++q) unpack8(w[j][q], wf[q]);
 #pragma unroll
-    for (int s = 0; s < S; ++s) {
-      float xf[8];
-      unpack8(xs[s * nvec + c], xf);
+        for (int s = 0; s < S; ++s) {
+          float xf[8];
+          unpack8(xs[s * nvec + c], xf);
 #pragma unroll
-      for (int q = 0; q < kRowsPerWarp; ++q)
+          for (int q = 0; q < kRowsPerWarp; ++q)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[q][s] = fmaf(wf[q][e], xf[e], acc[q][s]);
+            for (int e = 0; e < 8; ++e) acc[q][s] = fmaf(wf[q][e], xf[e], acc[q][s]);
+        }
+      }
+      load_group(w[j], g0 + j + kDepth);     // past the end of the row: no load, zeros
     }
-#pragma unroll
-    for (int q = 0; q < kRowsPerWarp; ++q) w[q] = nxt[q];
   }
 
   // warp sums in a fixed order; lane q finishes neuron i0 + q
