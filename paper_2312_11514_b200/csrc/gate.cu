@@ -5,20 +5,24 @@
 // a neuron is active iff g exceeds the activation's threshold for at least one stream, and the
 // FFN reuses g instead of recomputing it.  A dense fp16 GEMV over [d_ff][d_model] with fp32
 // accumulation: every gate row is read once with 16-byte loads.  A CTA owns 32 consecutive
-// neurons (one word of the bit mask), a warp four of them, so a thread keeps four independent
-// rows in flight.  Bound: HBM bandwidth, 2*d_model bytes per neuron.
+// neurons (one word of the bit mask; 8 or 16, whole bytes of it, are possible too), a warp four
+// of them, so a thread keeps four independent rows in flight.  Bound: HBM bandwidth,
+// 2*d_model bytes per neuron.
 #include "lif_internal.cuh"
 #include "mask_compact.cuh"
 
 namespace lif {
 namespace {
 
-constexpr int kGateTile = 32;          // neurons per CTA = one mask word
-constexpr int kRowsPerWarp = 4;
+#ifndef LIF_GATE_ROWS
+#define LIF_GATE_ROWS 4
+#endif
 #ifndef LIF_GATE_DEPTH
 #define LIF_GATE_DEPTH 2
 #endif
-constexpr int kDepth = LIF_GATE_DEPTH;   // load groups in flight per lane (4 x 16 bytes each)
+constexpr int kRowsPerWarp = LIF_GATE_ROWS;           // 1, 2 or 4
+constexpr int kGateTile = 8 * kRowsPerWarp;           // neurons per CTA: 1, 2 or 4 bytes of the mask
+constexpr int kDepth = LIF_GATE_DEPTH;   // load groups in flight per lane (one 16-byte piece per row each)
 
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   uint4 v;
@@ -55,7 +59,7 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
   const int i0 = blockIdx.x * kGateTile + warp * kRowsPerWarp;   // this warp's first neuron
 
   // Each lane keeps kDepth groups of loads in flight, a group being one 16-byte piece of each of
-  // its four rows.  The gate rows are weights: the first groups are issued before the
+  // its rows.  The gate rows are weights: the first groups are issued before the
   // dependency wait; x (possibly written by the previous kernel) comes after it.
   const int ngroups = (nvec + 31) >> 5;
   auto load_group = [&](uint4* dst, int g) {
@@ -132,8 +136,13 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
   }
   __syncthreads();
   if (warp == 0) {
-    const unsigned m = __ballot_sync(0xffffffffu, act_flag[lane] != 0);
-    if (lane == 0) mask_words[blockIdx.x] = m;
+    // the CTA's 8, 16 or 32 bits are whole bytes of the mask: a plain store, no merging
+    const unsigned m = __ballot_sync(0xffffffffu, lane < kGateTile && act_flag[lane] != 0);
+    if (lane == 0) {
+      if (kGateTile == 32) mask_words[blockIdx.x] = m;
+      else if (kGateTile == 16) reinterpret_cast<uint16_t*>(mask_words)[blockIdx.x] = (uint16_t)m;
+      else reinterpret_cast<uint8_t*>(mask_words)[blockIdx.x] = (uint8_t)m;
+    }
   }
   if (!compact) return;     // the consumer reads the bit mask itself
   compact_mask_last_cta(mask_words, nwords, ticket, active_idx, n_active, warp_sums, &is_last);
@@ -155,7 +164,7 @@ cudaError_t launch_gate_s(lif_layer* L, const __half* x, float* logits, int32_t*
                   (const __half*)D.dev_gate, (const __half*)D.dev_bias_up, theta, D.d_model,
                   D.d_ff, L->gate_val, logits, L->mask_words,
                   (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
-                  grid);
+                  (D.d_ff + 31) / 32);
 }
 
 }  // namespace

@@ -235,7 +235,8 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
   if (D.n_streams != 1) return cudaErrorInvalidValue;
   if (D.gate_mode == LIF_GATE_RESIDENT)
     return kernel == LIF_KERNEL_PREDICT_SCORES
-               ? launch_gate_predict(L, x, nullptr, L->active_idx, L->n_tmp, st, nullptr, 1)
+               ? launch_gate_predict(L, x, nullptr, L->active_idx, L->n_tmp, st, nullptr,
+                                     L->fused_plan ? 0 : 1)
                : cudaErrorInvalidValue;
   if (kernel == LIF_KERNEL_PREDICT_Z)
     return launch_k(predict_z_kernel<1>, dim3(L->z_ctas), dim3(kThreads), 0, st, L->use_pdl, x,
@@ -247,7 +248,8 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
                   (size_t)D.rank * sizeof(float), st, L->use_pdl, (const float*)L->z_partial,
                   L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit, D.rank,
                   D.d_ff, (float*)nullptr, L->mask_words, (int*)(L->counts + CNT_TICKET_PREDICT),
-                  (int*)L->active_idx, (int*)L->n_tmp, 1, L->keep_tok, D.spec_keep);
+                  (int*)L->active_idx, (int*)L->n_tmp, L->fused_plan ? 0 : 1, L->keep_tok,
+                  D.spec_keep);
 }
 
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,

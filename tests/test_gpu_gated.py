@@ -38,6 +38,8 @@ def _staged(cfg, **kw):
     (4096, 1408, 32, 2, 1, B.ACT_FATRELU, 0.1),       # Llama 2 7B row length
     (512, 4096, 40, 2, 3, B.ACT_FATRELU, 0.05),       # three streams
     (256, 1536, 16, 2, 8, B.ACT_RELU_SQUARED, 0.0),   # eight streams
+    (8192, 520, 16, 2, 1, B.ACT_FATRELU, 0.1),        # widest rows, last tile of 8 neurons
+    (2048, 2048, 16, 2, 8, B.ACT_FATRELU, 0.05),      # eight streams, tensor-core FFN
 ])
 def test_gated_staged(gate_mode, d, F, r, k, S, act, thr):
     cfg = W.LifConfig("gated", 1, d, F, r, k, S, 8, 0.08, 1.0, 0.8, 0.6, 21)
