@@ -311,7 +311,10 @@ def run_ours(args):
             "e2e": {"value": whole_job_tokens_per_s(K, world, ms_e2e), "unit": UNIT,
                     "h2d_bytes_per_step": S * d * 2, "d2h_bytes_per_step": L * S * d * 4,
                     "host_link_bytes_per_step": fetched / K},
-            "gpu_launches": 8 * n_launch,   # z, scores, window, moves, fetch, 2 x FFN (or up + down), sum
+            # per layer-step: z, scores (or the gate kernel alone), window, moves, fetch (one stream:
+            # with the new rows' FFN terms), FFN of cached rows (several streams: up + down), sum
+            "gpu_launches": ((7 if S == 1 else 8) - (1 if gate_mode == B.GATE_RESIDENT else 0)
+                             + (1 if gate_mode == B.GATE_BUNDLED else 0)) * n_launch,
             "roofline": {"kernel": "sparse_ffn_kernel" if S == 1 else
                                    "ffn_batched_up_kernel + ffn_batched_down_kernel + ffn_reduce_kernel",
                          "bound": "hbm",

@@ -291,8 +291,11 @@ enum {
                                     down-projection kernel, 1..16 */
   LIF_TUNE_BATCHED_UP_TWO_CTAS = 7, /* (0) multi-stream FFN, up-projection kernel: two light CTAs
                                     per SM instead of one with a deep ring */
-  LIF_TUNE_FUSED_PLAN = 6        /* (1 when d_ff <= 32768) lif_decode_step: the window update
+  LIF_TUNE_FUSED_PLAN = 6,       /* (1 when d_ff <= 32768) lif_decode_step: the window update
                                     reads the predictor's bit mask instead of its index list */
+  LIF_TUNE_FUSED_FETCH_FFN = 8   /* (1) lif_decode_step, one stream, with LIF_TUNE_SPLIT_FFN: the
+                                    fetch kernel also adds the FFN terms of the rows it brings
+                                    in (needs fetch CTAs = FFN CTAs, bundles of two vectors) */
 };
 lif_status lif_set_tuning(lif_layer* layer, int32_t key, int32_t value);
 
@@ -348,7 +351,8 @@ lif_status lif_timing_read(lif_layer* layer, float* host_us_sums /* [LIF_PHASE_L
 enum {
   LIF_KERNEL_PREDICT_Z = 0,  /* not with LIF_GATE_RESIDENT */
   LIF_KERNEL_PREDICT_SCORES = 1, /* LIF_GATE_RESIDENT: the gate-projection kernel */
-  LIF_KERNEL_FETCH = 2,      /* re-copies this step's new bundles */
+  LIF_KERNEL_FETCH = 2,      /* re-copies this step's new bundles (and, where the decode step
+                                fuses it, recomputes their FFN partials) */
   LIF_KERNEL_FFN_ACTIVE = 3, /* sparse FFN kernel over all active rows */
   LIF_KERNEL_FFN_HITS = 4,   /* ... over the active rows that were already cached */
   LIF_KERNEL_FFN_NEW = 5,    /* ... over the rows brought in this step */

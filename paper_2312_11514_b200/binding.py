@@ -30,7 +30,7 @@ EXPORTS = [
 ]
 KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ffn_new", "ffn_sum")
 (TUNE_DEPENDENT_LAUNCH, TUNE_SPLIT_FFN, TUNE_FETCH_CTAS, TUNE_FFN_CTAS, TUNE_FFN_STAGES,
- TUNE_BATCHED_COLUMN_PARTS, TUNE_FUSED_PLAN, TUNE_BATCHED_UP_TWO_CTAS) = range(8)
+ TUNE_BATCHED_COLUMN_PARTS, TUNE_FUSED_PLAN, TUNE_BATCHED_UP_TWO_CTAS, TUNE_FUSED_FETCH_FFN) = range(9)
 PHASES = ("predict_z", "predict_scores", "window", "moves", "fetch", "ffn", "ffn_sum")
 PHASE_LEN = 8
 

@@ -169,6 +169,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
     L->use_pdl = 1;
     L->split_ffn = 1;
     L->fused_plan = window_plan_supported(*desc) ? 1 : 0;
+    L->fused_fetch = 1;
     ok = cudaEventCreateWithFlags(&L->ev_plan, cudaEventDisableTiming) == cudaSuccess;
     if (ok && cudaEventCreateWithFlags(&L->ev_fetch, cudaEventDisableTiming) != cudaSuccess) {
       cudaEventDestroy(L->ev_plan);
@@ -436,8 +437,11 @@ lif_status lif_profile_launch(lif_layer* L, int32_t kernel, const void* dev_x, f
     case LIF_KERNEL_PREDICT_SCORES:
       e = launch_predict_one(L, kernel, (const __half*)dev_x, st);
       break;
-    case LIF_KERNEL_FETCH:
-      e = launch_fetch(L, st);
+    case LIF_KERNEL_FETCH:     // in the form the decode step launches it
+      e = (L->split_ffn && L->fused_fetch && fetch_ffn_supported(L))
+              ? launch_fetch_ffn(L, (const __half*)dev_x,
+                                 L->y_partial + (size_t)L->ffn_grid * L->desc.d_model, st)
+              : launch_fetch(L, st);
       break;
     case LIF_KERNEL_FFN_SUM:
       if (!dev_y) return LIF_ERR_INVALID_ARG;
@@ -462,6 +466,7 @@ lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
     case LIF_TUNE_FUSED_PLAN:
       L->fused_plan = value != 0 && window_plan_supported(L->desc);
       return LIF_OK;
+    case LIF_TUNE_FUSED_FETCH_FFN: L->fused_fetch = value != 0; return LIF_OK;
     case LIF_TUNE_FETCH_CTAS:
       if (value < 1 || value > 4096) return LIF_ERR_INVALID_ARG;
       L->fetch_grid = value;

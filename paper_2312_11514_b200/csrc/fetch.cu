@@ -58,6 +58,137 @@ fetch_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
   gather_rows(store, cache, load_ids, load_slots, counts[LIF_CNT_N_LOAD], row_vec);
 }
 
+// Fetch and FFN of the new rows in one kernel (single stream, row = up | down of at most
+// 32 KiB).  A CTA that brings a bundle in holds all of it in registers on its way from host
+// memory to the cache row, so it also computes that neuron's term of the FFN
+// (Section 3.3 item 3): h = act(<up, x> + bias) and partial += h * down.  The new rows then need
+// no second pass over HBM and no kernel of their own after the slowest step of the layer.  Rows
+// are dealt to CTAs in list order and each CTA adds its rows in that order, so the partials and
+// their sum do not depend on scheduling.  The first bundle's host loads are issued before the
+// dependency wait: the list and the counts were final before the preceding kernel (the row
+// moves) passed its own wait, while the cache rows may still be moving.
+constexpr int kFusedChunks = 4;     // 8-column chunks per thread and half row: d_model <= 8192
+
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __half22float2(h[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+
+struct FetchFfnArgs {
+  const uint4* store;
+  uint4* cache;
+  const int32_t* load_ids;
+  const int32_t* load_slots;
+  const int32_t* counts;
+  const __half* bias;        // per cache row
+  const __half* x;
+  const float* gate_val;     // resident gate: gate pre-activations by neuron id
+  float* y_partial;          // [gridDim.x][d]
+  int d, act;
+  float act_thr;
+};
+
+template <int kGate>
+__global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
+  __shared__ float part[kThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = a.d >> 3;                       // 16-byte chunks per half row
+  const int n = __ldcg(a.counts + LIF_CNT_N_LOAD);
+  if ((int)blockIdx.x >= n) {                      // the sum reads min(grid, n) partials
+    pdl_wait();
+    pdl_trigger();
+    return;
+  }
+  uint4 up[kFusedChunks], down[kFusedChunks];
+  auto host_loads = [&](int id) {
+    const uint4* src = a.store + (size_t)id * 2 * nvec;
+#pragma unroll
+    for (int k = 0; k < kFusedChunks; ++k) {
+      const int c = tid + k * kThreads;
+      if (c < nvec) {
+        up[k] = ld_host(src + c);
+        down[k] = ld_host(src + nvec + c);
+      }
+    }
+  };
+  int j = blockIdx.x;
+  int id = __ldcg(a.load_ids + j), slot = __ldcg(a.load_slots + j);
+  host_loads(id);
+  pdl_wait();
+  pdl_trigger();
+
+  uint4 xq[kFusedChunks];
+#pragma unroll
+  for (int k = 0; k < kFusedChunks; ++k) {
+    const int c = tid + k * kThreads;
+    xq[k] = c < nvec ? reinterpret_cast<const uint4*>(a.x)[c] : make_uint4(0, 0, 0, 0);
+  }
+  float acc[kFusedChunks][8];
+#pragma unroll
+  for (int k = 0; k < kFusedChunks; ++k)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[k][e] = 0.f;
+
+  while (true) {
+    const float b = kGate == LIF_GATE_RESIDENT ? a.gate_val[id] : __half2float(a.bias[slot]);
+    uint4* dst = a.cache + (size_t)slot * 2 * nvec;
+    float p = 0.f;
+#pragma unroll
+    for (int k = 0; k < kFusedChunks; ++k) {
+      const int c = tid + k * kThreads;
+      if (c < nvec) {
+        dst[c] = up[k];
+        dst[nvec + c] = down[k];
+        float uf[8], xf[8];
+        unpack8(up[k], uf);
+        unpack8(xq[k], xf);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) p = fmaf(uf[e], xf[e], p);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
+    if (lane == 0) part[warp] = p;
+    __syncthreads();
+    float v = 0.f;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) v += part[w];
+    const float h = kGate == LIF_GATE_RESIDENT ? apply_activation(b, a.act, a.act_thr) * v
+                                               : apply_activation(v + b, a.act, a.act_thr);
+    if (h != 0.f) {
+#pragma unroll
+      for (int k = 0; k < kFusedChunks; ++k) {
+        if (tid + k * kThreads < nvec) {
+          float df[8];
+          unpack8(down[k], df);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[k][e] = fmaf(h, df[e], acc[k][e]);
+        }
+      }
+    }
+    j += gridDim.x;
+    if (j >= n) break;
+    __syncthreads();                               // part[] is free again
+    id = a.load_ids[j];
+    slot = a.load_slots[j];
+    host_loads(id);
+  }
+  float4* out = reinterpret_cast<float4*>(a.y_partial + (size_t)blockIdx.x * a.d);
+#pragma unroll
+  for (int k = 0; k < kFusedChunks; ++k) {
+    const int c = tid + k * kThreads;
+    if (c < nvec) {
+      out[2 * c] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
+      out[2 * c + 1] = make_float4(acc[k][4], acc[k][5], acc[k][6], acc[k][7]);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads)
 probe_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n_chunks,
              int chunk_vec) {
@@ -86,6 +217,36 @@ cudaError_t launch_fetch(lif_layer* L, cudaStream_t st) {
                   (const uint4*)L->dev_bundles, (uint4*)L->desc.dev_cache,
                   (const int32_t*)L->load_ids, (const int32_t*)L->load_slots,
                   (const int32_t*)L->counts, row_elems(L->desc) / 8);
+}
+
+bool fetch_ffn_supported(const lif_layer* L) {
+  const lif_layer_desc& D = L->desc;
+  return D.n_streams == 1 && D.gate_mode != LIF_GATE_BUNDLED &&
+         D.d_model <= kFusedChunks * kThreads * 8 && L->fetch_grid == L->ffn_grid;
+}
+
+// Fetch of this step's new rows fused with their FFN terms; partials go to `partial`
+// ([fetch_grid][d_model], CTA c < min(grid, n_load) writes row c).
+cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st) {
+  const lif_layer_desc& D = L->desc;
+  FetchFfnArgs a;
+  a.store = (const uint4*)L->dev_bundles;
+  a.cache = (uint4*)D.dev_cache;
+  a.load_ids = L->load_ids;
+  a.load_slots = L->load_slots;
+  a.counts = L->counts;
+  a.bias = L->bias;
+  a.x = x;
+  a.gate_val = L->gate_val;
+  a.y_partial = partial;
+  a.d = D.d_model;
+  a.act = D.activation;
+  a.act_thr = D.activation_threshold;
+  return D.gate_mode == LIF_GATE_RESIDENT
+             ? launch_k(fetch_ffn_kernel<LIF_GATE_RESIDENT>, dim3(L->fetch_grid), dim3(kThreads), 0,
+                        st, L->use_pdl, a)
+             : launch_k(fetch_ffn_kernel<LIF_GATE_NONE>, dim3(L->fetch_grid), dim3(kThreads), 0, st,
+                        L->use_pdl, a);
 }
 
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,

@@ -451,12 +451,18 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
   if (ev) tm_record(ev[8], side);
   if (fork && (e = cudaEventRecord(L->ev_fetch, side)) != cudaSuccess) return e;
   if (ev) tm_record(ev[5], st);
-  if ((e = launch_fetch(L, st)) != cudaSuccess) return e;
-  if (ev) tm_record(ev[6], st);
   FfnArgs miss = ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
-  e = launch_k(ffn_kernel_for(D.gate_mode), dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
-               L->use_pdl, miss);
-  if (e != cudaSuccess) return e;
+  if (L->fused_fetch && fetch_ffn_supported(L)) {
+    // one kernel brings the new rows in and adds their FFN terms (CTA partials in p1)
+    if ((e = launch_fetch_ffn(L, x, p1, st)) != cudaSuccess) return e;
+    if (ev) tm_record(ev[6], st);
+  } else {
+    if ((e = launch_fetch(L, st)) != cudaSuccess) return e;
+    if (ev) tm_record(ev[6], st);
+    e = launch_k(ffn_kernel_for(D.gate_mode), dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
+                 L->use_pdl, miss);
+    if (e != cudaSuccess) return e;
+  }
   if (fork && (e = cudaStreamWaitEvent(st, L->ev_fetch, 0)) != cudaSuccess) return e;
   e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0,
                st, L->use_pdl, (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,

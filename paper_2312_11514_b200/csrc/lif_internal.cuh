@@ -77,6 +77,7 @@ struct lif_layer {
   int use_pdl;        // programmatic dependent launch along the compute stream
   int split_ffn;      // decode step: cached rows' FFN overlaps the fetch
   int fused_plan;     // decode step: window update reads the predictor's bit mask directly
+  int fused_fetch;    // decode step: the fetch kernel also computes the new rows' FFN terms
   cudaEvent_t ev_plan, ev_fetch;
   // optional per-kernel timing: kTimingEvents events per recorded step
   cudaEvent_t* tm_events;
@@ -116,6 +117,8 @@ cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = 
 cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st,
                           cudaEvent_t* ev = nullptr);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
+bool fetch_ffn_supported(const lif_layer* L);
+cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st);
 cudaError_t launch_refill(lif_layer* L, cudaStream_t st);
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,
                          int grid, cudaStream_t st);

@@ -387,3 +387,43 @@ def test_window_longer_than_the_sequence_never_evicts():
     used = [s["num_used"] for s in stats]
     assert used == sorted(used) and used[-1] > used[0]                # the cache only grows
     gpu.close()
+
+
+@pytest.mark.parametrize("d,F,k,act,thr,gate_mode,ffn_mode", [
+    (256, 1024, 3, B.ACT_RELU, 0.0, 0, 0),
+    (264, 1000, 2, B.ACT_FATRELU, 0.1, 0, 0),         # ragged row length
+    (8192, 520, 2, B.ACT_RELU_SQUARED, 0.0, 0, 0),    # widest row: four chunks per thread
+    (4096, 1408, 2, B.ACT_RELU, 0.0, 0, 1),           # whole-cache FFN
+    (512, 2048, 2, B.ACT_FATRELU, 0.05, 2, 0),        # resident gate
+    (512, 2048, 2, B.ACT_FATRELU, 0.05, 1, 0),        # bundled gate: falls back to two kernels
+])
+@pytest.mark.parametrize("fused_fetch", [1, 0])
+def test_decode_step_with_and_without_the_fused_fetch(d, F, k, act, thr, gate_mode, ffn_mode, fused_fetch):
+    # lif_decode_step either lets the fetch kernel add the new rows' FFN terms or runs the
+    # FFN kernel over them afterwards; both must match the oracle
+    cfg = W.LifConfig("fusedfetch", 1, d, F, 16, k, 1, 10, 0.08, 1.0, 0.8, 0.6, 31)
+    gpu, ora = P.make_layer_pair(cfg, 0, activation=act, act_threshold=thr, gate_mode=gate_mode,
+                                 ffn_mode=ffn_mode, b_down=True)
+    B.lif_set_tuning(gpu.handle, B.TUNE_FUSED_FETCH_FFN, fused_fetch)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(1, d, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    n_load = n_evict = 0
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        torch.cuda.synchronize()
+        x_np = X[t].cpu().numpy()
+        if ffn_mode == 0:
+            lists = P.check_decode_step(gpu, ora, x_np, y.cpu().numpy().astype(np.float64))
+        else:
+            g = gpu.lists()
+            lists = ora.cache.window_update(g["active_idx"])
+            ora.cache.insert(lists, ora.bundles, ora.bias_up)
+            P.compare_lists_and_state(gpu, ora, lists)
+            ref_y, flips = P.ffn_reference(ora, np.arange(ora.cache.num_used), x_np)
+            P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y, flips)
+        P.compare_cache_rows(gpu, ora)
+        n_load += len(lists["load_ids"]); n_evict += len(lists["evict_ids"])
+    assert n_load > 0 and n_evict > 0
+    gpu.close()
