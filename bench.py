@@ -281,8 +281,16 @@ def run_ours(args):
         row_extra = 8 if gate_mode == B.GATE_RESIDENT else 2    # bias, or neuron id + gate value
         peak, peak_kind = _peaks()
         # algorithmic bytes of one launch: bundle + bias per row, x in, partials out
-        ffn_bytes = (n_act_l * (beta + row_extra) + L * S * 6 * d) / L
-        ffn_gbs = ffn_bytes / (kernel_us["ffn_active"] * 1e-6) / 1e9
+        all_bytes = (n_act_l * (beta + row_extra) + L * S * 6 * d) / L
+        all_gbs = all_bytes / (kernel_us["ffn_active"] * 1e-6) / 1e9
+        if S == 1:
+            # the launch the decode step makes: the rows that were already cached (the new rows'
+            # terms are added by the fetch kernel, or by a second launch for three-vector bundles)
+            ffn_bytes = (n_hit_l * (beta + row_extra) + L * 6 * d) / L
+            ffn_us = kernel_us["ffn_hits"]
+        else:
+            ffn_bytes, ffn_us = all_bytes, kernel_us["ffn_active"]
+        ffn_gbs = ffn_bytes / (ffn_us * 1e-6) / 1e9
         fetch_bytes = n_load_l * beta / L
         fetch_gbs = fetch_bytes / (kernel_us["fetch"] * 1e-6) / 1e9
         if gate_mode == B.GATE_RESIDENT:       # gate matrix + bias in, gate values out
@@ -294,7 +302,8 @@ def run_ours(args):
         pred_gbs = pred_bytes / (pred_us * 1e-6) / 1e9
         split = None
         if S == 1:
-            split = {"already_cached_rows_GBs": (n_hit_l * (beta + row_extra) / L + 6 * d) / (kernel_us["ffn_hits"] * 1e-6) / 1e9,
+            split = {"all_active_rows": {"GBs": all_gbs, "us_per_launch": kernel_us["ffn_active"],
+                                         "bytes_per_launch": all_bytes, "frac": all_gbs / peak},
                      "new_rows_GBs": (n_load_l * (beta + row_extra) / L + 6 * d) / (kernel_us["ffn_new"] * 1e-6) / 1e9}
         out = {
             "metric": METRIC, "value": whole_job_tokens_per_s(K, world, ms_total), "unit": UNIT,
@@ -325,12 +334,15 @@ def run_ours(args):
                          "traffic_how": "dram read+write bytes per algorithmic byte from the ncu capture in "
                                         "profiles/sparse_ffn_kernel_opt6p7b_12layers.md (12 layers, "
                                         "451-529 rows per launch), scaled by this run's rows per launch",
-                         "us_per_launch": kernel_us["ffn_active"],
+                         "us_per_launch": ffn_us,
                          "bytes_per_launch": ffn_bytes,
-                         "how": "graph of this kernel on all layers' active rows of the last token, "
-                                f"{reps} replays, CUDA events",
-                         "split_launches": split},
-            "host_link": {"kernel": "fetch_kernel", "bound": "host_link", "achieved": fetch_gbs,
+                         "how": ("graph of this kernel on every layer, over the rows of the last token "
+                                 "that were already cached (the decode step's launch)" if S == 1 else
+                                 "graph of these kernels on every layer, over the active rows of the "
+                                 "last token") + f", {reps} replays, CUDA events",
+                         "other_launches": split},
+            "host_link": {"kernel": "fetch_ffn_kernel" if S == 1 and gate_mode != B.GATE_BUNDLED
+                                    else "fetch_kernel", "bound": "host_link", "achieved": fetch_gbs,
                           "peak": link_peak, "unit": "GB/s", "frac": fetch_gbs / link_peak,
                           "peak_kind": "of measured (1 GiB pinned cudaMemcpyAsync, this run)",
                           "bytes_per_launch": fetch_bytes, "us_per_launch": kernel_us["fetch"]},
