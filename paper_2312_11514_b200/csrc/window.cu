@@ -287,11 +287,31 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
   __shared__ int holes[kPlanMaxRows];
   __shared__ int newslot[kPlanMaxRows];
   const int tid = threadIdx.x;
-  pdl_wait();
-  pdl_trigger();
+  // The window state was last written by this layer's previous step, which is complete before
+  // the predictor of this step even starts: the slot side of the bookkeeping (row -> neuron,
+  // row bias, each cached neuron's stamp: three dependent round trips) is read before the
+  // dependency wait and overlaps the predictor's tail.  Only the mask waits.
   const int n = a.counts[LIF_CNT_NUM_USED];
   const int t = a.counts[LIF_CNT_STEP];
   const int t_end = t + a.keep - 1;   // the kept window ends at this token
+  const int seg = (n + kWindowThreads - 1) / kWindowThreads;   // <= kPlanSlots on the fast path
+  const int s0 = min(n, tid * seg);
+  const int my_slots = min(n, s0 + seg) - s0;
+  int pid[kPlanSlots], la[kPlanSlots];
+  __half pb[kPlanSlots];
+#pragma unroll
+  for (int j = 0; j < kPlanSlots; ++j) {
+    pid[j] = 0;
+    pb[j] = __half();
+    if (j < my_slots) {
+      pid[j] = a.pointers[s0 + j];
+      pb[j] = a.bias[s0 + j];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < kPlanSlots; ++j) la[j] = j < my_slots ? a.last_active[pid[j]] : 0;
+  pdl_wait();
+  pdl_trigger();
   const uint32_t w = tid < nwords ? mask_words[tid] : 0u;
   const int cnt = __popc(w);
   bits[tid] = w;
@@ -312,7 +332,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
     return;
   }
 
-  // ---- round trip 2: by neuron id (mine: bits of w) and by slot (mine: a contiguous run) ----
+  // ---- second round trip after the wait: by neuron id (mine: the bits of w) -------------------
   int so[kPlanBits];
   __half bu[kPlanBits];
   {
@@ -329,21 +349,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
       }
     }
   }
-  const int seg = (n + kWindowThreads - 1) / kWindowThreads;   // <= kPlanSlots
-  const int s0 = min(n, tid * seg);
-  const int my_slots = min(n, s0 + seg) - s0;
-  int pid[kPlanSlots];
-  __half pb[kPlanSlots];
-#pragma unroll
-  for (int j = 0; j < kPlanSlots; ++j) {
-    pid[j] = 0;
-    pb[j] = __half();
-    if (j < my_slots) {
-      pid[j] = a.pointers[s0 + j];
-      pb[j] = a.bias[s0 + j];
-    }
-  }
-  // ---- round trip 3: is each of my cached neurons still inside the window? ------------------
+  // ---- is each of my cached neurons still inside the window? -----------------------------------
   int age[kPlanSlots];          // steps since last active; 0 = active now
 #pragma unroll
   for (int j = 0; j < kPlanSlots; ++j) {
@@ -351,7 +357,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
     if (j < my_slots) {
       const int id = pid[j];
       const bool active_now = (bits[id >> 5] >> (id & 31)) & 1u;
-      if (!active_now) age[j] = max(1, t_end - a.last_active[id]);
+      if (!active_now) age[j] = max(1, t_end - la[j]);
     }
   }
   int c_load = 0;
