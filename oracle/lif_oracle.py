@@ -80,14 +80,21 @@ class NeuronCache:
     ``last_k_active`` is kept as ``last_active[i]`` = the last step at which neuron i was
     predicted active, so "still inside the window of k tokens" is last_active[i] > t - k."""
 
-    def __init__(self, d_model, d_ff, capacity, window_k, budget_rows=0, n_vec=2):
+    def __init__(self, d_model, d_ff, capacity, window_k, budget_rows=0, n_vec=2,
+                 append_first=False):
         """``budget_rows`` > 0 turns on the memory budget of Appendix C (Persimmon 8B, Phi-2):
         whenever the cache would pass the budget, the window is shrunk for that step.
         ``n_vec`` = vectors of d_model values per bundle: 2 (up row, down column; Section 3.2)
-        or 3 for a gated FFN (gate row, up row, down column; Appendix C, Llama 2)."""
+        or 3 for a gated FFN (gate row, up row, down column; Appendix C, Llama 2).
+        ``append_first`` applies the two operations of Section 3.3 in the other order: the new
+        neurons are stacked at the end first (item 2), then the deletions pull the last rows
+        into the freed ones (item 1) -- so a new neuron that would be moved straight away is
+        written into the freed row directly and only the deletions that outnumber the
+        arrivals move old rows.  Same cached set, different row order."""
         self.d_model, self.d_ff, self.capacity, self.k = d_model, d_ff, capacity, window_k
         self.budget_rows = budget_rows
         self.n_vec = n_vec
+        self.append_first = append_first
         self.k_eff = window_k
         self.matrix = np.zeros((capacity, n_vec * d_model), dtype=np.float16)
         self.pointers = np.full(capacity, -1, dtype=np.int32)
@@ -154,42 +161,58 @@ class NeuronCache:
         self.last_active[act] = stamps
         evict_ids = [int(self.pointers[s]) for s in evict_slots]
 
+        # With append_first the rows to bring in already stand at the end (rows n .. n + n_load,
+        # ascending neuron id) when the deletions are applied; their weights are not there yet,
+        # so "moving" one of them only decides where its bundle will be written.
+        n_load = len(load_ids)
+        end = n
+        ptr = np.concatenate([self.pointers, np.full(n_load, -1, dtype=np.int32)])   # room to stack
+        if self.append_first:
+            ptr[n:n + n_load] = load_ids
+            self.slot_of[load_ids] = np.arange(n, n + n_load)
+            end = n + n_load
+
         # Deleting: walk the freed rows in ascending order; the current last row replaces
         # the freed one unless the last row is itself to be deleted, in which case it is
         # simply dropped.
-        dead = np.zeros(self.capacity, dtype=bool)
+        dead = np.zeros(len(ptr), dtype=bool)
         dead[evict_slots] = True
+        for i in evict_ids:
+            self.slot_of[i] = -1
         move_src, move_dst = [], []
-        tail = n
+        tail = end
         for hole in evict_slots:
             while tail > 0 and dead[tail - 1]:
                 tail -= 1                                   # drop deleted rows off the end
             if hole >= tail:
                 break                                       # every remaining hole was dropped
             tail -= 1                                       # last surviving row
-            self.matrix[hole] = self.matrix[tail]
-            self.bias[hole] = self.bias[tail]
-            self.pointers[hole] = self.pointers[tail]
-            self.slot_of[self.pointers[hole]] = hole
+            ptr[hole] = ptr[tail]
+            self.slot_of[ptr[hole]] = hole
             dead[hole] = False
-            move_src.append(tail)
-            move_dst.append(hole)
-        for i in evict_ids:
-            self.slot_of[i] = -1
-        self.pointers[n_new:n] = -1
-        self.num_used = n_new
+            if tail < n:                                    # a cached row: its weights move
+                self.matrix[hole] = self.matrix[tail]
+                self.bias[hole] = self.bias[tail]
+                move_src.append(tail)
+                move_dst.append(hole)
         self.rows_moved += len(move_src)
+        n_new = n - len(evict_slots)                        # rows left of the old ones
 
-        # Bringing in new neurons: rows num_used .. num_used + num_new, ascending neuron id.
-        load_slots = list(range(n_new, n_new + len(load_ids)))
-        for i, s in zip(load_ids, load_slots):
-            self.pointers[s] = i
-            self.slot_of[i] = s
-        self.num_used = n_new + len(load_ids)
+        if self.append_first:
+            load_slots = [int(self.slot_of[i]) for i in load_ids]
+        else:
+            # Bringing in new neurons: rows num_used .. num_used + num_new, ascending neuron id.
+            load_slots = list(range(n_new, n_new + n_load))
+            for i, s in zip(load_ids, load_slots):
+                ptr[s] = i
+                self.slot_of[i] = s
+        self.num_used = n_new + n_load
+        ptr[self.num_used:] = -1
+        self.pointers[:] = ptr[:self.capacity]
         self.t = t0 + keep
 
         active_slots = self.slot_of[act].astype(np.int32)
-        hit_slots = active_slots[active_slots < n_new]
+        hit_slots = active_slots[~np.isin(act, np.asarray(load_ids, dtype=np.int32))]
         i32 = lambda v: np.asarray(v, dtype=np.int32)
         return {
             "evict_ids": i32(evict_ids), "move_src": i32(move_src), "move_dst": i32(move_dst),

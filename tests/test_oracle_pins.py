@@ -644,3 +644,97 @@ def test_gated_decode_step_three_vector_bundles():
         n_loaded += len(lists["load_ids"])
     assert cache.bytes_fetched == n_loaded * 3 * d * 2 and n_loaded > 0
     assert cache.matrix.shape == (F, 3 * d)
+
+
+# ------------------------------------------------------------------ append first, then delete
+@pytest.mark.parametrize("k", [1, 2, 5])
+def test_append_first_window_brute_force(k):
+    """Section 3.3 with its two operations in the other order (stack the new neurons, then
+    delete by pulling last rows into freed ones): same cached set, traffic and outputs as the
+    paper's order; new neurons land in freed rows; old rows move only when more are deleted
+    than arrive."""
+    F, d, T = 97, 4, 40
+    r = _rng(70 + k)
+    bundles = r.normal(size=(F, 2 * d)).astype(np.float16)
+    bias_up = r.normal(size=F).astype(np.float16)
+    sets = _random_active_sets(F, T, 0.08, seed=k)
+    cache = O.NeuronCache(d, F, capacity=F, window_k=k, append_first=True)
+    paper = O.NeuronCache(d, F, capacity=F, window_k=k)
+    saw_reuse = saw_append = saw_move = False
+    for t, act in enumerate(sets):
+        before = cache.cached_ids()
+        n = cache.num_used
+        slot_before = cache.slot_of.copy()
+        rows_before = {int(cache.pointers[s]): cache.matrix[s].copy() for s in range(n)}
+        freed = sorted(int(cache.slot_of[i]) for i in before
+                       if i not in set(act.tolist()) and cache.last_active[i] <= t - k)
+        lists = cache.window_update(act)
+        cache.insert(lists, bundles, bias_up)
+        ref = paper.window_update(act)
+        paper.insert(ref, bundles, bias_up)
+        _check_structure(cache)
+        union = set()
+        for u in range(max(0, t - k + 1), t + 1):
+            union |= set(sets[u].tolist())
+        assert cache.cached_ids() == union == paper.cached_ids()
+        for key in ("load_ids", "evict_ids"):
+            assert sorted(lists[key].tolist()) == sorted(ref[key].tolist())
+        e, l = len(freed), len(lists["load_ids"])
+        assert cache.num_used == n - e + l == paper.num_used
+        # brute-force statement of the placement: the last min(e, l) new neurons take the freed
+        # rows, lowest freed row <- highest id; the other new neurons stay stacked at n, n+1, ...
+        want = [n + j if j < l - min(e, l) else freed[l - 1 - j] for j in range(l)]
+        assert lists["load_slots"].tolist() == want
+        # old rows move only when deletions outnumber arrivals, never more than the paper's order
+        assert len(lists["move_src"]) <= max(0, e - l) and len(lists["move_src"]) <= len(ref["move_src"])
+        b = n - max(0, e - l)
+        assert all(src >= b > dst and dst in freed[min(e, l):] for src, dst in zip(lists["move_src"], lists["move_dst"]))
+        assert lists["move_src"].tolist() == sorted(lists["move_src"].tolist(), reverse=True)   # last row first
+        assert lists["move_dst"].tolist() == sorted(lists["move_dst"].tolist())
+        moved = {int(cache.pointers[dst]) for dst in lists["move_dst"]}
+        for i in before & union:
+            if i not in moved:
+                assert cache.slot_of[i] == slot_before[i]
+        for s in range(cache.num_used):
+            i = cache.pointers[s]
+            np.testing.assert_array_equal(cache.matrix[s], bundles[i])
+            assert cache.bias[s] == bias_up[i]
+            if i in rows_before:
+                np.testing.assert_array_equal(cache.matrix[s], rows_before[i])
+        assert [int(cache.pointers[s]) for s in lists["active_slots"]] == act.tolist()
+        assert sorted(lists["hit_slots"].tolist() + lists["load_slots"].tolist()) == \
+            sorted(lists["active_slots"].tolist())
+        # the FFN does not see the row order
+        x = r.normal(size=(1, d))
+        np.testing.assert_allclose(O.sparse_ffn(cache.matrix, cache.bias, lists["active_slots"], x),
+                                   O.sparse_ffn(paper.matrix, paper.bias, ref["active_slots"], x),
+                                   rtol=1e-12, atol=1e-12)
+        saw_reuse |= l > 0 and e > 0
+        saw_append |= l > e
+        saw_move |= len(lists["move_src"]) > 0
+    assert cache.bytes_fetched == paper.bytes_fetched and cache.rows_moved < paper.rows_moved
+    assert saw_reuse and saw_append and saw_move
+
+
+def test_append_first_worked_example_and_transient_overshoot():
+    # 6 rows cached (neurons 10..15 in rows 0..5), capacity 7.  Rows 1 and 4 are deleted and the
+    # neurons 3, 7, 20 arrive: stacked they would stand in rows 6, 7, 8 (beyond the capacity for a
+    # moment); the deletions pull 20 into row 1 and 7 into row 4; 3 stays in row 6.
+    cache = O.NeuronCache(2, 32, capacity=7, window_k=1, append_first=True)
+    cache.window_update(np.arange(10, 16))
+    lists = cache.window_update(np.array([3, 7, 10, 12, 13, 15, 20]))
+    assert lists["evict_ids"].tolist() == [11, 14]
+    assert lists["load_ids"].tolist() == [3, 7, 20] and lists["load_slots"].tolist() == [6, 4, 1]
+    assert lists["move_src"].size == 0
+    assert cache.pointers.tolist() == [10, 20, 12, 13, 7, 15, 3] and cache.num_used == 7
+    # more deletions than arrivals: 20, 12 and 3 go, 11 arrives.  Stacked, 11 stands in row 7 and
+    # goes to the first freed row (1); then the last row still in use, row 5 (15), goes to row 2;
+    # row 6 was freed itself and is dropped with the tail
+    lists = cache.window_update(np.array([7, 10, 11, 13, 15]))
+    assert sorted(lists["evict_ids"].tolist()) == [3, 12, 20]
+    assert lists["load_ids"].tolist() == [11] and lists["load_slots"].tolist() == [1]
+    assert lists["move_src"].tolist() == [5] and lists["move_dst"].tolist() == [2]
+    assert cache.pointers.tolist() == [10, 11, 15, 13, 7, -1, -1] and cache.num_used == 5
+    # capacity still refuses what does not fit at the end of the step
+    with pytest.raises(O.CapacityError):
+        cache.window_update(np.arange(0, 9))
