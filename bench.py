@@ -143,7 +143,7 @@ def run_ours(args):
     n_tok = Wm + K
     gate_mode, activation, act_thr = _gate_setup(args)
     layers = R.build_stack(cfg, dev, n_layers=args.layers, gate_mode=gate_mode, activation=activation,
-                           activation_threshold=act_thr)
+                           activation_threshold=act_thr, append_first=args.append_first)
     handles = [l.handle for l in layers]
     L, S, d = len(layers), cfg.n_streams, cfg.d_model
     X = _inputs(cfg, n_tok, dev, W)
@@ -313,6 +313,9 @@ def run_ours(args):
             "config": {"workload": f"{cfg.name}: {L} layers d_model={d} d_ff={cfg.d_ff} rank={cfg.rank} "
                                    f"window_k={cfg.window_k} streams={S}, AR(1) decode inputs"
                                    + (f", gated FFN ({args.gate} gate, FATReLU {act_thr})" if gate_mode else ""),
+                       "cache_order": "new neurons stacked first, then the deletions (bundles written "
+                                      "straight into freed rows)" if args.append_first else
+                                      "deletions first, then new neurons stacked (Section 3.3 as written)",
                        "l2": "per-token working set (all layers' window caches, "
                              f"{s1[3] / n_tok * beta / 2**20:.0f} MiB) exceeds the 126 MB L2",
                        "bundle_store": "pinned host memory, read by the fetch kernel",
@@ -380,7 +383,7 @@ def run_kernel_loop(args):
     cfg = W.CONFIGS[args.config]
     gate_mode, activation, act_thr = _gate_setup(args)
     layers = R.build_stack(cfg, dev, n_layers=args.layers, gate_mode=gate_mode, activation=activation,
-                           activation_threshold=act_thr)
+                           activation_threshold=act_thr, append_first=args.append_first)
     handles = [l.handle for l in layers]
     L, S, d = len(layers), cfg.n_streams, cfg.d_model
     X = _inputs(cfg, args.warmup, dev, W)
@@ -585,6 +588,9 @@ def main():
                     help="gated FFN: gate row inside the bundle, or resident gate projection as the "
                          "predictor (use with --config llama2_7b)")
     ap.add_argument("--act-threshold", type=float, default=0.05, help="FATReLU threshold of gated runs")
+    ap.add_argument("--append-first", type=int, default=1, choices=[0, 1],
+                    help="1: stack the new neurons before deleting, so their bundles go straight into "
+                         "freed rows; 0: the order of Section 3.3 as written (same cached set and outputs)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--cpu-layers", type=int, default=2)
     ap.add_argument("--cpu-tokens", type=int, default=30)

@@ -93,6 +93,13 @@ typedef struct {
                                step but gets the oldest stamp still inside the window.  The
                                step counter advances by spec_keep.  Not with budget_rows. */
   int32_t gate_mode;        /* LIF_GATE_*.  LIF_GATE_RESIDENT: not with spec_keep */
+  int32_t append_first;     /* 0: the order of Section 3.3 — delete (last rows move into the freed
+                               ones), then stack the new neurons at the end.  1: stack first,
+                               then delete: the last rows are then new neurons, so their bundles
+                               are written straight into freed rows and only deletions that
+                               outnumber the arrivals move cached rows.  Same cached set and
+                               outputs, fewer row copies, and row moves no longer touch the
+                               rows the fetch writes.  Not with ffn_mode = 1. */
   const void* dev_gate;     /* LIF_GATE_RESIDENT: fp16 [d_ff][d_model] gate projection, 16-byte
                                aligned; otherwise ignored */
   const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][V*d_model] */
@@ -129,6 +136,7 @@ enum {
  *   evict_ids[n_evict]     deleted neurons in ascending order of the slot they held
  *   move_src/dst[n_moves]  row move_src[j] was copied to row move_dst[j]
  *   load_ids[n_load]       neurons to bring in, ascending id; load_slots[j] = num_kept + j
+ *                          (append_first: the freed rows first, see lif_layer_desc)
  *   active_slots[n_active] cache row of active_idx[q] after the update
  *   hit_slots[n_hits]      rows of the active neurons that were already cached
  * State: pointers[capacity] (row -> neuron, -1 = free), slot_of[d_ff] (neuron -> row, -1 =

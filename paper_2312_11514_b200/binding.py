@@ -41,7 +41,7 @@ class LayerDesc(C.Structure):
         ("capacity", C.c_int32), ("n_streams", C.c_int32), ("threshold_logit", C.c_float),
         ("ffn_mode", C.c_int32), ("activation", C.c_int32), ("activation_threshold", C.c_float),
         ("budget_rows", C.c_int32), ("spec_keep", C.c_int32), ("gate_mode", C.c_int32),
-        ("dev_gate", C.c_void_p), ("host_bundles", C.c_void_p), ("dev_pred_A", C.c_void_p), ("dev_pred_B", C.c_void_p),
+        ("append_first", C.c_int32), ("dev_gate", C.c_void_p), ("host_bundles", C.c_void_p), ("dev_pred_A", C.c_void_p), ("dev_pred_B", C.c_void_p),
         ("dev_pred_c", C.c_void_p), ("dev_bias_up", C.c_void_p), ("dev_bias_down", C.c_void_p),
         ("dev_cache", C.c_void_p), ("dev_workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
     ]
@@ -140,7 +140,7 @@ def _stream(s) -> Optional[int]:
 
 def make_desc(*, d_model, d_ff, rank, window_k, capacity, n_streams=1, threshold_logit=0.0,
               ffn_mode=0, activation=0, activation_threshold=0.0, budget_rows=0, spec_keep=0,
-              gate_mode=0, gate=None, host_bundles=None, pred_A=None, pred_B=None, pred_c=None,
+              gate_mode=0, gate=None, append_first=0, host_bundles=None, pred_A=None, pred_B=None, pred_c=None,
               bias_up=None, bias_down=None, cache=None, workspace=None) -> LayerDesc:
     d = LayerDesc()
     d.d_model, d.d_ff, d.rank, d.window_k, d.capacity = d_model, d_ff, rank, window_k, capacity
@@ -149,6 +149,7 @@ def make_desc(*, d_model, d_ff, rank, window_k, capacity, n_streams=1, threshold
     d.budget_rows = budget_rows
     d.spec_keep = spec_keep
     d.gate_mode, d.dev_gate = gate_mode, _ptr(gate)
+    d.append_first = append_first
     d.host_bundles = _ptr(host_bundles)
     d.dev_pred_A, d.dev_pred_B, d.dev_pred_c = _ptr(pred_A), _ptr(pred_B), _ptr(pred_c)
     d.dev_bias_up, d.dev_bias_down = _ptr(bias_up), _ptr(bias_down)

@@ -69,6 +69,8 @@ static lif_status check_shape(const lif_layer_desc* d) {
   if (!(d->threshold_logit == d->threshold_logit)) return LIF_ERR_INVALID_ARG;   // NaN
   if (d->gate_mode < LIF_GATE_NONE || d->gate_mode > LIF_GATE_RESIDENT) return LIF_ERR_INVALID_ARG;
   if (d->gate_mode == LIF_GATE_RESIDENT && d->spec_keep > 0) return LIF_ERR_INVALID_ARG;
+  if (d->append_first != 0 && d->append_first != 1) return LIF_ERR_INVALID_ARG;
+  if (d->append_first && d->ffn_mode == 1) return LIF_ERR_INVALID_ARG;
   return LIF_OK;
 }
 
@@ -305,15 +307,18 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
     ev = L->tm_events + (size_t)(L->tm_cursor++) * kTimingEvents;
   if (ev) tm_record(ev[0], sc);
   bool ok;
+  // With append_first the row moves and the bundle writes touch different rows, so given a
+  // second stream the moves leave the critical chain (they only precede the cached rows' FFN).
+  const bool moves_aside = L->desc.append_first && sf != sc;
   if (L->fused_plan) {
     ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev, 0) == cudaSuccess;
-    ok = ok && launch_window_plan(L, sc, ev) == cudaSuccess;
+    ok = ok && launch_window_plan(L, sc, ev, !moves_aside) == cudaSuccess;
   } else {
     ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
-    ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
+    ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc, ev, !moves_aside) == cudaSuccess;
   }
   if (L->split_ffn && L->desc.n_streams == 1) {
-    ok = ok && launch_fetch_and_ffn_split(L, x, dev_y, sc, sf, ev) == cudaSuccess;
+    ok = ok && launch_fetch_and_ffn_split(L, x, dev_y, sc, sf, ev, moves_aside) == cudaSuccess;
     if (!ok) cudaGetLastError();
     return ok ? LIF_OK : LIF_ERR_CUDA;
   }
@@ -321,6 +326,7 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
     ok = ok && cudaEventRecord(L->ev_plan, sc) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(sf, L->ev_plan, 0) == cudaSuccess;
   }
+  if (moves_aside) ok = ok && launch_moves(L, sc, ev) == cudaSuccess;   // beside the fetch on sf
   if (ev) tm_record(ev[5], sf);
   ok = ok && launch_fetch(L, sf) == cudaSuccess;
   if (ev) tm_record(ev[6], sf);
@@ -440,7 +446,8 @@ lif_status lif_profile_launch(lif_layer* L, int32_t kernel, const void* dev_x, f
     case LIF_KERNEL_FETCH:     // in the form the decode step launches it
       e = (L->split_ffn && L->fused_fetch && fetch_ffn_supported(L))
               ? launch_fetch_ffn(L, (const __half*)dev_x,
-                                 L->y_partial + (size_t)L->ffn_grid * L->desc.d_model, st)
+                                 L->y_partial + (size_t)L->ffn_grid * L->desc.d_model, st,
+                                 !L->desc.append_first)
               : launch_fetch(L, st);
       break;
     case LIF_KERNEL_FFN_SUM:

@@ -64,9 +64,9 @@ fetch_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
 // (Section 3.3 item 3): h = act(<up, x> + bias) and partial += h * down.  The new rows then need
 // no second pass over HBM and no kernel of their own after the slowest step of the layer.  Rows
 // are dealt to CTAs in list order and each CTA adds its rows in that order, so the partials and
-// their sum do not depend on scheduling.  The first bundle's host loads are issued before the
-// dependency wait: the list and the counts were final before the preceding kernel (the row
-// moves) passed its own wait, while the cache rows may still be moving.
+// their sum do not depend on scheduling.  Where the kernel ahead is the row-move kernel, the
+// first bundle's host loads are issued before the dependency wait: the list and the counts were
+// final before that kernel passed its own wait, while the cache rows may still be moving.
 constexpr int kFusedChunks = 4;     // 8-column chunks per thread and half row: d_model <= 8192
 
 __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
@@ -93,15 +93,22 @@ struct FetchFfnArgs {
   float act_thr;
 };
 
-template <int kGate>
+// kEarly: the lists may be read, and the first host loads issued, before the dependency wait.
+template <int kGate, bool kEarly>
 __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   __shared__ float part[kThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = a.d >> 3;                       // 16-byte chunks per half row
-  const int n = __ldcg(a.counts + LIF_CNT_N_LOAD);
-  if ((int)blockIdx.x >= n) {                      // the sum reads min(grid, n) partials
+  if (!kEarly) {                                   // the kernel ahead wrote the lists
     pdl_wait();
     pdl_trigger();
+  }
+  const int n = __ldcg(a.counts + LIF_CNT_N_LOAD);
+  if ((int)blockIdx.x >= n) {                      // the sum reads min(grid, n) partials
+    if (kEarly) {
+      pdl_wait();
+      pdl_trigger();
+    }
     return;
   }
   uint4 up[kFusedChunks], down[kFusedChunks];
@@ -119,8 +126,10 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   int j = blockIdx.x;
   int id = __ldcg(a.load_ids + j), slot = __ldcg(a.load_slots + j);
   host_loads(id);
-  pdl_wait();
-  pdl_trigger();
+  if (kEarly) {
+    pdl_wait();
+    pdl_trigger();
+  }
 
   uint4 xq[kFusedChunks];
 #pragma unroll
@@ -227,7 +236,8 @@ bool fetch_ffn_supported(const lif_layer* L) {
 
 // Fetch of this step's new rows fused with their FFN terms; partials go to `partial`
 // ([fetch_grid][d_model], CTA c < min(grid, n_load) writes row c).
-cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st) {
+cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st,
+                             bool early_loads) {
   const lif_layer_desc& D = L->desc;
   FetchFfnArgs a;
   a.store = (const uint4*)L->dev_bundles;
@@ -242,11 +252,11 @@ cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cuda
   a.d = D.d_model;
   a.act = D.activation;
   a.act_thr = D.activation_threshold;
-  return D.gate_mode == LIF_GATE_RESIDENT
-             ? launch_k(fetch_ffn_kernel<LIF_GATE_RESIDENT>, dim3(L->fetch_grid), dim3(kThreads), 0,
-                        st, L->use_pdl, a)
-             : launch_k(fetch_ffn_kernel<LIF_GATE_NONE>, dim3(L->fetch_grid), dim3(kThreads), 0, st,
-                        L->use_pdl, a);
+  void (*kernel)(FetchFfnArgs) =
+      D.gate_mode == LIF_GATE_RESIDENT
+          ? (early_loads ? fetch_ffn_kernel<LIF_GATE_RESIDENT, true> : fetch_ffn_kernel<LIF_GATE_RESIDENT, false>)
+          : (early_loads ? fetch_ffn_kernel<LIF_GATE_NONE, true> : fetch_ffn_kernel<LIF_GATE_NONE, false>);
+  return launch_k(kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl, a);
 }
 
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,

@@ -403,7 +403,9 @@ cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cuda
       a = ffn_args(L, x, L->hit_slots, cnt + LIF_CNT_N_HITS, nullptr, p0, D.d_ff);
       break;
     case LIF_KERNEL_FFN_NEW:
-      a = ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
+      a = D.append_first
+              ? ffn_args(L, x, L->load_slots, cnt + LIF_CNT_N_LOAD, nullptr, p1, 0)
+              : ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
       break;
     case LIF_KERNEL_FFN_SUM:
       return launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st,
@@ -429,7 +431,7 @@ cudaError_t launch_partial_sum(lif_layer* L, const float* partial, const int32_t
 // were already cached does not depend on the fetch and runs on `side` meanwhile (forked after
 // the row moves, joined before the sum).
 cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream_t st,
-                                       cudaStream_t side, cudaEvent_t* ev) {
+                                       cudaStream_t side, cudaEvent_t* ev, bool moves_aside) {
   const lif_layer_desc& D = L->desc;
   const int d = D.d_model;
   const int32_t* cnt = L->counts;
@@ -441,6 +443,8 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
     if ((e = cudaEventRecord(L->ev_plan, st)) != cudaSuccess) return e;
     if ((e = cudaStreamWaitEvent(side, L->ev_plan, 0)) != cudaSuccess) return e;
   }
+  // append_first with a second stream: the row moves run there, ahead of the cached rows' FFN
+  if (moves_aside && (e = launch_moves(L, side, ev)) != cudaSuccess) return e;
   FfnArgs hit = D.ffn_mode == 0
                     ? ffn_args(L, x, L->hit_slots, cnt + LIF_CNT_N_HITS, nullptr, p0, D.d_ff)
                     : ffn_args(L, x, nullptr, cnt + LIF_CNT_NUM_KEPT, nullptr, p0, 0);
@@ -451,10 +455,13 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
   if (ev) tm_record(ev[8], side);
   if (fork && (e = cudaEventRecord(L->ev_fetch, side)) != cudaSuccess) return e;
   if (ev) tm_record(ev[5], st);
-  FfnArgs miss = ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
+  // the new rows: consecutive from num_kept, or (append_first) wherever load_slots says
+  FfnArgs miss = D.append_first
+                     ? ffn_args(L, x, L->load_slots, cnt + LIF_CNT_N_LOAD, nullptr, p1, 0)
+                     : ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
   if (L->fused_fetch && fetch_ffn_supported(L)) {
     // one kernel brings the new rows in and adds their FFN terms (CTA partials in p1)
-    if ((e = launch_fetch_ffn(L, x, p1, st)) != cudaSuccess) return e;
+    if ((e = launch_fetch_ffn(L, x, p1, st, !moves_aside)) != cudaSuccess) return e;
     if (ev) tm_record(ev[6], st);
   } else {
     if ((e = launch_fetch(L, st)) != cudaSuccess) return e;

@@ -113,12 +113,18 @@ cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t
 cudaError_t launch_gate_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
                                 int32_t* n_active, cudaStream_t st, cudaEvent_t* ev, int compact);
 bool window_plan_supported(const lif_layer_desc& D);
-cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr);
+// with_moves = false: the caller launches the row moves itself (launch_moves)
+cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr,
+                               bool with_moves = true);
 cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st,
-                          cudaEvent_t* ev = nullptr);
+                          cudaEvent_t* ev = nullptr, bool with_moves = true);
+cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
 bool fetch_ffn_supported(const lif_layer* L);
-cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st);
+// early_loads: the lists were final before the kernel ahead of this one passed its dependency
+// wait (so the first bundle's host loads may be issued before this kernel's own wait)
+cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st,
+                             bool early_loads);
 cudaError_t launch_refill(lif_layer* L, cudaStream_t st);
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,
                          int grid, cudaStream_t st);
@@ -127,7 +133,8 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
                        const int32_t* base, float* y, bool accumulate, cudaStream_t st,
                        cudaEvent_t* ev = nullptr);
 cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, cudaStream_t st,
-                                       cudaStream_t side, cudaEvent_t* ev = nullptr);
+                                       cudaStream_t side, cudaEvent_t* ev = nullptr,
+                                       bool moves_aside = false);
 cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cudaStream_t st);
 cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaStream_t st);
 cudaError_t ffn_configure(lif_layer* L);

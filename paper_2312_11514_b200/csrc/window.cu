@@ -12,6 +12,14 @@
 //   E  new neurons in ascending id get rows num_kept, num_kept + 1, ...
 //   F  slot lists for the FFN
 // The 4*d_model-byte row copies of step D run in a second, grid-wide kernel.
+//
+// append_first applies the two operations of Section 3.3 in the other order: the new neurons are
+// stacked at rows n, n + 1, ... first, then the deletions pull the last rows into the freed
+// ones.  A new neuron that would be moved straight away is simply given the freed row as the
+// place its bundle is written to: with e deleted and l new neurons, the r = min(e, l) last new
+// neurons take the r lowest freed rows (lowest row <- highest id), the others stay stacked, and
+// only the e - r freed rows left over are closed by moving old rows (those at or beyond
+// n - (e - r)).  Row moves and bundle writes then never touch the same row.
 #include "lif_internal.cuh"
 
 namespace lif {
@@ -69,6 +77,7 @@ struct WindowArgs {
   // with token `keep` of the step (keep = 1, keep_tok = nullptr: ordinary single-token update).
   const int8_t* keep_tok; // [F] last kept token per neuron, -1 if active only in later tokens
   int keep;
+  int append_first;       // stack the new neurons before deleting (see the header of this file)
   unsigned long long bundle_bytes;
 };
 
@@ -174,17 +183,20 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
 
   // ---- C: deleted rows (ascending slot) and surviving tail rows (descending slot) --------
   // Each thread owns a contiguous run of slots, so thread order is slot order.
+  // r freed rows are taken by new neurons directly; the others are closed by old rows from
+  // at or beyond `bound` (paper's order: r = 0, bound = n_kept)
+  const int reuse = a.append_first ? min(n_evict, n_load) : 0;
+  const int bound = n - (n_evict - reuse);
   const int seg = (n + kWindowThreads - 1) / kWindowThreads;
   const int s0 = min(n, tid * seg), s1 = min(n, s0 + seg);
-  int c_ev = 0, c_hole = 0, c_surv = 0;
+  int c_ev = 0, c_surv = 0;
   for (int s = s0; s < s1; ++s) {
     const int f = a.last_active[a.pointers[s]] <= stale_before;
     c_ev += f;
-    c_hole += f && s < n_kept;
-    c_surv += !f && s >= n_kept;
+    c_surv += !f && s >= bound;
   }
-  u64 pre = block_scan(pack3(c_ev, c_hole, c_surv), &tot, sc);
-  const int n_moves = field(tot, 1);          // == surviving tail rows
+  u64 pre = block_scan(pack3(c_ev, 0, c_surv), &tot, sc);
+  const int n_moves = field(tot, 2);          // surviving rows at or beyond the bound
   {
     int p_ev = field(pre, 0), p_surv = field(pre, 2);
     for (int s = s0; s < s1; ++s) {
@@ -194,7 +206,7 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
         a.evict_slots[p_ev] = s;
         a.evict_ids[p_ev] = id;
         ++p_ev;
-      } else if (s >= n_kept) {
+      } else if (s >= bound) {
         a.move_src[n_moves - 1 - p_surv] = s;   // last survivor first
         ++p_surv;
       }
@@ -205,7 +217,7 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   // ---- D: apply deletes to the bookkeeping ------------------------------------------------
   for (int j = tid; j < n_evict; j += kWindowThreads) a.slot_of[a.evict_ids[j]] = -1;
   for (int j = tid; j < n_moves; j += kWindowThreads) {
-    const int src = a.move_src[j], dst = a.evict_slots[j];
+    const int src = a.move_src[j], dst = a.evict_slots[reuse + j];
     const int id = a.pointers[src];
     a.move_dst[j] = dst;
     a.pointers[dst] = id;
@@ -213,7 +225,7 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
     a.bias[dst] = a.bias[src];
   }
   __syncthreads();
-  for (int s = n_kept + tid; s < n; s += kWindowThreads) a.pointers[s] = -1;
+  for (int s = bound + tid; s < n; s += kWindowThreads) a.pointers[s] = -1;
   __syncthreads();
 
   // ---- E + F: rows for the neurons to bring in, and the slot lists -----------------------
@@ -228,7 +240,9 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
       const int id = a.act[q];
       int s = a.slot_of[id];
       if (s < 0) {
-        s = n_kept + p_l;
+        // stacked new neurons keep rows bound, bound + 1, ...; the last `reuse` of them take
+        // the freed rows, lowest row <- highest id
+        s = p_l < n_load - reuse ? bound + p_l : a.evict_slots[n_load - 1 - p_l];
         a.load_ids[p_l] = id;
         a.load_slots[p_l] = s;
         a.slot_of[id] = s;
@@ -400,17 +414,17 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
     }
     return;
   }
-  int c_hole = 0, c_surv = 0;
+  // freed rows taken by new neurons directly, and where the rows that must move begin
+  // (paper's order: none, num_kept; see the header of this file)
+  const int reuse = a.append_first ? min(n_evict, n_load) : 0;
+  const int bound = n - (n_evict - reuse);
+  int c_surv = 0;
 #pragma unroll
   for (int j = 0; j < kPlanSlots; ++j)
-    if (j < my_slots) {
-      const bool e = (evm >> j) & 1u;
-      c_hole += e && (s0 + j) < n_kept;
-      c_surv += !e && (s0 + j) >= n_kept;
-    }
-  pre = block_scan(pack3(c_hole, c_surv, 0), &tot, sc);
-  const int n_moves = field(tot, 0);          // == surviving tail rows
-  int p_hole = field(pre, 0), p_surv = field(pre, 1);
+    if (j < my_slots) c_surv += !((evm >> j) & 1u) && (s0 + j) >= bound;
+  pre = block_scan(pack3(c_surv, 0, 0), &tot, sc);
+  const int n_moves = field(tot, 0);          // surviving rows at or beyond the bound
+  int p_surv = field(pre, 0);
 
   // ---- writes ---------------------------------------------------------------------------------
   {
@@ -424,24 +438,24 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
   for (int j = 0; j < kPlanSlots; ++j)
     if (j < my_slots && ((evm >> j) & 1u)) {                                     // deleted rows
       const int s = s0 + j;
-      a.evict_ids[p_ev++] = pid[j];
+      a.evict_ids[p_ev] = pid[j];
       a.slot_of[pid[j]] = -1;
-      if (s < n_kept) holes[p_hole++] = s;
+      holes[p_ev++] = s;                                 // freed rows, ascending
     }
   __syncthreads();
 #pragma unroll
   for (int j = 0; j < kPlanSlots; ++j)
     if (j < my_slots) {
       const int s = s0 + j;
-      if (!((evm >> j) & 1u) && s >= n_kept) {         // surviving tail row: last one first
+      if (!((evm >> j) & 1u) && s >= bound) {          // surviving tail row: last one first
         const int jm = n_moves - 1 - p_surv++;
-        const int dst = holes[jm];
+        const int dst = holes[reuse + jm];
         a.move_src[jm] = s;
         a.move_dst[jm] = dst;
         a.pointers[dst] = pid[j];
         a.slot_of[pid[j]] = dst;
         a.bias[dst] = pb[j];
-        newslot[s - n_kept] = dst;
+        newslot[s - bound] = dst;
       }
       if (s >= n_kept + n_load) a.pointers[s] = -1;    // tail beyond the rows to be loaded
     }
@@ -455,8 +469,8 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
         const int id = tid * 32 + __ffs(m) - 1;
         m &= m - 1;
         int s = so[i];
-        if (s < 0) {                                     // bring in: rows num_kept, num_kept + 1, ...
-          s = n_kept + p_load;
+        if (s < 0) {                                     // bring in: stacked rows, or freed ones
+          s = p_load < n_load - reuse ? bound + p_load : holes[n_load - 1 - p_load];
           a.load_ids[p_load] = id;
           a.load_slots[p_load] = s;
           ++p_load;
@@ -464,7 +478,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
           a.pointers[s] = id;
           a.bias[s] = bu[i];
         } else {
-          if (s >= n_kept) s = newslot[s - n_kept];      // it was moved into a hole
+          if (s >= bound) s = newslot[s - bound];        // it was moved into a freed row
           a.hit_slots[p_hit++] = s;
         }
         a.active_slots[q] = s;
@@ -493,7 +507,8 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
 }
 
 // Row moves of step D: cache row move_src[j] -> row move_dst[j].  Sources lie at or beyond
-// num_kept, destinations below it, so the copies never overlap.
+// num_kept (append_first: the bound above which old rows must move), destinations below it, so
+// the copies never overlap.
 __global__ void __launch_bounds__(kThreads)
 move_rows_kernel(uint4* __restrict__ cache, const int32_t* __restrict__ move_src,
                  const int32_t* __restrict__ move_dst, const int32_t* __restrict__ counts,
@@ -560,10 +575,11 @@ static WindowArgs window_args(lif_layer* L, const int32_t* act, const int32_t* n
   a.keep_tok = D.spec_keep > 0 ? L->keep_tok : nullptr;
   a.keep = D.spec_keep > 0 ? D.spec_keep : 1;
   a.bundle_bytes = 2ull * row_elems(D);
+  a.append_first = D.append_first;
   return a;
 }
 
-static cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev) {
+cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev) {
   const lif_layer_desc& D = L->desc;
   cudaError_t e;
   if (ev) tm_record(ev[3], st);
@@ -575,10 +591,10 @@ static cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev) 
 }
 
 cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act,
-                          cudaStream_t st, cudaEvent_t* ev) {
+                          cudaStream_t st, cudaEvent_t* ev, bool with_moves) {
   cudaError_t e = launch_k(window_update_kernel, dim3(1), dim3(kWindowThreads), 0, st, L->use_pdl,
                            window_args(L, act, n_act));
-  return e != cudaSuccess ? e : launch_moves(L, st, ev);
+  return (e != cudaSuccess || !with_moves) ? e : launch_moves(L, st, ev);
 }
 
 bool window_plan_supported(const lif_layer_desc& D) {
@@ -586,13 +602,13 @@ bool window_plan_supported(const lif_layer_desc& D) {
 }
 
 // Window update straight from the predictor's bit mask (see window_plan_kernel).
-cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev) {
+cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev, bool with_moves) {
   const lif_layer_desc& D = L->desc;
   const int nwords = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
   cudaError_t e = launch_k(window_plan_kernel, dim3(1), dim3(kWindowThreads), 0, st, L->use_pdl,
                            window_args(L, L->active_idx, L->n_tmp), (const uint32_t*)L->mask_words,
                            nwords, (int32_t*)L->n_tmp);
-  return e != cudaSuccess ? e : launch_moves(L, st, ev);
+  return (e != cudaSuccess || !with_moves) ? e : launch_moves(L, st, ev);
 }
 
 }  // namespace lif

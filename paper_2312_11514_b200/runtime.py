@@ -20,7 +20,8 @@ class Layer:
                  bias_down: Optional[torch.Tensor] = None, n_streams: int = 1,
                  threshold_logit: float = 0.0, ffn_mode: int = 0, activation: int = 0,
                  activation_threshold: float = 0.0, budget_rows: int = 0, spec_keep: int = 0,
-                 gate_mode: int = 0, gate: Optional[torch.Tensor] = None, device="cuda:0"):
+                 gate_mode: int = 0, gate: Optional[torch.Tensor] = None, append_first: int = 0,
+                 device="cuda:0"):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2312_11514_b200 needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
@@ -37,7 +38,8 @@ class Layer:
         shape = dict(d_model=d_model, d_ff=d_ff, rank=rank, window_k=window_k, capacity=capacity,
                      n_streams=n_streams, threshold_logit=threshold_logit, ffn_mode=ffn_mode,
                      activation=activation, activation_threshold=activation_threshold,
-                     budget_rows=budget_rows, spec_keep=spec_keep, gate_mode=gate_mode)
+                     budget_rows=budget_rows, spec_keep=spec_keep, gate_mode=gate_mode,
+                     append_first=append_first)
         self.spec_keep, self.gate_mode = spec_keep, gate_mode
         nbytes = B.lif_workspace_bytes(B.make_desc(**shape))
         self.workspace = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
@@ -100,7 +102,7 @@ def pinned_store(d_ff: int, d_model: int, n_vec: int = 2) -> torch.Tensor:
 
 def build_stack(cfg, device="cuda:0", n_layers: Optional[int] = None, capacity_margin: float = 8.0,
                 ffn_mode: int = 0, gen_device=None, gate_mode: int = 0, activation: int = 0,
-                activation_threshold: float = 0.0) -> List[Layer]:
+                activation_threshold: float = 0.0, append_first: int = 0) -> List[Layer]:
     """Generate the weights of a named synthetic configuration and create its layers."""
     from . import workloads as W
     layers = []
@@ -116,5 +118,5 @@ def build_stack(cfg, device="cuda:0", n_layers: Optional[int] = None, capacity_m
                             pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), n_streams=cfg.n_streams,
                             ffn_mode=ffn_mode, gate_mode=gate_mode, gate=dev(w.get("gate")),
                             activation=activation, activation_threshold=activation_threshold,
-                            device=device))
+                            append_first=append_first, device=device))
     return layers

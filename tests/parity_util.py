@@ -78,7 +78,7 @@ class OracleLayer:
     """Oracle-side twin of one layer, fed with the same tensors."""
 
     def __init__(self, w, d_model, d_ff, capacity, window_k, theta=0.0, b_down=None,
-                 activation=0, act_threshold=0.0, budget_rows=0, gate_mode=0):
+                 activation=0, act_threshold=0.0, budget_rows=0, gate_mode=0, append_first=False):
         self.activation, self.act_threshold, self.gate_mode = activation, act_threshold, gate_mode
         self.gate = w["gate"].cpu().numpy() if gate_mode == 2 else None
         self.A = w["A"].cpu().numpy().astype(np.float64)
@@ -91,7 +91,7 @@ class OracleLayer:
         if gate_mode == 2:        # the gate is the predictor: active iff it passes the activation
             self.theta = act_threshold if activation == O.FATRELU else 0.0
         self.cache = O.NeuronCache(d_model, d_ff, capacity, window_k, budget_rows,
-                                   n_vec=3 if gate_mode == 1 else 2)
+                                   n_vec=3 if gate_mode == 1 else 2, append_first=bool(append_first))
 
     def scores(self, x_np):
         """The predictor's scores: low-rank, or the resident gate's pre-activations."""
@@ -102,7 +102,7 @@ class OracleLayer:
 
 def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_down=False,
                     activation=0, act_threshold=0.0, budget_rows=0, spec_keep=0, gate_mode=0,
-                    device="cuda:0"):
+                    append_first=0, device="cuda:0"):
     store = R.pinned_store(cfg.d_ff, cfg.d_model, 3 if gate_mode == 1 else 2)
     w = W.make_layer(cfg, layer_idx, device=device, bundles_out=store, gate_mode=gate_mode,
                      act_threshold=act_threshold)
@@ -118,9 +118,10 @@ def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_d
                   n_streams=cfg.n_streams, threshold_logit=theta, ffn_mode=ffn_mode,
                   activation=activation, activation_threshold=act_threshold, budget_rows=budget_rows,
                   spec_keep=spec_keep, gate_mode=gate_mode,
-                  gate=dev(w["gate"]) if gate_mode == 2 else None, device=device)
+                  gate=dev(w["gate"]) if gate_mode == 2 else None, append_first=append_first,
+                  device=device)
     ora = OracleLayer(w, cfg.d_model, cfg.d_ff, cap, cfg.window_k, theta, bd, activation, act_threshold,
-                      budget_rows, gate_mode)
+                      budget_rows, gate_mode, append_first)
     return gpu, ora
 
 

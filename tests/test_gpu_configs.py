@@ -18,7 +18,8 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _run_config(name, n_tokens, sample_layers, oracle_tokens=None, gate_mode=0, activation=0, thr=0.0):
+def _run_config(name, n_tokens, sample_layers, oracle_tokens=None, gate_mode=0, activation=0, thr=0.0,
+                append_first=0):
     cfg = W.CONFIGS[name]
     n_vec = 3 if gate_mode == B.GATE_BUNDLED else 2
     bundle_bytes = n_vec * cfg.d_model * 2
@@ -36,10 +37,11 @@ def _run_config(name, n_tokens, sample_layers, oracle_tokens=None, gate_mode=0, 
         layers.append(R.Layer(d_model=d, d_ff=F, rank=cfg.rank, window_k=cfg.window_k, capacity=cap,
                               host_bundles=store, pred_A=w["A"], pred_B=w["B"], pred_c=w["c"],
                               bias_up=w["bias_up"], n_streams=S, gate_mode=gate_mode, gate=w.get("gate"),
-                              activation=activation, activation_threshold=thr, device=DEV))
+                              activation=activation, activation_threshold=thr,
+                              append_first=append_first, device=DEV))
         if l in sample_layers:
             oras[l] = P.OracleLayer(w, d, F, cap, cfg.window_k, activation=activation,
-                                    act_threshold=thr, gate_mode=gate_mode)
+                                    act_threshold=thr, gate_mode=gate_mode, append_first=append_first)
         del w
     X = W.make_inputs(cfg, device=DEV)
     dev_x = torch.empty(S, d, dtype=torch.float16, device=DEV)
@@ -91,6 +93,11 @@ def test_opt6p7b_full_stack_all_tokens():
     _run_config("opt6p7b", 128, sample_layers=(0, 15, 31))
 
 
+def test_opt6p7b_full_stack_new_neurons_stacked_first():
+    # the benchmark's default order of the cache operations: bundles go straight into freed rows
+    _run_config("opt6p7b", 48, sample_layers=(0, 15, 31), append_first=1)
+
+
 def test_falcon7b_full_stack():
     _run_config("falcon7b", 48, sample_layers=(3, 30), oracle_tokens=40)
 
@@ -100,7 +107,7 @@ def test_phi2_full_stack():
 
 
 def test_batched8_full_stack_eight_streams():
-    _run_config("batched8", 8, sample_layers=(1, 46), oracle_tokens=6)
+    _run_config("batched8", 8, sample_layers=(1, 46), oracle_tokens=6, append_first=1)
 
 
 @pytest.mark.parametrize("gate_mode", [B.GATE_BUNDLED, B.GATE_RESIDENT])

@@ -427,3 +427,68 @@ def test_decode_step_with_and_without_the_fused_fetch(d, F, k, act, thr, gate_mo
         n_load += len(lists["load_ids"]); n_evict += len(lists["evict_ids"])
     assert n_load > 0 and n_evict > 0
     gpu.close()
+
+
+# ---- append-first order of the cache operations (new neurons stacked, then the deletions) ----
+@pytest.mark.parametrize("d,F,r,k,S,fire", [
+    (256, 1024, 16, 3, 1, 0.05),
+    (264, 1000, 24, 1, 1, 0.08),      # window of one token: as many deletions as arrivals, roughly
+    (512, 4096, 40, 4, 3, 0.04),      # three streams
+    (2048, 8192, 32, 3, 1, 0.40),     # more than 4096 cached rows: the general window kernel
+])
+def test_append_first_staged(d, F, r, k, S, fire):
+    cfg = W.LifConfig("af", 1, d, F, r, k, S, 12, fire, 1.0, 0.8, 0.6, 41)
+    stats = _run_staged(cfg, 0, cfg.steps, b_down=True, append_first=1,
+                        capacity=F if fire > 0.2 else None)
+    assert sum(s["n_evict"] for s in stats) > 0
+
+
+@pytest.mark.parametrize("two_streams,fused_plan,fused_fetch,S,gate_mode", [
+    (True, 1, 1, 1, 0), (True, 0, 1, 1, 0), (True, 1, 0, 1, 0), (False, 1, 1, 1, 0),
+    (True, 1, 1, 4, 0), (True, 1, 1, 1, 2), (True, 1, 1, 1, 1)])
+def test_append_first_decode_step(two_streams, fused_plan, fused_fetch, S, gate_mode):
+    # with two streams the row moves run beside the fetch; all forms must match the oracle
+    cfg = W.LifConfig("afd", 1, 512, 4096, 32, 2, S, 14, 0.06, 1.0, 0.8, 0.6, 42)
+    act, thr = (B.ACT_FATRELU, 0.05) if gate_mode else (B.ACT_RELU, 0.0)
+    gpu, ora = P.make_layer_pair(cfg, 0, append_first=1, gate_mode=gate_mode, activation=act,
+                                 act_threshold=thr, b_down=True)
+    B.lif_set_tuning(gpu.handle, B.TUNE_FUSED_PLAN, fused_plan)
+    B.lif_set_tuning(gpu.handle, B.TUNE_FUSED_FETCH_FFN, fused_fetch)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(S, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = (torch.cuda.Stream(), torch.cuda.Stream()) if two_streams else (None, None)
+    torch.cuda.synchronize()
+    n_moves = n_reused = 0
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        torch.cuda.synchronize()
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        P.compare_cache_rows(gpu, ora)
+        n_moves += len(lists["move_src"])
+        n_reused += int((lists["load_slots"] < lists["num_used_before"]).sum())
+    st = B.lif_get_stats(gpu.handle)
+    assert st.status == B.LIF_OK and st.rows_moved == ora.cache.rows_moved == n_moves
+    assert n_reused > 0 and n_moves > 0
+    gpu.close()
+
+
+def test_append_first_with_memory_budget_and_speculative_window():
+    cfg = W.LifConfig("afb", 1, 256, 4096, 16, 5, 1, 24, 0.05, 1.0, 0.5, 0.87, 15)
+    stats = _run_staged(cfg, 0, cfg.steps, budget_rows=600, capacity=1024, append_first=1)
+    assert min(s["k_eff"] for s in stats) < cfg.window_k
+    S = 5
+    cfg = W.LifConfig("afs", 1, 256, 4096, 16, 3, S, 10, 0.03, 1.0, 0.8, 0.6, 16)
+    gpu, ora = P.make_layer_pair(cfg, 0, spec_keep=2, capacity=2048, append_first=1)
+    Xs = W.make_inputs(cfg.scaled(n_streams=1, steps=cfg.steps * S), device=DEV)
+    X = Xs.reshape(cfg.steps, S, cfg.d_model).contiguous()
+    bufs = P.make_bufs(gpu)
+    stats = [P.staged_step(gpu, ora, X[t], bufs) for t in range(cfg.steps)]
+    assert sum(s["n_evict"] for s in stats) > 0
+    gpu.close()
+
+
+def test_append_first_is_refused_with_the_whole_cache_ffn():
+    with pytest.raises(B.LifError) as e:
+        B.lif_workspace_bytes(B.make_desc(d_model=256, d_ff=1024, rank=16, window_k=2, capacity=512,
+                                          ffn_mode=1, append_first=1))
+    assert e.value.code == B.LIF_ERR_INVALID_ARG
