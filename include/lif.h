@@ -122,7 +122,8 @@ enum {
   LIF_CNT_N_LOAD = 3,       /* neurons to bring in */
   LIF_CNT_N_HITS = 4,       /* active neurons already cached */
   LIF_CNT_NUM_USED_BEFORE = 5,
-  LIF_CNT_NUM_KEPT = 6,     /* rows left after deleting = first slot of the new rows */
+  LIF_CNT_NUM_KEPT = 6,     /* rows left after deleting (without append_first also the first
+                               row of the new neurons) */
   LIF_CNT_NUM_USED = 7,     /* rows in use after the step */
   LIF_CNT_STEP = 8,         /* steps applied so far */
   LIF_CNT_STATUS = 9,       /* sticky lif_status written by kernels */
@@ -197,8 +198,8 @@ lif_status lif_predict(lif_layer* layer, const void* dev_x, float* dev_logits_or
 /* Sliding-window update (Section 3.1 "The Sliding Window Technique", Section 3.3 items 1-2):
  * stamps the active neurons, deletes the neurons not active in the last window_k steps by
  * moving tail rows into their slots (first freed slot <- last surviving row), assigns rows
- * num_kept.. to the neurons to bring in (ascending id), updates pointers / slot_of / bias /
- * num_used, writes every list of lif_lists, applies the row moves inside dev_cache, and
+ * num_kept.. (append_first: freed rows first) to the neurons to bring in (ascending id),
+ * updates pointers / slot_of / bias / num_used, writes every list of lif_lists, applies the row moves inside dev_cache, and
  * advances the step.  On overflow sets LIF_ERR_CAPACITY in the status word and changes
  * nothing.  dev_active_idx must be ascending and duplicate-free. */
 lif_status lif_window_update(lif_layer* layer, const int32_t* dev_active_idx,
