@@ -362,7 +362,7 @@ def run_ours(args):
         }
         if args.cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(cfg, layers, X, args.cpu_layers, args.cpu_tokens,
-                                               _gate_setup(args))
+                                               _gate_setup(args), args.append_first)
         print(json.dumps(out), flush=True)
     B.lif_graph_destroy(graph)
     for l in layers:
@@ -478,7 +478,7 @@ def _oracle_threads():
     return len(os.sched_getaffinity(0))
 
 
-def _oracle_layers(cfg, tensors, O, gate=(0, 0, 0.0)):
+def _oracle_layers(cfg, tensors, O, gate=(0, 0, 0.0), append_first=False):
     import numpy as np
     out = []
     for w, cap in tensors:
@@ -487,7 +487,8 @@ def _oracle_layers(cfg, tensors, O, gate=(0, 0, 0.0)):
                         bias_up=w["bias_up"].cpu().numpy(),
                         gate=w["gate"].cpu().numpy() if gate[0] == 2 else None,
                         cache=O.NeuronCache(cfg.d_model, cfg.d_ff, cap, cfg.window_k,
-                                            n_vec=3 if gate[0] == 1 else 2)))
+                                            n_vec=3 if gate[0] == 1 else 2,
+                                            append_first=bool(append_first))))
     return out
 
 
@@ -502,7 +503,7 @@ def _oracle_token(ol, x_np, O, gate=(0, 0, 0.0)):
                           activation=act, threshold=thr, gated=gm == 1)
 
 
-def cpu_baseline(cfg, layers, X, n_layers, n_tokens, gate=(0, 0, 0.0)):
+def cpu_baseline(cfg, layers, X, n_layers, n_tokens, gate=(0, 0, 0.0), append_first=False):
     """The oracle, as it stands, on a bounded sample: the first n_layers layers over the first
     n_tokens tokens; tokens/s scaled to the full stack by layers."""
     from oracle import lif_oracle as O
@@ -511,7 +512,7 @@ def cpu_baseline(cfg, layers, X, n_layers, n_tokens, gate=(0, 0, 0.0)):
                  "bundles": l.keep["host_bundles"], "bias_up": l.keep["bias_up"],
                  "gate": l.keep["gate"]}, l.capacity)
                for l in layers[:n_layers]]
-    ol = _oracle_layers(cfg, tensors, O, gate)
+    ol = _oracle_layers(cfg, tensors, O, gate, append_first)
     xs = X[:n_tokens].cpu().numpy()
     warm = min(cfg.window_k + 1, n_tokens - 1)
     for t in range(warm):
@@ -542,7 +543,7 @@ def run_reference(args):
     if not args.layers:
         # bound the run: time one layer-step, then keep as many layers as fit ~2 minutes
         w0 = {k: v.cpu() for k, v in mk(0).items()}
-        probe = _oracle_layers(cfg, [(w0, W.window_capacity(cfg, w0["p"]))], O, gate)
+        probe = _oracle_layers(cfg, [(w0, W.window_capacity(cfg, w0["p"]))], O, gate, args.append_first)
         x0 = _inputs(cfg, 2, gen, W).cpu().numpy()
         _oracle_token(probe, x0[0], O, gate)
         t0 = time.perf_counter()
@@ -554,7 +555,7 @@ def run_reference(args):
     for l in range(L):
         w = {k: v.cpu() for k, v in mk(l).items()}
         tensors.append((w, W.window_capacity(cfg, w["p"])))
-    ol = _oracle_layers(cfg, tensors, O, gate)
+    ol = _oracle_layers(cfg, tensors, O, gate, args.append_first)
     K, Wm = args.steps, args.warmup
     xs = _inputs(cfg, Wm + K, gen, W).cpu().numpy()
     for t in range(Wm):
