@@ -487,6 +487,25 @@ def test_append_first_with_memory_budget_and_speculative_window():
     gpu.close()
 
 
+def test_append_first_with_memory_budget_through_the_decode_step():
+    cfg = W.LifConfig("afbd", 1, 256, 4096, 16, 5, 1, 24, 0.05, 1.0, 0.5, 0.87, 15)
+    gpu, ora = P.make_layer_pair(cfg, 0, budget_rows=600, capacity=1024, append_first=1)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(1, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    ks = []
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        torch.cuda.synchronize()
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        P.compare_cache_rows(gpu, ora)
+        assert lists["num_used"] <= 600
+        ks.append(lists["k_eff"])
+    assert min(ks) < cfg.window_k and max(ks) == cfg.window_k, ks
+    gpu.close()
+
+
 def test_append_first_is_refused_with_the_whole_cache_ffn():
     with pytest.raises(B.LifError) as e:
         B.lif_workspace_bytes(B.make_desc(d_model=256, d_ff=1024, rank=16, window_k=2, capacity=512,
