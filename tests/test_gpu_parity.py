@@ -511,3 +511,38 @@ def test_append_first_is_refused_with_the_whole_cache_ffn():
         B.lif_workspace_bytes(B.make_desc(d_model=256, d_ff=1024, rank=16, window_k=2, capacity=512,
                                           ffn_mode=1, append_first=1))
     assert e.value.code == B.LIF_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("ffn_mode,split,gate_mode", [(0, 1, 0), (0, 0, 0), (1, 1, 0), (1, 0, 0), (0, 1, 1)])
+def test_multi_stream_decode_step_split_around_the_fetch(ffn_mode, split, gate_mode):
+    # several streams, two CUDA streams: the fetch runs on the second stream, one tensor-core FFN
+    # over all rows follows it (the split switch only concerns single-stream layers: splitting the
+    # multi-stream FFN around the fetch measured slower)
+    cfg = W.LifConfig("msplit", 1, 512, 4096, 32, 2, 3, 10, 0.06, 1.0, 0.8, 0.6, 43)
+    act, thr = (B.ACT_FATRELU, 0.05) if gate_mode else (B.ACT_RELU, 0.0)
+    gpu, ora = P.make_layer_pair(cfg, 0, ffn_mode=ffn_mode, gate_mode=gate_mode, activation=act,
+                                 act_threshold=thr, b_down=True)
+    B.lif_set_tuning(gpu.handle, B.TUNE_SPLIT_FFN, split)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(cfg.n_streams, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    n_evict = 0
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        torch.cuda.synchronize()
+        x_np = X[t].cpu().numpy()
+        if ffn_mode == 0:
+            lists = P.check_decode_step(gpu, ora, x_np, y.cpu().numpy().astype(np.float64))
+        else:
+            g = gpu.lists()
+            P.assert_mask_borderline(g["active_idx"], ora.scores(x_np), ora.theta)
+            lists = ora.cache.window_update(g["active_idx"])
+            ora.cache.insert(lists, ora.bundles, ora.bias_up)
+            P.compare_lists_and_state(gpu, ora, lists)
+            ref_y, flips = P.ffn_reference(ora, np.arange(ora.cache.num_used), x_np)
+            P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y, flips)
+        P.compare_cache_rows(gpu, ora)
+        n_evict += len(lists["evict_ids"])
+    assert n_evict > 0
+    gpu.close()
