@@ -31,6 +31,8 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes of sparse_ffn_kernel, from
 # the ncu capture summarised under profiles/ (set to None when that kernel changes)
 FFN_TRAFFIC_RATIO = 1.005
+# fetch_ffn_kernel: bytes read from system memory per bundle byte, same kind of capture
+FETCH_TRAFFIC_RATIO = 1.000
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -348,7 +350,11 @@ def run_ours(args):
                                     else "fetch_kernel", "bound": "host_link", "achieved": fetch_gbs,
                           "peak": link_peak, "unit": "GB/s", "frac": fetch_gbs / link_peak,
                           "peak_kind": "of measured (1 GiB pinned cudaMemcpyAsync, this run)",
-                          "bytes_per_launch": fetch_bytes, "us_per_launch": kernel_us["fetch"]},
+                          "bytes_per_launch": fetch_bytes, "us_per_launch": kernel_us["fetch"],
+                          "traffic": FETCH_TRAFFIC_RATIO * fetch_bytes if S == 1 and not gate_mode else None,
+                          "traffic_how": "system-memory bytes read per algorithmic byte from the ncu capture "
+                                         "in profiles/fetch_ffn_kernel_opt6p7b_12layers.md, scaled by this "
+                                         "run's rows per launch"},
             "predictor": {"bound": "hbm", "achieved": pred_gbs, "unit": "GB/s", "frac": pred_gbs / peak,
                           "bytes_per_launch": pred_bytes, "us_per_launch": pred_us},
             "kernel_us_per_launch": kernel_us,
