@@ -55,3 +55,27 @@ def test_inputs_ar1_and_capacity():
                                               lay["c"].numpy()), 0.0)
         cache.window_update(act)
     assert cache.num_used <= cap
+
+
+def test_gated_layers_shapes_and_gate_firing_rate():
+    cfg = W.CONFIGS["tiny"]
+    d, F, thr = cfg.d_model, cfg.d_ff, 0.05
+    plain = W.make_layer(cfg, 0)
+    bun = W.make_layer(cfg, 0, gate_mode=W.GATE_BUNDLED, act_threshold=thr)
+    res = W.make_layer(cfg, 0, gate_mode=W.GATE_RESIDENT, act_threshold=thr)
+    assert bun["bundles"].shape == (F, 3 * d) and "gate" not in bun
+    assert res["bundles"].shape == (F, 2 * d) and res["gate"].shape == (F, d)
+    # the same draws: the resident gate is the first vector of the three-vector bundle
+    assert torch.equal(res["gate"], bun["bundles"][:, :d])
+    assert torch.equal(res["bundles"], bun["bundles"][:, d:])
+    assert torch.equal(res["bias_up"], bun["bias_up"])
+    assert plain["bundles"].shape == (F, 2 * d)
+    assert W.CONFIGS["llama2_7b"].d_ff == 11008 and W.CONFIGS["llama2_7b"].window_k == 2
+    # N(0, I) inputs: the gate value passes the threshold at the configured mean rate, and the
+    # resident gate as predictor finds exactly those neurons
+    g = torch.Generator().manual_seed(7)
+    X = torch.randn(400, d, generator=g, dtype=torch.float64).numpy()
+    scores = O.gate_scores(X, res["gate"].numpy(), res["bias_up"].numpy())
+    assert abs((scores > thr).mean() - cfg.mean_fire) < 0.01
+    pre = X @ bun["bundles"][:, :d].double().numpy().T + bun["bias_up"].double().numpy()
+    np.testing.assert_allclose(pre, scores, rtol=1e-12, atol=1e-12)
