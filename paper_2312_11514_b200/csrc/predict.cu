@@ -133,11 +133,30 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
   const float my_c = (tid < kLogitTile && my_col < F) ? c[my_col] : 0.f;
   pdl_wait();
   pdl_trigger();
-  for (int i = tid; i < S * r; i += kThreads) {
-    float v = 0.f;
+  if (S == 1) {
+    for (int i = tid; i < S * r; i += kThreads) {
+      float v = 0.f;
 #pragma unroll 8
-    for (int p = 0; p < P; ++p) v += __ldcg(z_partial + (size_t)p * S * r + i);
-    zs[i] = v;
+      for (int p = 0; p < P; ++p) v += __ldcg(z_partial + (size_t)p * S * r + i);
+      zs[i] = v;
+    }
+  } else {
+    // several streams: S * r sums per CTA; four per thread at a time keep 32 loads in flight
+    // (same order of additions per sum)
+    for (int i0 = tid; i0 < S * r; i0 += 4 * kThreads) {
+      float v[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+      for (int p = 0; p < P; ++p) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * kThreads;
+          if (i < S * r) v[u] += __ldcg(z_partial + (size_t)p * S * r + i);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (i0 + u * kThreads < S * r) zs[i0 + u * kThreads] = v[u];
+    }
   }
   __syncthreads();
 
