@@ -506,6 +506,33 @@ def test_append_first_with_memory_budget_through_the_decode_step():
     gpu.close()
 
 
+def test_append_first_speculative_window_through_the_decode_step():
+    S, keep = 5, 2
+    cfg = W.LifConfig("afsd", 1, 256, 4096, 16, 3, S, 10, 0.03, 1.0, 0.8, 0.6, 16)
+    gpu, ora = P.make_layer_pair(cfg, 0, spec_keep=keep, capacity=2048, append_first=1)
+    Xs = W.make_inputs(cfg.scaled(n_streams=1, steps=cfg.steps * S), device=DEV)
+    X = Xs.reshape(cfg.steps, S, cfg.d_model).contiguous()
+    y = torch.empty(S, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    n_evict = 0
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        g = gpu.lists()
+        x_np = X[t].cpu().numpy()
+        logits = O.predictor_logits(x_np, ora.A, ora.B, ora.c)
+        P.assert_mask_borderline(g["active_idx"], logits, 0.0)
+        kt = P.keep_tokens_checked(gpu, g["active_idx"], logits, 0.0)
+        _, _, lists, ref_y = O.decode_step(ora.cache, x_np, ora.A, ora.B, ora.c, 0.0, ora.bundles,
+                                           ora.bias_up, act=g["active_idx"], keep_token=kt, keep=keep)
+        P.compare_lists_and_state(gpu, ora, lists)
+        P.compare_cache_rows(gpu, ora)
+        P.assert_y_close(y.cpu().numpy().astype(np.float64), ref_y)
+        n_evict += len(lists["evict_ids"])
+    assert n_evict > 0 and gpu.lists()["step"] == cfg.steps * keep
+    gpu.close()
+
+
 def test_append_first_is_refused_with_the_whole_cache_ffn():
     with pytest.raises(B.LifError) as e:
         B.lif_workspace_bytes(B.make_desc(d_model=256, d_ff=1024, rank=16, window_k=2, capacity=512,
