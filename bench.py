@@ -514,13 +514,14 @@ def cpu_baseline(cfg, layers, X, n_layers, n_tokens, gate=(0, 0, 0.0), append_fi
     n_tokens tokens; tokens/s scaled to the full stack by layers."""
     from oracle import lif_oracle as O
     n_layers = min(n_layers, len(layers))
+    n_tokens = min(n_tokens, X.shape[0])          # a short run has fewer tokens than the sample asks for
     tensors = [({"A": l.keep["pred_A"], "B": l.keep["pred_B"], "c": l.keep["pred_c"],
                  "bundles": l.keep["host_bundles"], "bias_up": l.keep["bias_up"],
                  "gate": l.keep["gate"]}, l.capacity)
                for l in layers[:n_layers]]
     ol = _oracle_layers(cfg, tensors, O, gate, append_first)
     xs = X[:n_tokens].cpu().numpy()
-    warm = min(cfg.window_k + 1, n_tokens - 1)
+    warm = max(0, min(cfg.window_k + 1, n_tokens - 1))
     for t in range(warm):
         _oracle_token(ol, xs[t], O, gate)
     t0 = time.perf_counter()
