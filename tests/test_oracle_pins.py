@@ -738,3 +738,40 @@ def test_append_first_worked_example_and_transient_overshoot():
     # capacity still refuses what does not fit at the end of the step
     with pytest.raises(O.CapacityError):
         cache.window_update(np.arange(0, 9))
+
+
+def test_append_first_agrees_with_the_papers_order_under_budget_and_multi_token_updates():
+    # the order of the two cache operations changes rows, never sets, window choices or traffic
+    F, d, T = 120, 3, 40
+    r = _rng(90)
+    bundles = r.normal(size=(F, 2 * d)).astype(np.float16)
+    bias_up = r.normal(size=F).astype(np.float16)
+    sets = _random_active_sets(F, T, 0.10, seed=9)
+    a = O.NeuronCache(d, F, F, window_k=5, budget_rows=34, append_first=True)
+    b = O.NeuronCache(d, F, F, window_k=5, budget_rows=34)
+    ks = []
+    for act in sets:
+        la, lb = a.window_update(act), b.window_update(act)
+        a.insert(la, bundles, bias_up); b.insert(lb, bundles, bias_up)
+        _check_structure(a)
+        assert la["k_eff"] == lb["k_eff"] and a.cached_ids() == b.cached_ids()
+        assert sorted(la["evict_ids"].tolist()) == sorted(lb["evict_ids"].tolist())
+        assert la["load_ids"].tolist() == lb["load_ids"].tolist() and a.num_used <= 34
+        ks.append(la["k_eff"])
+    assert min(ks) < 5 and a.bytes_fetched == b.bytes_fetched and a.rows_moved <= b.rows_moved
+    # several tokens per update (speculative decoding), window ending at the second token
+    a = O.NeuronCache(d, F, F, window_k=3, append_first=True)
+    b = O.NeuronCache(d, F, F, window_k=3)
+    for t in range(0, T - 4, 4):
+        logits = np.full((4, F), -1.0)
+        for j in range(4):
+            logits[j, sets[t + j]] = 1.0
+        act = O.active_set(logits, 0.0)
+        kt = O.keep_tokens(logits, 0.0, act, 2)
+        la, lb = a.window_update(act, kt, 2), b.window_update(act, kt, 2)
+        a.insert(la, bundles, bias_up); b.insert(lb, bundles, bias_up)
+        _check_structure(a)
+        assert a.cached_ids() == b.cached_ids() and a.t == b.t
+        np.testing.assert_array_equal(a.last_active, b.last_active)
+        for s in range(a.num_used):
+            np.testing.assert_array_equal(a.matrix[s], bundles[a.pointers[s]])
