@@ -196,11 +196,12 @@ def test_decode_token_host_matches_per_layer_decode_steps():
         l.close()
 
 
-def test_graph_replay_matches_direct_decode_steps_bitwise():
+@pytest.mark.parametrize("append_first", [0, 1])
+def test_graph_replay_matches_direct_decode_steps_bitwise(append_first):
     cfg = W.CONFIGS["tiny"]
     X = W.make_inputs(cfg, device=DEV)
-    a = R.build_stack(cfg, DEV)
-    b = R.build_stack(cfg, DEV)
+    a = R.build_stack(cfg, DEV, append_first=append_first)
+    b = R.build_stack(cfg, DEV, append_first=append_first)
     L, S, d = cfg.n_layers, cfg.n_streams, cfg.d_model
     dev_x = torch.empty(S, d, dtype=torch.float16, device=DEV)
     y_g = torch.zeros(L, S, d, dtype=torch.float32, device=DEV)
@@ -572,4 +573,44 @@ def test_multi_stream_decode_step_split_around_the_fetch(ffn_mode, split, gate_m
         P.compare_cache_rows(gpu, ora)
         n_evict += len(lists["evict_ids"])
     assert n_evict > 0
+    gpu.close()
+
+
+@pytest.mark.parametrize("append_first", [0, 1])
+def test_phase_timing_and_snapshot_with_both_cache_orders(append_first):
+    cfg = W.CONFIGS["tiny"]
+    X = W.make_inputs(cfg, device=DEV)
+    gpu, ora = P.make_layer_pair(cfg, 0, append_first=append_first)
+    y = torch.empty(1, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for t in range(6):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+    # event nodes around every kernel of the next three steps (the row moves may run on sf)
+    B.lif_timing_enable(gpu.handle, 3)
+    for t in range(6, 10):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+    us, n = B.lif_timing_read(gpu.handle)
+    assert n == 3 and set(us) == set(B.PHASES)
+    assert all(v >= 0.0 for v in us.values()) and us["fetch"] > 0 and us["ffn"] > 0 and us["window"] > 0
+    B.lif_timing_enable(gpu.handle, 0)
+    # snapshot, run on, wreck, restore, run on again: bitwise the same
+    snap = B.lif_snapshot(gpu.handle)
+    def run():
+        out = []
+        for t in range(10, 16):
+            B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+            torch.cuda.synchronize()
+            out.append((y.cpu().numpy().copy(), gpu.lists()["pointers"].copy()))
+        return out
+    first = run()
+    B.lif_reset(gpu.handle)
+    gpu.cache.zero_()
+    torch.cuda.synchronize()
+    B.lif_restore(gpu.handle, snap)
+    again = run()
+    for (ya, pa), (yb, pb) in zip(first, again):
+        assert np.array_equal(ya.view(np.uint32), yb.view(np.uint32))
+        np.testing.assert_array_equal(pa, pb)
+    assert gpu.lists()["status"] == B.LIF_OK
     gpu.close()
