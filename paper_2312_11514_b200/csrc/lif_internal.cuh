@@ -152,7 +152,11 @@ size_t ffn_smem_for(const lif_layer* L, int stages);
 // Launch with (pdl) or without the programmatic-stream-serialization attribute.  A kernel
 // launched with it may start while the previous kernel of the stream is still running; it
 // must execute pdl_wait() before it touches anything an earlier kernel wrote (every kernel of
-// this library does so on every path, which also keeps the ordering transitive).
+// this library does so on every path, which also keeps the ordering transitive).  Inside a
+// captured graph the attribute can make every incoming dependency of the launch programmatic,
+// a cross-stream event wait included (measured: a kernel that read another stream's output
+// ahead of its wait raced in graph replay only).  So what a kernel reads before pdl_wait() must
+// be weights, or data that was final before each kernel ahead of it passed its own wait.
 template <typename... KArgs, typename... Args>
 cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                      cudaStream_t st, int pdl, Args... args) {
