@@ -220,6 +220,7 @@ def check_decode_step(gpu, ora, x_np, y_np):
     oracle's only at borderline scores; from that list on, the oracle reproduces lists, window
     state and (within tolerance) the output ``y_np`` [S][d].  Returns the step's lists."""
     g = gpu.lists()
+    assert g["status"] == B.LIF_OK, f"device status {g['status']}"
     scores = ora.scores(x_np)
     assert_mask_borderline(g["active_idx"], scores, ora.theta)
     lists = ora.cache.window_update(g["active_idx"])

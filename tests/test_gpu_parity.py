@@ -614,3 +614,28 @@ def test_phase_timing_and_snapshot_with_both_cache_orders(append_first):
         np.testing.assert_array_equal(pa, pb)
     assert gpu.lists()["status"] == B.LIF_OK
     gpu.close()
+
+
+@pytest.mark.parametrize("gate_mode,append_first", [(0, 0), (0, 1), (2, 1)])
+def test_more_neurons_than_the_mask_fed_window_kernel_takes(gate_mode, append_first):
+    # d_ff = 40960 > 32768: the decode step uses the list-fed window kernel (the predictor
+    # compacts its mask itself); also the widest index range of the gate kernel's mask words
+    cfg = W.LifConfig("wide", 1, 256, 40960, 16, 2, 1, 8, 0.02, 1.0, 0.8, 0.6, 51)
+    act, thr = (B.ACT_FATRELU, 0.05) if gate_mode else (B.ACT_RELU, 0.0)
+    # (a rank-16 predictor makes the active count swing widely from token to token: roomy cache)
+    gpu, ora = P.make_layer_pair(cfg, 0, gate_mode=gate_mode, activation=act, act_threshold=thr,
+                                 append_first=append_first, capacity=16384)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(1, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    n_evict = 0
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        torch.cuda.synchronize()
+        assert gpu.lists()["status"] == B.LIF_OK
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        P.compare_cache_rows(gpu, ora)
+        n_evict += len(lists["evict_ids"])
+    assert n_evict > 0 and gpu.lists()["active_idx"].max() > 32768
+    gpu.close()
