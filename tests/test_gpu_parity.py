@@ -639,3 +639,27 @@ def test_more_neurons_than_the_mask_fed_window_kernel_takes(gate_mode, append_fi
         n_evict += len(lists["evict_ids"])
     assert n_evict > 0 and gpu.lists()["active_idx"].max() > 32768
     gpu.close()
+
+
+@pytest.mark.parametrize("d,F,r,k,S", [
+    (8, 64, 8, 1, 1),          # the smallest shapes the header allows
+    (8, 64, 8, 2, 8),
+    (64, 256, 2048, 2, 1),     # the largest predictor rank
+    (64, 256, 2048, 2, 8),     # ... with eight streams: 64 KB of stage-1 sums per CTA
+    (8192, 264, 8, 2, 2),      # the widest rows, two streams (per-stream FFN: d_model % 16 == 0 but few rows)
+])
+def test_extreme_shapes(d, F, r, k, S):
+    cfg = W.LifConfig("edge", 1, d, F, r, k, S, 8, 0.10, 1.0, 0.8, 0.6, 61)
+    stats = _run_staged(cfg, 0, cfg.steps, b_down=True, capacity=F)
+    assert max(s["n_active"] for s in stats) > 0
+    gpu, ora = P.make_layer_pair(cfg, 0, capacity=F, append_first=1)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(S, d, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        torch.cuda.synchronize()
+        P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        P.compare_cache_rows(gpu, ora)
+    gpu.close()
