@@ -12,7 +12,10 @@
 //   phase B: CTAs own (row partition, column part); the down halves of the part stream through
 //            the ring, 16 rows per MMA k-step; H = relu(sum of the K-slice partials), split into
 //            fp16 high + low parts (so the product keeps fp32 accuracy), is the B operand; each
-//            warp keeps its column tiles' accumulators in registers for the whole kernel.
+//            warp keeps its column tiles' accumulators in registers for the whole kernel.  H is
+//            scaled by a power of two before the split (the largest magnitude seen so far maps
+//            near 2^10; accumulators are rescaled exactly when it grows), so the result does not
+//            depend on where the activations sit in fp16's narrow exponent range.
 // Partition partials are added in a fixed order by the partial-sum kernel.  Bound: HBM.
 // Gated layers (Appendix C, Llama 2): with the gate row in the bundle, phase A runs twice (gate
 // rows with the bias, then up rows) and phase B uses H = act(gate) * up; with the gate
@@ -266,6 +269,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   __half* h_hi = reinterpret_cast<__half*>(bars + stages);             // [8][16]
   __half* h_lo = h_hi + 128;
   int* slot_all = reinterpret_cast<int*>(h_lo + 128);                  // [kRowCacheB]
+  // per group parity: max |H| of the four warps that load H
+  float (*gmax)[4] = reinterpret_cast<float (*)[4]>(slot_all + kRowCacheB);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
@@ -330,6 +335,21 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   pdl_trigger();
   float h_next = 0.f;
   if (tid < 128 && hk < my_cnt) h_next = load_h(hk);
+  // max |H| of a group is published one group ahead (after the MMAs, when the prefetched values
+  // have landed), so that scaling costs no extra barrier
+  auto publish_max = [&](int parity) {
+    if (tid < 128) {
+      float m = fabsf(h_next);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      if (lane == 0) gmax[parity][warp] = m;
+    }
+  };
+  publish_max(0);
+  __syncthreads();
+  constexpr int kUnset = -1000;
+  int h_exp = kUnset;              // H is scaled by 2^(10 - h_exp); kUnset: only zeros so far
+  auto pow2 = [](int e) { return __int_as_float((127 + max(-126, min(127, e))) << 23); };
 
   int timed_out = 0;
   const int n_groups = (my_cnt + 15) >> 4;
@@ -338,8 +358,25 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     const int st0 = (g & 1) * 16;
     const unsigned parity = (unsigned)(g >> 1) & 1u;
     const int valid = min(16, my_cnt - g * 16);
+    {
+      // the same for every thread: exponent of the largest |H| so far; accumulators follow
+      const float m = fmaxf(fmaxf(gmax[g & 1][0], gmax[g & 1][1]), fmaxf(gmax[g & 1][2], gmax[g & 1][3]));
+      if (m > 0.f && m < 3.0e38f) {
+        const int e = (int)((__float_as_uint(m) >> 23) & 0xff) - 127;
+        if (e > h_exp) {
+          if (h_exp != kUnset) {
+            const float f = pow2(h_exp - e);
+#pragma unroll
+            for (int t = 0; t < kMaxTilesPerWarp; ++t)
+#pragma unroll
+              for (int q = 0; q < 4; ++q) acc[t][q] *= f;
+          }
+          h_exp = e;
+        }
+      }
+    }
     if (tid < 128) {
-      const float h = hk < valid ? h_next : 0.f;
+      const float h = (hk < valid ? h_next : 0.f) * (h_exp == kUnset ? 1.f : pow2(10 - h_exp));
       const __half hi = __float2half_rn(h);
       h_hi[hs * 16 + hk] = hi;
       h_lo[hs * 16 + hk] = __float2half_rn(h - __half2float(hi));
@@ -373,6 +410,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
         mma16816(acc[t], af, bl0, bl1);
       }
     }
+    publish_max((g + 1) & 1);                      // of the group just prefetched
     __syncthreads();                               // stages of this group and h_hi/h_lo are free
     if (tid < 16) {
       const int i = (g + 2) * 16 + tid;
@@ -388,6 +426,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   }
   // epilogue: acc[t] = (column gq (+8) of the tile, streams 2*tq, 2*tq + 1)
   float* out = a.y_partial + (size_t)prt * a.S * d;
+  const float unscale = h_exp == kUnset ? 1.f : pow2(h_exp - 10);
 #pragma unroll
   for (int t = 0; t < kMaxTilesPerWarp; ++t) {
     const int tile = warp + t * 8;
@@ -396,7 +435,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
       for (int e = 0; e < 4; ++e) {
         const int m = tile * 16 + gq + (e >> 1) * 8;
         const int s = tq * 2 + (e & 1);
-        if (m < ncols && s < a.S) out[(size_t)s * d + col0 + m] = acc[t][e];
+        if (m < ncols && s < a.S) out[(size_t)s * d + col0 + m] = acc[t][e] * unscale;
       }
     }
   }
@@ -408,7 +447,7 @@ size_t up_smem(int k_per_split, int stages) {
 }
 size_t down_smem(int cols_per_part, int stages) {
   return stages * (2 * (size_t)cols_per_part + kPad) + stages * 8 + 2 * 128 * 2 + kRowCacheB * 4 +
-         16;
+         2 * 4 * 4 + 16;
 }
 
 }  // namespace

@@ -215,11 +215,14 @@ def staged_step(gpu, ora, x_dev, bufs, whole_cache=False):
                 n_border=n_border, k_eff=ref_lists["k_eff"], num_used=ref_lists["num_used"])
 
 
-def check_decode_step(gpu, ora, x_np, y_np):
+def check_decode_step(gpu, ora, x_np, y):
     """After one lif_decode_step of ``gpu`` on ``x_np``: the active list may differ from the
     oracle's only at borderline scores; from that list on, the oracle reproduces lists, window
-    state and (within tolerance) the output ``y_np`` [S][d].  Returns the step's lists."""
-    g = gpu.lists()
+    state and (within tolerance) the output ``y`` [S][d] (a device tensor, read here after the
+    device has been synchronised, or an array the caller read after synchronising).  Returns
+    the step's lists."""
+    g = gpu.lists()                    # synchronises the device
+    y_np = y.cpu().numpy().astype(np.float64) if isinstance(y, torch.Tensor) else y
     assert g["status"] == B.LIF_OK, f"device status {g['status']}"
     scores = ora.scores(x_np)
     assert_mask_borderline(g["active_idx"], scores, ora.theta)

@@ -69,7 +69,7 @@ def test_gated_decode_step(gate_mode, S, two_streams, fused):
     n_evict = 0
     for t in range(cfg.steps):
         B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
-        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
         P.compare_cache_rows(gpu, ora)
         n_evict += len(lists["evict_ids"])
     assert n_evict > 0

@@ -416,7 +416,7 @@ def test_decode_step_with_and_without_the_fused_fetch(d, F, k, act, thr, gate_mo
         torch.cuda.synchronize()
         x_np = X[t].cpu().numpy()
         if ffn_mode == 0:
-            lists = P.check_decode_step(gpu, ora, x_np, y.cpu().numpy().astype(np.float64))
+            lists = P.check_decode_step(gpu, ora, x_np, y)
         else:
             g = gpu.lists()
             lists = ora.cache.window_update(g["active_idx"])
@@ -463,7 +463,7 @@ def test_append_first_decode_step(two_streams, fused_plan, fused_fetch, S, gate_
     for t in range(cfg.steps):
         B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
         torch.cuda.synchronize()
-        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
         P.compare_cache_rows(gpu, ora)
         n_moves += len(lists["move_src"])
         n_reused += int((lists["load_slots"] < lists["num_used_before"]).sum())
@@ -499,7 +499,7 @@ def test_append_first_with_memory_budget_through_the_decode_step():
     for t in range(cfg.steps):
         B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
         torch.cuda.synchronize()
-        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
         P.compare_cache_rows(gpu, ora)
         assert lists["num_used"] <= 600
         ks.append(lists["k_eff"])
@@ -561,7 +561,7 @@ def test_multi_stream_decode_step_split_around_the_fetch(ffn_mode, split, gate_m
         torch.cuda.synchronize()
         x_np = X[t].cpu().numpy()
         if ffn_mode == 0:
-            lists = P.check_decode_step(gpu, ora, x_np, y.cpu().numpy().astype(np.float64))
+            lists = P.check_decode_step(gpu, ora, x_np, y)
         else:
             g = gpu.lists()
             P.assert_mask_borderline(g["active_idx"], ora.scores(x_np), ora.theta)
@@ -634,7 +634,7 @@ def test_more_neurons_than_the_mask_fed_window_kernel_takes(gate_mode, append_fi
         B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
         torch.cuda.synchronize()
         assert gpu.lists()["status"] == B.LIF_OK
-        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
         P.compare_cache_rows(gpu, ora)
         n_evict += len(lists["evict_ids"])
     assert n_evict > 0 and gpu.lists()["active_idx"].max() > 32768
@@ -660,6 +660,22 @@ def test_extreme_shapes(d, F, r, k, S):
     for t in range(cfg.steps):
         B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
         torch.cuda.synchronize()
-        P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y.cpu().numpy().astype(np.float64))
+        P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
         P.compare_cache_rows(gpu, ora)
+    gpu.close()
+
+
+@pytest.mark.parametrize("gate_mode,act", [(1, B.ACT_RELU_SQUARED), (0, B.ACT_RELU_SQUARED), (0, B.ACT_RELU)])
+def test_multi_stream_ffn_with_tiny_activations(gate_mode, act):
+    # d_model = 16 and squared ReLU give activations around 1e-5 and below: the tensor-core FFN
+    # splits them into fp16 parts and must not lose them to fp16's narrow exponent range
+    cfg = W.LifConfig("tinyact", 1, 16, 2000, 40, 6, 8, 10, 0.01, 1.0, 0.8, 0.6, 551)
+    gpu, ora = P.make_layer_pair(cfg, 0, gate_mode=gate_mode, activation=act, capacity=2000)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(8, 16, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
     gpu.close()
