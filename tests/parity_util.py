@@ -35,7 +35,7 @@ def assert_y_close(got, ref, flips=()):
     """``flips``: (stream, delta[d]) pairs, one per FATReLU decision that sits within rounding of
     its threshold: the activation jumps there, so either side of it is a correct result and
     ``got`` may match ``ref`` with any subset of the deltas added."""
-    assert len(flips) <= 6, "too many borderline activations to enumerate"
+    assert len(flips) <= 14, "too many borderline activations to enumerate"
     worst = None
     for subset in range(1 << len(flips)):
         r = ref.copy()
@@ -51,7 +51,9 @@ def assert_y_close(got, ref, flips=()):
     raise AssertionError(f"outputs off, worst ratio {worst:.3f}")
 
 
-ACT_BORDER = 1e-4   # |pre-activation - FATReLU threshold| below this: the decision may differ
+# |pre-activation - FATReLU threshold| below this: the decision may differ (fp32 accumulation of
+# up to 8192 fp16 products of O(1) size is off by about 1e-6)
+ACT_BORDER = 2e-5
 
 
 def ffn_reference(ora, slots, x_np, gate_pre=None):
