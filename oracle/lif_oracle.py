@@ -336,6 +336,44 @@ def decode_step_gate_predictor(cache, x, gate_matrix, gate_bias, bundles, b_down
 
 
 # --------------------------------------------------------------------------------------
+# Neuron sharding over several devices (not in the paper, which runs on one device: it follows
+# from Section 3.3 item 3 -- the FFN output is a sum of one term per cached neuron, in any row
+# order -- and from the window rule of Section 3.1 being a per-neuron rule)
+# --------------------------------------------------------------------------------------
+def neuron_shard_range(d_ff, rank, world):
+    """Contiguous id range [lo, hi) of the neurons device ``rank`` of ``world`` owns: equal
+    shares of d_ff / world neurons (d_ff must divide evenly)."""
+    if world < 1 or not 0 <= rank < world or d_ff % world:
+        raise ValueError("d_ff must be a multiple of the number of shards")
+    per = d_ff // world
+    return rank * per, (rank + 1) * per
+
+
+def sharded_decode_step(caches, x, A, B, c, theta, bundles, bias_up, b_down=None,
+                        whole_cache=False, activation=RELU, threshold=0.0):
+    """One layer, one token with the neurons split over len(caches) devices.  Device g owns the
+    bundles, predictor columns, offsets and biases of its id range and its own window cache
+    (local ids = global id - lo); the input x and the factor A are on every device.  Each
+    device runs the ordinary step on its share and produces a partial output; the layer's
+    output is the sum of the partials (the one exchange of the step), with the down-projection
+    bias added once.  Returns the per-device (logits, act, lists, partial y) and the sum."""
+    world = len(caches)
+    F = np.asarray(B).shape[1]
+    parts = []
+    y = None
+    for g, cache in enumerate(caches):
+        lo, hi = neuron_shard_range(F, g, world)
+        part = decode_step(cache, x, A, np.asarray(B)[:, lo:hi], np.asarray(c)[lo:hi], theta,
+                           np.asarray(bundles)[lo:hi], np.asarray(bias_up)[lo:hi], None,
+                           whole_cache, None, activation, threshold)
+        parts.append(part)
+        y = part[3] if y is None else y + part[3]
+    if b_down is not None:
+        y = y + np.asarray(b_down, dtype=np.float64)[None, :]
+    return parts, y
+
+
+# --------------------------------------------------------------------------------------
 # The paper's latency / memory accounting (Section 3 intro, Table 1, Appendix C)
 # --------------------------------------------------------------------------------------
 def io_latency_ms(gigabytes, throughput_gb_per_s):

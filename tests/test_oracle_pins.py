@@ -775,3 +775,74 @@ def test_append_first_agrees_with_the_papers_order_under_budget_and_multi_token_
         np.testing.assert_array_equal(a.last_active, b.last_active)
         for s in range(a.num_used):
             np.testing.assert_array_equal(a.matrix[s], bundles[a.pointers[s]])
+
+
+# ------------------------------------------------------------------ neuron sharding
+def test_neuron_shard_ranges_tile_the_ids():
+    for F, G in ((24, 1), (24, 2), (24, 3), (1024, 8)):
+        ranges = [O.neuron_shard_range(F, g, G) for g in range(G)]
+        assert ranges[0][0] == 0 and ranges[-1][1] == F
+        assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
+        assert len({hi - lo for lo, hi in ranges}) == 1
+    with pytest.raises(ValueError):
+        O.neuron_shard_range(10, 0, 3)
+    with pytest.raises(ValueError):
+        O.neuron_shard_range(12, 3, 3)
+
+
+@pytest.mark.parametrize("G", [2, 4])
+def test_sharded_step_with_true_mask_predictor_equals_dense_ffn(G):
+    # Same construction as the single-device pin: the predictor reproduces the up projection,
+    # so the summed partial outputs must equal the dense FFN (bias of the down projection
+    # added once, not once per device) at every step.
+    r = _rng(70 + G)
+    F, d, T = 48, 8, 10
+    W_up = r.normal(size=(F, d)).astype(np.float16)
+    W_down = r.normal(size=(d, F)).astype(np.float16)
+    b_up = (r.normal(size=F) - 1.0).astype(np.float16)
+    b_down = r.normal(size=d).astype(np.float16)
+    bundles = np.concatenate([W_up, W_down.T], axis=1)
+    caches = [O.NeuronCache(d, F // G, F // G, window_k=3) for _ in range(G)]
+    x = r.normal(size=(1, d))
+    for _ in range(T):
+        x = (0.8 * x + 0.6 * r.normal(size=(1, d))).astype(np.float16)
+        _, y = O.sharded_decode_step(caches, x, W_up.T, np.eye(F), b_up, 0.0, bundles, b_up, b_down)
+        xd = x[0].astype(np.float64)
+        dense = W_down.astype(np.float64) @ np.maximum(W_up.astype(np.float64) @ xd + b_up, 0.0)
+        np.testing.assert_allclose(y[0], dense + b_down, rtol=1e-10, atol=1e-10)
+
+
+@pytest.mark.parametrize("G,append_first", [(1, False), (2, False), (3, True)])
+def test_sharded_step_partitions_the_single_device_step(G, append_first):
+    # Random low-rank predictor: the devices' active lists, cached sets and fetched bytes
+    # partition those of one device holding every neuron, and the partial outputs sum to its
+    # output.  One shard is the single-device step itself, bit for bit.
+    r = _rng(80 + G)
+    F, d, rank, S, T, k = 60, 16, 4, 2, 14, 3
+    bundles = r.normal(scale=0.3, size=(F, 2 * d)).astype(np.float16)
+    bias_up = r.normal(scale=0.2, size=F).astype(np.float16)
+    A = r.normal(size=(d, rank)).astype(np.float16)
+    B = r.normal(size=(rank, F)).astype(np.float16)
+    c = (r.normal(size=F) - 1.2).astype(np.float32)
+    b_down = r.normal(size=d).astype(np.float16)
+    one = O.NeuronCache(d, F, F, window_k=k, append_first=append_first)
+    caches = [O.NeuronCache(d, F // G, F // G, window_k=k, append_first=append_first) for _ in range(G)]
+    x = r.normal(size=(S, d))
+    for _ in range(T):
+        x = (0.7 * x + 0.7 * r.normal(size=(S, d))).astype(np.float16)
+        logits, act, lists, y_one = O.decode_step(one, x, A, B, c, 0.0, bundles, bias_up, b_down)
+        parts, y = O.sharded_decode_step(caches, x, A, B, c, 0.0, bundles, bias_up, b_down)
+        if G == 1:
+            np.testing.assert_array_equal(y, y_one)
+            np.testing.assert_array_equal(parts[0][2]["load_slots"], lists["load_slots"])
+        np.testing.assert_allclose(y, y_one, rtol=1e-11, atol=1e-11)
+        got_act, got_cached = [], set()
+        for g, (lg, a, _, _) in enumerate(parts):
+            lo, hi = O.neuron_shard_range(F, g, G)
+            np.testing.assert_array_equal(lg, logits[:, lo:hi])
+            got_act.extend((a + lo).tolist())
+            got_cached |= {i + lo for i in caches[g].cached_ids()}
+        assert got_act == act.tolist()
+        assert got_cached == one.cached_ids()
+        assert sum(ch.bytes_fetched for ch in caches) == one.bytes_fetched
+        assert sum(ch.num_used for ch in caches) == one.num_used
