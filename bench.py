@@ -139,13 +139,18 @@ def run_ours(args):
 
     # every rank decodes its own sequence with its own replica of the stack (weak scaling,
     # no exchange between ranks)
+    # --shard neurons (N > 1): all ranks decode ONE sequence, each with its share of every
+    # layer's neurons, and sum their partial outputs after every layer (strong scaling)
+    # (at N = 1 the same layer-by-layer path runs with the whole layer as the only share)
+    sharded = args.shard == "neurons"
     cfg = W.CONFIGS[args.config]
-    cfg = rank_config(cfg, rank)
+    cfg = cfg if sharded else rank_config(cfg, rank)
     K, Wm = args.steps, args.warmup
     n_tok = Wm + K
     gate_mode, activation, act_thr = _gate_setup(args)
     layers = R.build_stack(cfg, dev, n_layers=args.layers, gate_mode=gate_mode, activation=activation,
-                           activation_threshold=act_thr, append_first=args.append_first)
+                           activation_threshold=act_thr, append_first=args.append_first,
+                           shard=(rank, world) if sharded else None)
     handles = [l.handle for l in layers]
     L, S, d = len(layers), cfg.n_streams, cfg.d_model
     X = _inputs(cfg, n_tok, dev, W)
@@ -177,10 +182,30 @@ def run_ours(args):
     dev_x = torch.empty(S, d, dtype=torch.float16, device=dev)
     graph = B.lif_graph_capture(handles, dev_x, Y, sc, sf)
 
+    def layers_then_sums():
+        # neuron-sharded token: a layer's output exists only after the exchange, so the layers
+        # are launched one by one with the sum over ranks between them (no whole-token graph)
+        for l in range(L):
+            B.lif_decode_step(handles[l], dev_x, Y[l], sc, sf)
+            R.sum_partial_outputs(Y[l])
+
     def token(t):
         with torch.cuda.stream(sc):
             dev_x.copy_(X[t], non_blocking=True)
-        B.lif_graph_launch(graph, sc)
+            if sharded:
+                layers_then_sums()
+        if not sharded:
+            B.lif_graph_launch(graph, sc)
+
+    def token_host(t):
+        if not sharded:
+            B.lif_graph_launch_host(graph, host_x[t], host_y, sc)
+            return
+        with torch.cuda.stream(sc):
+            dev_x.copy_(host_x[t], non_blocking=True)
+            layers_then_sums()
+            host_y.copy_(Y, non_blocking=True)
+        sc.synchronize()
 
     # ---- pass 1: device-resident inputs ------------------------------------------------------
     reset()
@@ -212,11 +237,11 @@ def run_ours(args):
     host_y = torch.empty(L, S, d, dtype=torch.float32, pin_memory=True)
     reset()
     for t in range(Wm):
-        B.lif_graph_launch_host(graph, host_x[t], host_y, sc)
+        token_host(t)
     barrier()
     e0.record(sc)
     for t in range(Wm, n_tok):
-        B.lif_graph_launch_host(graph, host_x[t], host_y, sc)
+        token_host(t)
     e1.record(sc)
     barrier()
     ms_e2e = slowest(e0.elapsed_time(e1))
@@ -308,10 +333,10 @@ def run_ours(args):
                                          "bytes_per_launch": all_bytes, "frac": all_gbs / peak},
                      "new_rows_GBs": (n_load_l * (beta + row_extra) / L + 6 * d) / (kernel_us["ffn_new"] * 1e-6) / 1e9}
         out = {
-            "metric": METRIC, "value": whole_job_tokens_per_s(K, world, ms_total), "unit": UNIT,
+            "metric": METRIC, "value": whole_job_tokens_per_s(K, 1 if sharded else world, ms_total), "unit": UNIT,
             "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms_total / K,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
-            "data": "synthetic",
+            "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
+            "dtype": "f16", "data": "synthetic",
             "config": {"workload": f"{cfg.name}: {L} layers d_model={d} d_ff={cfg.d_ff} rank={cfg.rank} "
                                    f"window_k={cfg.window_k} streams={S}, AR(1) decode inputs"
                                    + (f", gated FFN ({args.gate} gate, FATReLU {act_thr})" if gate_mode else ""),
@@ -321,8 +346,10 @@ def run_ours(args):
                        "l2": "per-token working set (all layers' window caches, "
                              f"{s1[3] / n_tok * beta / 2**20:.0f} MiB) exceeds the 126 MB L2",
                        "bundle_store": "pinned host memory, read by the fetch kernel",
-                       "parallelism": "independent sequence per GPU"},
-            "e2e": {"value": whole_job_tokens_per_s(K, world, ms_e2e), "unit": UNIT,
+                       "parallelism": f"one sequence, neurons of every layer split over {world} GPUs, "
+                                      "partial outputs summed (all-reduce) after every layer"
+                                      if sharded else "independent sequence per GPU"},
+            "e2e": {"value": whole_job_tokens_per_s(K, 1 if sharded else world, ms_e2e), "unit": UNIT,
                     "h2d_bytes_per_step": S * d * 2, "d2h_bytes_per_step": L * S * d * 4,
                     "host_link_bytes_per_step": fetched / K},
             # per layer-step: z, scores (or the gate kernel alone), window, moves, fetch (one stream:
@@ -599,6 +626,10 @@ def main():
     ap.add_argument("--append-first", type=int, default=1, choices=[0, 1],
                     help="1: stack the new neurons before deleting, so their bundles go straight into "
                          "freed rows; 0: the order of Section 3.3 as written (same cached set and outputs)")
+    ap.add_argument("--shard", default="sequences", choices=["sequences", "neurons"],
+                    help="N > 1: 'sequences' = one independent sequence and stack per GPU (default); "
+                         "'neurons' = one sequence, every layer's neurons split over the GPUs, partial "
+                         "outputs all-reduced after every layer")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--cpu-layers", type=int, default=2)
     ap.add_argument("--cpu-tokens", type=int, default=30)

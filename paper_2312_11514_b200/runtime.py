@@ -100,22 +100,60 @@ def pinned_store(d_ff: int, d_model: int, n_vec: int = 2) -> torch.Tensor:
     return torch.empty(d_ff, n_vec * d_model, dtype=torch.float16, pin_memory=True)
 
 
+def neuron_shard(d_ff: int, rank: int, world: int):
+    """Ids [lo, hi) of the neurons that device ``rank`` of ``world`` owns when one layer's
+    neurons are split over several devices: equal contiguous shares, each a multiple of 8
+    (the layer description's rule for d_ff)."""
+    if world < 1 or not 0 <= rank < world or d_ff % (8 * world):
+        raise ValueError(f"d_ff={d_ff} does not split into {world} shares that are multiples of 8")
+    per = d_ff // world
+    return rank * per, (rank + 1) * per
+
+
+def sum_partial_outputs(y: torch.Tensor, group=None) -> torch.Tensor:
+    """The one exchange of a neuron-sharded layer-step: every device holds the FFN terms of its
+    own neurons in ``y`` (fp32 ``[n_streams][d_model]``); afterwards every device holds their
+    sum.  In place, on the current stream (NCCL) or on the host (gloo).  One device: no-op."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(y, op=dist.ReduceOp.SUM, group=group)
+    return y
+
+
 def build_stack(cfg, device="cuda:0", n_layers: Optional[int] = None, capacity_margin: float = 8.0,
                 ffn_mode: int = 0, gen_device=None, gate_mode: int = 0, activation: int = 0,
-                activation_threshold: float = 0.0, append_first: int = 0) -> List[Layer]:
-    """Generate the weights of a named synthetic configuration and create its layers."""
+                activation_threshold: float = 0.0, append_first: int = 0,
+                shard=None, bias_down: Optional[List[torch.Tensor]] = None) -> List[Layer]:
+    """Generate the weights of a named synthetic configuration and create its layers.
+
+    ``shard = (rank, world)`` keeps only this device's share of every layer's neurons (its rows
+    of the bundle store, its predictor columns, offsets and biases, a window cache sized for its
+    share): the layer's output is then the sum over devices of the outputs computed here
+    (``sum_partial_outputs``).  ``bias_down`` (one fp16 ``[d_model]`` tensor per layer) is given
+    to the first device only, so that the sum holds it once."""
     from . import workloads as W
     layers = []
     gen_device = gen_device or device
+    n_vec = 3 if gate_mode == B.GATE_BUNDLED else 2
     for l in range(n_layers or cfg.n_layers):
-        store = pinned_store(cfg.d_ff, cfg.d_model, 3 if gate_mode == B.GATE_BUNDLED else 2)
-        w = W.make_layer(cfg, l, device=gen_device, bundles_out=store, gate_mode=gate_mode,
-                         act_threshold=activation_threshold)
-        cap = W.window_capacity(cfg, w["p"], capacity_margin)
+        if shard is None:
+            lo, hi = 0, cfg.d_ff
+            store = pinned_store(cfg.d_ff, cfg.d_model, n_vec)
+            w = W.make_layer(cfg, l, device=gen_device, bundles_out=store, gate_mode=gate_mode,
+                             act_threshold=activation_threshold)
+        else:
+            lo, hi = neuron_shard(cfg.d_ff, *shard)
+            w = W.slice_layer(W.make_layer(cfg, l, device=gen_device, gate_mode=gate_mode,
+                                           act_threshold=activation_threshold), lo, hi)
+            store = pinned_store(hi - lo, cfg.d_model, n_vec)
+            store.copy_(w["bundles"])
+        cap = min(hi - lo, W.window_capacity(cfg, w["p"], capacity_margin))
         dev = lambda t: None if t is None else t.to(device).contiguous()
-        layers.append(Layer(d_model=cfg.d_model, d_ff=cfg.d_ff, rank=cfg.rank, window_k=cfg.window_k,
+        b_down = bias_down[l] if bias_down is not None and (shard is None or shard[0] == 0) else None
+        layers.append(Layer(d_model=cfg.d_model, d_ff=hi - lo, rank=cfg.rank, window_k=cfg.window_k,
                             capacity=cap, host_bundles=store, pred_A=dev(w["A"]), pred_B=dev(w["B"]),
-                            pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), n_streams=cfg.n_streams,
+                            pred_c=dev(w["c"]), bias_up=dev(w["bias_up"]), bias_down=dev(b_down),
+                            n_streams=cfg.n_streams,
                             ffn_mode=ffn_mode, gate_mode=gate_mode, gate=dev(w.get("gate")),
                             activation=activation, activation_threshold=activation_threshold,
                             append_first=append_first, device=device))

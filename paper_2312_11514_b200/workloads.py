@@ -151,6 +151,23 @@ def make_layer(cfg: LifConfig, layer: int, device: Optional[torch.device] = None
     return out
 
 
+def slice_layer(w: Dict[str, torch.Tensor], lo: int, hi: int) -> Dict[str, torch.Tensor]:
+    """The tensors of neurons ``lo`` .. ``hi - 1`` of a generated layer, as contiguous copies:
+    rows of the bundle store (and of the gate projection), columns of the predictor's second
+    factor, the per-neuron offsets, biases and popularities.  The first factor ``A`` is shared
+    by every neuron and returned as it is.  Slicing only: no arithmetic."""
+    per_neuron_rows = ("bundles", "gate", "bias_up", "c", "p")
+    out = {}
+    for name, t in w.items():
+        if name in per_neuron_rows:
+            out[name] = t[lo:hi].contiguous()
+        elif name == "B":
+            out[name] = t[:, lo:hi].contiguous()
+        else:
+            out[name] = t
+    return out
+
+
 def make_inputs(cfg: LifConfig, device: Optional[torch.device] = None) -> torch.Tensor:
     """Decode inputs ``X[steps][n_streams][d_model]`` fp16: independent AR(1) sequences."""
     device = torch.device(device or "cpu")
