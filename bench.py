@@ -182,12 +182,26 @@ def run_ours(args):
     dev_x = torch.empty(S, d, dtype=torch.float16, device=dev)
     graph = B.lif_graph_capture(handles, dev_x, Y, sc, sf)
 
+    exchange = None
+    if sharded and args.exchange == "peer":
+        if world == 1 and not dist.is_initialized():      # the buffer mapping needs a group
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29517")
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device(dev))
+        exchange = R.PeerExchange(L, S, d, dev)
+
     def layers_then_sums():
         # neuron-sharded token: a layer's output exists only after the exchange, so the layers
         # are launched one by one with the sum over ranks between them (no whole-token graph)
         for l in range(L):
-            B.lif_decode_step(handles[l], dev_x, Y[l], sc, sf)
-            R.sum_partial_outputs(Y[l])
+            if exchange is None:                          # library all-reduce, in place
+                B.lif_decode_step(handles[l], dev_x, Y[l], sc, sf)
+                R.sum_partial_outputs(Y[l])
+            else:                                         # peers' partials read by our kernel
+                B.lif_decode_step(handles[l], dev_x, exchange.partials[l], sc, sf)
+                exchange.sum_layer(l, Y[l], sc)
+        if exchange is not None:
+            exchange.end_token()
 
     def token(t):
         with torch.cuda.stream(sc):
@@ -347,7 +361,7 @@ def run_ours(args):
                              f"{s1[3] / n_tok * beta / 2**20:.0f} MiB) exceeds the 126 MB L2",
                        "bundle_store": "pinned host memory, read by the fetch kernel",
                        "parallelism": f"one sequence, neurons of every layer split over {world} GPUs, "
-                                      "partial outputs summed (all-reduce) after every layer"
+                                      f"partial outputs summed after every layer ({args.exchange})"
                                       if sharded else "independent sequence per GPU"},
             "e2e": {"value": whole_job_tokens_per_s(K, 1 if sharded else world, ms_e2e), "unit": UNIT,
                     "h2d_bytes_per_step": S * d * 2, "d2h_bytes_per_step": L * S * d * 4,
@@ -400,7 +414,8 @@ def run_ours(args):
     B.lif_graph_destroy(graph)
     for l in layers:
         l.close()
-    if world > 1:
+    del exchange
+    if dist.is_initialized():
         dist.destroy_process_group()
 
 
@@ -630,6 +645,9 @@ def main():
                     help="N > 1: 'sequences' = one independent sequence and stack per GPU (default); "
                          "'neurons' = one sequence, every layer's neurons split over the GPUs, partial "
                          "outputs all-reduced after every layer")
+    ap.add_argument("--exchange", default="nccl", choices=["nccl", "peer"],
+                    help="--shard neurons: sum the partial outputs with an NCCL all-reduce, or with "
+                         "lif_sum_peer_outputs reading the peers' partials from peer-mapped memory")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--cpu-layers", type=int, default=2)
     ap.add_argument("--cpu-tokens", type=int, default=30)

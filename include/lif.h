@@ -251,6 +251,31 @@ lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* dev_bias, c
                                  const void* dev_bias_down, float* dev_y, int32_t d_model,
                                  void* stream);
 
+/* Neuron sharding over several devices (not in the paper, which runs on one device; it rests
+ * on Section 3.3 item 3: the FFN output is a sum of one term per cached neuron, in any order).
+ * Each device creates its layers over its own share of the neurons (its rows of the bundle
+ * store, its columns of dev_pred_B, its entries of dev_pred_c and dev_bias_up; dev_bias_down on
+ * one device only), runs the calls above on them, and the layer's output is the sum over devices
+ * of the outputs computed there.
+ * lif_sum_peer_outputs forms that sum on the calling device:
+ *   dev_y[i] = dev_partials[0][i] + dev_partials[1][i] + ... (in this order), i < n_floats.
+ *   dev_partials  HOST array of n_peers device pointers, fp32, 16-byte aligned; each is the
+ *                 partial output of one device ([n_streams][d_model] of one layer, or several
+ *                 layers' worth): memory of the current device, or of a peer device that is
+ *                 mapped into this one (peer access enabled, or a shared mapping).  Read with
+ *                 plain loads.  The array itself is read during the call only.
+ *   n_peers       1 .. LIF_MAX_PEERS
+ *   dev_y         fp32 [n_floats] on the current device, 16-byte aligned; may be exactly one of
+ *                 the partials (the sum then replaces it), but not a shifted overlap of one.
+ *   n_floats      multiple of 4
+ * Enqueue only.  The caller orders the call after the work that produced every partial (on
+ * other devices: an event or barrier across devices before this call) and keeps the partials
+ * unchanged until the kernel has run.  Given the same partials in the same order every device
+ * computes the same bits.  Errors: LIF_ERR_INVALID_ARG, LIF_ERR_ALIGNMENT, LIF_ERR_CUDA. */
+#define LIF_MAX_PEERS 16
+lif_status lif_sum_peer_outputs(const float* const* dev_partials, int32_t n_peers, float* dev_y,
+                                size_t n_floats, void* stream);
+
 /* One token through the layer: predict -> window update -> fetch -> sparse FFN (ffn_mode
  * selects the rows).  Two streams let the bundle fetch overlap the part of the FFN that does
  * not need the new rows; which of the two kernels runs on `fetch_stream` is the library's

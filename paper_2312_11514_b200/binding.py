@@ -26,7 +26,7 @@ EXPORTS = [
     "lif_probe_host_read", "lif_timing_enable", "lif_timing_read",
     "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
     "lif_sparse_ffn_static", "lif_set_tuning", "lif_profile_launch",
-    "lif_read_state", "lif_snapshot_bytes", "lif_snapshot", "lif_restore",
+    "lif_read_state", "lif_snapshot_bytes", "lif_snapshot", "lif_restore", "lif_sum_peer_outputs",
 ]
 KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ffn_new", "ffn_sum")
 (TUNE_DEPENDENT_LAUNCH, TUNE_SPLIT_FFN, TUNE_FETCH_CTAS, TUNE_FFN_CTAS, TUNE_FFN_STAGES,
@@ -100,6 +100,7 @@ def lib() -> C.CDLL:
         "lif_graph_launch_host": [vp, vp, vp, vp],
         "lif_graph_destroy": [vp],
         "lif_sparse_ffn_static": [vp, vp, vp, vp, vp, vp, vp, i32, vp],
+        "lif_sum_peer_outputs": [C.POINTER(vp), i32, vp, sz, vp],
         "lif_set_tuning": [vp, i32, i32],
         "lif_read_state": [vp, vp, vp, vp, vp],
         "lif_snapshot_bytes": [vp, C.POINTER(sz)],
@@ -272,6 +273,14 @@ def lif_sparse_ffn_static(matrix, bias, x, slots, n_slots, bias_down, y, d_model
     _check(lib().lif_sparse_ffn_static(_ptr(matrix), _ptr(bias), _ptr(x), _ptr(slots),
                                        _ptr(n_slots), _ptr(bias_down), _ptr(y), d_model,
                                        _stream(stream)), "lif_sparse_ffn_static")
+
+
+def lif_sum_peer_outputs(partials, y, stream=None) -> None:
+    """y = partials[0] + partials[1] + ... (fp32 tensors of equal size, this device's or mapped
+    peers'; integers are taken as device addresses); see include/lif.h."""
+    ptrs = (C.c_void_p * len(partials))(*[p if isinstance(p, int) else _ptr(p) for p in partials])
+    _check(lib().lif_sum_peer_outputs(ptrs, len(partials), _ptr(y), y.numel(), _stream(stream)),
+           "lif_sum_peer_outputs")
 
 
 def lif_set_tuning(layer: int, key: int, value: int) -> None:

@@ -120,6 +120,36 @@ def sum_partial_outputs(y: torch.Tensor, group=None) -> torch.Tensor:
     return y
 
 
+class PeerExchange:
+    """The exchange of a neuron-sharded token over peer-mapped device memory instead of a
+    library all-reduce.  Every rank writes its partial output of layer l into slot l of a
+    buffer that all ranks of the group have mapped (torch symmetric memory: allocation and
+    address exchange only); after a barrier across the ranks, ``lif_sum_peer_outputs`` reads
+    all ranks' slots with plain loads and adds them in rank order, so every rank gets the same
+    bits.  A slot is rewritten only in the next token, after ``end_token``'s barrier, so one
+    barrier per layer is enough.  Call the methods with the compute stream current."""
+
+    def __init__(self, n_layers: int, n_streams: int, d_model: int, device, group=None):
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm
+        group = group if group is not None else dist.group.WORLD
+        self.partials = symm.empty(n_layers, n_streams, d_model, dtype=torch.float32,
+                                   device=torch.device(device))
+        self.handle = symm.rendezvous(self.partials, group)
+        self.slot_bytes = n_streams * d_model * 4
+        self.peer_ptrs = [int(p) for p in self.handle.buffer_ptrs]     # rank order
+        assert self.peer_ptrs[self.handle.rank] == self.partials.data_ptr()
+
+    def sum_layer(self, l: int, y: torch.Tensor, stream=None) -> None:
+        """y = sum over ranks of slot l, once every rank's slot l is complete."""
+        self.handle.barrier(channel=0)
+        B.lif_sum_peer_outputs([p + l * self.slot_bytes for p in self.peer_ptrs], y, stream)
+
+    def end_token(self) -> None:
+        """No rank starts the next token (and rewrites its slots) while a peer still reads."""
+        self.handle.barrier(channel=1)
+
+
 def build_stack(cfg, device="cuda:0", n_layers: Optional[int] = None, capacity_margin: float = 8.0,
                 ffn_mode: int = 0, gen_device=None, gate_mode: int = 0, activation: int = 0,
                 activation_threshold: float = 0.0, append_first: int = 0,

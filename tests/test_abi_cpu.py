@@ -101,3 +101,4 @@ def test_graph_and_profiling_calls_reject_null_handles():
     assert lib.lif_set_tuning(None, 0, 0) == B.LIF_ERR_INVALID_ARG
     assert lib.lif_timing_enable(None, 1) == B.LIF_ERR_INVALID_ARG
     assert lib.lif_sparse_ffn_static(None, None, None, None, None, None, None, 256, None) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_sum_peer_outputs(None, 2, None, 16, None) == B.LIF_ERR_INVALID_ARG

@@ -82,3 +82,35 @@ def test_shares_follow_their_oracles_and_sum_to_the_unsplit_layer(name, scale, G
         for layer in st:
             layer.close()
 
+
+
+@pytest.mark.parametrize("G,n", [(1, 8), (2, 4096), (5, 4 * 7168 + 4), (16, 300_000)])
+def test_peer_sum_adds_the_partials_in_rank_order(G, n):
+    # The partials of G devices stand on this one device (a peer's mapped memory is read the
+    # same way).  fp32 sums in the stated order are exact to compute on the CPU, so the
+    # comparison is bit for bit; in place over the first partial gives the same bits.
+    g = torch.Generator(device="cpu").manual_seed(G * 1000 + n)
+    parts = [(torch.randn(n, generator=g) * 10 ** float(torch.randint(-3, 3, (1,), generator=g)))
+             .to(DEV) for _ in range(G)]
+    y = torch.full((n,), float("nan"), device=DEV)
+    B.lif_sum_peer_outputs(parts, y)
+    torch.cuda.synchronize()
+    want = np.zeros(n, dtype=np.float32)
+    for p in parts:
+        want = (want + p.cpu().numpy()).astype(np.float32)
+    np.testing.assert_array_equal(y.cpu().numpy(), want)
+    B.lif_sum_peer_outputs(parts, parts[0])
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(parts[0].cpu().numpy(), want)
+
+
+def test_peer_sum_argument_checks():
+    y = torch.zeros(16, device=DEV)
+    a = torch.zeros(20, device=DEV)
+    with pytest.raises(B.LifError):
+        B.lif_sum_peer_outputs([a[1:17]], y)                 # misaligned partial
+    with pytest.raises(B.LifError):
+        B.lif_sum_peer_outputs([a[:16]] * 17, y)             # more than LIF_MAX_PEERS
+    with pytest.raises(B.LifError):
+        B.lif_sum_peer_outputs([a[:14]], y[:14])             # not a multiple of 4
+    assert B.lib().lif_sum_peer_outputs(None, 1, None, 4, None) == B.LIF_ERR_INVALID_ARG
