@@ -23,6 +23,7 @@ inline int z_rows_per_cta(int d_model) {
   const int rows = ((d_model + 31) / 32 + 31) / 32 * 32;
   return rows < 32 ? 32 : rows;
 }
+constexpr int kMaxZPartials = 32;   // z_cta_count() never exceeds it
 inline int z_cta_count(int d_model) {
   return (d_model + z_rows_per_cta(d_model) - 1) / z_rows_per_cta(d_model);
 }

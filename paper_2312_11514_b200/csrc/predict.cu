@@ -134,10 +134,17 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
   pdl_wait();
   pdl_trigger();
   if (S == 1) {
+    // one stream: every partial of a sum is requested before the first is used (one memory
+    // round trip instead of several); the additions keep their order
     for (int i = tid; i < S * r; i += kThreads) {
+      float t[kMaxZPartials];
+#pragma unroll
+      for (int p = 0; p < kMaxZPartials; ++p)
+        t[p] = p < P ? __ldcg(z_partial + (size_t)p * S * r + i) : 0.f;
       float v = 0.f;
-#pragma unroll 8
-      for (int p = 0; p < P; ++p) v += __ldcg(z_partial + (size_t)p * S * r + i);
+#pragma unroll
+      for (int p = 0; p < kMaxZPartials; ++p)
+        if (p < P) v += t[p];
       zs[i] = v;
     }
   } else {
