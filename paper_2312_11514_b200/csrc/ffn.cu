@@ -275,11 +275,24 @@ ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
   const int v0 = min(G, *n0), v1 = p1 ? min(G, *n1) : 0;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
   if (in) {
-#pragma unroll 4
-    for (int g = gs; g < v0 + v1; g += 32) {
-      const float* src = g < v0 ? p0 + (size_t)g * d : p1 + (size_t)(g - v0) * d;
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(src) + col4);
-      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    // batches of 10 partials per thread (two sets of up to 148 over 32 slices), a batch's loads
+    // in flight together; the additions keep their order
+    for (int g0 = gs; g0 < v0 + v1; g0 += 32 * 10) {
+      float4 v[10];
+#pragma unroll
+      for (int k = 0; k < 10; ++k) {
+        const int g = g0 + 32 * k;
+        if (g < v0 + v1) {
+          const float* src = g < v0 ? p0 + (size_t)g * d : p1 + (size_t)(g - v0) * d;
+          v[k] = __ldcg(reinterpret_cast<const float4*>(src) + col4);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 10; ++k) {
+        if (g0 + 32 * k < v0 + v1) {
+          s.x += v[k].x; s.y += v[k].y; s.z += v[k].z; s.w += v[k].w;
+        }
+      }
     }
   }
   red[gs][c4] = s;
