@@ -94,6 +94,8 @@ __device__ __forceinline__ int active_stamp(const WindowArgs& a, int id, int t, 
 }
 
 constexpr int kMaxBudgetWindow = 32;
+constexpr int kSegRegs = 12;    // general path: cached rows per thread kept in registers
+constexpr int kActRegs = 8;     // and active-list entries per thread
 __device__ __forceinline__ int widest_window_that_fits(const int* hist, int k, int n, int n_load,
                                                        int limit) {
   int evicted = 0;          // rows deleted under window kk = sum of hist[a], a >= kk
@@ -141,9 +143,54 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   const int limit = a.budget > 0 ? min(a.cap, a.budget) : a.cap;
   const int stale_before = t_end - k_eff;   // last_active <= stale_before: outside the window
 
+  // Register path: when a thread's run of cached rows and its run of the active list are
+  // short (kSegRegs rows, kActRegs list entries), their ids are read once, and every pass below
+  // issues its dependent loads (stamp, slot) for the whole run together instead of one entry
+  // at a time between stores.  Same decisions, same lists.
+  const int seg = (n + kWindowThreads - 1) / kWindowThreads;
+  const int s0 = min(n, tid * seg), s1 = min(n, s0 + seg);
+  const int na_ok = bad ? 0 : na;
+  const int qseg = (na_ok + kWindowThreads - 1) / kWindowThreads;
+  const int q0 = min(na_ok, tid * qseg), q1 = min(na_ok, q0 + qseg);
+  const bool in_regs = seg <= kSegRegs && qseg <= kActRegs;     // uniform over the CTA
+  int row_id[kSegRegs], act_id[kActRegs];
+  if (in_regs) {
+#pragma unroll
+    for (int j = 0; j < kSegRegs; ++j) row_id[j] = s0 + j < s1 ? a.pointers[s0 + j] : 0;
+#pragma unroll
+    for (int j = 0; j < kActRegs; ++j) act_id[j] = q0 + j < q1 ? a.act[q0 + j] : 0;
+  }
+
   // ---- A: what would happen ------------------------------------------------------------
   int c_load = 0, c_back = 0, c_stale = 0;
-  if (!bad) {
+  if (!bad && in_regs) {
+    int so[kActRegs], la[kActRegs];
+#pragma unroll
+    for (int j = 0; j < kActRegs; ++j) {
+      so[j] = 0;
+      la[j] = 0;
+      if (q0 + j < q1) {
+        if (act_id[j] < 0 || act_id[j] >= a.F) {
+          bad = 1;
+        } else {
+          so[j] = a.slot_of[act_id[j]];
+          la[j] = a.last_active[act_id[j]];
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kActRegs; ++j) {
+      if (q0 + j < q1 && act_id[j] >= 0 && act_id[j] < a.F) {
+        if (so[j] < 0) ++c_load;
+        else if (la[j] <= stale_before) ++c_back;
+      }
+    }
+    int ls[kSegRegs];
+#pragma unroll
+    for (int j = 0; j < kSegRegs; ++j) ls[j] = s0 + j < s1 ? a.last_active[row_id[j]] : 0;
+#pragma unroll
+    for (int j = 0; j < kSegRegs; ++j) c_stale += (s0 + j < s1 && ls[j] <= stale_before);
+  } else if (!bad) {
     for (int q = tid; q < na; q += kWindowThreads) {
       const int id = a.act[q];
       if (id < 0 || id >= a.F) { bad = 1; continue; }
@@ -175,9 +222,15 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   }
 
   // ---- B: stamp --------------------------------------------------------------------------
-  for (int q = tid; q < na; q += kWindowThreads) {
-    const int id = a.act[q];
-    a.last_active[id] = active_stamp(a, id, t, t_end);
+  if (in_regs) {
+#pragma unroll
+    for (int j = 0; j < kActRegs; ++j)
+      if (q0 + j < q1) a.last_active[act_id[j]] = active_stamp(a, act_id[j], t, t_end);
+  } else {
+    for (int q = tid; q < na; q += kWindowThreads) {
+      const int id = a.act[q];
+      a.last_active[id] = active_stamp(a, id, t, t_end);
+    }
   }
   __syncthreads();
 
@@ -187,17 +240,47 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   // at or beyond `bound` (paper's order: r = 0, bound = n_kept)
   const int reuse = a.append_first ? min(n_evict, n_load) : 0;
   const int bound = n - (n_evict - reuse);
-  const int seg = (n + kWindowThreads - 1) / kWindowThreads;
-  const int s0 = min(n, tid * seg), s1 = min(n, s0 + seg);
   int c_ev = 0, c_surv = 0;
-  for (int s = s0; s < s1; ++s) {
-    const int f = a.last_active[a.pointers[s]] <= stale_before;
-    c_ev += f;
-    c_surv += !f && s >= bound;
+  unsigned stale_rows = 0;                    // register path: bit j = row s0 + j is deleted
+  if (in_regs) {
+    int ls[kSegRegs];
+#pragma unroll
+    for (int j = 0; j < kSegRegs; ++j) ls[j] = s0 + j < s1 ? a.last_active[row_id[j]] : 0;
+#pragma unroll
+    for (int j = 0; j < kSegRegs; ++j) {
+      if (s0 + j < s1) {
+        const int f = ls[j] <= stale_before;
+        stale_rows |= (unsigned)f << j;
+        c_ev += f;
+        c_surv += !f && s0 + j >= bound;
+      }
+    }
+  } else {
+    for (int s = s0; s < s1; ++s) {
+      const int f = a.last_active[a.pointers[s]] <= stale_before;
+      c_ev += f;
+      c_surv += !f && s >= bound;
+    }
   }
   u64 pre = block_scan(pack3(c_ev, 0, c_surv), &tot, sc);
   const int n_moves = field(tot, 2);          // surviving rows at or beyond the bound
-  {
+  if (in_regs) {
+    int p_ev = field(pre, 0), p_surv = field(pre, 2);
+#pragma unroll
+    for (int j = 0; j < kSegRegs; ++j) {
+      const int s = s0 + j;
+      if (s < s1) {
+        if ((stale_rows >> j) & 1u) {
+          a.evict_slots[p_ev] = s;
+          a.evict_ids[p_ev] = row_id[j];
+          ++p_ev;
+        } else if (s >= bound) {
+          a.move_src[n_moves - 1 - p_surv] = s;   // last survivor first
+          ++p_surv;
+        }
+      }
+    }
+  } else {
     int p_ev = field(pre, 0), p_surv = field(pre, 2);
     for (int s = s0; s < s1; ++s) {
       const int id = a.pointers[s];
@@ -229,12 +312,49 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   __syncthreads();
 
   // ---- E + F: rows for the neurons to bring in, and the slot lists -----------------------
-  const int qseg = (na + kWindowThreads - 1) / kWindowThreads;
-  const int q0 = min(na, tid * qseg), q1 = min(na, q0 + qseg);
   int c_l = 0;
-  for (int q = q0; q < q1; ++q) c_l += a.slot_of[a.act[q]] < 0;
+  int so_now[kActRegs];
+  __half bu[kActRegs];
+  if (in_regs) {
+#pragma unroll
+    for (int j = 0; j < kActRegs; ++j) {
+      so_now[j] = 0;
+      bu[j] = __half();
+      if (q0 + j < q1) {
+        so_now[j] = a.slot_of[act_id[j]];
+        bu[j] = a.bias_up[act_id[j]];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kActRegs; ++j) c_l += (q0 + j < q1 && so_now[j] < 0);
+  } else {
+    for (int q = q0; q < q1; ++q) c_l += a.slot_of[a.act[q]] < 0;
+  }
   pre = block_scan(pack3(c_l, (q1 - q0) - c_l, 0), &tot, sc);
-  {
+  if (in_regs) {
+    int p_l = field(pre, 0), p_h = field(pre, 1);
+#pragma unroll
+    for (int j = 0; j < kActRegs; ++j) {
+      const int q = q0 + j;
+      if (q < q1) {
+        const int id = act_id[j];
+        int sl = so_now[j];
+        if (sl < 0) {
+          sl = p_l < n_load - reuse ? bound + p_l : a.evict_slots[n_load - 1 - p_l];
+          a.load_ids[p_l] = id;
+          a.load_slots[p_l] = sl;
+          a.slot_of[id] = sl;
+          a.pointers[sl] = id;
+          a.bias[sl] = bu[j];
+          ++p_l;
+        } else {
+          a.hit_slots[p_h++] = sl;
+        }
+        a.active_slots[q] = sl;
+        if (a.active_idx != a.act) a.active_idx[q] = id;
+      }
+    }
+  } else {
     int p_l = field(pre, 0), p_h = field(pre, 1);
     for (int q = q0; q < q1; ++q) {
       const int id = a.act[q];
