@@ -410,7 +410,7 @@ __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArg
 // kPlanBits active neurons per mask word.  Otherwise the CTA compacts the mask into the list
 // and runs the general path.
 constexpr int kPlanSlots = 4;
-constexpr int kPlanBits = 8;
+constexpr int kPlanBits = 12;
 constexpr int kPlanMaxRows = kPlanSlots * kWindowThreads;
 
 __global__ void __launch_bounds__(kWindowThreads)
