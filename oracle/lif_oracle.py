@@ -398,6 +398,13 @@ def flash_to_dram_gb(model_gb, ffn_percent_of_model, fraction_of_ffn_per_token):
     return model_gb * ffn_percent_of_model / 100.0 * fraction_of_ffn_per_token
 
 
+def average_predictor_rank(layer_counts, ranks):
+    """Mean predictor rank over the layers when groups of layers use different ranks
+    (Appendix B, overhead of predictors: most layers rank 128, the last four rank 1024)."""
+    layer_counts = np.asarray(layer_counts, dtype=np.float64)
+    return float((layer_counts * np.asarray(ranks, dtype=np.float64)).sum() / layer_counts.sum())
+
+
 def predictor_weight_fraction(rank, d_model, d_ff, non_embedding_per_layer=None):
     """Predictor parameters r*(d_model + d_ff) relative to a transformer layer's
     4*d^2 (attention) + 2*d*d_ff (FFN) weights (Appendix B, overhead of predictors)."""

@@ -335,7 +335,7 @@ def test_cost_model_reproduces_paper_values(kind, inputs, value, tol, cite):
         got = O.flash_to_dram_gb(*map(float, inputs.split(",")))
     elif kind == "avg_rank":
         n1, r1, n2, r2 = map(float, inputs.split(","))
-        got = (n1 * r1 + n2 * r2) / (n1 + n2)
+        got = O.average_predictor_rank([n1, n2], [r1, r2])
     elif kind == "predictor_fraction":
         got = O.predictor_weight_fraction(*map(int, inputs.split(",")))
     elif kind == "kv_fraction":
@@ -492,6 +492,83 @@ def test_multi_token_update_keeps_the_window_ending_at_the_kept_token():
             probe.window_update(act2, kt2, keep=m)
             assert not (late_only - set(act2.tolist())) & probe.cached_ids()
         _check_structure(cache)
+
+
+def _clone_cache(cache):
+    twin = O.NeuronCache(cache.d_model, cache.d_ff, cache.capacity, cache.k)
+    twin.__dict__.update({k_: (v.copy() if isinstance(v, np.ndarray) else v)
+                          for k_, v in cache.__dict__.items()})
+    return twin
+
+
+@pytest.mark.parametrize("k,S,m", [(2, 5, 5), (2, 5, 4), (3, 5, 5), (1, 4, 3), (3, 8, 7), (2, 5, 2)])
+def test_multi_token_pass_longer_than_the_window(k, S, m):
+    # A pass that keeps more tokens than the window holds (m > k; Section 4, "Speculative
+    # Decoding": the window is updated with several tokens at once).  Everything is derived
+    # from the per-token history, nothing from the oracle's stamp expression:
+    #   cached set  = neurons active in the last k kept tokens, plus every neuron the pass used
+    #                 (a pass does not delete what it uses);
+    #   window invariant in stamp form (Section 3.1): cached  <=>  last_active > t - k;
+    #   horizon     = with no further activity a cached neuron leaves at the first single-token
+    #                 step whose window no longer holds a kept token in which it was active,
+    #                 and not before the step after the pass that used it.
+    # Invariant and horizon together leave one value for each stamp: horizon - k.
+    F = 240
+    T = 6 * S
+    sets = _random_active_sets(F, T, 0.05, seed=100 + 10 * k + m)
+    cache = O.NeuronCache(2, F, F, k)
+    kept = []                                    # (time, active set) of every kept token
+    for p in range(0, T, S):
+        chunk = sets[p:p + S]
+        act, kt = _pass_info(chunk, F, m)
+        before = cache.cached_ids()
+        ls = cache.window_update(act, kt, keep=m)
+        t0 = len(kept)
+        kept += [(t0 + j, set(chunk[j].tolist())) for j in range(m)]
+        t = len(kept) - 1                        # time of the kept token that ends the window
+        assert cache.t == t + 1
+        used = set(act.tolist())
+        in_window = set().union(*[a for (tau, a) in kept if tau > t - k])
+        expect = (before & in_window) | used
+        assert cache.cached_ids() == expect
+        assert ls["load_ids"].tolist() == sorted(used - before)
+        assert set(ls["evict_ids"].tolist()) == before - expect
+        # window invariant in stamp form
+        by_stamp = set(np.nonzero(cache.last_active > t - k)[0].tolist())
+        assert by_stamp == expect
+        # horizon of every cached neuron, by brute force over the kept history
+        last_kept = {i: max([tau for (tau, a) in kept if i in a], default=None) for i in expect}
+        horizon = {i: max(t + 1, (last_kept[i] + k) if last_kept[i] is not None else t + 1)
+                   for i in expect}
+        probe = _clone_cache(cache)
+        left_at = {}
+        for step in range(t + 1, t + k + 2):     # empty single-token steps
+            gone = probe.cached_ids()
+            probe.window_update(np.zeros(0, dtype=np.int32))
+            gone -= probe.cached_ids()
+            for i in gone:
+                left_at[i] = step
+        assert left_at == horizon
+        for i in expect:
+            assert cache.last_active[i] == horizon[i] - k
+        _check_structure(cache)
+
+
+def test_stamps_of_a_long_pass_worked_example():
+    # k = 2, one pass of 5 kept tokens (times 0..4).  Neuron 7 is active in token 0 only,
+    # neuron 8 in token 3, neuron 9 in token 4, neuron 6 in tokens 1 and 3.  The window after
+    # the pass is {3, 4}.  7 was used by the pass, so it is still cached, but no token of the
+    # window holds it: it must leave at the very next step, i.e. carry the oldest stamp of the
+    # window (3); 6 and 8 carry 3, 9 carries 4.
+    cache = O.NeuronCache(2, 16, 16, 2)
+    act = np.array([6, 7, 8, 9], dtype=np.int32)
+    cache.window_update(act, np.array([3, 0, 3, 4]), keep=5)
+    assert cache.t == 5 and cache.cached_ids() == {6, 7, 8, 9}
+    assert cache.last_active[[6, 7, 8, 9]].tolist() == [3, 3, 3, 4]
+    cache.window_update(np.zeros(0, dtype=np.int32))         # time 5: window {4, 5}
+    assert cache.cached_ids() == {9}
+    cache.window_update(np.zeros(0, dtype=np.int32))         # time 6: window {5, 6}
+    assert cache.cached_ids() == set()
 
 
 def test_keep_tokens_helper():
