@@ -4,19 +4,12 @@
 // contiguous bytes of one bundle with 16-byte loads, and each thread keeps several loads in
 // flight so the link sees enough outstanding requests.  Bound: host-link bandwidth.
 #include "lif_internal.cuh"
+#include "mask_compact.cuh"
 
 namespace lif {
 namespace {
 
 constexpr int kFetchUnroll = 8;   // 16-byte loads in flight per thread
-
-__device__ __forceinline__ uint4 ld_host(const uint4* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
 
 // Copies `row_vec` 16-byte vectors per row.  Work unit = (row, slice of kThreads*kFetchUnroll
 // vectors); units are dealt round-robin to CTAs so a short list still spreads over the grid.
@@ -39,7 +32,7 @@ __device__ __forceinline__ void gather_rows(const uint4* __restrict__ src_base,
 #pragma unroll
     for (int i = 0; i < kFetchUnroll; ++i) {
       const int v = v0 + i * kThreads;
-      if (v < row_vec) buf[i] = ld_host(src + v);
+      if (v < row_vec) buf[i] = ld_stream16(src + v);
     }
 #pragma unroll
     for (int i = 0; i < kFetchUnroll; ++i) {
@@ -69,16 +62,6 @@ fetch_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
 // final before that kernel passed its own wait, while the cache rows may still be moving.
 constexpr int kFusedChunks = 4;     // 8-column chunks per thread and half row: d_model <= 8192
 
-__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
-  const __half2* h = reinterpret_cast<const __half2*>(&v);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float2 t = __half22float2(h[i]);
-    f[2 * i] = t.x;
-    f[2 * i + 1] = t.y;
-  }
-}
-
 struct FetchFfnArgs {
   const uint4* store;
   uint4* cache;
@@ -91,21 +74,66 @@ struct FetchFfnArgs {
   float* y_partial;          // [gridDim.x][d]
   int d, act;
   float act_thr;
+  const uint32_t* new_mask_words;   // kEarlyMask: the predictor's mask of neurons to bring in
+  int nwords;
 };
 
-// kEarly: the lists may be read, and the first host loads issued, before the dependency wait.
-template <int kGate, bool kEarly>
+// How much of the kernel may run before its dependency wait:
+//   kEarlyNone   nothing: the kernel ahead wrote the lists.
+//   kEarlyLists  the lists were final before the kernel ahead passed its own wait (it is the
+//                row-move kernel): count, ids and rows are read and the first bundle's host
+//                loads issued ahead of the wait.
+//   kEarlyMask   the kernel ahead is the window kernel, whose lists are not final yet, but the
+//                predictor's mask of neurons to bring in is: the load list is exactly the set
+//                bits of that mask in ascending order (the window kernel derives it from the
+//                same state), so CTA c finds the id of its first bundle, the c-th set bit,
+//                itself and its host loads travel while the window kernel runs.  After the
+//                wait the count is compared with the window kernel's (it is 0 when that
+//                kernel refused the step) and the rows come from its list.
+template <int kGate, int kEarly>
 __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   __shared__ float part[kThreads / 32];
+  __shared__ int scan_sums[kThreads / 32];
+  __shared__ int first_id;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = a.d >> 3;                       // 16-byte chunks per half row
-  if (!kEarly) {                                   // the kernel ahead wrote the lists
+  if (kEarly == kEarlyNone) {
     pdl_wait();
     pdl_trigger();
   }
-  const int n = __ldcg(a.counts + LIF_CNT_N_LOAD);
+  int n;
+  if (kEarly == kEarlyMask) {
+    // thread t owns a run of consecutive mask words; block-wide prefix of their bit counts
+    const int wpt = (a.nwords + kThreads - 1) / kThreads;
+    const int w0 = min(a.nwords, tid * wpt), w1 = min(a.nwords, w0 + wpt);
+    uint32_t mw[4];                                // nwords <= 1024 in this mode
+    int cnt = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      mw[i] = w0 + i < w1 ? __ldcg(a.new_mask_words + w0 + i) : 0u;
+      cnt += __popc(mw[i]);
+    }
+    if (tid == 0) first_id = -1;
+    int off = block_exclusive_scan_256(cnt, &n, scan_sums);   // also orders the first_id store
+    const int want = blockIdx.x;
+    if (want >= off && want < off + cnt) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int c = __popc(mw[i]);
+        if (want >= off && want < off + c) {
+          uint32_t m = mw[i];
+          for (int s = want - off; s > 0; --s) m &= m - 1;
+          first_id = (w0 + i) * 32 + __ffs(m) - 1;
+        }
+        off += c;
+      }
+    }
+    __syncthreads();
+  } else {
+    n = __ldcg(a.counts + LIF_CNT_N_LOAD);
+  }
   if ((int)blockIdx.x >= n) {                      // the sum reads min(grid, n) partials
-    if (kEarly) {
+    if (kEarly != kEarlyNone) {
       pdl_wait();
       pdl_trigger();
     }
@@ -118,17 +146,34 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
     for (int k = 0; k < kFusedChunks; ++k) {
       const int c = tid + k * kThreads;
       if (c < nvec) {
-        up[k] = ld_host(src + c);
-        down[k] = ld_host(src + nvec + c);
+        up[k] = ld_stream16(src + c);
+        down[k] = ld_stream16(src + nvec + c);
       }
     }
   };
   int j = blockIdx.x;
-  int id = __ldcg(a.load_ids + j), slot = __ldcg(a.load_slots + j);
+  int id, slot = 0;
+  if (kEarly == kEarlyMask) {
+    id = first_id;
+  } else {
+    id = __ldcg(a.load_ids + j);
+    slot = __ldcg(a.load_slots + j);
+  }
   host_loads(id);
-  if (kEarly) {
+  if (kEarly != kEarlyNone) {
     pdl_wait();
     pdl_trigger();
+  }
+  if (kEarly == kEarlyMask) {
+    // the window kernel is complete: its count is this one unless it refused the step (0, window
+    // state unchanged), in which case nothing is written
+    const int n_plan = __ldcg(a.counts + LIF_CNT_N_LOAD);
+    if (n_plan != n) {
+      if (n_plan != 0 && tid == 0)      // cannot happen: both counts come from the same state
+        atomicCAS(const_cast<int32_t*>(a.counts) + LIF_CNT_STATUS, LIF_OK, LIF_ERR_STATE);
+      return;
+    }
+    slot = __ldcg(a.load_slots + j);
   }
 
   uint4 xq[kFusedChunks];
@@ -237,7 +282,7 @@ bool fetch_ffn_supported(const lif_layer* L) {
 // Fetch of this step's new rows fused with their FFN terms; partials go to `partial`
 // ([fetch_grid][d_model], CTA c < min(grid, n_load) writes row c).
 cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st,
-                             bool early_loads) {
+                             int early) {
   const lif_layer_desc& D = L->desc;
   FetchFfnArgs a;
   a.store = (const uint4*)L->dev_bundles;
@@ -252,10 +297,18 @@ cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cuda
   a.d = D.d_model;
   a.act = D.activation;
   a.act_thr = D.activation_threshold;
-  void (*kernel)(FetchFfnArgs) =
-      D.gate_mode == LIF_GATE_RESIDENT
-          ? (early_loads ? fetch_ffn_kernel<LIF_GATE_RESIDENT, true> : fetch_ffn_kernel<LIF_GATE_RESIDENT, false>)
-          : (early_loads ? fetch_ffn_kernel<LIF_GATE_NONE, true> : fetch_ffn_kernel<LIF_GATE_NONE, false>);
+  a.new_mask_words = L->new_mask_words;
+  a.nwords = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
+  if (early == kEarlyMask && a.nwords > 4 * kThreads) early = kEarlyNone;
+  void (*kernel)(FetchFfnArgs);
+  if (D.gate_mode == LIF_GATE_RESIDENT)
+    kernel = early == kEarlyMask    ? fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyMask>
+             : early == kEarlyLists ? fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyLists>
+                                    : fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyNone>;
+  else
+    kernel = early == kEarlyMask    ? fetch_ffn_kernel<LIF_GATE_NONE, kEarlyMask>
+             : early == kEarlyLists ? fetch_ffn_kernel<LIF_GATE_NONE, kEarlyLists>
+                                    : fetch_ffn_kernel<LIF_GATE_NONE, kEarlyNone>;
   return launch_k(kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl, a);
 }
 

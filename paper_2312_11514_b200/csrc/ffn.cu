@@ -19,53 +19,6 @@ namespace lif {
 namespace {
 
 constexpr int kMaxChunks = 4;            // 8-column chunks per thread: d_model <= 8192
-constexpr unsigned kWaitLimit = 1u << 22;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
-               "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
-  unsigned ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: false if the barrier did not complete within kWaitLimit polls.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
-  for (unsigned i = 0; i < kWaitLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, unsigned bytes,
-                                         uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
-      : "memory");
-}
-
-__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
-  const __half2* h = reinterpret_cast<const __half2*>(&v);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float2 t = __half22float2(h[i]);
-    f[2 * i] = t.x;
-    f[2 * i + 1] = t.y;
-  }
-}
 
 struct FfnArgs {
   const __half* cache;
@@ -474,7 +427,7 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
                      : ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
   if (L->fused_fetch && fetch_ffn_supported(L)) {
     // one kernel brings the new rows in and adds their FFN terms (CTA partials in p1)
-    if ((e = launch_fetch_ffn(L, x, p1, st, !moves_aside)) != cudaSuccess) return e;
+    if ((e = launch_fetch_ffn(L, x, p1, st, moves_aside ? kEarlyMask : kEarlyLists)) != cudaSuccess) return e;
     if (ev) tm_record(ev[6], st);
   } else {
     if ((e = launch_fetch(L, st)) != cudaSuccess) return e;

@@ -24,34 +24,17 @@ constexpr int kRowsPerWarp = LIF_GATE_ROWS;           // 1, 2 or 4
 constexpr int kGateTile = 8 * kRowsPerWarp;           // neurons per CTA: 1, 2 or 4 bytes of the mask
 constexpr int kDepth = LIF_GATE_DEPTH;   // load groups in flight per lane (one 16-byte piece per row each)
 
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
-
-__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
-  const __half2* h = reinterpret_cast<const __half2*>(&v);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float2 t = __half22float2(h[i]);
-    f[2 * i] = t.x;
-    f[2 * i + 1] = t.y;
-  }
-}
-
 template <int S>
 __global__ void __launch_bounds__(kThreads)
 gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate,
                    const __half* __restrict__ bias, float theta, int d, int F,
                    float* __restrict__ gate_val, float* __restrict__ logits,
                    uint32_t* mask_words, int* ticket, int* __restrict__ active_idx,
-                   int* __restrict__ n_active, int compact, int nwords) {
+                   int* __restrict__ n_active, int compact, int nwords,
+                   const int32_t* __restrict__ slot_of, uint32_t* new_mask_words) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* xs = reinterpret_cast<uint4*>(smem_raw);          // [S][d / 8]
-  __shared__ int act_flag[kGateTile];
+  __shared__ int act_flag[kGateTile];     // bit 0: active, bit 1: active and not cached yet
   __shared__ int warp_sums[kThreads / 32];
   __shared__ int is_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -66,7 +49,7 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
     const int c = lane + 32 * g;
 #pragma unroll
     for (int q = 0; q < kRowsPerWarp; ++q)
-      dst[q] = (i0 + q < F && c < nvec) ? ldg_stream(gate + (size_t)(i0 + q) * d + c * 8)
+      dst[q] = (i0 + q < F && c < nvec) ? ld_stream16(gate + (size_t)(i0 + q) * d + c * 8)
                                         : make_uint4(0, 0, 0, 0);
   };
   uint4 w[kDepth][kRowsPerWarp];
@@ -132,16 +115,25 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
         active = active || (v > theta);
       }
     }
-    act_flag[warp * kRowsPerWarp + lane] = active ? 1 : 0;
+    // (the window state of the previous step is final long before this kernel starts)
+    act_flag[warp * kRowsPerWarp + lane] = active ? (slot_of[i] < 0 ? 3 : 1) : 0;
   }
   __syncthreads();
   if (warp == 0) {
     // the CTA's 8, 16 or 32 bits are whole bytes of the mask: a plain store, no merging
     const unsigned m = __ballot_sync(0xffffffffu, lane < kGateTile && act_flag[lane] != 0);
+    const unsigned mn = __ballot_sync(0xffffffffu, lane < kGateTile && (act_flag[lane] & 2));
     if (lane == 0) {
-      if (kGateTile == 32) mask_words[blockIdx.x] = m;
-      else if (kGateTile == 16) reinterpret_cast<uint16_t*>(mask_words)[blockIdx.x] = (uint16_t)m;
-      else reinterpret_cast<uint8_t*>(mask_words)[blockIdx.x] = (uint8_t)m;
+      if (kGateTile == 32) {
+        mask_words[blockIdx.x] = m;
+        new_mask_words[blockIdx.x] = mn;
+      } else if (kGateTile == 16) {
+        reinterpret_cast<uint16_t*>(mask_words)[blockIdx.x] = (uint16_t)m;
+        reinterpret_cast<uint16_t*>(new_mask_words)[blockIdx.x] = (uint16_t)mn;
+      } else {
+        reinterpret_cast<uint8_t*>(mask_words)[blockIdx.x] = (uint8_t)m;
+        reinterpret_cast<uint8_t*>(new_mask_words)[blockIdx.x] = (uint8_t)mn;
+      }
     }
   }
   if (!compact) return;     // the consumer reads the bit mask itself
@@ -164,7 +156,7 @@ cudaError_t launch_gate_s(lif_layer* L, const __half* x, float* logits, int32_t*
                   (const __half*)D.dev_gate, (const __half*)D.dev_bias_up, theta, D.d_model,
                   D.d_ff, L->gate_val, logits, L->mask_words,
                   (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
-                  (D.d_ff + 31) / 32);
+                  (D.d_ff + 31) / 32, (const int32_t*)L->slot_of, L->new_mask_words);
 }
 
 }  // namespace

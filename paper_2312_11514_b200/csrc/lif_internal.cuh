@@ -35,7 +35,7 @@ struct Workspace {
   // offsets in bytes from the workspace base; every block 256-byte aligned
   size_t counts, pointers, slot_of, last_active, bias, active_idx, evict_ids, evict_slots,
       move_src, move_dst, load_ids, load_slots, active_slots, hit_slots, n_tmp, z_partial,
-      mask_words, keep_tok, h_rows, gate_val, y_partial, total;
+      mask_words, new_mask_words, keep_tok, h_rows, gate_val, y_partial, total;
 };
 
 // fp16 elements per bundle / cache row: up | down, preceded by the gate row when it is bundled
@@ -58,6 +58,7 @@ struct lif_layer {
       *active_slots, *hit_slots, *n_tmp;
   float* z_partial;
   uint32_t* mask_words;
+  uint32_t* new_mask_words;   // bit i: neuron i is predicted active and has no cache row yet
   int8_t* keep_tok;   // [d_ff] last kept token per neuron (speculative mode)
   float* y_partial;
   float* h_rows;      // [K slices][d_ff][8] fp32: phase-A output of the multi-stream FFN
@@ -122,10 +123,14 @@ cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act
 cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
 bool fetch_ffn_supported(const lif_layer* L);
-// early_loads: the lists were final before the kernel ahead of this one passed its dependency
-// wait (so the first bundle's host loads may be issued before this kernel's own wait)
+// early: what the kernel may do before its own dependency wait.  kEarlyLists: the lists were
+// final before the kernel ahead of this one passed its wait, so the first bundle's host loads
+// are issued from them; kEarlyMask: the kernel ahead is the window kernel of the same step and
+// the predictor ran just before that: the first bundle's id comes from the predictor's mask of
+// neurons to bring in; kEarlyNone: nothing.
+enum { kEarlyNone = 0, kEarlyLists = 1, kEarlyMask = 2 };
 cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st,
-                             bool early_loads);
+                             int early);
 cudaError_t launch_refill(lif_layer* L, cudaStream_t st);
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,
                          int grid, cudaStream_t st);
@@ -189,6 +194,76 @@ __device__ __forceinline__ float apply_activation(float v, int act, float thr) {
 // Let the next kernel of the stream start its prologue.
 __device__ __forceinline__ void pdl_trigger() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// 16-byte streaming load (no L1 allocation) of data that is read once: weights, bundles in
+// mapped host memory.  Deliberately not the non-coherent (.nc) form: a load of memory the
+// assembler knows to be read-only may be scheduled after a later griddepcontrol.wait, next to
+// its first use, which silently turns a prefetch issued ahead of the dependency wait into a load
+// behind it (measured: the predictor kernels 0.7-1 us slower each, the fetch kernel's early
+// host loads without effect).  An ordinary load stays where it is written.
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p)
+               : "memory");
+  return v;
+}
+
+// eight fp16 values -> fp32
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __half22float2(h[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+
+// ---- mbarrier + bulk asynchronous copy (TMA, CTA-local, no multicast) -------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within `limit` polls.
+constexpr unsigned kWaitLimit = 1u << 22;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity,
+                                          unsigned limit = kWaitLimit) {
+  for (unsigned i = 0; i < limit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// global -> this CTA's shared memory, completion counted in bytes on `bar`; src, dst and bytes
+// are multiples of 16
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, unsigned bytes,
+                                         uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
 }
 #endif
 

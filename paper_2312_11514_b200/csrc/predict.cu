@@ -13,24 +13,6 @@
 namespace lif {
 namespace {
 
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
-
-__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
-  const __half2* h = reinterpret_cast<const __half2*>(&v);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float2 t = __half22float2(h[i]);
-    f[2 * i] = t.x;
-    f[2 * i + 1] = t.y;
-  }
-}
-
 // ---- stage 1: z_partial[cta][s][j] = sum_{m in rows(cta)} x[s][m] * A[m][j] -------------
 template <int S>
 __global__ void __launch_bounds__(kThreads)
@@ -56,7 +38,7 @@ predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
     const int m = m0 + rl + u * nrl;
-    aq[u] = (rl < nrl && m < m1) ? ldg_stream(A + (size_t)m * r + cg * 8) : make_uint4(0, 0, 0, 0);
+    aq[u] = (rl < nrl && m < m1) ? ld_stream16(A + (size_t)m * r + cg * 8) : make_uint4(0, 0, 0, 0);
   }
   pdl_wait();
   pdl_trigger();
@@ -78,7 +60,7 @@ predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int
 #pragma unroll 4
     for (int m = m0 + rl + 8 * nrl; m < m1; m += nrl) {
       float af[8];
-      unpack8(ldg_stream(A + (size_t)m * r + cg * 8), af);
+      unpack8(ld_stream16(A + (size_t)m * r + cg * 8), af);
 #pragma unroll
       for (int s = 0; s < S; ++s) {
         const float xs = __half2float(x[(size_t)s * d + m]);
@@ -112,7 +94,8 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
                       const float* __restrict__ c, float theta, int r, int F,
                       float* __restrict__ logits, uint32_t* mask_words, int* ticket,
                       int* __restrict__ active_idx, int* __restrict__ n_active, int compact,
-                      int8_t* __restrict__ keep_tok, int keep) {
+                      int8_t* __restrict__ keep_tok, int keep, const int32_t* __restrict__ slot_of,
+                      uint32_t* new_mask_words) {
   extern __shared__ float zs[];                 // [S][r]
   __shared__ float red[16][kLogitTile];
   __shared__ int warp_sums[kThreads / 32];
@@ -127,10 +110,14 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
     const int j = rs + 16 * u;
-    bq[u] = (col < F && j < r) ? ldg_stream(B + (size_t)j * F + col) : make_uint4(0, 0, 0, 0);
+    bq[u] = (col < F && j < r) ? ld_stream16(B + (size_t)j * F + col) : make_uint4(0, 0, 0, 0);
   }
   const int my_col = blockIdx.x * kLogitTile + tid;   // used by threads < kLogitTile
   const float my_c = (tid < kLogitTile && my_col < F) ? c[my_col] : 0.f;
+  // The window state was last written by this layer's previous step, complete long before this
+  // kernel could start: whether the neuron already has a cache row is read here, so the mask of
+  // neurons to bring in (active and not cached) costs no round trip of its own.
+  const int my_row = (tid < kLogitTile && my_col < F) ? slot_of[my_col] : 0;
   pdl_wait();
   pdl_trigger();
   if (S == 1) {
@@ -177,7 +164,7 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int j = j0 + rs + 16 * u;
-        bq[u] = (col < F && j < r) ? ldg_stream(B + (size_t)j * F + col) : make_uint4(0, 0, 0, 0);
+        bq[u] = (col < F && j < r) ? ld_stream16(B + (size_t)j * F + col) : make_uint4(0, 0, 0, 0);
       }
     }
 #pragma unroll
@@ -217,7 +204,11 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
   if (kSpec && tid < kLogitTile && my_col < F) keep_tok[my_col] = (int8_t)last_kept;
   if (tid < kLogitTile) {
     const unsigned m = __ballot_sync(0xffffffffu, active);
-    if ((tid & 31) == 0) mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = m;
+    const unsigned mn = __ballot_sync(0xffffffffu, active && my_row < 0);
+    if ((tid & 31) == 0) {
+      mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = m;
+      new_mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = mn;
+    }
   }
 
   if (!compact) return;     // the consumer reads the bit mask itself
@@ -249,7 +240,7 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
                (const float*)L->z_partial, L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c,
                D.threshold_logit, D.rank, D.d_ff, logits, L->mask_words,
                (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
-               L->keep_tok, D.spec_keep);
+               L->keep_tok, D.spec_keep, (const int32_t*)L->slot_of, L->new_mask_words);
   if (ev) tm_record(ev[2], st);
   return e;
 }
@@ -275,7 +266,7 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
                   L->z_ctas, (const __half*)D.dev_pred_B, D.dev_pred_c, D.threshold_logit, D.rank,
                   D.d_ff, (float*)nullptr, L->mask_words, (int*)(L->counts + CNT_TICKET_PREDICT),
                   (int*)L->active_idx, (int*)L->n_tmp, L->fused_plan ? 0 : 1, L->keep_tok,
-                  D.spec_keep);
+                  D.spec_keep, (const int32_t*)L->slot_of, L->new_mask_words);
 }
 
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
