@@ -272,8 +272,14 @@ def run_ours(args):
     reps = 20
     if S == 1:
         launchers = {name: (lambda l, kind=kind: B.lif_profile_launch(handles[l], kind, dev_x, Y[l], sc))
-                     for kind, name in enumerate(B.KERNELS)
-                     if not (gate_mode == B.GATE_RESIDENT and name == "predict_z")}
+                     for kind, name in enumerate(B.KERNELS)}
+        try:        # the first predictor stage is a kernel of its own only in some configurations
+            launchers["predict_z"](0)
+        except B.LifError as err:
+            if err.code != B.LIF_ERR_STATE:
+                raise
+            del launchers["predict_z"]
+        torch.cuda.synchronize()
     else:
         # several streams: the staged entry points (predictor = 2 kernels; FFN = the tensor-core
         # up, down and partial-sum kernels over all active rows)
@@ -339,7 +345,7 @@ def run_ours(args):
             pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_scores"]
         else:
             pred_bytes = 2 * cfg.rank * (d + cfg.d_ff) + 4 * cfg.d_ff
-            pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_z"] + kernel_us["predict_scores"]
+            pred_us = kernel_us["predict"] if S > 1 else kernel_us.get("predict_z", 0.0) + kernel_us["predict_scores"]
         pred_gbs = pred_bytes / (pred_us * 1e-6) / 1e9
         split = None
         if S == 1:

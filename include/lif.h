@@ -13,9 +13,13 @@
  *    only the opaque handle (plus two CUDA events inside it).
  *  - `stream` arguments are `cudaStream_t` values passed as `void*` (NULL = default stream).
  *  - Calls that take a stream only enqueue work and never synchronise.  Argument errors are
- *    returned immediately.  Conditions only the device can see (cache overflow, a bounded
- *    wait that ran out) are written to the layer's device status word, leave the window
- *    state of that step untouched, and are reported by lif_get_stats.
+ *    returned immediately.  Conditions only the device can see are written to the layer's
+ *    sticky device status word and reported by lif_get_stats: a cache overflow or a bad neuron
+ *    id (the window update of that step is refused, the window state untouched); a row index
+ *    outside the cache given to the sparse FFN (the row is not read and contributes nothing); a
+ *    bounded wait on a copy that ran out (LIF_ERR_TIMEOUT: that call's output lacks some rows'
+ *    terms; the window bookkeeping stays consistent, and while this status stands every
+ *    further window update is refused — lif_clear_status resumes).
  *  - fp16 = IEEE binary16; accumulations are fp32.
  *  - All counts the kernels need (n_active, n_load, ...) stay in device memory; no call
  *    needs them on the host to launch the next one.
@@ -215,7 +219,10 @@ lif_status lif_fetch_bundles(lif_layer* layer, void* fetch_stream);
  * lif_predict / lif_decode_step of the layer, which must have been given the same x)
  *   dev_slots    int32 rows to use, or NULL for rows [0, *dev_n_slots)
  *   dev_n_slots  int32 [1] (device)
- *   dev_y        fp32 [n_streams][d_model] */
+ *   dev_y        fp32 [n_streams][d_model]
+ * A row outside [0, capacity) or a count outside [0, capacity] is never used to address the
+ * cache: the row contributes nothing, the count is clamped, and the status word becomes
+ * LIF_ERR_INVALID_ARG. */
 lif_status lif_sparse_ffn(lif_layer* layer, const void* dev_x, const int32_t* dev_slots,
                           const int32_t* dev_n_slots, float* dev_y, void* stream);
 
@@ -228,8 +235,12 @@ lif_status lif_sparse_ffn(lif_layer* layer, const void* dev_x, const int32_t* de
  * instead: the partial sums live in a fixed 2 MiB array inside the library's device image
  * (held on every GPU that loads the library until the process exits), and the call allocates
  * nothing, on the host or the device.
- *   dev_matrix     fp16 [rows][2*d_model] cache rows (up half, down half), 16-byte aligned
- *   dev_bias       fp16 [rows] up-projection bias of each row
+ *   dev_matrix     fp16 [n_rows][2*d_model] cache rows (up half, down half), 16-byte aligned
+ *   n_rows         rows of dev_matrix (>= 1): a row index outside [0, n_rows), or a count
+ *                  outside [0, n_rows], is never used to address memory; it contributes
+ *                  nothing (the count is clamped) and is reported as LIF_ERR_INVALID_ARG by
+ *                  lif_sparse_ffn_static_status
+ *   dev_bias       fp16 [n_rows] up-projection bias of each row
  *   dev_x          fp16 [d_model], one stream
  *   dev_slots      int32 rows to use, or NULL for rows [0, *dev_n_slots)
  *   dev_n_slots    int32 [1] on the device
@@ -239,17 +250,23 @@ lif_status lif_sparse_ffn(lif_layer* layer, const void* dev_x, const int32_t* de
  * at most one per SM) and therefore the order of the partial sums can differ, so results
  * agree to rounding, not bitwise.  d_model above LIF_STATIC_MAX_D_MODEL, or not a multiple of
  * 8, is refused with LIF_ERR_INVALID_ARG; misaligned pointers with LIF_ERR_ALIGNMENT.
- * The first call on each device looks up the array's device address and opts the kernel in
- * to large shared memory; make that first call with the device current and outside any
- * stream capture.  All calls on a device share the one array and it keeps the previous
- * call's contents: every call overwrites the part it reads and clears its own status word,
- * but two calls whose kernels overlap on the GPU (different streams) race on it — keep calls
- * on one device ordered. */
+ * The first call on each device (of either function below) looks up the array's device
+ * address and opts the kernel in to large shared memory; make that first call with the device
+ * current and outside any stream capture.  All calls on a device share the one array and it
+ * keeps the previous call's contents: every call overwrites the part it reads, but two calls
+ * whose kernels overlap on the GPU (different streams) race on it — keep calls on one device
+ * ordered.
+ * Conditions only the kernels can see go to a status word inside the same array, which stays
+ * set until it is read: lif_sparse_ffn_static_status synchronises the device, copies the word
+ * (a lif_status: LIF_OK, LIF_ERR_INVALID_ARG for a refused row or count, LIF_ERR_TIMEOUT for a
+ * bounded wait that ran out — the output of that call then lacks some rows' terms) to
+ * *host_status and, with clear != 0, resets it.  It allocates nothing either. */
 #define LIF_STATIC_MAX_D_MODEL 8192
-lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* dev_bias, const void* dev_x,
-                                 const int32_t* dev_slots, const int32_t* dev_n_slots,
-                                 const void* dev_bias_down, float* dev_y, int32_t d_model,
-                                 void* stream);
+lif_status lif_sparse_ffn_static(const void* dev_matrix, int32_t n_rows, const void* dev_bias,
+                                 const void* dev_x, const int32_t* dev_slots,
+                                 const int32_t* dev_n_slots, const void* dev_bias_down,
+                                 float* dev_y, int32_t d_model, void* stream);
+lif_status lif_sparse_ffn_static_status(int32_t* host_status, int32_t clear);
 
 /* Neuron sharding over several devices (not in the paper, which runs on one device; it rests
  * on Section 3.3 item 3: the FFN output is a sum of one term per cached neuron, in any order).
@@ -311,28 +328,6 @@ lif_status lif_graph_launch_host(lif_graph* graph, const void* host_x, float* ho
                                  void* stream);
 lif_status lif_graph_destroy(lif_graph* graph);
 
-/* Launch-shape knobs (defaults in parentheses); they change speed, never results beyond the
- * order of floating-point partial sums.  Set them before capturing a graph. */
-enum {
-  LIF_TUNE_DEPENDENT_LAUNCH = 0, /* (1) programmatic dependent launch along the compute stream */
-  LIF_TUNE_SPLIT_FFN = 1,        /* (1) lif_decode_step runs the FFN of already-cached rows
-                                    while the fetch copies, then the FFN of the new rows */
-  LIF_TUNE_FETCH_CTAS = 2,       /* (SM count) CTAs of the fetch kernel, 1..4096 */
-  LIF_TUNE_FFN_CTAS = 3,         /* (SM count) CTAs of the sparse-FFN kernel, 1..256 */
-  LIF_TUNE_FFN_STAGES = 4,       /* (as many as fit, at most 16) bundles in flight per CTA;
-                                    fewer stages let several CTAs share an SM */
-  LIF_TUNE_BATCHED_COLUMN_PARTS = 5, /* (fewest that fit) column parts of the multi-stream FFN's
-                                    down-projection kernel, 1..16 */
-  LIF_TUNE_BATCHED_UP_TWO_CTAS = 7, /* (0) multi-stream FFN, up-projection kernel: two light CTAs
-                                    per SM instead of one with a deep ring */
-  LIF_TUNE_FUSED_PLAN = 6,       /* (1 when d_ff <= 32768) lif_decode_step: the window update
-                                    reads the predictor's bit mask instead of its index list */
-  LIF_TUNE_FUSED_FETCH_FFN = 8   /* (1) lif_decode_step, one stream, with LIF_TUNE_SPLIT_FFN: the
-                                    fetch kernel also adds the FFN terms of the rows it brings
-                                    in (needs fetch CTAs = FFN CTAs, bundles of two vectors) */
-};
-lif_status lif_set_tuning(lif_layer* layer, int32_t key, int32_t value);
-
 /* Device addresses of lists and state (valid for the layer's lifetime). */
 lif_status lif_get_lists(lif_layer* layer, lif_lists* host_out);
 
@@ -349,57 +344,16 @@ lif_status lif_read_state(lif_layer* layer, int32_t* host_pointers, int32_t* hos
  * lif_restore copies it back and re-reads rows 0..num_used-1 from the host bundle store, so a
  * restored layer continues exactly as the snapshotted one would have.  Both synchronise the
  * device; the buffer is plain host memory of at least lif_snapshot_bytes() bytes and is only
- * valid for a layer of the same description.  LIF_ERR_STATE: the buffer's counters do not fit
- * this layer. */
+ * valid for a layer of the same description.  lif_restore checks the buffer on the host
+ * before anything reaches the device (counters in range, pointers and slot_of inverse maps of
+ * each other over exactly num_used rows, free rows marked -1, stamps older than the step);
+ * LIF_ERR_STATE: it does not describe a state of this layer, and the layer is left as it was. */
 lif_status lif_snapshot_bytes(lif_layer* layer, size_t* out_bytes);
 lif_status lif_snapshot(lif_layer* layer, void* host_buf, size_t bytes);
 lif_status lif_restore(lif_layer* layer, const void* host_buf, size_t bytes);
 
 /* Clears the sticky device status word. */
 lif_status lif_clear_status(lif_layer* layer, void* stream);
-
-/* Phases timed by lif_timing_* (one CUDA event pair each, inside lif_decode_step). */
-enum {
-  LIF_PHASE_PREDICT_Z = 0,      /* x.A partial sums */
-  LIF_PHASE_PREDICT_SCORES = 1, /* scores, threshold, compaction */
-  LIF_PHASE_WINDOW = 2,         /* window bookkeeping kernel */
-  LIF_PHASE_MOVES = 3,          /* row moves */
-  LIF_PHASE_FETCH = 4,          /* bundle fetch (on the fetch stream) */
-  LIF_PHASE_FFN = 5,            /* sparse FFN gather kernel(s) */
-  LIF_PHASE_FFN_SUM = 6,        /* partial-sum kernel(s) */
-  LIF_PHASE_LEN = 8
-};
-
-/* Profiling aid: with n_steps > 0, the next n_steps calls of lif_decode_step record CUDA
- * events around every kernel (host-side event objects, no device memory); n_steps = 0 turns
- * it off and frees the events.  lif_timing_read synchronises the device and returns, per
- * phase, the summed device time in microseconds over the steps recorded since enabling. */
-lif_status lif_timing_enable(lif_layer* layer, int32_t n_steps);
-lif_status lif_timing_read(lif_layer* layer, float* host_us_sums /* [LIF_PHASE_LEN] */,
-                           int32_t* host_n_steps);
-
-/* Profiling aid: enqueue exactly one kernel of the decode step, with the launch shape
- * lif_decode_step uses, on the layer's current lists (valid after a completed step; these
- * kernels do not change the window state, so they can be replayed).  dev_x as for
- * lif_decode_step; dev_y is written only by LIF_KERNEL_FFN_SUM.  n_streams must be 1. */
-enum {
-  LIF_KERNEL_PREDICT_Z = 0,  /* not with LIF_GATE_RESIDENT */
-  LIF_KERNEL_PREDICT_SCORES = 1, /* LIF_GATE_RESIDENT: the gate-projection kernel */
-  LIF_KERNEL_FETCH = 2,      /* re-copies this step's new bundles (and, where the decode step
-                                fuses it, recomputes their FFN partials) */
-  LIF_KERNEL_FFN_ACTIVE = 3, /* sparse FFN kernel over all active rows */
-  LIF_KERNEL_FFN_HITS = 4,   /* ... over the active rows that were already cached */
-  LIF_KERNEL_FFN_NEW = 5,    /* ... over the rows brought in this step */
-  LIF_KERNEL_FFN_SUM = 6     /* partial-sum kernel over the hits + new partials */
-};
-lif_status lif_profile_launch(lif_layer* layer, int32_t kernel, const void* dev_x, float* dev_y,
-                              void* stream);
-
-/* Bandwidth probe for the host link: a kernel reads `bytes` of mapped pinned host memory
- * into device memory with the same access pattern as lif_fetch_bundles (chunk_bytes-sized
- * pieces; chunk_bytes a multiple of 16, bytes a multiple of chunk_bytes).  Enqueue only. */
-lif_status lif_probe_host_read(const void* host_src, void* dev_dst, size_t bytes,
-                               size_t chunk_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -25,12 +25,13 @@ EXPORTS = [
     "lif_decode_token_host", "lif_get_lists", "lif_get_stats", "lif_clear_status",
     "lif_probe_host_read", "lif_timing_enable", "lif_timing_read",
     "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
-    "lif_sparse_ffn_static", "lif_set_tuning", "lif_profile_launch",
+    "lif_sparse_ffn_static", "lif_sparse_ffn_static_status", "lif_set_tuning", "lif_profile_launch",
     "lif_read_state", "lif_snapshot_bytes", "lif_snapshot", "lif_restore", "lif_sum_peer_outputs",
 ]
 KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ffn_new", "ffn_sum")
 (TUNE_DEPENDENT_LAUNCH, TUNE_SPLIT_FFN, TUNE_FETCH_CTAS, TUNE_FFN_CTAS, TUNE_FFN_STAGES,
- TUNE_BATCHED_COLUMN_PARTS, TUNE_FUSED_PLAN, TUNE_BATCHED_UP_TWO_CTAS, TUNE_FUSED_FETCH_FFN) = range(9)
+ TUNE_BATCHED_COLUMN_PARTS, TUNE_FUSED_PLAN, TUNE_BATCHED_UP_TWO_CTAS, TUNE_FUSED_FETCH_FFN,
+ TUNE_WAIT_POLLS) = range(10)
 PHASES = ("predict_z", "predict_scores", "window", "moves", "fetch", "ffn", "ffn_sum")
 PHASE_LEN = 8
 
@@ -99,7 +100,8 @@ def lib() -> C.CDLL:
         "lif_graph_launch": [vp, vp],
         "lif_graph_launch_host": [vp, vp, vp, vp],
         "lif_graph_destroy": [vp],
-        "lif_sparse_ffn_static": [vp, vp, vp, vp, vp, vp, vp, i32, vp],
+        "lif_sparse_ffn_static": [vp, i32, vp, vp, vp, vp, vp, vp, i32, vp],
+        "lif_sparse_ffn_static_status": [C.POINTER(C.c_int32), i32],
         "lif_sum_peer_outputs": [C.POINTER(vp), i32, vp, sz, vp],
         "lif_set_tuning": [vp, i32, i32],
         "lif_read_state": [vp, vp, vp, vp, vp],
@@ -266,13 +268,22 @@ def lif_graph_destroy(graph: int) -> None:
     _check(lib().lif_graph_destroy(graph), "lif_graph_destroy")
 
 
-def lif_sparse_ffn_static(matrix, bias, x, slots, n_slots, bias_down, y, d_model: int,
+def lif_sparse_ffn_static(matrix, n_rows: int, bias, x, slots, n_slots, bias_down, y, d_model: int,
                           stream=None) -> None:
     """Sparse FFN without a layer or workspace: the partial sums use the library's built-in
     2 MiB device array, so nothing is allocated (see include/lif.h for the sharing rules)."""
-    _check(lib().lif_sparse_ffn_static(_ptr(matrix), _ptr(bias), _ptr(x), _ptr(slots),
+    _check(lib().lif_sparse_ffn_static(_ptr(matrix), n_rows, _ptr(bias), _ptr(x), _ptr(slots),
                                        _ptr(n_slots), _ptr(bias_down), _ptr(y), d_model,
                                        _stream(stream)), "lif_sparse_ffn_static")
+
+
+def lif_sparse_ffn_static_status(clear: bool = True) -> int:
+    """Synchronises the device and returns the sticky status word of lif_sparse_ffn_static on
+    the current device (a LIF_* code), resetting it when ``clear``."""
+    out = C.c_int32(-1)
+    _check(lib().lif_sparse_ffn_static_status(C.byref(out), 1 if clear else 0),
+           "lif_sparse_ffn_static_status")
+    return int(out.value)
 
 
 def lif_sum_peer_outputs(partials, y, stream=None) -> None:

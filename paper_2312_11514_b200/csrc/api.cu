@@ -171,6 +171,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
     L->fetch_grid = L->n_sm;
     L->move_grid = L->n_sm;
     L->use_pdl = 1;
+    L->wait_polls = kWaitLimit;
     L->split_ffn = 1;
     L->fused_plan = window_plan_supported(*desc) ? 1 : 0;
     L->fused_fetch = 1;
@@ -441,7 +442,9 @@ lif_status lif_profile_launch(lif_layer* L, int32_t kernel, const void* dev_x, f
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
   switch (kernel) {
-    case LIF_KERNEL_PREDICT_Z:
+    case LIF_KERNEL_PREDICT_Z:     // only where the first stage is a kernel of its own
+      if (L->desc.gate_mode == LIF_GATE_RESIDENT) return LIF_ERR_STATE;
+      /* fall through */
     case LIF_KERNEL_PREDICT_SCORES:
       e = launch_predict_one(L, kernel, (const __half*)dev_x, st);
       break;
@@ -491,6 +494,10 @@ lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
     case LIF_TUNE_BATCHED_UP_TWO_CTAS:
       L->fb_up_two_ctas = value != 0;
       return ffn_batched_configure(L) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+    case LIF_TUNE_WAIT_POLLS:
+      if (value < 0) return LIF_ERR_INVALID_ARG;
+      L->wait_polls = (unsigned)value;
+      return LIF_OK;
     case LIF_TUNE_FFN_STAGES:
       if (value < 1 || value > L->ffn_stages_max) return LIF_ERR_INVALID_ARG;
       L->ffn_stages = value;
@@ -586,11 +593,32 @@ lif_status lif_restore(lif_layer* L, const void* host_buf, size_t bytes) {
   size_t need = 0;
   if (!L || !host_buf || lif_snapshot_bytes(L, &need) != LIF_OK || bytes < need)
     return LIF_ERR_INVALID_ARG;
-  // a snapshot of another shape or a damaged one: check the counters it carries
-  const int32_t* cnt = (const int32_t*)host_buf;
-  if (cnt[LIF_CNT_NUM_USED] < 0 || cnt[LIF_CNT_NUM_USED] > L->desc.capacity ||
-      cnt[LIF_CNT_STEP] < 0)
-    return LIF_ERR_STATE;
+  // A snapshot of another shape, a truncated or a damaged one: everything the kernels will
+  // use as an index is checked here, on the host, before any of it reaches the device.
+  {
+    const int F = L->desc.d_ff, cap = L->desc.capacity;
+    const int32_t* cnt = (const int32_t*)host_buf;
+    const int32_t* ptr = cnt + LIF_CNT_LEN;
+    const int32_t* slot_of = ptr + cap;
+    const int32_t* last = slot_of + F;
+    const int n = cnt[LIF_CNT_NUM_USED], step = cnt[LIF_CNT_STEP];
+    if (n < 0 || n > cap || step < 0) return LIF_ERR_STATE;
+    for (int s = 0; s < cap; ++s) {
+      if (s < n ? (ptr[s] < 0 || ptr[s] >= F || slot_of[ptr[s]] != s) : ptr[s] != -1)
+        return LIF_ERR_STATE;
+    }
+    int cached = 0;
+    for (int i = 0; i < F; ++i) {
+      if (slot_of[i] >= 0) {
+        if (slot_of[i] >= n || ptr[slot_of[i]] != i) return LIF_ERR_STATE;
+        ++cached;
+      } else if (slot_of[i] != -1) {
+        return LIF_ERR_STATE;
+      }
+      if (last[i] >= step && last[i] != kNever) return LIF_ERR_STATE;   // stamps lie in the past
+    }
+    if (cached != n) return LIF_ERR_STATE;
+  }
   if (cudaDeviceSynchronize() != cudaSuccess) return LIF_ERR_CUDA;
   StatePart p[5];
   const unsigned char* in = (const unsigned char*)host_buf;

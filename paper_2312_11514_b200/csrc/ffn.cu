@@ -36,6 +36,8 @@ struct FfnArgs {
   float act_thr;
   const float* gate_val;  // resident gate: this stream's gate pre-activations, by neuron id
   const int32_t* pointers;  // resident gate: row -> neuron id
+  int rows;               // rows of `cache`: a slot outside [0, rows) is refused, not read
+  unsigned wait_polls;    // poll limit of the first wait on each copy (kWaitLimit)
 };
 
 // kGate = LIF_GATE_*: none (row = up | down), bundled (gate | up | down), resident (up | down,
@@ -78,8 +80,19 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
     const int q = cta + tid * G;
     if (q < a.slots_len) my_slot = a.slots[q];
   }
-  const int n = *a.n;
-  if (cta >= n) return;                       // the reduction only reads min(G, n) partials
+  // Row count and rows come from the caller (or from lists the caller could have overwritten):
+  // a count outside [0, rows] is clamped and a row outside [0, rows) contributes nothing and is
+  // never read; either sets LIF_ERR_INVALID_ARG in the status word.
+  int n = *a.n;
+  int bad_input = 0;
+  if (n < 0 || n > a.rows) {
+    bad_input = 1;
+    n = n < 0 ? 0 : a.rows;
+  }
+  if (cta >= n) {                             // the reduction only reads min(G, n) partials
+    if (bad_input && cta == 0 && tid == 0) atomicCAS(a.status, LIF_OK, LIF_ERR_INVALID_ARG);
+    return;
+  }
   const int base = a.base ? *a.base : 0;
   const int my_cnt = (n - cta + G - 1) / G;
   __syncthreads();                            // barrier init visible
@@ -95,12 +108,18 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
   for (int r0 = 0; r0 < my_cnt; r0 += stages) {
     const int rc = min(stages, my_cnt - r0);
     // thread i issues the copy of row i of this round and fetches its bias
+    bool row_ok = true;                       // (thread i also finishes row i below)
     if (tid < rc) {
       const int q = cta + (r0 + tid) * G;
       int slot;
       if (!a.slots) slot = base + q;
       else if (r0 == 0 && q < a.slots_len) slot = my_slot;
       else slot = a.slots[q];
+      if (slot < 0 || slot >= a.rows) {       // refused: row 0 travels in its place, weight 0
+        row_ok = false;
+        bad_input = 1;
+        slot = 0;
+      }
       mbar_expect_tx(bars + tid, row_bytes);
       bulk_g2s(rows + (size_t)tid * row_bytes, a.cache + (size_t)slot * kVec * d, row_bytes,
                bars + tid);
@@ -114,7 +133,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
     }
     // up projection: partial dot products as rows land
     for (int i = 0; i < rc; ++i) {
-      if (!mbar_wait(bars + i, parity)) timed_out = 1;
+      if (!mbar_wait(bars + i, parity, a.wait_polls)) timed_out = 1;
       const uint4* up = reinterpret_cast<const uint4*>(rows + (size_t)i * row_bytes);
       float p = 0.f, p2 = 0.f;
       for (int c = tid; c < nvec; c += kThreads) {
@@ -165,6 +184,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
       } else {
         hs[tid] = apply_activation(bias_s[tid], a.act, a.act_thr) * v;
       }
+      if (!row_ok) hs[tid] = 0.f;
     }
     __syncthreads();
     // down projection: y += h * down half
@@ -188,6 +208,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
     parity ^= 1u;
   }
 
+  if (bad_input) atomicCAS(a.status, LIF_OK, LIF_ERR_INVALID_ARG);
   float4* out = reinterpret_cast<float4*>(a.y_partial + (size_t)cta * d);
 #pragma unroll
   for (int k = 0; k < kMaxChunks; ++k) {
@@ -209,7 +230,7 @@ __global__ void __launch_bounds__(kSumThreads)
 ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
                   const float* __restrict__ p1, const int32_t* __restrict__ n1, int G,
                   const __half* __restrict__ b_down, int b_period, float* __restrict__ y, int d,
-                  int accumulate) {
+                  int accumulate, int n_cap) {
   __shared__ float4 red[32][kSumCols];
   const int tid = threadIdx.x;
   const int c4 = tid & (kSumCols - 1), gs = tid / kSumCols;
@@ -225,7 +246,8 @@ ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
   }
   pdl_wait();
   pdl_trigger();
-  const int v0 = min(G, *n0), v1 = p1 ? min(G, *n1) : 0;
+  // counts as the kernels that wrote the partials clamp them: [0, n_cap]
+  const int v0 = min(G, max(0, min(*n0, n_cap))), v1 = p1 ? min(G, max(0, min(*n1, n_cap))) : 0;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
   if (in) {
     // batches of 10 partials per thread (two sets of up to 148 over 32 slices), a batch's loads
@@ -317,6 +339,8 @@ static FfnArgs ffn_args(lif_layer* L, const __half* x, const int32_t* slots, con
   a.act_thr = L->desc.activation_threshold;
   a.gate_val = L->gate_val;
   a.pointers = L->pointers;
+  a.rows = L->desc.capacity;
+  a.wait_polls = L->wait_polls;
   return a;
 }
 
@@ -347,7 +371,7 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
     e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st, L->use_pdl,
                  (const float*)L->y_partial, n, (const float*)nullptr, (const int32_t*)nullptr,
                  L->ffn_grid, (const __half*)D.dev_bias_down, d, y + (size_t)s * d, d,
-                 accumulate ? 1 : 0);
+                 accumulate ? 1 : 0, D.capacity);
     if (e != cudaSuccess) return e;
   }
   if (ev) tm_record(ev[9], st);
@@ -376,7 +400,8 @@ cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cuda
     case LIF_KERNEL_FFN_SUM:
       return launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st,
                       L->use_pdl, (const float*)p0, cnt + LIF_CNT_N_HITS, (const float*)p1,
-                      cnt + LIF_CNT_N_LOAD, L->ffn_grid, (const __half*)D.dev_bias_down, d, y, d, 0);
+                      cnt + LIF_CNT_N_LOAD, L->ffn_grid, (const __half*)D.dev_bias_down, d, y, d, 0,
+                      D.capacity);
     default:
       return cudaErrorInvalidValue;
   }
@@ -389,7 +414,7 @@ cudaError_t launch_partial_sum(lif_layer* L, const float* partial, const int32_t
   return launch_k(ffn_reduce_kernel, dim3((width / 4 + kSumCols - 1) / kSumCols),
                   dim3(kSumThreads), 0, st, L->use_pdl, partial, n, (const float*)nullptr,
                   (const int32_t*)nullptr, partitions, (const __half*)L->desc.dev_bias_down,
-                  L->desc.d_model, y, width, 0);
+                  L->desc.d_model, y, width, 0, L->desc.capacity);
 }
 
 // Fetch + FFN of a single-stream decode step.  The critical chain stays on `st` with dependent
@@ -439,7 +464,7 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
   if (fork && (e = cudaStreamWaitEvent(st, L->ev_fetch, 0)) != cudaSuccess) return e;
   e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0,
                st, L->use_pdl, (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,
-               (const __half*)D.dev_bias_down, d, y, d, 0);
+               (const __half*)D.dev_bias_down, d, y, d, 0, D.capacity);
   if (ev) tm_record(ev[9], st);
   return e;
 }
@@ -459,7 +484,8 @@ constexpr int kStaticFloats = 512 * 1024;   // 2 MiB of partials, resident on ev
 constexpr int kStaticMaxDevices = 64;
 
 struct StaticScratch {
-  int32_t status;                // sink for the kernel's timeout flag; cleared by every call
+  int32_t status;                // sticky lif_status of the kernels (bad row, wait that ran out);
+                                 // read and cleared by lif_sparse_ffn_static_status
   int32_t pad[63];
   float partial[kStaticFloats];  // [ctas][d_model]
 };
@@ -479,23 +505,20 @@ std::mutex g_static_mutex;
 }  // namespace
 }  // namespace lif
 
-extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* dev_bias,
-                                            const void* dev_x, const int32_t* dev_slots,
-                                            const int32_t* dev_n_slots, const void* dev_bias_down,
-                                            float* dev_y, int32_t d_model, void* stream) {
-  using namespace lif;
-  if (!dev_matrix || !dev_bias || !dev_x || !dev_n_slots || !dev_y) return LIF_ERR_INVALID_ARG;
-  // the scratch holds at least 64 CTA partials of this width
-  if (d_model < 8 || d_model % 8 || d_model > LIF_STATIC_MAX_D_MODEL) return LIF_ERR_INVALID_ARG;
-  auto mis = [](const void* p, size_t a) { return ((uintptr_t)p % a) != 0; };
-  if (mis(dev_matrix, 16) || mis(dev_x, 16) || mis(dev_y, 16) || mis(dev_bias, 2) ||
-      mis(dev_n_slots, 4) || (dev_slots && mis(dev_slots, 4)) ||
-      (dev_bias_down && mis(dev_bias_down, 8)))
-    return LIF_ERR_ALIGNMENT;
-
+namespace lif {
+namespace {
+// First use on the current device: resolve the scratch array's device address and opt the
+// kernel in to large shared memory.  Returns nullptr (and leaves `err`) on failure.
+StaticDevice* static_device(lif_status* err) {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return LIF_ERR_CUDA;
-  if (dev < 0 || dev >= kStaticMaxDevices) return LIF_ERR_STATE;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    *err = LIF_ERR_CUDA;
+    return nullptr;
+  }
+  if (dev < 0 || dev >= kStaticMaxDevices) {
+    *err = LIF_ERR_STATE;
+    return nullptr;
+  }
   StaticDevice& sd = g_static_dev[dev];
   std::lock_guard<std::mutex> setup_lock(g_static_mutex);   // first calls from several threads
   if (!sd.ready) {
@@ -508,11 +531,51 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                              sd.max_smem) != cudaSuccess) {
       cudaGetLastError();
-      return LIF_ERR_CUDA;
+      *err = LIF_ERR_CUDA;
+      return nullptr;
     }
     sd.scratch = static_cast<StaticScratch*>(p);
     sd.ready = true;
   }
+  return &sd;
+}
+}  // namespace
+}  // namespace lif
+
+extern "C" lif_status lif_sparse_ffn_static_status(int32_t* host_status, int32_t clear) {
+  using namespace lif;
+  if (!host_status) return LIF_ERR_INVALID_ARG;
+  lif_status err = LIF_OK;
+  StaticDevice* sd = static_device(&err);
+  if (!sd) return err;
+  bool ok = cudaDeviceSynchronize() == cudaSuccess &&
+            cudaMemcpy(host_status, &sd->scratch->status, sizeof(int32_t),
+                       cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (ok && clear) ok = cudaMemset(&sd->scratch->status, 0, sizeof(int32_t)) == cudaSuccess;
+  if (!ok) cudaGetLastError();
+  return ok ? LIF_OK : LIF_ERR_CUDA;
+}
+
+extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, int32_t n_rows,
+                                            const void* dev_bias, const void* dev_x,
+                                            const int32_t* dev_slots, const int32_t* dev_n_slots,
+                                            const void* dev_bias_down, float* dev_y,
+                                            int32_t d_model, void* stream) {
+  using namespace lif;
+  if (!dev_matrix || !dev_bias || !dev_x || !dev_n_slots || !dev_y || n_rows < 1)
+    return LIF_ERR_INVALID_ARG;
+  // the scratch holds at least 64 CTA partials of this width
+  if (d_model < 8 || d_model % 8 || d_model > LIF_STATIC_MAX_D_MODEL) return LIF_ERR_INVALID_ARG;
+  auto mis = [](const void* p, size_t a) { return ((uintptr_t)p % a) != 0; };
+  if (mis(dev_matrix, 16) || mis(dev_x, 16) || mis(dev_y, 16) || mis(dev_bias, 2) ||
+      mis(dev_n_slots, 4) || (dev_slots && mis(dev_slots, 4)) ||
+      (dev_bias_down && mis(dev_bias_down, 8)))
+    return LIF_ERR_ALIGNMENT;
+
+  lif_status err = LIF_OK;
+  StaticDevice* sdp = static_device(&err);
+  if (!sdp) return err;
+  StaticDevice& sd = *sdp;
 
   int stages = 16;
   while (stages > 1 && ffn_smem_bytes(d_model, stages) > (size_t)sd.max_smem) --stages;
@@ -521,10 +584,6 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
   if (grid > sd.n_sm) grid = sd.n_sm;
 
   cudaStream_t st = (cudaStream_t)stream;
-  if (cudaMemsetAsync(&sd.scratch->status, 0, sizeof(int32_t), st) != cudaSuccess) {
-    cudaGetLastError();
-    return LIF_ERR_CUDA;
-  }
   FfnArgs a;
   a.cache = (const __half*)dev_matrix;
   a.bias = (const __half*)dev_bias;
@@ -541,10 +600,12 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, const void* 
   a.act_thr = 0.f;
   a.gate_val = nullptr;
   a.pointers = nullptr;
+  a.rows = n_rows;
+  a.wait_polls = kWaitLimit;
   sparse_ffn_kernel<LIF_GATE_NONE><<<grid, kThreads, ffn_smem_bytes(d_model, stages), st>>>(a);
   if (cudaGetLastError() != cudaSuccess) return LIF_ERR_CUDA;
   ffn_reduce_kernel<<<(d_model / 4 + kSumCols - 1) / kSumCols, kSumThreads, 0, st>>>(
       sd.scratch->partial, dev_n_slots, nullptr, nullptr, grid, (const __half*)dev_bias_down,
-      d_model, dev_y, d_model, 0);
+      d_model, dev_y, d_model, 0, n_rows);
   return cudaGetLastError() == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
 }

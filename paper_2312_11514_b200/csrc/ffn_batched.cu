@@ -81,10 +81,30 @@ struct BatchedArgs {
   const float* H2;        // bundled gate: phase-A output of the up rows (H holds the gate rows)
   const float* gate_val;  // resident gate: [S][F] gate pre-activations by neuron id
   const int32_t* pointers;  // resident gate: row -> neuron id
+  int rows;               // rows of `cache`: a slot outside [0, rows) is refused, not read
+  unsigned wait_polls;    // poll limit of the first wait on each group of copies
 };
 
+// Cache row of list position q, or -1 when the list names a row outside the cache (such a row is
+// never read: row 0 travels in its place and its activations are forced to zero).
 __device__ __forceinline__ int row_slot(const BatchedArgs& a, int q, int base) {
-  return a.slots ? a.slots[q] : base + q;
+  const int slot = a.slots ? a.slots[q] : base + q;
+  return (slot < 0 || slot >= a.rows) ? -1 : slot;
+}
+// Row count as every kernel of this path clamps it: [0, rows].
+__device__ __forceinline__ int row_count(const BatchedArgs& a) {
+  const int n = *a.n;
+  return n < 0 ? 0 : (n > a.rows ? a.rows : n);
+}
+// After a wait ran out: one more bounded chance for every copy still in flight to land in this
+// CTA's shared memory (a barrier is re-polled with the parity of its current phase; one whose
+// phase already completed returns at once).
+__device__ __forceinline__ void drain_ring(uint64_t* bars, int stages, int group, int g,
+                                           int groups_in_ring) {
+  for (int k = 0; k < groups_in_ring; ++k) {
+    const int gg = g + k;                              // groups g .. g + ring - 1 may be armed
+    mbar_wait(bars + (gg % groups_in_ring) * group, (unsigned)(gg / groups_in_ring) & 1u);
+  }
 }
 
 // ---- phase A: partial pre-activations  Hp[slice][q][s] = <Up[q, slice], x[s, slice]> (+ bias) --
@@ -114,7 +134,8 @@ __global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs
   }
   pdl_wait();
   pdl_trigger();
-  const int n = *a.n;
+  const int n = row_count(a);
+  if (n != *a.n && blockIdx.x == 0 && tid == 0) atomicCAS(a.status, LIF_OK, LIF_ERR_INVALID_ARG);
   if (prt >= n) return;
   const int base = a.base ? *a.base : 0;
   const int P = a.up_partitions;
@@ -124,15 +145,23 @@ __global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs
   // Slots and biases of this CTA's rows go to shared memory once, so the group loop below has
   // no dependent global loads; the first copies are issued on the way.  Then the x slice
   // (streams beyond S are zero).
+  // a refused row is remembered as a NaN bias: its pre-activations are written as zero
+  const float kRefused = __int_as_float(0x7fc00000);
   for (int i = tid; i < min(my_cnt, kRowCacheA); i += kThreads) {
-    const int slot = row_slot(a, prt + i * P, base);
+    int slot = row_slot(a, prt + i * P, base);
+    const bool refused = slot < 0;
+    if (refused) {
+      atomicCAS(a.status, LIF_OK, LIF_ERR_INVALID_ARG);
+      slot = 0;
+    }
     slot_all[i] = slot;
     if (i < stages) {
       mbar_expect_tx(group_bar(bars, i, G), seg_bytes);
       bulk_g2s(rows + (size_t)i * pitch, a.cache + (size_t)slot * a.row_elems + a.vec_off + k0,
                seg_bytes, group_bar(bars, i, G));
     }
-    const float b = (ks == 0 && a.add_bias) ? __half2float(a.bias[slot]) : 0.f;
+    const float b = refused ? kRefused
+                            : ((ks == 0 && a.add_bias) ? __half2float(a.bias[slot]) : 0.f);
     bias_all[i] = b;
     if (i < stages) bias_s[i] = b;
   }
@@ -166,7 +195,7 @@ __global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs
     const int st0 = (g % groups_in_ring) * G;
     const unsigned parity = (unsigned)(g / groups_in_ring) & 1u;
     const int valid = min(G, my_cnt - g * G);
-    if (!mbar_wait(bars + st0, parity)) timed_out = 1;
+    if (!mbar_wait(bars + st0, parity, a.wait_polls)) timed_out = 1;
     // D[row][stream] over this warp's part of the slice
     float c[4] = {0.f, 0.f, 0.f, 0.f};
     const unsigned char* ab = rows + (size_t)(st0 + a_row) * pitch + a_off;
@@ -183,7 +212,7 @@ __global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs
     if (__syncthreads_or(timed_out)) {
       if (tid == 0) {
         atomicCAS(a.status, LIF_OK, LIF_ERR_TIMEOUT);
-        mbar_wait(bars + st0, parity);
+        drain_ring(bars, stages, G, g, groups_in_ring);
       }
       __syncthreads();
       return;
@@ -196,7 +225,8 @@ __global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs
 #pragma unroll
         for (int w = 0; w < 8; ++w) v += red[w * 128 + src];
         const int q = prt + (g * G + r) * P;
-        Hp[(size_t)q * 8 + s] = v + bias_s[st0 + r];
+        const float b = bias_s[st0 + r];
+        Hp[(size_t)q * 8 + s] = b == b ? v + b : 0.f;     // NaN marks a refused row
       }
     }
     __syncthreads();                                    // stages st0.. , bias_s and red are free
@@ -205,12 +235,19 @@ __global__ void __launch_bounds__(kThreads, 2) ffn_batched_up_kernel(BatchedArgs
       const int i = (g + groups_in_ring) * G + tid;
       if (i < my_cnt) {
         const bool cached = i < kRowCacheA;
-        const int slot = cached ? slot_all[i] : row_slot(a, prt + i * P, base);
+        int slot = cached ? slot_all[i] : row_slot(a, prt + i * P, base);
+        const bool refused = slot < 0;
+        if (refused) {
+          atomicCAS(a.status, LIF_OK, LIF_ERR_INVALID_ARG);
+          slot = 0;
+        }
         mbar_expect_tx(bars + st0, seg_bytes);
         bulk_g2s(rows + (size_t)(st0 + tid) * pitch,
                  a.cache + (size_t)slot * a.row_elems + a.vec_off + k0, seg_bytes, bars + st0);
         bias_s[st0 + tid] =
-            cached ? bias_all[i] : ((ks == 0 && a.add_bias) ? __half2float(a.bias[slot]) : 0.f);
+            cached ? bias_all[i]
+                   : (refused ? kRefused
+                              : ((ks == 0 && a.add_bias) ? __half2float(a.bias[slot]) : 0.f));
       } else {
         mbar_arrive(bars + st0);
       }
@@ -245,7 +282,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   // through H.  Rows, slots and counters were final before that kernel passed its own
   // dependency wait (it signals its dependents only afterwards), so they are read, and the
   // first copies issued, before the wait below: the prologue overlaps the up kernel's tail.
-  const int n = *a.n;
+  const int n = row_count(a);
   const int base = a.base ? *a.base : 0;
   const int P = a.partitions;
   const int my_cnt = prt < n ? (n - prt + P - 1) / P : 0;       // rows q = prt + i * P
@@ -259,8 +296,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
   __syncthreads();
   const size_t col_off = (size_t)a.down_off + col0;
 
+  // (a refused row was reported by the up kernel and has H = 0: row 0 stands in for it)
   for (int i = tid; i < min(my_cnt, kRowCacheB); i += kThreads) {   // slots once, first copies
-    const int slot = row_slot(a, prt + i * P, base);
+    const int slot = max(0, row_slot(a, prt + i * P, base));
     slot_all[i] = slot;
     if (i < stages) {
       mbar_expect_tx(group_bar(bars, i), seg_bytes);
@@ -290,7 +328,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     }
     if (a.gate_mode == LIF_GATE_RESIDENT) {      // H = up value, gate from the score array
       if (hs >= a.S) return 0.f;
-      const int id = a.pointers[row_slot(a, prt + i * P, base)];
+      const int id = a.pointers[max(0, row_slot(a, prt + i * P, base))];
       return apply_activation(a.gate_val[(size_t)hs * a.F + id], a.act, a.act_thr) * v;
     }
     return apply_activation(v, a.act, a.act_thr);
@@ -347,11 +385,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
       const int i = (g + 1) * 16 + hk;
       h_next = i < my_cnt ? load_h(i) : 0.f;
     }
-    if (!mbar_wait(bars + st0, parity)) timed_out = 1;
+    if (!mbar_wait(bars + st0, parity, a.wait_polls)) timed_out = 1;
     if (__syncthreads_or(timed_out)) {
       if (tid == 0) {
         atomicCAS(a.status, LIF_OK, LIF_ERR_TIMEOUT);
-        mbar_wait(bars + st0, parity);
+        drain_ring(bars, stages, kGroup, g, stages / kGroup);
       }
       __syncthreads();
       return;
@@ -379,7 +417,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_down_kernel(BatchedAr
     if (tid < 16) {
       const int i = (g + 2) * 16 + tid;
       if (i < my_cnt) {
-        const int slot = i < kRowCacheB ? slot_all[i] : row_slot(a, prt + i * P, base);
+        const int slot = i < kRowCacheB ? slot_all[i] : max(0, row_slot(a, prt + i * P, base));
         mbar_expect_tx(bars + st0, seg_bytes);
         bulk_g2s(rows + (size_t)(st0 + tid) * pitch,
                  a.cache + (size_t)slot * a.row_elems + col_off, seg_bytes, bars + st0);
@@ -507,6 +545,8 @@ cudaError_t launch_ffn_batched(lif_layer* L, const __half* x, const int32_t* slo
   a.H2 = nullptr;
   a.gate_val = L->gate_val;
   a.pointers = L->pointers;
+  a.rows = D.capacity;
+  a.wait_polls = L->wait_polls;
   a.stages = L->fb_up_stages;
   cudaError_t e = launch_k(ffn_batched_up_kernel, dim3(L->fb_up_partitions * L->fb_ksplit),
                            dim3(kThreads), L->fb_up_smem, st, L->use_pdl, a);

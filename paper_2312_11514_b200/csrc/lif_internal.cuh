@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include "lif.h"
+#include "lif_profile.h"
 
 namespace lif {
 
@@ -76,6 +77,7 @@ struct lif_layer {
   size_t ffn_smem;    // dynamic shared memory of the sparse-FFN kernel
   int fetch_grid;     // CTAs of the fetch kernel
   int move_grid;
+  unsigned wait_polls; // poll limit of the first wait on each bulk copy in the FFN kernels
   int use_pdl;        // programmatic dependent launch along the compute stream
   int split_ffn;      // decode step: cached rows' FFN overlaps the fetch
   int fused_plan;     // decode step: window update reads the predictor's bit mask directly

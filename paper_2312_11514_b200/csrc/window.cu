@@ -116,6 +116,8 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   const int t_end = t + a.keep - 1;   // the kept window ends at this token
   u64 tot;
   int bad = (na < 0 || na > a.F) ? 1 : 0;
+  // a predictor input that never arrived left an incomplete active set: no update from it
+  const int stale_input = a.counts[LIF_CNT_STATUS] == LIF_ERR_TIMEOUT;
   int k_eff = a.k;
   if (a.budget > 0) {
     // age histogram of the cached rows, minus those that are active again now
@@ -206,7 +208,7 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
   const int n_evict = field(tot, 2) - field(tot, 1);
   const int n_kept = n - n_evict;
 
-  if (any_bad || n_kept + n_load > limit) {
+  if (any_bad || stale_input || n_kept + n_load > limit) {
     if (tid == 0) {
       if (a.counts[LIF_CNT_STATUS] == LIF_OK)
         a.counts[LIF_CNT_STATUS] = any_bad ? LIF_ERR_INVALID_ARG : LIF_ERR_CAPACITY;
@@ -447,6 +449,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
   pdl_wait();
   pdl_trigger();
   const uint32_t w = tid < nwords ? mask_words[tid] : 0u;
+  const int stale_input = a.counts[LIF_CNT_STATUS] == LIF_ERR_TIMEOUT;   // see the general path
   const int cnt = __popc(w);
   bits[tid] = w;
   u64 tot;
@@ -521,7 +524,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
   const int n_kept = n - n_evict;
   int p_load = field(pre, 0), p_ev = field(pre, 1), p_hit = field(pre, 2);
 
-  if (n_kept + n_load > limit) {            // refuse before anything is changed
+  if (stale_input || n_kept + n_load > limit) {            // refuse before anything is changed
     if (tid == 0) {
       if (a.counts[LIF_CNT_STATUS] == LIF_OK) a.counts[LIF_CNT_STATUS] = LIF_ERR_CAPACITY;
       a.counts[LIF_CNT_N_ACTIVE] = 0;

@@ -8,13 +8,16 @@ import pytest
 
 from paper_2312_11514_b200 import binding as B
 
-HEADER = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "lif.h")
+INCLUDE = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
 
 
 def _declared():
-    text = open(HEADER).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(lif_[a-z_]+)\s*\(", text)))
+    names = set()
+    for header in sorted(os.listdir(INCLUDE)):
+        text = open(os.path.join(INCLUDE, header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(lif_[a-z_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol():
@@ -100,5 +103,6 @@ def test_graph_and_profiling_calls_reject_null_handles():
     assert lib.lif_profile_launch(None, 0, None, None, None) == B.LIF_ERR_INVALID_ARG
     assert lib.lif_set_tuning(None, 0, 0) == B.LIF_ERR_INVALID_ARG
     assert lib.lif_timing_enable(None, 1) == B.LIF_ERR_INVALID_ARG
-    assert lib.lif_sparse_ffn_static(None, None, None, None, None, None, None, 256, None) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_sparse_ffn_static(None, 1, None, None, None, None, None, None, 256, None) == B.LIF_ERR_INVALID_ARG
+    assert lib.lif_sparse_ffn_static_status(None, 0) == B.LIF_ERR_INVALID_ARG
     assert lib.lif_sum_peer_outputs(None, 2, None, 16, None) == B.LIF_ERR_INVALID_ARG
