@@ -76,6 +76,8 @@ struct FetchFfnArgs {
   float act_thr;
   const uint32_t* new_mask_words;   // kEarlyMask: the predictor's mask of neurons to bring in
   int nwords;
+  const int* tiles_done;            // kEarlyWatch: mask words the score kernel has written
+  int n_tiles;                      // ... out of this many
 };
 
 // How much of the kernel may run before its dependency wait:
@@ -90,13 +92,39 @@ struct FetchFfnArgs {
 //                itself and its host loads travel while the window kernel runs.  After the
 //                wait the count is compared with the window kernel's (it is 0 when that
 //                kernel refused the step) and the rows come from its list.
-template <int kGate, int kEarly>
+constexpr int kWatchPolls = 64;     // about 30 us of polling at most
+
+template <int kGate, int kEarlyT>
 __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   __shared__ float part[kThreads / 32];
   __shared__ int scan_sums[kThreads / 32];
   __shared__ int first_id;
+  __shared__ int watch_ok;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = a.d >> 3;                       // 16-byte chunks per half row
+  int kEarly = kEarlyT;
+  if (kEarlyT == kEarlyWatch) {
+    // Resident while the score kernel may still be running (all of its CTAs are: it released
+    // the window kernel, which released this one, only after every one of them had started).
+    // One thread polls the count of finished tiles.  The count was cleared by this step's first
+    // predictor stage; a count beyond the tiles means other launches of the score kernel came
+    // between and nothing can be told from it.  Whatever the outcome, no result depends on it:
+    // without the count the kernel simply waits for its predecessors like kEarlyNone.
+    if (tid == 0) {
+      int ok = 0;
+      for (int i = 0; i < kWatchPolls; ++i) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(a.tiles_done) : "memory");
+        if (v >= a.n_tiles) {
+          ok = v == a.n_tiles;
+          break;
+        }
+      }
+      watch_ok = ok;
+    }
+    __syncthreads();
+    kEarly = watch_ok ? kEarlyMask : kEarlyNone;
+  }
   if (kEarly == kEarlyNone) {
     pdl_wait();
     pdl_trigger();
@@ -299,14 +327,19 @@ cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cuda
   a.act_thr = D.activation_threshold;
   a.new_mask_words = L->new_mask_words;
   a.nwords = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
-  if (early == kEarlyMask && a.nwords > 4 * kThreads) early = kEarlyNone;
+  a.tiles_done = L->counts + CNT_TILES_DONE;
+  a.n_tiles = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);   // counted per word pair
+  if (early >= kEarlyMask && a.nwords > 4 * kThreads) early = kEarlyNone;
+  // only the low-rank predictor counts its tiles
+  if (early == kEarlyWatch && D.gate_mode == LIF_GATE_RESIDENT) early = kEarlyMask;
   void (*kernel)(FetchFfnArgs);
   if (D.gate_mode == LIF_GATE_RESIDENT)
     kernel = early == kEarlyMask    ? fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyMask>
              : early == kEarlyLists ? fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyLists>
                                     : fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyNone>;
   else
-    kernel = early == kEarlyMask    ? fetch_ffn_kernel<LIF_GATE_NONE, kEarlyMask>
+    kernel = early == kEarlyWatch   ? fetch_ffn_kernel<LIF_GATE_NONE, kEarlyWatch>
+             : early == kEarlyMask  ? fetch_ffn_kernel<LIF_GATE_NONE, kEarlyMask>
              : early == kEarlyLists ? fetch_ffn_kernel<LIF_GATE_NONE, kEarlyLists>
                                     : fetch_ffn_kernel<LIF_GATE_NONE, kEarlyNone>;
   return launch_k(kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl, a);

@@ -452,7 +452,7 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
                      : ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
   if (L->fused_fetch && fetch_ffn_supported(L)) {
     // one kernel brings the new rows in and adds their FFN terms (CTA partials in p1)
-    if ((e = launch_fetch_ffn(L, x, p1, st, moves_aside ? kEarlyMask : kEarlyLists)) != cudaSuccess) return e;
+    if ((e = launch_fetch_ffn(L, x, p1, st, moves_aside ? kEarlyWatch : kEarlyLists)) != cudaSuccess) return e;
     if (ev) tm_record(ev[6], st);
   } else {
     if ((e = launch_fetch(L, st)) != cudaSuccess) return e;

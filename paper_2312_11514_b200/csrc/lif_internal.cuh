@@ -13,6 +13,7 @@ namespace lif {
 // Private entries of the counts block (public ones: LIF_CNT_* in lif.h).
 enum {
   CNT_TICKET_PREDICT = 16,  // "last block done" counter of the score kernel
+  CNT_TILES_DONE = 17,      // mask words the score kernel has written so far in this step
   CNT_TOTALS = 32           // four uint64: bytes_fetched, rows_moved, rows_active, rows_cached
 };
 
@@ -130,7 +131,10 @@ bool fetch_ffn_supported(const lif_layer* L);
 // are issued from them; kEarlyMask: the kernel ahead is the window kernel of the same step and
 // the predictor ran just before that: the first bundle's id comes from the predictor's mask of
 // neurons to bring in; kEarlyNone: nothing.
-enum { kEarlyNone = 0, kEarlyLists = 1, kEarlyMask = 2 };
+// kEarlyWatch: like kEarlyMask, but the window kernel ahead releases its dependents as soon as it
+// starts, so this kernel is resident while the score kernel still runs and watches that kernel's
+// count of finished tiles (bounded; it falls back to kEarlyNone when the count does not come).
+enum { kEarlyNone = 0, kEarlyLists = 1, kEarlyMask = 2, kEarlyWatch = 3 };
 cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st,
                              int early);
 cudaError_t launch_refill(lif_layer* L, cudaStream_t st);

@@ -78,6 +78,7 @@ struct WindowArgs {
   const int8_t* keep_tok; // [F] last kept token per neuron, -1 if active only in later tokens
   int keep;
   int append_first;       // stack the new neurons before deleting (see the header of this file)
+  int release_early;      // release the dependent kernel before this kernel's own wait
   unsigned long long bundle_bytes;
 };
 
@@ -399,8 +400,9 @@ __device__ void window_update_generic(const WindowArgs& a, Scan& sc) {
 
 __global__ void __launch_bounds__(kWindowThreads) window_update_kernel(WindowArgs a) {
   __shared__ Scan sc;
+  if (a.release_early) pdl_trigger();     // see window_plan_kernel
   pdl_wait();
-  pdl_trigger();
+  if (!a.release_early) pdl_trigger();
   window_update_generic(a, sc);
 }
 
@@ -423,6 +425,12 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
   __shared__ int holes[kPlanMaxRows];
   __shared__ int newslot[kPlanMaxRows];
   const int tid = threadIdx.x;
+  // With the low-rank predictor the kernel behind this one is released at once: every kernel of
+  // the library waits for its predecessor's completion before it touches that kernel's output,
+  // and the fetch kernel uses the time to become resident and to watch the score kernel finish
+  // (kEarlyWatch).  Otherwise the release follows this kernel's own wait, which is what lets a
+  // dependent read the predictor's masks ahead of its wait (kEarlyMask).
+  if (a.release_early) pdl_trigger();
   // The window state was last written by this layer's previous step, which is complete before
   // the predictor of this step even starts: the slot side of the bookkeeping (row -> neuron,
   // row bias, each cached neuron's stamp: three dependent round trips) is read before the
@@ -447,7 +455,7 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
 #pragma unroll
   for (int j = 0; j < kPlanSlots; ++j) la[j] = j < my_slots ? a.last_active[pid[j]] : 0;
   pdl_wait();
-  pdl_trigger();
+  if (!a.release_early) pdl_trigger();
   const uint32_t w = tid < nwords ? mask_words[tid] : 0u;
   const int stale_input = a.counts[LIF_CNT_STATUS] == LIF_ERR_TIMEOUT;   // see the general path
   const int cnt = __popc(w);
@@ -703,6 +711,7 @@ static WindowArgs window_args(lif_layer* L, const int32_t* act, const int32_t* n
   a.keep = D.spec_keep > 0 ? D.spec_keep : 1;
   a.bundle_bytes = 2ull * row_elems(D);
   a.append_first = D.append_first;
+  a.release_early = D.gate_mode != LIF_GATE_RESIDENT;
   return a;
 }
 
