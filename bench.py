@@ -1,15 +1,17 @@
 """Benchmark of the sparse-decode FFN stack (predict -> window update -> bundle fetch ->
 sparse FFN, every layer, one token per step) on seeded synthetic data.
 
-  python bench.py --gpus 1 --steps K --warmup W           CUDA path, one JSON line
+  python bench.py --gpus N --steps K --warmup W           CUDA path, one JSON line
   python bench.py --impl reference ...                     CPU oracle on the host cores
+  python bench.py --floors                                 link and launch reference points
 
 One step = one decode token through all layers of the configuration.  `value` is tokens/s
 with the decode inputs resident in HBM (the bundle store stays in pinned host memory: reading
 it is part of the method); `e2e` passes pinned HOST inputs/outputs through
 lif_graph_launch_host.  A token is one CUDA graph (lif_graph_capture).  Per-kernel durations
-for the roofline come from a further timed pass over the same tokens with a CUDA event node
-around every kernel of the graph.
+for the roofline come from a further pass after the timed tokens: for each kernel, a graph of
+that one kernel on every layer (the lists of the last token) is replayed and timed with CUDA
+events.  With --gpus N > 1 and no torchrun environment the script starts its own N ranks.
 """
 from __future__ import annotations
 
@@ -34,6 +36,7 @@ FFN_TRAFFIC_RATIO = 1.005
 # fetch_ffn_kernel: bytes read from system memory per bundle byte, same kind of capture
 FETCH_TRAFFIC_RATIO = 1.000
 FALLBACK_HBM_GBS = 6650.0
+_LINK_PEAK = {}          # measured pinned host -> device rate per local device, GB/s
 
 
 def _peaks():
@@ -108,6 +111,12 @@ def whole_job_tokens_per_s(steps, world, ms_slowest):
 GATE_MODES = {"none": 0, "bundled": 1, "resident": 2}
 
 
+def workload_string(cfg, n_layers, gate_name, gate_mode, act_thr):
+    return (f"{cfg.name}: {n_layers} layers d_model={cfg.d_model} d_ff={cfg.d_ff} rank={cfg.rank} "
+            f"window_k={cfg.window_k} streams={cfg.n_streams}, AR(1) decode inputs"
+            + (f", gated FFN ({gate_name} gate, FATReLU {act_thr})" if gate_mode else ""))
+
+
 def _gate_setup(args):
     """(gate_mode, activation, threshold): gated runs use FATReLU on the gate value (Appendix C,
     Llama 2); ungated runs use ReLU."""
@@ -123,9 +132,6 @@ def _inputs(cfg, n_tokens, device, W):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2312_11514_b200 import binding as B
-    from paper_2312_11514_b200 import runtime as R
-    from paper_2312_11514_b200 import workloads as W
 
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
@@ -136,6 +142,32 @@ def run_ours(args):
     dev = f"cuda:{local}"
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
+    out = measure(args, args.config, args.steps, args.warmup, rank, world, local, detail=True)
+    if rank == 0:
+        if args.other_configs and world == 1 and args.config == "opt6p7b" and not args.layers \
+                and args.gate == "none" and args.shard == "sequences":
+            # the other single-GPU configurations at reduced length, so that their numbers are
+            # in the same record (batched8 keeps 36.75 GiB of bundles in pinned host memory)
+            out["other_configs"] = []
+            for name in ("falcon7b", "phi2", "batched8"):
+                o = measure(args, name, 24, 8, rank, world, local, detail=False)
+                out["other_configs"].append({k: o[k] for k in (
+                    "value", "unit", "ms_per_step", "steps", "warmup", "config", "e2e", "roofline",
+                    "host_link", "per_token", "kernel_us_per_launch")})
+        print(json.dumps(out), flush=True)
+    if dist.is_initialized():
+        dist.destroy_process_group()
+
+
+def measure(args, config_name, steps, warmup, rank, world, local, detail):
+    """Build the stack of one configuration, time it, and return the record (rank 0)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2312_11514_b200 import binding as B
+    from paper_2312_11514_b200 import runtime as R
+    from paper_2312_11514_b200 import workloads as W
+
+    dev = f"cuda:{local}"
 
     # every rank decodes its own sequence with its own replica of the stack (weak scaling,
     # no exchange between ranks)
@@ -143,9 +175,9 @@ def run_ours(args):
     # layer's neurons, and sum their partial outputs after every layer (strong scaling)
     # (at N = 1 the same layer-by-layer path runs with the whole layer as the only share)
     sharded = args.shard == "neurons"
-    cfg = W.CONFIGS[args.config]
+    cfg = W.CONFIGS[config_name]
     cfg = cfg if sharded else rank_config(cfg, rank)
-    K, Wm = args.steps, args.warmup
+    K, Wm = steps, warmup
     n_tok = Wm + K
     gate_mode, activation, act_thr = _gate_setup(args)
     layers = R.build_stack(cfg, dev, n_layers=args.layers, gate_mode=gate_mode, activation=activation,
@@ -267,19 +299,18 @@ def run_ours(args):
     with torch.cuda.stream(sc):
         dev_x.copy_(X[last])
     cnts = torch.stack([l.counts[:16] for l in layers]).cpu()
-    n_act_l, n_load_l, n_hit_l = (cnts[:, i].sum().item() for i in (B.CNT_N_ACTIVE, B.CNT_N_LOAD, B.CNT_N_HITS))
+    n_act_l, n_load_l, n_hit_l, n_used_l = (cnts[:, i].sum().item() for i in (
+        B.CNT_N_ACTIVE, B.CNT_N_LOAD, B.CNT_N_HITS, B.CNT_NUM_USED))
     kernel_us = {}
     reps = 20
     if S == 1:
         launchers = {name: (lambda l, kind=kind: B.lif_profile_launch(handles[l], kind, dev_x, Y[l], sc))
-                     for kind, name in enumerate(B.KERNELS)}
-        try:        # the first predictor stage is a kernel of its own only in some configurations
-            launchers["predict_z"](0)
-        except B.LifError as err:
-            if err.code != B.LIF_ERR_STATE:
-                raise
-            del launchers["predict_z"]
-        torch.cuda.synchronize()
+                     for kind, name in enumerate(B.KERNELS)
+                     if not (gate_mode == B.GATE_RESIDENT and name == "predict_z")}
+        if not detail:
+            launchers = {k: v for k, v in launchers.items() if k in ("fetch", "ffn_active", "ffn_hits", "ffn_new")}
+        if args.append_first == 0 and "ffn_cache" in launchers:
+            pass      # rows [0, num_used) are the cache in both orders once a step is complete
     else:
         # several streams: the staged entry points (predictor = 2 kernels; FFN = the tensor-core
         # up, down and partial-sum kernels over all active rows)
@@ -310,8 +341,8 @@ def run_ours(args):
     n_launch = K * L
 
     # host-link peak: pinned host -> device cudaMemcpyAsync of 1 GiB, best of 5
-    link_peak = None
-    if rank == 0:
+    link_peak = _LINK_PEAK.get(local)
+    if rank == 0 and link_peak is None:
         nb = 1 << 30
         hbuf = torch.empty(nb, dtype=torch.uint8, pin_memory=True)
         dbuf = torch.empty(nb, dtype=torch.uint8, device=dev)
@@ -321,6 +352,7 @@ def run_ours(args):
             torch.cuda.synchronize()
             best = min(best, e0.elapsed_time(e1))
         link_peak = nb / best / 1e6
+        _LINK_PEAK[local] = link_peak
         del hbuf, dbuf
 
     if rank == 0:
@@ -340,26 +372,35 @@ def run_ours(args):
         ffn_gbs = ffn_bytes / (ffn_us * 1e-6) / 1e9
         fetch_bytes = n_load_l * beta / L
         fetch_gbs = fetch_bytes / (kernel_us["fetch"] * 1e-6) / 1e9
-        if gate_mode == B.GATE_RESIDENT:       # gate matrix + bias in, gate values out
-            pred_bytes = 2 * cfg.d_ff * d + 2 * cfg.d_ff + 4 * S * cfg.d_ff
-            pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_scores"]
-        else:
-            pred_bytes = 2 * cfg.rank * (d + cfg.d_ff) + 4 * cfg.d_ff
-            pred_us = kernel_us["predict"] if S > 1 else kernel_us.get("predict_z", 0.0) + kernel_us["predict_scores"]
-        pred_gbs = pred_bytes / (pred_us * 1e-6) / 1e9
+        predictor = None
+        if detail or S > 1:
+            if gate_mode == B.GATE_RESIDENT:       # gate matrix + bias in, gate values out
+                pred_bytes = 2 * cfg.d_ff * d + 2 * cfg.d_ff + 4 * S * cfg.d_ff
+                pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_scores"]
+            else:
+                pred_bytes = 2 * cfg.rank * (d + cfg.d_ff) + 4 * cfg.d_ff
+                pred_us = kernel_us["predict"] if S > 1 else kernel_us["predict_z"] + kernel_us["predict_scores"]
+            pred_gbs = pred_bytes / (pred_us * 1e-6) / 1e9
+            predictor = {"bound": "hbm", "achieved": pred_gbs, "unit": "GB/s", "frac": pred_gbs / peak,
+                         "bytes_per_launch": pred_bytes, "us_per_launch": pred_us}
         split = None
         if S == 1:
             split = {"all_active_rows": {"GBs": all_gbs, "us_per_launch": kernel_us["ffn_active"],
                                          "bytes_per_launch": all_bytes, "frac": all_gbs / peak},
                      "new_rows_GBs": (n_load_l * (beta + row_extra) / L + 6 * d) / (kernel_us["ffn_new"] * 1e-6) / 1e9}
+            if "ffn_cache" in kernel_us:
+                # the same kernel over every cached row (Section 3.3 item 3 as written)
+                cache_bytes = (n_used_l * (beta + row_extra) + L * 6 * d) / L
+                cache_gbs = cache_bytes / (kernel_us["ffn_cache"] * 1e-6) / 1e9
+                split["whole_cache"] = {"GBs": cache_gbs, "us_per_launch": kernel_us["ffn_cache"],
+                                        "bytes_per_launch": cache_bytes, "frac": cache_gbs / peak,
+                                        "rows_per_launch": n_used_l / L}
         out = {
             "metric": METRIC, "value": whole_job_tokens_per_s(K, 1 if sharded else world, ms_total), "unit": UNIT,
             "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms_total / K,
             "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
             "dtype": "f16", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: {L} layers d_model={d} d_ff={cfg.d_ff} rank={cfg.rank} "
-                                   f"window_k={cfg.window_k} streams={S}, AR(1) decode inputs"
-                                   + (f", gated FFN ({args.gate} gate, FATReLU {act_thr})" if gate_mode else ""),
+            "config": {"workload": workload_string(cfg, L, args.gate, gate_mode, act_thr),
                        "cache_order": "new neurons stacked first, then the deletions (bundles written "
                                       "straight into freed rows)" if args.append_first else
                                       "deletions first, then new neurons stacked (Section 3.3 as written)",
@@ -402,8 +443,7 @@ def run_ours(args):
                           "traffic_how": "system-memory bytes read per algorithmic byte from the ncu capture "
                                          "in profiles/fetch_ffn_kernel_opt6p7b_12layers.md, scaled by this "
                                          "run's rows per launch"},
-            "predictor": {"bound": "hbm", "achieved": pred_gbs, "unit": "GB/s", "frac": pred_gbs / peak,
-                          "bytes_per_launch": pred_bytes, "us_per_launch": pred_us},
+            "predictor": predictor,
             "kernel_us_per_launch": kernel_us,
             "per_token": {"rows_active": rows_active / K, "rows_loaded": fetched / beta / K,
                           "rows_moved": rows_moved / K},
@@ -413,16 +453,24 @@ def run_ours(args):
                                    f"{Wm} warm-up tokens"},
             "clocks": clock_info,
         }
-        if args.cpu_baseline:
-            out["cpu_baseline"] = cpu_baseline(cfg, layers, X, args.cpu_layers, args.cpu_tokens,
+        out["host_link_whole_token"] = {
+            "achieved": fetched / K / (ms_total / K) / 1e6, "peak": link_peak, "unit": "GB/s",
+            "frac": fetched / K / (ms_total / K) / 1e6 / link_peak,
+            "what": "bundle bytes fetched per token over the token's time: the share of a token "
+                    "during which the host link is busy at its measured peak"}
+        if detail and args.cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(cfg, layers, X, args.cpu_seconds,
                                                _gate_setup(args), args.append_first)
-        print(json.dumps(out), flush=True)
+    else:
+        out = None
     B.lif_graph_destroy(graph)
     for l in layers:
         l.close()
-    del exchange
-    if dist.is_initialized():
-        dist.destroy_process_group()
+    del exchange, layers, handles, graph, X
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return out
 
 
 def run_kernel_loop(args):
@@ -557,30 +605,31 @@ def _oracle_token(ol, x_np, O, gate=(0, 0, 0.0)):
                           activation=act, threshold=thr, gated=gm == 1)
 
 
-def cpu_baseline(cfg, layers, X, n_layers, n_tokens, gate=(0, 0, 0.0), append_first=False):
-    """The oracle, as it stands, on a bounded sample: the first n_layers layers over the first
-    n_tokens tokens; tokens/s scaled to the full stack by layers."""
+def cpu_baseline(cfg, layers, X, seconds, gate=(0, 0, 0.0), append_first=False):
+    """The oracle, as it stands, on a bounded sample of the same workload: EVERY layer of the
+    stack (a few layers alone stay in the host caches and run almost twice as fast per layer),
+    as many tokens as fit about `seconds` of CPU time after window_k + 1 warm-up tokens."""
     from oracle import lif_oracle as O
-    n_layers = min(n_layers, len(layers))
-    n_tokens = min(n_tokens, X.shape[0])          # a short run has fewer tokens than the sample asks for
     tensors = [({"A": l.keep["pred_A"], "B": l.keep["pred_B"], "c": l.keep["pred_c"],
                  "bundles": l.keep["host_bundles"], "bias_up": l.keep["bias_up"],
                  "gate": l.keep["gate"]}, l.capacity)
-               for l in layers[:n_layers]]
+               for l in layers]
     ol = _oracle_layers(cfg, tensors, O, gate, append_first)
-    xs = X[:n_tokens].cpu().numpy()
-    warm = max(0, min(cfg.window_k + 1, n_tokens - 1))
+    xs = X.cpu().numpy()
+    warm = max(1, min(cfg.window_k + 1, xs.shape[0] - 1))
     for t in range(warm):
         _oracle_token(ol, xs[t], O, gate)
     t0 = time.perf_counter()
-    for t in range(warm, n_tokens):
+    done = 0
+    for t in range(warm, xs.shape[0]):
         _oracle_token(ol, xs[t], O, gate)
+        done += 1
+        if time.perf_counter() - t0 > seconds:
+            break
     dt = time.perf_counter() - t0
-    per_layer_step = dt / ((n_tokens - warm) * n_layers)
-    return {"value": 1.0 / (per_layer_step * cfg.n_layers), "unit": UNIT, "cores": _oracle_threads(),
-            "kind": "oracle",
-            "sample": f"layers 0..{n_layers - 1} of {cfg.n_layers}, tokens {warm}..{n_tokens - 1} after "
-                      f"{warm} warm-up tokens; per-layer time x {cfg.n_layers}"}
+    return {"value": done / dt, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
+            "sample": f"all {len(layers)} layers, tokens {warm}..{warm + done - 1} after {warm} warm-up "
+                      f"tokens ({dt:.1f} s of CPU time)"}
 
 
 def run_reference(args):
@@ -625,11 +674,138 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
         "steps": K, "warmup": Wm, "ms_per_step": dt / K * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: {L} of {cfg.n_layers} layers, CPU oracle (numpy, float64)"},
+        "config": {"workload": workload_string(cfg, cfg.n_layers if not args.layers else L, args.gate,
+                                               gate[0], gate[2]),
+                   "arm": "CPU oracle (numpy, float64)" + ("" if L == (args.layers or cfg.n_layers) else
+                          f": {L} of {cfg.n_layers} layers timed, tokens/s scaled by layers")},
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{L} of {cfg.n_layers} layers, every timed token"},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }), flush=True)
+
+
+def run_stub(args):
+    """Stand-in arm without a device, for testing the multi-rank plumbing on CPU: every rank
+    'decodes' its K tokens by sleeping (1 + rank) ms per token, the ranks meet at a barrier, the
+    slowest rank's time is taken, and rank 0 prints the line with the whole-job rate."""
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    for _ in range(args.warmup):
+        time.sleep(0.001)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.001 * (1 + rank))
+    ms = (time.perf_counter() - t0) * 1e3
+    if world > 1:
+        dist.barrier()
+    ms_slowest = max_over_ranks(ms, world, "cpu")
+    if rank == 0:
+        print(json.dumps({"impl": "stub", "metric": METRIC, "unit": UNIT, "n_gpus": world,
+                          "value": whole_job_tokens_per_s(args.steps, world, ms_slowest),
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_slowest / args.steps,
+                          "higher_is_better": True, "scaling": "weak", "data": "none",
+                          "config": {"workload": "stub", "parallelism": "independent sequence per rank"}}),
+              flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def launch_ranks(args):
+    """`--gpus N` with N > 1 outside torchrun: start N ranks of this script on this node (one per
+    GPU, rendezvous on 127.0.0.1) and pass their output through.  Returns the exit code."""
+    import socket
+    if args.impl == "ours":
+        import torch
+        have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+        if have < args.gpus:
+            print(f"bench.py: --gpus {args.gpus} needs {args.gpus} CUDA devices on this node, found {have}",
+                  file=sys.stderr)
+            return 2
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")            # the communicator's set-up goes to stderr
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
+def run_floors(args):
+    """Reference points that the kernels are judged against, measured with calls the library
+    exports: the host link (copy engine, and a kernel reading mapped host memory), and what a
+    kernel that does nothing but read a few MB of HBM achieves per launch when it is launched the
+    way the decode step launches its kernels (a graph of dependent launches, L2-cold)."""
+    import torch
+    from paper_2312_11514_b200 import binding as B
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    st = torch.cuda.Stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    out = {"mode": "floors", "hbm_peak_GBs": _peaks()[0], "hbm_peak_kind": _peaks()[1]}
+
+    def timed(fn, reps):
+        with torch.cuda.stream(st):
+            fn()
+            e0.record(st)
+            for _ in range(reps):
+                fn()
+            e1.record(st)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / reps          # us
+
+    # ---- host link
+    nb = 1 << 30
+    hbuf = torch.empty(nb, dtype=torch.uint8, pin_memory=True)
+    dbuf = torch.empty(nb, dtype=torch.uint8, device=dev)
+    best = min(timed(lambda: dbuf.copy_(hbuf, non_blocking=True), 1) for _ in range(5))
+    link = {"cudaMemcpyAsync_1GiB_GBs": nb / best / 1e3}
+    best = min(timed(lambda: B.lif_probe_host_read(hbuf, dbuf, nb, 16384, st), 1) for _ in range(3))
+    link["kernel_read_1GiB_16KiB_chunks_GBs"] = nb / best / 1e3
+    for mb in (1, 2, 4, 8):
+        n = mb << 20
+        offs = [(i * 97 % 509) * (2 << 20) for i in range(24)]      # different regions: no reuse
+        it = iter(range(10 ** 9))
+        us = timed(lambda: B.lif_probe_host_read(hbuf[offs[next(it) % 24]:], dbuf, n, 16384, st), 24)
+        it = iter(range(10 ** 9))
+        us_cp = timed(lambda: dbuf[:n].copy_(hbuf[offs[next(it) % 24]:][:n], non_blocking=True), 24)
+        link[f"{mb}MiB_per_launch"] = {"kernel_read_us": us, "kernel_read_GBs": n / us / 1e3,
+                                       "cudaMemcpyAsync_us": us_cp, "cudaMemcpyAsync_GBs": n / us_cp / 1e3}
+    out["host_link"] = link
+    del hbuf
+
+    # ---- HBM streaming read per launch, launched like the decode step's kernels
+    pool = torch.empty(2 << 30, dtype=torch.uint8, device=dev)       # 2 GiB: every launch is L2-cold
+    pool.zero_()
+    sink = torch.zeros(16, dtype=torch.uint8, device=dev)
+    reads = {}
+    for mb in (1, 2, 4, 6, 8, 16, 64):
+        n = mb << 20
+        n_regions = min(64, (2 << 30) // n)
+        for ctas in (1, 2, 4):
+            for pdl in (1, 0):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=st):
+                    for i in range(32):
+                        off = (i * 37 % n_regions) * n
+                        B.lif_probe_device_read(pool[off:], n, sink, ctas, bool(pdl), st)
+                us = timed(g.replay, 10) / 32
+                reads[f"{mb}MiB_{ctas}cta_per_sm_{'dependent' if pdl else 'plain'}"] = {
+                    "us_per_launch": us, "GBs": n / us / 1e3, "frac_of_hbm_peak": n / us / 1e3 / out["hbm_peak_GBs"]}
+                del g
+    out["hbm_read_per_launch_in_graph"] = reads
+    # the same kernel launched on a stream, one launch at a time (what a graph saves)
+    n = 8 << 20
+    it = iter(range(10 ** 9))
+    us = timed(lambda: B.lif_probe_device_read(pool[(next(it) % 64) * n:], n, sink, 2, True, st), 64)
+    out["hbm_read_8MiB_stream_launches_us"] = us
+    print(json.dumps(out), flush=True)
 
 
 def main():
@@ -637,7 +813,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=16)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "stub"],
+                    help="'stub': no device, for testing the multi-rank plumbing on CPU")
     ap.add_argument("--config", default="opt6p7b")
     ap.add_argument("--layers", type=int, default=None, help="use only the first N layers")
     ap.add_argument("--gate", default="none", choices=sorted(GATE_MODES),
@@ -655,8 +832,12 @@ def main():
                     help="--shard neurons: sum the partial outputs with an NCCL all-reduce, or with "
                          "lif_sum_peer_outputs reading the peers' partials from peer-mapped memory")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
-    ap.add_argument("--cpu-layers", type=int, default=2)
-    ap.add_argument("--cpu-tokens", type=int, default=30)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0,
+                    help="CPU time the oracle baseline may take after its warm-up tokens")
+    ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
+                    help="leave out the reduced-length runs of the other configurations")
+    ap.add_argument("--floors", action="store_true",
+                    help="measure the reference points (host link, HBM read per launch) and exit")
     ap.add_argument("--kernel-loop", default=None,
                     help="profiling aid: after the warm-up tokens launch this kernel once per layer "
                          "(predict_z, predict_scores, fetch, ffn_active, ffn_hits, ffn_new, ffn_sum; "
@@ -667,7 +848,13 @@ def main():
     if args.warmup < 3:     # fewer than 3 warm-up steps would make the timing invalid: do 3
         print(f"bench.py: --warmup {args.warmup} raised to 3", file=sys.stderr)
         args.warmup = 3
-    if args.sweep_k:
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(launch_ranks(args))
+    if args.impl == "stub":
+        run_stub(args)
+    elif args.floors:
+        run_floors(args)
+    elif args.sweep_k:
         run_sweep_k(args)
     elif args.kernel_loop:
         run_kernel_loop(args)

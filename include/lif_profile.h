@@ -73,7 +73,9 @@ enum {
   LIF_KERNEL_FFN_ACTIVE = 3, /* sparse FFN kernel over all active rows */
   LIF_KERNEL_FFN_HITS = 4,   /* ... over the active rows that were already cached */
   LIF_KERNEL_FFN_NEW = 5,    /* ... over the rows brought in this step */
-  LIF_KERNEL_FFN_SUM = 6     /* partial-sum kernel over the hits + new partials */
+  LIF_KERNEL_FFN_SUM = 6,    /* partial-sum kernel over the hits + new partials */
+  LIF_KERNEL_FFN_CACHE = 7   /* sparse FFN kernel over every cached row, [0, num_used): what
+                                Section 3.3 item 3 writes (matrix[:num_rows]) */
 };
 lif_status lif_profile_launch(lif_layer* layer, int32_t kernel, const void* dev_x, float* dev_y,
                               void* stream);
@@ -83,6 +85,14 @@ lif_status lif_profile_launch(lif_layer* layer, int32_t kernel, const void* dev_
  * pieces; chunk_bytes a multiple of 16, bytes a multiple of chunk_bytes).  Enqueue only. */
 lif_status lif_probe_host_read(const void* host_src, void* dev_dst, size_t bytes,
                                size_t chunk_bytes, void* stream);
+
+/* Reference point for kernels that read a few megabytes per launch: a kernel that does nothing
+ * but read `bytes` (a multiple of 16) of device memory with 16-byte loads from ctas_per_sm CTAs
+ * on every SM (1..8), launched with (dependent_launch != 0) or without the programmatic
+ * dependent-launch attribute the decode step's kernels use.  dev_sink: 16 bytes of device memory
+ * that are (practically never) written.  Enqueue only. */
+lif_status lif_probe_device_read(const void* dev_src, size_t bytes, void* dev_sink,
+                                 int32_t ctas_per_sm, int32_t dependent_launch, void* stream);
 
 #ifdef __cplusplus
 }

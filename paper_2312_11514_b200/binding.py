@@ -23,12 +23,13 @@ EXPORTS = [
     "lif_status_str", "lif_workspace_bytes", "lif_create_layer", "lif_destroy_layer", "lif_reset",
     "lif_predict", "lif_window_update", "lif_fetch_bundles", "lif_sparse_ffn", "lif_decode_step",
     "lif_decode_token_host", "lif_get_lists", "lif_get_stats", "lif_clear_status",
-    "lif_probe_host_read", "lif_timing_enable", "lif_timing_read",
+    "lif_probe_host_read", "lif_probe_device_read", "lif_timing_enable", "lif_timing_read",
     "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
     "lif_sparse_ffn_static", "lif_sparse_ffn_static_status", "lif_set_tuning", "lif_profile_launch",
     "lif_read_state", "lif_snapshot_bytes", "lif_snapshot", "lif_restore", "lif_sum_peer_outputs",
 ]
-KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ffn_new", "ffn_sum")
+KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ffn_new", "ffn_sum",
+           "ffn_cache")
 (TUNE_DEPENDENT_LAUNCH, TUNE_SPLIT_FFN, TUNE_FETCH_CTAS, TUNE_FFN_CTAS, TUNE_FFN_STAGES,
  TUNE_BATCHED_COLUMN_PARTS, TUNE_FUSED_PLAN, TUNE_BATCHED_UP_TWO_CTAS, TUNE_FUSED_FETCH_FFN,
  TUNE_WAIT_POLLS) = range(10)
@@ -96,6 +97,7 @@ def lib() -> C.CDLL:
         "lif_get_stats": [vp, C.POINTER(Stats)],
         "lif_clear_status": [vp, vp],
         "lif_probe_host_read": [vp, vp, sz, sz, vp],
+        "lif_probe_device_read": [vp, sz, vp, i32, i32, vp],
         "lif_graph_capture": [C.POINTER(vp), i32, vp, vp, vp, vp, C.POINTER(vp)],
         "lif_graph_launch": [vp, vp],
         "lif_graph_launch_host": [vp, vp, vp, vp],
@@ -227,6 +229,13 @@ def lif_get_stats(layer: int) -> Stats:
 
 def lif_clear_status(layer: int, stream=None) -> None:
     _check(lib().lif_clear_status(layer, _stream(stream)), "lif_clear_status")
+
+
+def lif_probe_device_read(dev_src, nbytes: int, dev_sink, ctas_per_sm: int = 2,
+                          dependent_launch: bool = True, stream=None) -> None:
+    _check(lib().lif_probe_device_read(_ptr(dev_src), nbytes, _ptr(dev_sink), ctas_per_sm,
+                                       1 if dependent_launch else 0, _stream(stream)),
+           "lif_probe_device_read")
 
 
 def lif_probe_host_read(host_src, dev_dst, nbytes: int, chunk_bytes: int, stream=None) -> None:

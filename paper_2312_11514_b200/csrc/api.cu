@@ -461,6 +461,7 @@ lif_status lif_profile_launch(lif_layer* L, int32_t kernel, const void* dev_x, f
     case LIF_KERNEL_FFN_ACTIVE:
     case LIF_KERNEL_FFN_HITS:
     case LIF_KERNEL_FFN_NEW:
+    case LIF_KERNEL_FFN_CACHE:
       e = launch_one(L, kernel, (const __half*)dev_x, dev_y, st);
       break;
     default:
@@ -679,6 +680,21 @@ lif_status lif_probe_host_read(const void* host_src, void* dev_dst, size_t bytes
     return LIF_ERR_CUDA;
   return launch_probe(alias, dev_dst, bytes, chunk_bytes, n_sm, (cudaStream_t)stream) ==
                  cudaSuccess
+             ? LIF_OK
+             : LIF_ERR_CUDA;
+}
+
+lif_status lif_probe_device_read(const void* dev_src, size_t bytes, void* dev_sink,
+                                 int32_t ctas_per_sm, int32_t dependent_launch, void* stream) {
+  if (!dev_src || !dev_sink || !bytes || bytes % 16 || ctas_per_sm < 1 || ctas_per_sm > 8)
+    return LIF_ERR_INVALID_ARG;
+  if (!aligned(dev_src, 16) || !aligned(dev_sink, 16)) return LIF_ERR_ALIGNMENT;
+  int dev = 0, n_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return LIF_ERR_CUDA;
+  return launch_probe_read(dev_src, bytes, dev_sink, n_sm * ctas_per_sm, dependent_launch != 0,
+                           (cudaStream_t)stream) == cudaSuccess
              ? LIF_OK
              : LIF_ERR_CUDA;
 }

@@ -277,6 +277,33 @@ probe_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n_chunk
   gather_rows(src, dst, nullptr, nullptr, n_chunks, chunk_vec);
 }
 
+// Streaming read of `n_vec` 16-byte vectors of device memory, eight loads in flight per thread,
+// nothing else: the time such a launch takes is what any kernel that has to read that many bytes
+// after its predecessor has finished can at best approach.  The xor of everything read goes to
+// `sink` so that the loads cannot be dropped.
+__global__ void __launch_bounds__(kThreads)
+probe_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint4* __restrict__ sink) {
+  pdl_wait();
+  pdl_trigger();
+  uint4 acc = make_uint4(0, 0, 0, 0);
+  const size_t stride = (size_t)gridDim.x * kThreads;
+  size_t v = (size_t)blockIdx.x * kThreads + threadIdx.x;
+  for (; v + 7 * stride < n_vec; v += 8 * stride) {
+    uint4 q[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[i] = ld_stream16(src + v + i * stride);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      acc.x ^= q[i].x; acc.y ^= q[i].y; acc.z ^= q[i].z; acc.w ^= q[i].w;
+    }
+  }
+  for (; v < n_vec; v += stride) {
+    const uint4 q = ld_stream16(src + v);
+    acc.x ^= q.x; acc.y ^= q.y; acc.z ^= q.z; acc.w ^= q.w;
+  }
+  if ((acc.x ^ acc.y ^ acc.z ^ acc.w) == 0x9e3779b9u) *sink = acc;   // practically never
+}
+
 // Refill after a restore: cache row s <- bundle pointers[s] for s < num_used.
 __global__ void __launch_bounds__(kThreads)
 refill_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
@@ -343,6 +370,12 @@ cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cuda
              : early == kEarlyLists ? fetch_ffn_kernel<LIF_GATE_NONE, kEarlyLists>
                                     : fetch_ffn_kernel<LIF_GATE_NONE, kEarlyNone>;
   return launch_k(kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl, a);
+}
+
+cudaError_t launch_probe_read(const void* dev_src, size_t bytes, void* dev_sink, int grid, int pdl,
+                              cudaStream_t st) {
+  return launch_k(probe_read_kernel, dim3(grid), dim3(kThreads), 0, st, pdl, (const uint4*)dev_src,
+                  bytes / 16, (uint4*)dev_sink);
 }
 
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,

@@ -397,6 +397,9 @@ cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cuda
               ? ffn_args(L, x, L->load_slots, cnt + LIF_CNT_N_LOAD, nullptr, p1, 0)
               : ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
       break;
+    case LIF_KERNEL_FFN_CACHE:      // every cached row: rows [0, num_used) after a completed step
+      a = ffn_args(L, x, nullptr, cnt + LIF_CNT_NUM_USED, nullptr, p0, 0);
+      break;
     case LIF_KERNEL_FFN_SUM:
       return launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st,
                       L->use_pdl, (const float*)p0, cnt + LIF_CNT_N_HITS, (const float*)p1,

@@ -140,6 +140,8 @@ cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cuda
 cudaError_t launch_refill(lif_layer* L, cudaStream_t st);
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,
                          int grid, cudaStream_t st);
+cudaError_t launch_probe_read(const void* dev_src, size_t bytes, void* dev_sink, int grid, int pdl,
+                              cudaStream_t st);
 // slots == nullptr: rows base[0] .. base[0] + n[0] (base == nullptr: 0)
 cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
                        const int32_t* base, float* y, bool accumulate, cudaStream_t st,

@@ -20,9 +20,7 @@ def _draw(rng):
     r = int(rng.choice([8, 16, 40, 128, 256]))
     k = int(rng.integers(1, 7))
     S = int(rng.choice([1, 1, 1, 2, 3, 5, 8]))
-    # firing rates from 5 % up: with one or two active rows the output can be a single
-    # near-zero pre-activation, where fp32 and float64 differ by more than any relative bound
-    fire = float(rng.choice([0.05, 0.2, 0.5]))
+    fire = float(rng.choice([0.01, 0.02, 0.05, 0.2, 0.5]))
     gate_mode = int(rng.choice([0, 0, 1, 2]))
     act = int(rng.choice([0, 1, 2]))
     append_first = int(rng.integers(0, 2))
@@ -33,7 +31,7 @@ def _draw(rng):
     return cfg, kw
 
 
-@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 4, 5])
 def test_random_configurations(seed):
     rng = np.random.default_rng(1000 + seed)
     for _ in range(12):

@@ -1,8 +1,12 @@
 """The N > 1 path of the benchmark on CPU: two gloo ranks shard by sequence (independent
 replicas, no data-path exchange), time is the slowest rank's, throughput is the whole job's."""
+import json
 import os
 import socket
+import subprocess
 import sys
+
+import pytest
 
 import torch
 import torch.distributed as dist
@@ -134,3 +138,34 @@ def test_neuron_shares_are_equal_multiples_of_eight():
         R.neuron_shard(1024, 2, 2)
     assert R.neuron_shard(1024, 3, 4) == (768, 1024)
     assert R.sum_partial_outputs(torch.ones(2, 4)).tolist() == [[1.0] * 4] * 2   # one device: no-op
+
+
+def test_bench_starts_its_own_ranks_for_gpus_above_one():
+    # `bench.py --gpus 2` outside torchrun starts two ranks itself (here: the device-free stub arm
+    # over gloo); rank 0 prints one line for the whole job, with the slowest rank's time
+    bench = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "bench.py")
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, bench, "--gpus", "2", "--impl", "stub", "--steps", "6", "--warmup", "3"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2 and rec["steps"] == 6 and rec["scaling"] == "weak"
+    # rank 1 sleeps 2 ms per token: the job's time is the slowest rank's, the rate counts both ranks
+    assert rec["ms_per_step"] >= 2.0
+    assert rec["value"] == pytest.approx(2 * 6 / (rec["ms_per_step"] * 6 / 1e3), rel=1e-9)
+    # one rank: no launcher involved, same line shape
+    res1 = subprocess.run([sys.executable, bench, "--gpus", "1", "--impl", "stub", "--steps", "4", "--warmup", "3"],
+                          capture_output=True, text=True, timeout=120, env=env)
+    assert res1.returncode == 0 and json.loads(res1.stdout.splitlines()[-1])["n_gpus"] == 1
+
+
+def test_bench_refuses_more_gpus_than_the_node_has():
+    import torch
+    have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+    bench = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "bench.py")
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, bench, "--gpus", str(have + 2), "--steps", "3"],
+                         capture_output=True, text=True, timeout=120, env=env)
+    assert res.returncode == 2 and "CUDA devices" in res.stderr and not res.stdout.strip()
