@@ -184,6 +184,10 @@ def measure(args, config_name, steps, warmup, rank, world, local, detail):
                            activation_threshold=act_thr, append_first=args.append_first,
                            shard=(rank, world) if sharded else None)
     handles = [l.handle for l in layers]
+    for item in args.tune:                 # launch-shape knobs of include/lif_profile.h
+        key, value = item.split("=")
+        for h in handles:
+            B.lif_set_tuning(h, getattr(B, "TUNE_" + key.upper()), int(value))
     L, S, d = len(layers), cfg.n_streams, cfg.d_model
     X = _inputs(cfg, n_tok, dev, W)
     Y = torch.empty(L, S, d, dtype=torch.float32, device=dev)
@@ -487,6 +491,10 @@ def run_kernel_loop(args):
     layers = R.build_stack(cfg, dev, n_layers=args.layers, gate_mode=gate_mode, activation=activation,
                            activation_threshold=act_thr, append_first=args.append_first)
     handles = [l.handle for l in layers]
+    for item in args.tune:
+        key, value = item.split("=")
+        for h in handles:
+            B.lif_set_tuning(h, getattr(B, "TUNE_" + key.upper()), int(value))
     L, S, d = len(layers), cfg.n_streams, cfg.d_model
     X = _inputs(cfg, args.warmup, dev, W)
     Y = torch.empty(L, S, d, dtype=torch.float32, device=dev)
@@ -836,6 +844,9 @@ def main():
                     help="CPU time the oracle baseline may take after its warm-up tokens")
     ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
                     help="leave out the reduced-length runs of the other configurations")
+    ap.add_argument("--tune", action="append", default=[], metavar="KNOB=VALUE",
+                    help="set a LIF_TUNE_* knob on every layer before capture, e.g. "
+                         "--tune batched_up_whole_rows=0 (repeatable)")
     ap.add_argument("--floors", action="store_true",
                     help="measure the reference points (host link, HBM read per launch) and exit")
     ap.add_argument("--kernel-loop", default=None,
