@@ -32,7 +32,7 @@ UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes of sparse_ffn_kernel, from
 # the ncu capture summarised under profiles/ (set to None when that kernel changes)
-FFN_TRAFFIC_RATIO = 1.005
+FFN_TRAFFIC_RATIO = 1.003
 # fetch_ffn_kernel: bytes read from system memory per bundle byte, same kind of capture
 FETCH_TRAFFIC_RATIO = 1.000
 FALLBACK_HBM_GBS = 6650.0
@@ -430,7 +430,7 @@ def measure(args, config_name, steps, warmup, rank, world, local, detail):
                                     if FFN_TRAFFIC_RATIO and S == 1 and not gate_mode else None,
                          "traffic_how": "dram read+write bytes per algorithmic byte from the ncu capture in "
                                         "profiles/sparse_ffn_kernel_opt6p7b_12layers.md (12 layers, "
-                                        "451-529 rows per launch), scaled by this run's rows per launch",
+                                        "277-463 rows per launch), scaled by this run's rows per launch",
                          "us_per_launch": ffn_us,
                          "bytes_per_launch": ffn_bytes,
                          "how": ("graph of this kernel on every layer, over the rows of the last token "
