@@ -34,7 +34,11 @@ class Layer:
         self.n_streams = n_streams
         self.keep = dict(host_bundles=host_bundles, pred_A=pred_A, pred_B=pred_B, pred_c=pred_c,
                          bias_up=bias_up, bias_down=bias_down, gate=gate)
-        self.cache = torch.zeros(capacity, n_vec * d_model, dtype=torch.float16, device=self.device)
+        # One guard row past the cache and a guard block past the workspace, filled with a bit
+        # pattern no kernel writes: `guards_intact()` tells whether anything ran past the end.
+        self._cache_all = torch.zeros(capacity + 1, n_vec * d_model, dtype=torch.float16, device=self.device)
+        self._cache_all[capacity].view(torch.int16).fill_(self._GUARD)
+        self.cache = self._cache_all[:capacity]
         shape = dict(d_model=d_model, d_ff=d_ff, rank=rank, window_k=window_k, capacity=capacity,
                      n_streams=n_streams, threshold_logit=threshold_logit, ffn_mode=ffn_mode,
                      activation=activation, activation_threshold=activation_threshold,
@@ -42,7 +46,9 @@ class Layer:
                      append_first=append_first)
         self.spec_keep, self.gate_mode = spec_keep, gate_mode
         nbytes = B.lif_workspace_bytes(B.make_desc(**shape))
-        self.workspace = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
+        self._workspace_all = torch.zeros(nbytes + 256, dtype=torch.uint8, device=self.device)
+        self._workspace_all[nbytes:].fill_(self._GUARD & 0xFF)
+        self.workspace = self._workspace_all[:nbytes]
         with torch.cuda.device(self.device):
             self.handle = B.lif_create_layer(B.make_desc(
                 **shape, host_bundles=host_bundles, pred_A=pred_A, pred_B=pred_B, pred_c=pred_c,
@@ -51,6 +57,16 @@ class Layer:
             torch.cuda.synchronize()   # the reset ran on the default stream
         self._lists = B.lif_get_lists(self.handle)
         self.counts = self._view("counts", B.CNT_LEN)
+
+    _GUARD = 0x7B7B
+
+    def guards_intact(self) -> bool:
+        """True while the row after the cache and the block after the workspace still hold the
+        pattern they were created with (synchronises)."""
+        torch.cuda.synchronize(self.device)
+        row_ok = bool((self._cache_all[self.capacity].view(torch.int16) == self._GUARD).all())
+        ws_ok = bool((self._workspace_all[self.workspace.numel():] == (self._GUARD & 0xFF)).all())
+        return row_ok and ws_ok
 
     def _view(self, name: str, n: int, dtype=torch.int32) -> torch.Tensor:
         off = getattr(self._lists, name) - self.workspace.data_ptr()
@@ -83,9 +99,11 @@ class Layer:
 
     def close(self) -> None:
         if getattr(self, "handle", None):
-            torch.cuda.synchronize(self.device)
+            intact = self.guards_intact()
             B.lif_destroy_layer(self.handle)
             self.handle = None
+            if not intact:
+                raise RuntimeError("a kernel wrote past the end of the cache or of the workspace")
 
     def __del__(self):
         try:

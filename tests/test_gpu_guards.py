@@ -156,3 +156,22 @@ def test_restore_refuses_a_damaged_snapshot_on_the_host():
     B.lif_decode_step(gpu.handle, X[4], y)
     P.check_decode_step(gpu, ora, X[4].cpu().numpy(), y)
     gpu.close()
+
+
+def test_guard_row_and_guard_block_survive_a_run_that_fills_the_cache():
+    # a threshold below every score makes all neurons active: the first step loads d_ff bundles
+    # into a cache of exactly d_ff rows, every list of the workspace is filled to its last
+    # element, and nothing is written past the cache or the workspace
+    cfg = W.LifConfig("full", 1, 264, 512, 16, 4, 1, 4, 0.30, 0.3, 0.5, 0.6, 5)
+    gpu, ora = P.make_layer_pair(cfg, 0, capacity=cfg.d_ff, theta=-1e30, b_down=True)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(1, cfg.d_model, dtype=torch.float32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for t in range(cfg.steps):
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
+        assert lists["num_used"] == cfg.d_ff and len(lists["active_slots"]) == cfg.d_ff
+        assert gpu.guards_intact()
+    assert len(gpu.lists()["hit_slots"]) == cfg.d_ff
+    gpu.close()          # raises if a guard was touched
