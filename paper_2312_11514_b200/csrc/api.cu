@@ -313,6 +313,10 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   // With append_first the row moves and the bundle writes touch different rows, so given a
   // second stream the moves leave the critical chain (they only precede the cached rows' FFN).
   const bool moves_aside = L->desc.append_first && sf != sc;
+  // The fetch kernel can watch the predictor when it directly follows the window kernel (or the
+  // row moves behind it) on the compute stream: two streams, one input stream, fused fetch.
+  L->watch_chain = sf != sc && L->use_pdl && L->split_ffn && L->desc.n_streams == 1 && L->fused_fetch &&
+                   fetch_ffn_supported(L) && fetch_ffn_can_watch(L);
   if (L->fused_plan) {
     ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev, 0) == cudaSuccess;
     ok = ok && launch_window_plan(L, sc, ev, !moves_aside) == cudaSuccess;
@@ -322,9 +326,11 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   }
   if (L->split_ffn && L->desc.n_streams == 1) {
     ok = ok && launch_fetch_and_ffn_split(L, x, dev_y, sc, sf, ev, moves_aside) == cudaSuccess;
+    L->watch_chain = 0;
     if (!ok) cudaGetLastError();
     return ok ? LIF_OK : LIF_ERR_CUDA;
   }
+  L->watch_chain = 0;
   if (sf != sc) {
     ok = ok && cudaEventRecord(L->ev_plan, sc) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(sf, L->ev_plan, 0) == cudaSuccess;

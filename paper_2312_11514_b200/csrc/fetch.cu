@@ -106,9 +106,10 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   if (kEarlyT == kEarlyWatch) {
     // Resident while the score kernel may still be running (all of its CTAs are: it released
     // the window kernel, which released this one, only after every one of them had started).
-    // One thread polls the count of finished tiles.  The count was cleared by this step's first
-    // predictor stage; a count beyond the tiles means other launches of the score kernel came
-    // between and nothing can be told from it.  Whatever the outcome, no result depends on it:
+    // One thread polls the predictor's count of written mask words.  The count was cleared
+    // before this step's predictor ran (by its first stage, or by the previous step's last sum);
+    // a count beyond the total means other launches of the predictor came between and nothing
+    // can be told from it.  Whatever the outcome, no result depends on it:
     // without the count the kernel simply waits for its predecessors like kEarlyNone.
     if (tid == 0) {
       int ok = 0;
@@ -334,6 +335,11 @@ bool fetch_ffn_supported(const lif_layer* L) {
          D.d_model <= kFusedChunks * kThreads * 8 && L->fetch_grid == L->ffn_grid;
 }
 
+// The mask-driven forms scan at most four mask words per thread.
+bool fetch_ffn_can_watch(const lif_layer* L) {
+  return (L->desc.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32) <= 4 * kThreads;
+}
+
 // Fetch of this step's new rows fused with their FFN terms; partials go to `partial`
 // ([fetch_grid][d_model], CTA c < min(grid, n_load) writes row c).
 cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cudaStream_t st,
@@ -355,13 +361,13 @@ cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cuda
   a.new_mask_words = L->new_mask_words;
   a.nwords = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
   a.tiles_done = L->counts + CNT_TILES_DONE;
-  a.n_tiles = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);   // counted per word pair
-  if (early >= kEarlyMask && a.nwords > 4 * kThreads) early = kEarlyNone;
-  // only the low-rank predictor counts its tiles
-  if (early == kEarlyWatch && D.gate_mode == LIF_GATE_RESIDENT) early = kEarlyMask;
+  // what the predictor counts: word pairs (low-rank score kernel) or CTAs (gate kernel)
+  a.n_tiles = D.gate_mode == LIF_GATE_RESIDENT ? gate_predict_ctas(D) : a.nwords;
+  if (early >= kEarlyMask && !fetch_ffn_can_watch(L)) early = kEarlyNone;
   void (*kernel)(FetchFfnArgs);
   if (D.gate_mode == LIF_GATE_RESIDENT)
-    kernel = early == kEarlyMask    ? fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyMask>
+    kernel = early == kEarlyWatch   ? fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyWatch>
+             : early == kEarlyMask  ? fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyMask>
              : early == kEarlyLists ? fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyLists>
                                     : fetch_ffn_kernel<LIF_GATE_RESIDENT, kEarlyNone>;
   else

@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(kSumThreads)
 ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
                   const float* __restrict__ p1, const int32_t* __restrict__ n1, int G,
                   const __half* __restrict__ b_down, int b_period, float* __restrict__ y, int d,
-                  int accumulate, int n_cap) {
+                  int accumulate, int n_cap, int* clear_after_wait) {
   __shared__ float4 red[32][kSumCols];
   const int tid = threadIdx.x;
   const int c4 = tid & (kSumCols - 1), gs = tid / kSumCols;
@@ -246,6 +246,9 @@ ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
   }
   pdl_wait();
   pdl_trigger();
+  // every earlier kernel of the step is complete: the predictor's count of written mask words
+  // has no watcher left and is cleared for the next step
+  if (clear_after_wait && blockIdx.x == 0 && tid == 0) *clear_after_wait = 0;
   // counts as the kernels that wrote the partials clamp them: [0, n_cap]
   const int v0 = min(G, max(0, min(*n0, n_cap))), v1 = p1 ? min(G, max(0, min(*n1, n_cap))) : 0;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -371,7 +374,7 @@ cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, cons
     e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st, L->use_pdl,
                  (const float*)L->y_partial, n, (const float*)nullptr, (const int32_t*)nullptr,
                  L->ffn_grid, (const __half*)D.dev_bias_down, d, y + (size_t)s * d, d,
-                 accumulate ? 1 : 0, D.capacity);
+                 accumulate ? 1 : 0, D.capacity, (int*)nullptr);
     if (e != cudaSuccess) return e;
   }
   if (ev) tm_record(ev[9], st);
@@ -404,7 +407,7 @@ cudaError_t launch_one(lif_layer* L, int kernel, const __half* x, float* y, cuda
       return launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0, st,
                       L->use_pdl, (const float*)p0, cnt + LIF_CNT_N_HITS, (const float*)p1,
                       cnt + LIF_CNT_N_LOAD, L->ffn_grid, (const __half*)D.dev_bias_down, d, y, d, 0,
-                      D.capacity);
+                      D.capacity, (int*)nullptr);
     default:
       return cudaErrorInvalidValue;
   }
@@ -417,7 +420,7 @@ cudaError_t launch_partial_sum(lif_layer* L, const float* partial, const int32_t
   return launch_k(ffn_reduce_kernel, dim3((width / 4 + kSumCols - 1) / kSumCols),
                   dim3(kSumThreads), 0, st, L->use_pdl, partial, n, (const float*)nullptr,
                   (const int32_t*)nullptr, partitions, (const __half*)L->desc.dev_bias_down,
-                  L->desc.d_model, y, width, 0, L->desc.capacity);
+                  L->desc.d_model, y, width, 0, L->desc.capacity, (int*)nullptr);
 }
 
 // Fetch + FFN of a single-stream decode step.  The critical chain stays on `st` with dependent
@@ -455,7 +458,7 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
                      : ffn_args(L, x, nullptr, cnt + LIF_CNT_N_LOAD, cnt + LIF_CNT_NUM_KEPT, p1, 0);
   if (L->fused_fetch && fetch_ffn_supported(L)) {
     // one kernel brings the new rows in and adds their FFN terms (CTA partials in p1)
-    if ((e = launch_fetch_ffn(L, x, p1, st, moves_aside ? kEarlyWatch : kEarlyLists)) != cudaSuccess) return e;
+    if ((e = launch_fetch_ffn(L, x, p1, st, L->watch_chain ? kEarlyWatch : (moves_aside ? kEarlyMask : kEarlyLists))) != cudaSuccess) return e;
     if (ev) tm_record(ev[6], st);
   } else {
     if ((e = launch_fetch(L, st)) != cudaSuccess) return e;
@@ -467,7 +470,8 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
   if (fork && (e = cudaStreamWaitEvent(st, L->ev_fetch, 0)) != cudaSuccess) return e;
   e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0,
                st, L->use_pdl, (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,
-               (const __half*)D.dev_bias_down, d, y, d, 0, D.capacity);
+               (const __half*)D.dev_bias_down, d, y, d, 0, D.capacity,
+               (int*)(L->counts + CNT_TILES_DONE));
   if (ev) tm_record(ev[9], st);
   return e;
 }
@@ -609,6 +613,6 @@ extern "C" lif_status lif_sparse_ffn_static(const void* dev_matrix, int32_t n_ro
   if (cudaGetLastError() != cudaSuccess) return LIF_ERR_CUDA;
   ffn_reduce_kernel<<<(d_model / 4 + kSumCols - 1) / kSumCols, kSumThreads, 0, st>>>(
       sd.scratch->partial, dev_n_slots, nullptr, nullptr, grid, (const __half*)dev_bias_down,
-      d_model, dev_y, d_model, 0, n_rows);
+      d_model, dev_y, d_model, 0, n_rows, (int*)nullptr);
   return cudaGetLastError() == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
 }

@@ -31,7 +31,7 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
                    float* __restrict__ gate_val, float* __restrict__ logits,
                    uint32_t* mask_words, int* ticket, int* __restrict__ active_idx,
                    int* __restrict__ n_active, int compact, int nwords,
-                   const int32_t* __restrict__ slot_of, uint32_t* new_mask_words) {
+                   const int32_t* __restrict__ slot_of, uint32_t* new_mask_words, int* tiles_done) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* xs = reinterpret_cast<uint4*>(smem_raw);          // [S][d / 8]
   __shared__ int act_flag[kGateTile];     // bit 0: active, bit 1: active and not cached yet
@@ -134,6 +134,8 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
         reinterpret_cast<uint8_t*>(mask_words)[blockIdx.x] = (uint8_t)m;
         reinterpret_cast<uint8_t*>(new_mask_words)[blockIdx.x] = (uint8_t)mn;
       }
+      // count this CTA's mask bits as written (release), for a fetch kernel that watches
+      asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(tiles_done) : "memory");
     }
   }
   if (!compact) return;     // the consumer reads the bit mask itself
@@ -156,10 +158,13 @@ cudaError_t launch_gate_s(lif_layer* L, const __half* x, float* logits, int32_t*
                   (const __half*)D.dev_gate, (const __half*)D.dev_bias_up, theta, D.d_model,
                   D.d_ff, L->gate_val, logits, L->mask_words,
                   (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
-                  (D.d_ff + 31) / 32, (const int32_t*)L->slot_of, L->new_mask_words);
+                  (D.d_ff + 31) / 32, (const int32_t*)L->slot_of, L->new_mask_words,
+                  (int*)(L->counts + CNT_TILES_DONE));
 }
 
 }  // namespace
+
+int gate_predict_ctas(const lif_layer_desc& D) { return (D.d_ff + kGateTile - 1) / kGateTile; }
 
 cudaError_t launch_gate_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
                                 int32_t* n_active, cudaStream_t st, cudaEvent_t* ev, int compact) {

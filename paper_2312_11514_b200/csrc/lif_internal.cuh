@@ -79,6 +79,8 @@ struct lif_layer {
   int fetch_grid;     // CTAs of the fetch kernel
   int move_grid;
   unsigned wait_polls; // poll limit of the first wait on each bulk copy in the FFN kernels
+  int watch_chain;    // set by lif_decode_step while it launches a step whose fetch kernel watches
+                      // the predictor: window and row-move kernels release their dependents at entry
   int use_pdl;        // programmatic dependent launch along the compute stream
   int split_ffn;      // decode step: cached rows' FFN overlaps the fetch
   int fused_plan;     // decode step: window update reads the predictor's bit mask directly
@@ -123,9 +125,14 @@ cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = 
                                bool with_moves = true);
 cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act, cudaStream_t st,
                           cudaEvent_t* ev = nullptr, bool with_moves = true);
-cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr);
+// release_early: the row-move kernel releases its dependent at entry (only ahead of a fetch
+// kernel in its watching form)
+cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr,
+                         bool release_early = false);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
 bool fetch_ffn_supported(const lif_layer* L);
+bool fetch_ffn_can_watch(const lif_layer* L);
+int gate_predict_ctas(const lif_layer_desc& D);    // CTAs of the resident-gate predictor
 // early: what the kernel may do before its own dependency wait.  kEarlyLists: the lists were
 // final before the kernel ahead of this one passed its wait, so the first bundle's host loads
 // are issued from them; kEarlyMask: the kernel ahead is the window kernel of the same step and

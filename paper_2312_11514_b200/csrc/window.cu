@@ -425,11 +425,12 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
   __shared__ int holes[kPlanMaxRows];
   __shared__ int newslot[kPlanMaxRows];
   const int tid = threadIdx.x;
-  // With the low-rank predictor the kernel behind this one is released at once: every kernel of
-  // the library waits for its predecessor's completion before it touches that kernel's output,
-  // and the fetch kernel uses the time to become resident and to watch the score kernel finish
-  // (kEarlyWatch).  Otherwise the release follows this kernel's own wait, which is what lets a
-  // dependent read the predictor's masks ahead of its wait (kEarlyMask).
+  // Inside a decode step whose fetch kernel watches the predictor (kEarlyWatch) the kernel behind
+  // this one is released at once: every kernel of the library waits for its predecessor's
+  // completion before it touches that kernel's output, and the fetch kernel uses the time to
+  // become resident and to watch the predictor finish.  Otherwise the release follows this
+  // kernel's own wait, which is what lets a dependent read lists or masks ahead of its wait
+  // (kEarlyLists, kEarlyMask).
   if (a.release_early) pdl_trigger();
   // The window state was last written by this layer's previous step, which is complete before
   // the predictor of this step even starts: the slot side of the bookkeeping (row -> neuron,
@@ -643,9 +644,12 @@ window_plan_kernel(WindowArgs a, const uint32_t* __restrict__ mask_words, int nw
 __global__ void __launch_bounds__(kThreads)
 move_rows_kernel(uint4* __restrict__ cache, const int32_t* __restrict__ move_src,
                  const int32_t* __restrict__ move_dst, const int32_t* __restrict__ counts,
-                 int row_vec) {
+                 int row_vec, int release_early) {
+  // release_early: the kernel behind is the fetch kernel in its watching form, which reads
+  // nothing of this step's lists or rows before its own wait (see window_plan_kernel)
+  if (release_early) pdl_trigger();
   pdl_wait();
-  pdl_trigger();
+  if (!release_early) pdl_trigger();
   const int n = counts[LIF_CNT_N_MOVES];
   for (int j = blockIdx.x; j < n; j += gridDim.x) {
     const uint4* src = cache + (size_t)move_src[j] * row_vec;
@@ -711,17 +715,17 @@ static WindowArgs window_args(lif_layer* L, const int32_t* act, const int32_t* n
   a.keep = D.spec_keep > 0 ? D.spec_keep : 1;
   a.bundle_bytes = 2ull * row_elems(D);
   a.append_first = D.append_first;
-  a.release_early = D.gate_mode != LIF_GATE_RESIDENT;
+  a.release_early = L->watch_chain;
   return a;
 }
 
-cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev) {
+cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev, bool release_early) {
   const lif_layer_desc& D = L->desc;
   cudaError_t e;
   if (ev) tm_record(ev[3], st);
   e = launch_k(move_rows_kernel, dim3(L->move_grid), dim3(kThreads), 0, st, L->use_pdl,
                (uint4*)D.dev_cache, (const int32_t*)L->move_src, (const int32_t*)L->move_dst,
-               (const int32_t*)L->counts, row_elems(D) / 8);
+               (const int32_t*)L->counts, row_elems(D) / 8, release_early ? 1 : 0);
   if (ev) tm_record(ev[4], st);
   return e;
 }
@@ -730,7 +734,7 @@ cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act
                           cudaStream_t st, cudaEvent_t* ev, bool with_moves) {
   cudaError_t e = launch_k(window_update_kernel, dim3(1), dim3(kWindowThreads), 0, st, L->use_pdl,
                            window_args(L, act, n_act));
-  return (e != cudaSuccess || !with_moves) ? e : launch_moves(L, st, ev);
+  return (e != cudaSuccess || !with_moves) ? e : launch_moves(L, st, ev, L->watch_chain != 0);
 }
 
 bool window_plan_supported(const lif_layer_desc& D) {
@@ -744,7 +748,7 @@ cudaError_t launch_window_plan(lif_layer* L, cudaStream_t st, cudaEvent_t* ev, b
   cudaError_t e = launch_k(window_plan_kernel, dim3(1), dim3(kWindowThreads), 0, st, L->use_pdl,
                            window_args(L, L->active_idx, L->n_tmp), (const uint32_t*)L->mask_words,
                            nwords, (int32_t*)L->n_tmp);
-  return (e != cudaSuccess || !with_moves) ? e : launch_moves(L, st, ev);
+  return (e != cudaSuccess || !with_moves) ? e : launch_moves(L, st, ev, L->watch_chain != 0);
 }
 
 }  // namespace lif
