@@ -808,6 +808,25 @@ def run_floors(args):
                     "us_per_launch": us, "GBs": n / us / 1e3, "frac_of_hbm_peak": n / us / 1e3 / out["hbm_peak_GBs"]}
                 del g
     out["hbm_read_per_launch_in_graph"] = reads
+    # ---- streaming through a shared-memory ring of bulk copies (how the FFN kernels bring rows in)
+    rings = {}
+    tmo = torch.zeros(1, dtype=torch.int32, device=dev)
+    nbytes = 160 << 20
+    for chunk, stages, group, ctas, every in (
+            (3584, 48, 16, 1, 0), (7168, 32, 16, 1, 0), (14336, 16, 8, 1, 0), (14336, 12, 4, 1, 0),
+            (28672, 8, 4, 1, 0), (7168, 14, 7, 2, 0), (3584, 14, 7, 4, 0), (16384, 3, 1, 4, 0),
+            (3584, 48, 16, 1, 2), (7168, 32, 16, 1, 2), (3584, 48, 16, 1, 1), (7168, 32, 16, 1, 1),
+            (7168, 28, 14, 1, 2), (14336, 16, 8, 1, 2)):
+        it = iter(range(10 ** 9))
+        us = min(timed(lambda: B.lif_probe_bulk_ring(pool[(next(it) % 12) * nbytes:], nbytes, chunk, stages,
+                                                     group, ctas, every, sink, tmo, st), 1)
+                 for _ in range(5))
+        how = "bulk copies" if every == 0 else ("16-byte async copies" if every == 1 else
+                                                f"every {every}nd stage by 16-byte async copies")
+        rings[f"{chunk}B_x{stages}_refill{group}_{ctas}cta_per_sm_{how}"] = {
+            "us": us, "GBs": nbytes / us / 1e3, "frac_of_hbm_peak": nbytes / us / 1e3 / out["hbm_peak_GBs"]}
+    assert int(tmo.item()) == 0, "a ring probe's wait ran out"
+    out["bulk_copy_ring_160MiB"] = rings
     # the same kernel launched on a stream, one launch at a time (what a graph saves)
     n = 8 << 20
     it = iter(range(10 ** 9))

@@ -94,6 +94,20 @@ lif_status lif_probe_host_read(const void* host_src, void* dev_dst, size_t bytes
 lif_status lif_probe_device_read(const void* dev_src, size_t bytes, void* dev_sink,
                                  int32_t ctas_per_sm, int32_t dependent_launch, void* stream);
 
+/* Reference point for the kernels that stream rows through a ring of bulk copies: every CTA
+ * (ctas_per_sm on every SM, 256 threads) streams an equal share of `bytes` of device memory in
+ * pieces of chunk_bytes (multiple of 16) through a shared-memory ring of `stages` stages,
+ * refilled refill_group stages at a time (stages a multiple of it, at most 256 per group) with
+ * one mbarrier per group and bounded waits.  threads_every = 0: every stage is filled by one bulk copy; n > 0: every n-th
+ * stage is filled by 16-byte asynchronous copies of all threads instead.  The data is only
+ * touched (4 bytes per thread and stage).  dev_timeouts: int32 on the device, incremented by a
+ * CTA whose wait ran out (it then lets its copies land and leaves).  stages * (chunk_bytes + 8)
+ * must fit the shared memory of a CTA.  Enqueue only. */
+lif_status lif_probe_bulk_ring(const void* dev_src, size_t bytes, uint32_t chunk_bytes,
+                               int32_t stages, int32_t refill_group, int32_t ctas_per_sm,
+                               int32_t threads_every, void* dev_sink, int32_t* dev_timeouts,
+                               void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,7 @@ EXPORTS = [
     "lif_status_str", "lif_workspace_bytes", "lif_create_layer", "lif_destroy_layer", "lif_reset",
     "lif_predict", "lif_window_update", "lif_fetch_bundles", "lif_sparse_ffn", "lif_decode_step",
     "lif_decode_token_host", "lif_get_lists", "lif_get_stats", "lif_clear_status",
-    "lif_probe_host_read", "lif_probe_device_read", "lif_timing_enable", "lif_timing_read",
+    "lif_probe_host_read", "lif_probe_device_read", "lif_probe_bulk_ring", "lif_timing_enable", "lif_timing_read",
     "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
     "lif_sparse_ffn_static", "lif_sparse_ffn_static_status", "lif_set_tuning", "lif_profile_launch",
     "lif_read_state", "lif_snapshot_bytes", "lif_snapshot", "lif_restore", "lif_sum_peer_outputs",
@@ -98,6 +98,7 @@ def lib() -> C.CDLL:
         "lif_clear_status": [vp, vp],
         "lif_probe_host_read": [vp, vp, sz, sz, vp],
         "lif_probe_device_read": [vp, sz, vp, i32, i32, vp],
+        "lif_probe_bulk_ring": [vp, sz, C.c_uint32, i32, i32, i32, i32, vp, vp, vp],
         "lif_graph_capture": [C.POINTER(vp), i32, vp, vp, vp, vp, C.POINTER(vp)],
         "lif_graph_launch": [vp, vp],
         "lif_graph_launch_host": [vp, vp, vp, vp],
@@ -236,6 +237,13 @@ def lif_probe_device_read(dev_src, nbytes: int, dev_sink, ctas_per_sm: int = 2,
     _check(lib().lif_probe_device_read(_ptr(dev_src), nbytes, _ptr(dev_sink), ctas_per_sm,
                                        1 if dependent_launch else 0, _stream(stream)),
            "lif_probe_device_read")
+
+
+def lif_probe_bulk_ring(dev_src, nbytes: int, chunk_bytes: int, stages: int, refill_group: int,
+                        ctas_per_sm: int, threads_every: int, dev_sink, dev_timeouts, stream=None) -> None:
+    _check(lib().lif_probe_bulk_ring(_ptr(dev_src), nbytes, chunk_bytes, stages, refill_group,
+                                     ctas_per_sm, threads_every, _ptr(dev_sink), _ptr(dev_timeouts),
+                                     _stream(stream)), "lif_probe_bulk_ring")
 
 
 def lif_probe_host_read(host_src, dev_dst, nbytes: int, chunk_bytes: int, stream=None) -> None:

@@ -705,4 +705,30 @@ lif_status lif_probe_device_read(const void* dev_src, size_t bytes, void* dev_si
              : LIF_ERR_CUDA;
 }
 
+lif_status lif_probe_bulk_ring(const void* dev_src, size_t bytes, uint32_t chunk_bytes,
+                               int32_t stages, int32_t refill_group, int32_t ctas_per_sm,
+                               int32_t threads_every, void* dev_sink, int32_t* dev_timeouts,
+                               void* stream) {
+  if (!dev_src || !dev_sink || !dev_timeouts || !bytes) return LIF_ERR_INVALID_ARG;
+  if (chunk_bytes < 16 || chunk_bytes % 16 || stages < 1 || stages > 256 || refill_group < 1 ||
+      refill_group > stages || stages % refill_group || ctas_per_sm < 1 || ctas_per_sm > 8 ||
+      threads_every < 0)
+    return LIF_ERR_INVALID_ARG;
+  if (!aligned(dev_src, 16) || !aligned(dev_sink, 16) || !aligned(dev_timeouts, 4))
+    return LIF_ERR_ALIGNMENT;
+  int dev = 0, n_sm = 0, max_smem = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+    return LIF_ERR_CUDA;
+  if ((size_t)stages * chunk_bytes + (size_t)stages * 8 > (size_t)max_smem) return LIF_ERR_INVALID_ARG;
+  const int grid = n_sm * ctas_per_sm;
+  const size_t per_cta = bytes / grid / chunk_bytes * chunk_bytes;   // whole chunks, 16-byte aligned
+  if (per_cta == 0) return LIF_ERR_INVALID_ARG;
+  return launch_probe_ring(dev_src, per_cta, chunk_bytes, stages, refill_group, threads_every, grid,
+                           dev_sink, dev_timeouts, (cudaStream_t)stream) == cudaSuccess
+             ? LIF_OK
+             : LIF_ERR_CUDA;
+}
+
 }  // extern "C"

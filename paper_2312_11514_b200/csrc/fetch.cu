@@ -305,6 +305,78 @@ probe_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint4* __restrict
   if ((acc.x ^ acc.y ^ acc.z ^ acc.w) == 0x9e3779b9u) *sink = acc;   // practically never
 }
 
+// Streaming read through a shared-memory ring, the way the FFN kernels bring rows in: CTA c
+// streams its share of `src` in pieces of `chunk` bytes through `stages` stages, refilled `group`
+// stages at a time with one mbarrier per group (bounded waits); the only use of the data is one
+// 4-byte read per thread and stage.  Stage s is filled by one bulk copy when mix_every == 0 or
+// s % mix_every != 0, else by 16-byte asynchronous copies issued by all threads (cp.async, which
+// goes through the load/store path instead of the bulk-copy engine).
+__global__ void __launch_bounds__(kThreads)
+probe_ring_kernel(const unsigned char* __restrict__ src, size_t bytes_per_cta, unsigned chunk,
+                  int stages, int group, int mix_every, uint4* __restrict__ sink,
+                  int32_t* __restrict__ timeouts) {
+  extern __shared__ __align__(128) unsigned char ring[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)stages * chunk);   // one per group
+  const int tid = threadIdx.x;
+  const unsigned char* mine = src + (size_t)blockIdx.x * bytes_per_cta;
+  const int n_chunks = (int)(bytes_per_cta / chunk);
+  const int n_groups = (n_chunks + group - 1) / group;
+  const int ring_groups = stages / group;
+  auto by_threads = [&](int s) { return mix_every > 0 && s % mix_every == 0; };
+  if (tid == 0) {
+    for (int g = 0; g < ring_groups; ++g) {
+      int arrivals = 0;                       // per stage: one (bulk copy or skip) or one per thread
+      for (int s = g * group; s < (g + 1) * group; ++s) arrivals += by_threads(s) ? kThreads : 1;
+      mbar_init(bars + g, arrivals);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  pdl_wait();
+  pdl_trigger();
+  __syncthreads();
+  auto fill_group = [&](int g) {              // chunks of group g -> ring group g % ring_groups
+    uint64_t* bar = bars + g % ring_groups;
+    for (int j = 0; j < group; ++j) {
+      const int c = g * group + j, s = (g % ring_groups) * group + j;
+      const bool live = c < n_chunks;
+      if (by_threads(s)) {
+        if (live)
+          for (unsigned off = (unsigned)tid * 16; off < chunk; off += kThreads * 16)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(ring + (size_t)s * chunk + off)),
+                         "l"(mine + (size_t)c * chunk + off) : "memory");
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+      } else if (tid == j % kThreads) {
+        if (live) {
+          mbar_expect_tx(bar, chunk);
+          bulk_g2s(ring + (size_t)s * chunk, mine + (size_t)c * chunk, chunk, bar);
+        } else {
+          mbar_arrive(bar);
+        }
+      }
+    }
+  };
+  int issued = 0;                             // groups whose copies have been issued (uniform)
+  for (; issued < min(ring_groups, n_groups); ++issued) fill_group(issued);
+  unsigned acc = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    const int lost = mbar_wait(bars + g % ring_groups, (unsigned)(g / ring_groups) & 1u) ? 0 : 1;
+    for (int j = 0; j < group && g * group + j < n_chunks; ++j)
+      acc ^= *reinterpret_cast<const unsigned*>(ring + (size_t)((g % ring_groups) * group + j) * chunk +
+                                                (tid * 4) % chunk);
+    if (__syncthreads_or(lost)) {             // give up: flag, let what is in flight land, leave
+      if (tid == 0) atomicAdd(timeouts, 1);
+      for (int gg = g + 1; gg < issued; ++gg)
+        mbar_wait(bars + gg % ring_groups, (unsigned)(gg / ring_groups) & 1u);
+      return;
+    }
+    // the generic-proxy reads of this group's stages are done: refill them
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (issued < n_groups) fill_group(issued++);
+  }
+  if (acc == 0x9e3779b9u) *sink = make_uint4(acc, 0, 0, 0);   // practically never
+}
+
 // Refill after a restore: cache row s <- bundle pointers[s] for s < num_used.
 __global__ void __launch_bounds__(kThreads)
 refill_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
@@ -382,6 +454,18 @@ cudaError_t launch_probe_read(const void* dev_src, size_t bytes, void* dev_sink,
                               cudaStream_t st) {
   return launch_k(probe_read_kernel, dim3(grid), dim3(kThreads), 0, st, pdl, (const uint4*)dev_src,
                   bytes / 16, (uint4*)dev_sink);
+}
+
+cudaError_t launch_probe_ring(const void* dev_src, size_t bytes_per_cta, unsigned chunk, int stages,
+                              int group, int mix_every, int grid, void* dev_sink,
+                              int32_t* dev_timeouts, cudaStream_t st) {
+  const size_t smem = (size_t)stages * chunk + (size_t)(stages / group) * 8;
+  cudaError_t e = cudaFuncSetAttribute(probe_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  return launch_k(probe_ring_kernel, dim3(grid), dim3(kThreads), smem, st, 1,
+                  (const unsigned char*)dev_src, bytes_per_cta, chunk, stages, group, mix_every,
+                  (uint4*)dev_sink, dev_timeouts);
 }
 
 cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes, size_t chunk,

@@ -149,6 +149,9 @@ cudaError_t launch_probe(const void* dev_src_alias, void* dev_dst, size_t bytes,
                          int grid, cudaStream_t st);
 cudaError_t launch_probe_read(const void* dev_src, size_t bytes, void* dev_sink, int grid, int pdl,
                               cudaStream_t st);
+cudaError_t launch_probe_ring(const void* dev_src, size_t bytes_per_cta, unsigned chunk, int stages,
+                              int group, int mix_every, int grid, void* dev_sink,
+                              int32_t* dev_timeouts, cudaStream_t st);
 // slots == nullptr: rows base[0] .. base[0] + n[0] (base == nullptr: 0)
 cudaError_t launch_ffn(lif_layer* L, const __half* x, const int32_t* slots, const int32_t* n,
                        const int32_t* base, float* y, bool accumulate, cudaStream_t st,
