@@ -692,6 +692,84 @@ def run_reference(args):
     }), flush=True)
 
 
+def run_file_store(args):
+    """The bundle store in files (the paper's storage tier: reader threads, one read per bundle,
+    uncached where the file system allows) instead of pinned host memory: one JSON line per
+    thread count with tokens/s, the bytes read per token and the rate the reads reached.  The
+    loads are managed on the host, so every layer-step synchronises twice; compare with the same
+    --layers through the default (pinned-memory) path."""
+    import numpy as np
+    import torch
+    from paper_2312_11514_b200 import binding as B
+    from paper_2312_11514_b200 import runtime as R
+    from paper_2312_11514_b200 import workloads as W
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    cfg = W.CONFIGS[args.config]
+    L = args.layers or min(cfg.n_layers, 8)
+    S, d = cfg.n_streams, cfg.d_model
+    K, Wm = args.steps, args.warmup
+    os.makedirs(args.store_dir, exist_ok=True)
+    layers, paths = [], []
+    for l in range(L):
+        full = R.pinned_store(cfg.d_ff, d)
+        w = W.make_layer(cfg, l, device=dev, bundles_out=full)
+        path = os.path.join(args.store_dir, f"lif_bundles_{cfg.name}_{l}.bin")
+        with open(path, "wb") as f:
+            full.numpy().tofile(f)
+            f.flush()
+            os.fsync(f.fileno())
+        paths.append(path)
+        cap = min(cfg.d_ff, W.window_capacity(cfg, w["p"]))
+        staging = torch.zeros(cap, 2 * d, dtype=torch.float16).pin_memory()
+        to = lambda t: t.to(dev).contiguous()
+        layers.append(R.Layer(d_model=d, d_ff=cfg.d_ff, rank=cfg.rank, window_k=cfg.window_k, capacity=cap,
+                              host_bundles=staging, pred_A=to(w["A"]), pred_B=to(w["B"]), pred_c=to(w["c"]),
+                              bias_up=to(w["bias_up"]), n_streams=S, append_first=args.append_first,
+                              staging_rows=cap, device=dev))
+        del full, w
+    X = _inputs(cfg, Wm + K, dev, W)
+    Y = torch.empty(L, S, d, dtype=torch.float32, device=dev)
+    sc = torch.cuda.Stream()
+    try:
+        for n_threads in [int(v) for v in args.store_threads.split(",")]:
+            stores = [B.lif_store_open(p, cfg.d_ff, cfg.bundle_bytes, n_threads, not args.store_cached)
+                      for p in paths]
+            for l in layers:
+                B.lif_reset(l.handle, sc)
+            torch.cuda.synchronize()
+            t0 = None
+            for t in range(Wm + K):
+                if t == Wm:
+                    s0 = [B.lif_store_get_stats(s) for s in stores]
+                    t0 = time.perf_counter()
+                for l in range(L):
+                    B.lif_decode_step_store(layers[l].handle, stores[l], X[t], Y[l], sc)
+            dt = time.perf_counter() - t0
+            s1 = [B.lif_store_get_stats(s) for s in stores]
+            req = sum(b.bytes_requested - a.bytes_requested for a, b in zip(s0, s1))
+            got = sum(b.bytes_read - a.bytes_read for a, b in zip(s0, s1))
+            secs = sum(b.seconds_reading - a.seconds_reading for a, b in zip(s0, s1))
+            reads = sum(b.reads - a.reads for a, b in zip(s0, s1))
+            assert all(B.lif_get_stats(l.handle).status == B.LIF_OK for l in layers)
+            print(json.dumps({
+                "mode": "file_store", "config": cfg.name, "layers": L, "steps": K, "warmup": Wm,
+                "reader_threads": n_threads, "direct_io": bool(s1[0].direct_io),
+                "tokens_per_s_these_layers": K / dt, "ms_per_layer_step": dt / (K * L) * 1e3,
+                "bundle_MB_per_token": req / K / 1e6, "bytes_read_over_requested": got / max(req, 1),
+                "read_GBs_while_reading": req / max(secs, 1e-9) / 1e9,
+                "read_calls_per_s_while_reading": reads / max(secs, 1e-9),
+                "share_of_time_in_reads": secs / dt, "bundle_bytes": cfg.bundle_bytes,
+                "store_dir": args.store_dir}), flush=True)
+            for s in stores:
+                B.lif_store_close(s)
+    finally:
+        for l in layers:
+            l.close()
+        for p in paths:
+            os.remove(p)
+
+
 def run_stub(args):
     """Stand-in arm without a device, for testing the multi-rank plumbing on CPU: every rank
     'decodes' its K tokens by sleeping (1 + rank) ms per token, the ranks meet at a barrier, the
@@ -866,6 +944,12 @@ def main():
     ap.add_argument("--tune", action="append", default=[], metavar="KNOB=VALUE",
                     help="set a LIF_TUNE_* knob on every layer before capture, e.g. "
                          "--tune batched_up_whole_rows=0 (repeatable)")
+    ap.add_argument("--store", default="pinned", choices=["pinned", "file"],
+                    help="'file': the bundles of --layers layers (default 8) are written to files under "
+                         "--store-dir and read by reader threads (lif_decode_step_store)")
+    ap.add_argument("--store-dir", default="/tmp/lif_store")
+    ap.add_argument("--store-threads", default="32", help="comma-separated reader thread counts")
+    ap.add_argument("--store-cached", action="store_true", help="read through the page cache (no O_DIRECT)")
     ap.add_argument("--floors", action="store_true",
                     help="measure the reference points (host link, HBM read per launch) and exit")
     ap.add_argument("--kernel-loop", default=None,
@@ -884,6 +968,8 @@ def main():
         run_stub(args)
     elif args.floors:
         run_floors(args)
+    elif args.store == "file":
+        run_file_store(args)
     elif args.sweep_k:
         run_sweep_k(args)
     elif args.kernel_loop:

@@ -104,9 +104,16 @@ typedef struct {
                                outnumber the arrivals move cached rows.  Same cached set and
                                outputs, fewer row copies, and row moves no longer touch the
                                rows the fetch writes.  Not with ffn_mode = 1. */
+  int32_t staging_rows;     /* 0: host_bundles is the whole bundle store.  > 0 (>= capacity): the
+                               bundles live in a file (lif_store_*) and host_bundles is only a
+                               staging buffer of this many rows; the layer then steps through
+                               lif_decode_step_store, and the calls that read the store by
+                               neuron id (lif_fetch_bundles, lif_decode_step, graphs, lif_restore)
+                               return LIF_ERR_STATE */
   const void* dev_gate;     /* LIF_GATE_RESIDENT: fp16 [d_ff][d_model] gate projection, 16-byte
                                aligned; otherwise ignored */
-  const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][V*d_model] */
+  const void* host_bundles; /* HOST, pinned + mapped: fp16 [d_ff][V*d_model]
+                               (staging_rows > 0: [staging_rows][V*d_model]) */
   const void* dev_pred_A;   /* fp16 [d_model][rank] */
   const void* dev_pred_B;   /* fp16 [rank][d_ff] */
   const float* dev_pred_c;  /* fp32 [d_ff] per-neuron score offset */
@@ -267,6 +274,41 @@ lif_status lif_sparse_ffn_static(const void* dev_matrix, int32_t n_rows, const v
                                  const int32_t* dev_n_slots, const void* dev_bias_down,
                                  float* dev_y, int32_t d_model, void* stream);
 lif_status lif_sparse_ffn_static_status(int32_t* host_status, int32_t clear);
+
+/* The bundle store in a file: the paper's storage tier.  Section 2.2 ("Read Throughput"),
+ * Section 4.1 ("Implementation Details") and Appendix C ("Caching Considerations for Data Loading
+ * from Flash Memory"): the bundles of the newly needed neurons are read from flash by many
+ * threads (32 in the paper), one read per bundle, bypassing the operating system's cache, and
+ * the loads are managed on the CPU.
+ * lif_store_open: `path` holds n_bundles bundles of bundle_bytes bytes each (multiple of 16),
+ * bundle i at byte i * bundle_bytes; n_threads reader threads (1..256) are started.  direct_io != 0
+ * asks for uncached reads (O_DIRECT); where the file system refuses, the file is read through the
+ * cache and lif_store_stats.direct_io says so.  Bundles whose size or destination is not a
+ * multiple of 4096 bytes are read through an aligned window and copied.
+ * lif_store_read: bundles host_ids[0..n) into host_dst[j * bundle_bytes], with the store's
+ * threads; returns when all are read.  LIF_ERR_INVALID_ARG for an id outside the store,
+ * LIF_ERR_STATE for a failed read.  One call at a time per store.
+ * lif_decode_step_store: one token through a layer created with staging_rows > 0 — predict and
+ * window update on the device, the load list copied to the host (the stream is synchronised),
+ * the bundles read from the file into the staging buffer, copied to their cache rows by a kernel,
+ * and the sparse FFN; the stream is synchronised again before the call returns (the staging
+ * buffer is free for the next step).  Same results as lif_decode_step on a pinned store. */
+typedef struct lif_store lif_store;
+typedef struct {
+  uint64_t reads;           /* read calls issued */
+  uint64_t bytes_read;      /* bytes those calls returned (aligned windows included) */
+  uint64_t bytes_requested; /* bundles asked for x bundle_bytes */
+  double seconds_reading;   /* wall time inside batches of reads */
+  int32_t direct_io;        /* 1: the file is open for uncached reads */
+  int32_t n_threads;
+} lif_store_stats;
+lif_status lif_store_open(const char* path, int64_t n_bundles, int64_t bundle_bytes,
+                          int32_t n_threads, int32_t direct_io, lif_store** out);
+lif_status lif_store_close(lif_store* store);
+lif_status lif_store_read(lif_store* store, const int32_t* host_ids, int32_t n, void* host_dst);
+lif_status lif_store_get_stats(lif_store* store, lif_store_stats* host_out);
+lif_status lif_decode_step_store(lif_layer* layer, lif_store* store, const void* dev_x, float* dev_y,
+                                 void* stream);
 
 /* Neuron sharding over several devices (not in the paper, which runs on one device; it rests
  * on Section 3.3 item 3: the FFN output is a sum of one term per cached neuron, in any order).

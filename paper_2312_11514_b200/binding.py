@@ -27,6 +27,7 @@ EXPORTS = [
     "lif_graph_capture", "lif_graph_launch", "lif_graph_launch_host", "lif_graph_destroy",
     "lif_sparse_ffn_static", "lif_sparse_ffn_static_status", "lif_set_tuning", "lif_profile_launch",
     "lif_read_state", "lif_snapshot_bytes", "lif_snapshot", "lif_restore", "lif_sum_peer_outputs",
+    "lif_store_open", "lif_store_close", "lif_store_read", "lif_store_get_stats", "lif_decode_step_store",
 ]
 KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ffn_new", "ffn_sum",
            "ffn_cache")
@@ -43,7 +44,7 @@ class LayerDesc(C.Structure):
         ("capacity", C.c_int32), ("n_streams", C.c_int32), ("threshold_logit", C.c_float),
         ("ffn_mode", C.c_int32), ("activation", C.c_int32), ("activation_threshold", C.c_float),
         ("budget_rows", C.c_int32), ("spec_keep", C.c_int32), ("gate_mode", C.c_int32),
-        ("append_first", C.c_int32), ("dev_gate", C.c_void_p), ("host_bundles", C.c_void_p), ("dev_pred_A", C.c_void_p), ("dev_pred_B", C.c_void_p),
+        ("append_first", C.c_int32), ("staging_rows", C.c_int32), ("dev_gate", C.c_void_p), ("host_bundles", C.c_void_p), ("dev_pred_A", C.c_void_p), ("dev_pred_B", C.c_void_p),
         ("dev_pred_c", C.c_void_p), ("dev_bias_up", C.c_void_p), ("dev_bias_down", C.c_void_p),
         ("dev_cache", C.c_void_p), ("dev_workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
     ]
@@ -59,6 +60,11 @@ class Stats(C.Structure):
     _fields_ = [("counts", C.c_int32 * 16), ("bytes_fetched", C.c_uint64),
                 ("rows_moved", C.c_uint64), ("rows_active", C.c_uint64),
                 ("rows_cached", C.c_uint64), ("status", C.c_int32), ("reserved", C.c_int32)]
+
+
+class StoreStats(C.Structure):
+    _fields_ = [("reads", C.c_uint64), ("bytes_read", C.c_uint64), ("bytes_requested", C.c_uint64),
+                ("seconds_reading", C.c_double), ("direct_io", C.c_int32), ("n_threads", C.c_int32)]
 
 
 class LifError(RuntimeError):
@@ -106,6 +112,11 @@ def lib() -> C.CDLL:
         "lif_sparse_ffn_static": [vp, i32, vp, vp, vp, vp, vp, vp, i32, vp],
         "lif_sparse_ffn_static_status": [C.POINTER(C.c_int32), i32],
         "lif_sum_peer_outputs": [C.POINTER(vp), i32, vp, sz, vp],
+        "lif_store_open": [C.c_char_p, C.c_int64, C.c_int64, i32, i32, C.POINTER(vp)],
+        "lif_store_close": [vp],
+        "lif_store_read": [vp, vp, i32, vp],
+        "lif_store_get_stats": [vp, C.POINTER(StoreStats)],
+        "lif_decode_step_store": [vp, vp, vp, vp, vp],
         "lif_set_tuning": [vp, i32, i32],
         "lif_read_state": [vp, vp, vp, vp, vp],
         "lif_snapshot_bytes": [vp, C.POINTER(sz)],
@@ -138,6 +149,15 @@ def _ptr(t) -> Optional[int]:
     return t if isinstance(t, int) else t.data_ptr()
 
 
+def _host_ptr(a) -> Optional[int]:
+    """Address of a host array: numpy array or CPU tensor."""
+    if a is None:
+        return None
+    if hasattr(a, "ctypes"):
+        return a.ctypes.data
+    return a.data_ptr()
+
+
 def _stream(s) -> Optional[int]:
     if s is None:
         return None
@@ -146,7 +166,7 @@ def _stream(s) -> Optional[int]:
 
 def make_desc(*, d_model, d_ff, rank, window_k, capacity, n_streams=1, threshold_logit=0.0,
               ffn_mode=0, activation=0, activation_threshold=0.0, budget_rows=0, spec_keep=0,
-              gate_mode=0, gate=None, append_first=0, host_bundles=None, pred_A=None, pred_B=None, pred_c=None,
+              gate_mode=0, gate=None, append_first=0, staging_rows=0, host_bundles=None, pred_A=None, pred_B=None, pred_c=None,
               bias_up=None, bias_down=None, cache=None, workspace=None) -> LayerDesc:
     d = LayerDesc()
     d.d_model, d.d_ff, d.rank, d.window_k, d.capacity = d_model, d_ff, rank, window_k, capacity
@@ -156,6 +176,7 @@ def make_desc(*, d_model, d_ff, rank, window_k, capacity, n_streams=1, threshold
     d.spec_keep = spec_keep
     d.gate_mode, d.dev_gate = gate_mode, _ptr(gate)
     d.append_first = append_first
+    d.staging_rows = staging_rows
     d.host_bundles = _ptr(host_bundles)
     d.dev_pred_A, d.dev_pred_B, d.dev_pred_c = _ptr(pred_A), _ptr(pred_B), _ptr(pred_c)
     d.dev_bias_up, d.dev_bias_down = _ptr(bias_up), _ptr(bias_down)
@@ -301,6 +322,35 @@ def lif_sparse_ffn_static_status(clear: bool = True) -> int:
     _check(lib().lif_sparse_ffn_static_status(C.byref(out), 1 if clear else 0),
            "lif_sparse_ffn_static_status")
     return int(out.value)
+
+
+def lif_store_open(path: str, n_bundles: int, bundle_bytes: int, n_threads: int = 32,
+                   direct_io: bool = True) -> int:
+    out = C.c_void_p(None)
+    _check(lib().lif_store_open(path.encode(), n_bundles, bundle_bytes, n_threads,
+                                1 if direct_io else 0, C.byref(out)), "lif_store_open")
+    return out.value
+
+
+def lif_store_close(store: int) -> None:
+    _check(lib().lif_store_close(store), "lif_store_close")
+
+
+def lif_store_read(store: int, ids, dst) -> None:
+    """Bundles ``ids`` (int32 numpy array or CPU tensor) into ``dst`` (host numpy array or CPU
+    tensor of len(ids) * bundle_bytes bytes)."""
+    _check(lib().lif_store_read(store, _host_ptr(ids), len(ids), _host_ptr(dst)), "lif_store_read")
+
+
+def lif_store_get_stats(store: int) -> StoreStats:
+    out = StoreStats()
+    _check(lib().lif_store_get_stats(store, C.byref(out)), "lif_store_get_stats")
+    return out
+
+
+def lif_decode_step_store(layer: int, store: int, x, y, stream=None) -> None:
+    _check(lib().lif_decode_step_store(layer, store, _ptr(x), _ptr(y), _stream(stream)),
+           "lif_decode_step_store")
 
 
 def lif_sum_peer_outputs(partials, y, stream=None) -> None:

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "liblif.so")
-SOURCES = ["api.cu", "predict.cu", "gate.cu", "window.cu", "fetch.cu", "ffn.cu", "ffn_batched.cu", "exchange.cu"]
+SOURCES = ["api.cu", "predict.cu", "gate.cu", "window.cu", "fetch.cu", "ffn.cu", "ffn_batched.cu", "exchange.cu", "store.cu"]
 
 
 def _nvcc() -> str:

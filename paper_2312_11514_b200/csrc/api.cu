@@ -72,6 +72,8 @@ static lif_status check_shape(const lif_layer_desc* d) {
   if (d->gate_mode == LIF_GATE_RESIDENT && d->spec_keep > 0) return LIF_ERR_INVALID_ARG;
   if (d->append_first != 0 && d->append_first != 1) return LIF_ERR_INVALID_ARG;
   if (d->append_first && d->ffn_mode == 1) return LIF_ERR_INVALID_ARG;
+  if (d->staging_rows != 0 && (d->staging_rows < d->capacity || d->staging_rows > d->d_ff))
+    return LIF_ERR_INVALID_ARG;
   return LIF_OK;
 }
 
@@ -284,6 +286,7 @@ lif_status lif_window_update(lif_layer* L, const int32_t* dev_active_idx,
 
 lif_status lif_fetch_bundles(lif_layer* L, void* fetch_stream) {
   if (!L) return LIF_ERR_INVALID_ARG;
+  if (L->desc.staging_rows) return LIF_ERR_STATE;     // host_bundles is not the store
   return launch_fetch(L, (cudaStream_t)fetch_stream) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
 }
 
@@ -302,6 +305,7 @@ lif_status lif_sparse_ffn(lif_layer* L, const void* dev_x, const int32_t* dev_sl
 lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* compute_stream,
                            void* fetch_stream) {
   if (!L || !dev_x || !dev_y) return LIF_ERR_INVALID_ARG;
+  if (L->desc.staging_rows) return LIF_ERR_STATE;     // host_bundles is not the store
   if (!aligned(dev_x, 16) || !aligned(dev_y, 16)) return LIF_ERR_ALIGNMENT;
   cudaStream_t sc = (cudaStream_t)compute_stream, sf = (cudaStream_t)fetch_stream;
   const __half* x = (const __half*)dev_x;
@@ -455,6 +459,7 @@ lif_status lif_profile_launch(lif_layer* L, int32_t kernel, const void* dev_x, f
       e = launch_predict_one(L, kernel, (const __half*)dev_x, st);
       break;
     case LIF_KERNEL_FETCH:     // in the form the decode step launches it
+      if (L->desc.staging_rows) return LIF_ERR_STATE;
       e = (L->split_ffn && L->fused_fetch && fetch_ffn_supported(L))
               ? launch_fetch_ffn(L, (const __half*)dev_x,
                                  L->y_partial + (size_t)L->ffn_grid * L->desc.d_model, st,
@@ -600,6 +605,7 @@ lif_status lif_restore(lif_layer* L, const void* host_buf, size_t bytes) {
   size_t need = 0;
   if (!L || !host_buf || lif_snapshot_bytes(L, &need) != LIF_OK || bytes < need)
     return LIF_ERR_INVALID_ARG;
+  if (L->desc.staging_rows) return LIF_ERR_STATE;     // the rows cannot be re-read by neuron id
   // A snapshot of another shape, a truncated or a damaged one: everything the kernels will
   // use as an index is checked here, on the host, before any of it reaches the device.
   {

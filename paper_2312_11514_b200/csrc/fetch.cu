@@ -401,6 +401,13 @@ cudaError_t launch_fetch(lif_layer* L, cudaStream_t st) {
                   (const int32_t*)L->counts, row_elems(L->desc) / 8);
 }
 
+// File-backed store: staging row j (bundle load_ids[j], read by the host) -> cache row load_slots[j].
+cudaError_t launch_fetch_staged(lif_layer* L, cudaStream_t st) {
+  return launch_k(fetch_kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl,
+                  (const uint4*)L->dev_bundles, (uint4*)L->desc.dev_cache, (const int32_t*)nullptr,
+                  (const int32_t*)L->load_slots, (const int32_t*)L->counts, row_elems(L->desc) / 8);
+}
+
 bool fetch_ffn_supported(const lif_layer* L) {
   const lif_layer_desc& D = L->desc;
   return D.n_streams == 1 && D.gate_mode != LIF_GATE_BUNDLED &&

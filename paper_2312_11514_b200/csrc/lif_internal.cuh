@@ -130,6 +130,7 @@ cudaError_t launch_window(lif_layer* L, const int32_t* act, const int32_t* n_act
 cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullptr,
                          bool release_early = false);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
+cudaError_t launch_fetch_staged(lif_layer* L, cudaStream_t st);
 bool fetch_ffn_supported(const lif_layer* L);
 bool fetch_ffn_can_watch(const lif_layer* L);
 int gate_predict_ctas(const lif_layer_desc& D);    // CTAs of the resident-gate predictor

@@ -21,13 +21,14 @@ class Layer:
                  threshold_logit: float = 0.0, ffn_mode: int = 0, activation: int = 0,
                  activation_threshold: float = 0.0, budget_rows: int = 0, spec_keep: int = 0,
                  gate_mode: int = 0, gate: Optional[torch.Tensor] = None, append_first: int = 0,
-                 device="cuda:0"):
+                 staging_rows: int = 0, device="cuda:0"):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2312_11514_b200 needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
         assert host_bundles.is_pinned() and host_bundles.dtype == torch.float16
         n_vec = 3 if gate_mode == B.GATE_BUNDLED else 2      # d_model-vectors per bundle
-        assert host_bundles.shape == (d_ff, n_vec * d_model) and host_bundles.is_contiguous()
+        # staging_rows > 0: the bundles live in a file and host_bundles is the staging buffer
+        assert host_bundles.shape == (staging_rows or d_ff, n_vec * d_model) and host_bundles.is_contiguous()
         assert gate is None or (gate.shape == (d_ff, d_model) and gate.dtype == torch.float16
                                 and gate.is_contiguous())
         self.d_model, self.d_ff, self.rank, self.capacity = d_model, d_ff, rank, capacity
@@ -43,7 +44,7 @@ class Layer:
                      n_streams=n_streams, threshold_logit=threshold_logit, ffn_mode=ffn_mode,
                      activation=activation, activation_threshold=activation_threshold,
                      budget_rows=budget_rows, spec_keep=spec_keep, gate_mode=gate_mode,
-                     append_first=append_first)
+                     append_first=append_first, staging_rows=staging_rows)
         self.spec_keep, self.gate_mode = spec_keep, gate_mode
         nbytes = B.lif_workspace_bytes(B.make_desc(**shape))
         self._workspace_all = torch.zeros(nbytes + 256, dtype=torch.uint8, device=self.device)

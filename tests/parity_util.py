@@ -107,11 +107,19 @@ class OracleLayer:
 
 def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_down=False,
                     activation=0, act_threshold=0.0, budget_rows=0, spec_keep=0, gate_mode=0,
-                    append_first=0, device="cuda:0"):
-    store = R.pinned_store(cfg.d_ff, cfg.d_model, 3 if gate_mode == 1 else 2)
+                    append_first=0, store_file=None, device="cuda:0"):
+    """``store_file``: write the bundles to this file and give the layer a staging buffer of
+    ``capacity`` rows instead of the whole store (it then steps through lif_decode_step_store)."""
+    n_vec = 3 if gate_mode == 1 else 2
+    store = R.pinned_store(cfg.d_ff, cfg.d_model, n_vec)
     w = W.make_layer(cfg, layer_idx, device=device, bundles_out=store, gate_mode=gate_mode,
                      act_threshold=act_threshold)
     cap = capacity or W.window_capacity(cfg, w["p"])
+    staging_rows = 0
+    if store_file is not None:
+        store.numpy().tofile(store_file)
+        staging_rows = cap
+        store = torch.zeros(cap, n_vec * cfg.d_model, dtype=torch.float16).pin_memory()
     bd = None
     if b_down:
         g = torch.Generator(device="cpu").manual_seed(77 + layer_idx)
@@ -124,7 +132,7 @@ def make_layer_pair(cfg, layer_idx, *, capacity=None, theta=0.0, ffn_mode=0, b_d
                   activation=activation, activation_threshold=act_threshold, budget_rows=budget_rows,
                   spec_keep=spec_keep, gate_mode=gate_mode,
                   gate=dev(w["gate"]) if gate_mode == 2 else None, append_first=append_first,
-                  device=device)
+                  staging_rows=staging_rows, device=device)
     ora = OracleLayer(w, cfg.d_model, cfg.d_ff, cap, cfg.window_k, theta, bd, activation, act_threshold,
                       budget_rows, gate_mode, append_first)
     return gpu, ora
