@@ -6,9 +6,10 @@
 // A bundle is one contiguous 4*d_model-byte row (Section 3.2), so the unit of HBM traffic is
 // one bulk asynchronous copy (TMA, cp.async.bulk) of a whole row into shared memory.  Each
 // CTA owns rows q = cta, cta + G, ...; it issues the copies for all its rows up front (up to
-// `stages` in flight), and as each row's mbarrier completes the 256 threads dot the up half
-// with x (16-byte shared loads, warp-shuffle + 8-way shared reduction), apply bias + ReLU, and
-// axpy the down half into fp32 register accumulators.  Rows whose ReLU is zero skip the axpy.
+// `stages` in flight); each of the 8 warps takes a row of the round and, when that row's
+// mbarrier completes, dots the whole up half with x (16-byte shared loads, warp-shuffle sum)
+// and applies bias + ReLU; then all 256 threads axpy the down halves into fp32 register
+// accumulators.  Rows whose ReLU is zero skip the axpy.
 // CTA partials go to a [G][d] fp32 scratch; a second kernel adds them in CTA order, so the
 // result does not depend on scheduling.  Bound: HBM bandwidth, 4*d_model bytes per row.
 #include <mutex>
@@ -42,22 +43,24 @@ struct FfnArgs {
 
 // kGate = LIF_GATE_*: none (row = up | down), bundled (gate | up | down), resident (up | down,
 // gate value looked up by neuron id).
+// (registers capped at 128 per thread, not for a second CTA of this kernel — shared memory allows
+// one — but so that a CTA of it fits on an SM beside a CTA of the fetch kernel, which holds
+// every SM for the length of the host-link transfer)
 template <int kGate>
-__global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) sparse_ffn_kernel(FfnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int d = a.d;
   constexpr int kVec = kGate == LIF_GATE_BUNDLED ? 3 : 2;       // d-vectors per row
-  constexpr int kParts = kGate == LIF_GATE_BUNDLED ? 16 : 8;    // warp partials per row
   const unsigned row_bytes = 2u * kVec * d;
   const int stages = a.stages;
-  // shared layout: rows[stages][row_bytes] | x[d] fp16 | bars[stages] | part[stages][kParts] |
+  // shared layout: rows[stages][row_bytes] | x[d] fp16 | bars[stages] | row flags[stages] |
   //                h[stages] | bias[stages]
   unsigned char* rows = smem;
   __half* xs = reinterpret_cast<__half*>(rows + (size_t)stages * row_bytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(xs) +
                                                (((size_t)d * 2 + 15) & ~(size_t)15));
-  float* part = reinterpret_cast<float*>(bars + stages);
-  float* hs = part + stages * kParts;
+  int* ok_s = reinterpret_cast<int*>(bars + stages);      // 0: the row's index was refused
+  float* hs = reinterpret_cast<float*>(ok_s + stages);
   float* bias_s = hs + stages;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -108,7 +111,7 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
   for (int r0 = 0; r0 < my_cnt; r0 += stages) {
     const int rc = min(stages, my_cnt - r0);
     // thread i issues the copy of row i of this round and fetches its bias
-    bool row_ok = true;                       // (thread i also finishes row i below)
+    bool row_ok = true;
     if (tid < rc) {
       const int q = cta + (r0 + tid) * G;
       int slot;
@@ -125,18 +128,22 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
                bars + tid);
       bias_s[tid] = kGate == LIF_GATE_RESIDENT ? a.gate_val[a.pointers[slot]]
                                                : __half2float(a.bias[slot]);
+      ok_s[tid] = row_ok ? 1 : 0;
     }
     if (r0 == 0) {
       const uint4* xg = reinterpret_cast<const uint4*>(a.x);
       for (int c = tid; c < nvec; c += kThreads) reinterpret_cast<uint4*>(xs)[c] = xg[c];
-      __syncthreads();
     }
-    // up projection: partial dot products as rows land
-    for (int i = 0; i < rc; ++i) {
+    __syncthreads();                          // x, biases and row flags of this round
+    // up projection: warp w takes rows w, w + 8, ... of the round, each as soon as it has landed
+    // (a whole dot product per warp: no partial sums to exchange, and the rows of a round are
+    // worked on side by side instead of one after the other)
+    for (int i = warp; i < rc; i += kThreads / 32) {
       if (!mbar_wait(bars + i, parity, a.wait_polls)) timed_out = 1;
       const uint4* up = reinterpret_cast<const uint4*>(rows + (size_t)i * row_bytes);
       float p = 0.f, p2 = 0.f;
-      for (int c = tid; c < nvec; c += kThreads) {
+#pragma unroll 4
+      for (int c = lane; c < nvec; c += 32) {
         float uf[8], xf[8];
         unpack8(up[c], uf);
         unpack8(reinterpret_cast<const uint4*>(xs)[c], xf);
@@ -155,11 +162,14 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
         for (int o = 16; o > 0; o >>= 1) p2 += __shfl_xor_sync(0xffffffffu, p2, o);
       }
       if (lane == 0) {
-        part[i * kParts + warp] = p;
-        if (kGate == LIF_GATE_BUNDLED) part[i * kParts + 8 + warp] = p2;
+        float h;
+        if (kGate == LIF_GATE_NONE) h = apply_activation(p + bias_s[i], a.act, a.act_thr);
+        else if (kGate == LIF_GATE_BUNDLED) h = apply_activation(p + bias_s[i], a.act, a.act_thr) * p2;
+        else h = apply_activation(bias_s[i], a.act, a.act_thr) * p;
+        hs[i] = ok_s[i] ? h : 0.f;            // a refused row contributes nothing
       }
     }
-    if (__syncthreads_or(timed_out)) {
+    if (__syncthreads_or(timed_out)) {        // also publishes hs[]
       // A copy did not arrive in time: flag it, give the copies still in flight one more
       // bounded chance to land (they target this CTA's shared memory), and leave.  The
       // partial is not written.
@@ -170,23 +180,6 @@ __global__ void __launch_bounds__(kThreads, 1) sparse_ffn_kernel(FfnArgs a) {
       __syncthreads();
       return;
     }
-    if (tid < rc) {
-      float v = 0.f;
-#pragma unroll
-      for (int w = 0; w < 8; ++w) v += part[tid * kParts + w];
-      if (kGate == LIF_GATE_NONE) {
-        hs[tid] = apply_activation(v + bias_s[tid], a.act, a.act_thr);
-      } else if (kGate == LIF_GATE_BUNDLED) {
-        float u = 0.f;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) u += part[tid * kParts + 8 + w];
-        hs[tid] = apply_activation(v + bias_s[tid], a.act, a.act_thr) * u;
-      } else {
-        hs[tid] = apply_activation(bias_s[tid], a.act, a.act_thr) * v;
-      }
-      if (!row_ok) hs[tid] = 0.f;
-    }
-    __syncthreads();
     // down projection: y += h * down half
     for (int i = 0; i < rc; ++i) {
       const float h = hs[i];
