@@ -36,7 +36,7 @@ Workspace plan_workspace(const lif_layer_desc& d, int ffn_grid_max) {
   w.n_tmp = take(64);
   w.z_partial = take(z_ctas * S * d.rank * 4);
   w.mask_words = take(n_mask * 4);
-  w.new_mask_words = take(n_mask * 4);
+  w.new_mask_words = take((size_t)new_mask_entries(d) * 8);
   w.keep_tok = take(d.spec_keep > 0 ? F : 0);
   w.h_rows = take(d.n_streams > 1 ? (size_t)kBatchedMaxKSplit * F * 8 * 4 *
                                         (d.gate_mode == LIF_GATE_BUNDLED ? 2 : 1)
@@ -155,7 +155,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
   L->n_tmp = (int32_t*)(b + ws.n_tmp);
   L->z_partial = (float*)(b + ws.z_partial);
   L->mask_words = (uint32_t*)(b + ws.mask_words);
-  L->new_mask_words = (uint32_t*)(b + ws.new_mask_words);
+  L->new_mask_words = (unsigned long long*)(b + ws.new_mask_words);
   L->keep_tok = desc->spec_keep > 0 ? (int8_t*)(b + ws.keep_tok) : nullptr;
   L->y_partial = (float*)(b + ws.y_partial);
   L->h_rows = (float*)(b + ws.h_rows);

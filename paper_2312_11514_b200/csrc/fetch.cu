@@ -74,10 +74,10 @@ struct FetchFfnArgs {
   float* y_partial;          // [gridDim.x][d]
   int d, act;
   float act_thr;
-  const uint32_t* new_mask_words;   // kEarlyMask: the predictor's mask of neurons to bring in
-  int nwords;
-  const int* tiles_done;            // kEarlyWatch: mask words the score kernel has written
-  int n_tiles;                      // ... out of this many
+  const unsigned long long* new_mask_words;   // neurons to bring in: entries {bits, run}
+  int nwords;                       // entries ...
+  int word_bits;                    // ... and the consecutive neurons each one covers
+  const int* predictor_run;         // kEarlyWatch: number of the predictor run of this step
 };
 
 // How much of the kernel may run before its dependency wait:
@@ -86,12 +86,15 @@ struct FetchFfnArgs {
 //                row-move kernel): count, ids and rows are read and the first bundle's host
 //                loads issued ahead of the wait.
 //   kEarlyMask   the kernel ahead is the window kernel, whose lists are not final yet, but the
-//                predictor's mask of neurons to bring in is: the load list is exactly the set
-//                bits of that mask in ascending order (the window kernel derives it from the
-//                same state), so CTA c finds the id of its first bundle, the c-th set bit,
-//                itself and its host loads travel while the window kernel runs.  After the
-//                wait the count is compared with the window kernel's (it is 0 when that
-//                kernel refused the step) and the rows come from its list.
+//                predictor's entries of neurons to bring in are: the load list is exactly their
+//                set bits in ascending order (the window kernel derives it from the same
+//                state), so CTA c finds the id of its first bundle, the c-th set bit, itself
+//                and its host loads travel while the window kernel runs.
+//   kEarlyWatch  as kEarlyMask, but the kernel may be resident while the predictor still runs
+//                and reads the entries as they arrive (see the kernel).
+// In the last two forms nothing depends on what was read ahead of the wait: after it the count
+// and the id are compared with the window kernel's list, and a CTA whose early reading differs
+// (the window kernel refused the step, the entries were another run's) starts over from the list.
 constexpr int kWatchPolls = 64;     // about 30 us of polling at most
 
 template <int kGate, int kEarlyT>
@@ -99,32 +102,43 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   __shared__ float part[kThreads / 32];
   __shared__ int scan_sums[kThreads / 32];
   __shared__ int first_id;
-  __shared__ int watch_ok;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = a.d >> 3;                       // 16-byte chunks per half row
   int kEarly = kEarlyT;
-  if (kEarlyT == kEarlyWatch) {
-    // Resident while the score kernel may still be running (all of its CTAs are: it released
-    // the window kernel, which released this one, only after every one of them had started).
-    // One thread polls the predictor's count of written mask words.  The count was cleared
-    // before this step's predictor ran (by its first stage, or by the previous step's last sum);
-    // a count beyond the total means other launches of the predictor came between and nothing
-    // can be told from it.  Whatever the outcome, no result depends on it:
-    // without the count the kernel simply waits for its predecessors like kEarlyNone.
-    if (tid == 0) {
-      int ok = 0;
-      for (int i = 0; i < kWatchPolls; ++i) {
-        int v;
-        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(a.tiles_done) : "memory");
-        if (v >= a.n_tiles) {
-          ok = v == a.n_tiles;
-          break;
-        }
+  // thread t owns a run of consecutive words of the mask of neurons to bring in
+  const int wpt = (a.nwords + kThreads - 1) / kThreads;
+  const int w0 = min(a.nwords, tid * wpt), w1 = min(a.nwords, w0 + wpt);
+  uint32_t mw[4] = {0u, 0u, 0u, 0u};               // nwords <= 1024 in the mask-driven forms
+  auto read_words = [&](int want_tag, bool check) {
+    bool all_mine = true;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      mw[i] = 0u;
+      if (w0 + i < w1) {
+        unsigned long long v;
+        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(a.new_mask_words + w0 + i)
+                     : "memory");
+        mw[i] = (uint32_t)v;
+        all_mine = all_mine && (!check || (int)(v >> 32) == want_tag);
       }
-      watch_ok = ok;
     }
-    __syncthreads();
-    kEarly = watch_ok ? kEarlyMask : kEarlyNone;
+    return all_mine;
+  };
+  if (kEarlyT == kEarlyWatch) {
+    // Resident while the predictor may still be running (all of its CTAs are: it released the
+    // window kernel, which released this one, only after every one of them had started).  Every
+    // mask word is stored together with the number of the predictor run that wrote it (one
+    // 8-byte store), and that number was fixed before the run began, so each thread simply
+    // re-reads its own words until all of them carry it: one read tells both that the words are
+    // there and what they hold.  Bounded; if the words do not come the kernel waits for its
+    // predecessors like kEarlyNone, and whatever it read is checked against the window kernel's
+    // list after the wait, so no result depends on this phase.
+    const int run = __ldcg(a.predictor_run);
+    int ok = 0;
+    for (int i = 0; i < kWatchPolls && !ok; ++i) ok = __syncthreads_and(read_words(run, true) ? 1 : 0);
+    kEarly = ok ? kEarlyMask : kEarlyNone;
+  } else if (kEarlyT == kEarlyMask) {
+    read_words(0, false);                          // final before the kernel ahead passed its wait
   }
   if (kEarly == kEarlyNone) {
     pdl_wait();
@@ -132,16 +146,10 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   }
   int n;
   if (kEarly == kEarlyMask) {
-    // thread t owns a run of consecutive mask words; block-wide prefix of their bit counts
-    const int wpt = (a.nwords + kThreads - 1) / kThreads;
-    const int w0 = min(a.nwords, tid * wpt), w1 = min(a.nwords, w0 + wpt);
-    uint32_t mw[4];                                // nwords <= 1024 in this mode
+    // block-wide prefix of the words' bit counts; CTA c takes the c-th set bit
     int cnt = 0;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      mw[i] = w0 + i < w1 ? __ldcg(a.new_mask_words + w0 + i) : 0u;
-      cnt += __popc(mw[i]);
-    }
+    for (int i = 0; i < 4; ++i) cnt += __popc(mw[i]);
     if (tid == 0) first_id = -1;
     int off = block_exclusive_scan_256(cnt, &n, scan_sums);   // also orders the first_id store
     const int want = blockIdx.x;
@@ -152,7 +160,7 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
         if (want >= off && want < off + c) {
           uint32_t m = mw[i];
           for (int s = want - off; s > 0; --s) m &= m - 1;
-          first_id = (w0 + i) * 32 + __ffs(m) - 1;
+          first_id = (w0 + i) * a.word_bits + __ffs(m) - 1;
         }
         off += c;
       }
@@ -160,13 +168,6 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
     __syncthreads();
   } else {
     n = __ldcg(a.counts + LIF_CNT_N_LOAD);
-  }
-  if ((int)blockIdx.x >= n) {                      // the sum reads min(grid, n) partials
-    if (kEarly != kEarlyNone) {
-      pdl_wait();
-      pdl_trigger();
-    }
-    return;
   }
   uint4 up[kFusedChunks], down[kFusedChunks];
   auto host_loads = [&](int id) {
@@ -181,29 +182,38 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
     }
   };
   int j = blockIdx.x;
-  int id, slot = 0;
-  if (kEarly == kEarlyMask) {
-    id = first_id;
-  } else {
-    id = __ldcg(a.load_ids + j);
-    slot = __ldcg(a.load_slots + j);
+  int id = -1, slot = 0;
+  const bool mine = j < n;                         // this CTA has a first bundle
+  if (mine) {
+    if (kEarly == kEarlyMask) {
+      id = first_id;
+    } else {
+      id = __ldcg(a.load_ids + j);
+      slot = __ldcg(a.load_slots + j);
+    }
+    host_loads(id);
   }
-  host_loads(id);
   if (kEarly != kEarlyNone) {
     pdl_wait();
     pdl_trigger();
   }
   if (kEarly == kEarlyMask) {
-    // the window kernel is complete: its count is this one unless it refused the step (0, window
-    // state unchanged), in which case nothing is written
+    // The window kernel is complete.  Its list is the reference: the masks read ahead of the
+    // wait are this step's exactly when count and id agree with it (they do not when the window
+    // kernel refused the step — count 0, nothing is written — or when the masks were another
+    // predictor run's); otherwise the CTA starts over from the list.
     const int n_plan = __ldcg(a.counts + LIF_CNT_N_LOAD);
-    if (n_plan != n) {
-      if (n_plan != 0 && tid == 0)      // cannot happen: both counts come from the same state
-        atomicCAS(const_cast<int32_t*>(a.counts) + LIF_CNT_STATUS, LIF_OK, LIF_ERR_STATE);
-      return;
+    const bool stale = n_plan != n || (mine && __ldcg(a.load_ids + j) != id);
+    n = n_plan;
+    if (j < n) {
+      slot = __ldcg(a.load_slots + j);
+      if (stale) {
+        id = __ldcg(a.load_ids + j);
+        host_loads(id);
+      }
     }
-    slot = __ldcg(a.load_slots + j);
   }
+  if (j >= n) return;                              // the sum reads min(grid, n) partials
 
   uint4 xq[kFusedChunks];
 #pragma unroll
@@ -416,7 +426,7 @@ bool fetch_ffn_supported(const lif_layer* L) {
 
 // The mask-driven forms scan at most four mask words per thread.
 bool fetch_ffn_can_watch(const lif_layer* L) {
-  return (L->desc.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32) <= 4 * kThreads;
+  return new_mask_entries(L->desc) <= 4 * kThreads;
 }
 
 // Fetch of this step's new rows fused with their FFN terms; partials go to `partial`
@@ -438,10 +448,9 @@ cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cuda
   a.act = D.activation;
   a.act_thr = D.activation_threshold;
   a.new_mask_words = L->new_mask_words;
-  a.nwords = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
-  a.tiles_done = L->counts + CNT_TILES_DONE;
-  // what the predictor counts: word pairs (low-rank score kernel) or CTAs (gate kernel)
-  a.n_tiles = D.gate_mode == LIF_GATE_RESIDENT ? gate_predict_ctas(D) : a.nwords;
+  a.nwords = new_mask_entries(D);
+  a.word_bits = new_mask_entry_bits(D);
+  a.predictor_run = L->counts + CNT_PREDICTOR_RUN;
   if (early >= kEarlyMask && !fetch_ffn_can_watch(L)) early = kEarlyNone;
   void (*kernel)(FetchFfnArgs);
   if (D.gate_mode == LIF_GATE_RESIDENT)

@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kSumThreads)
 ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
                   const float* __restrict__ p1, const int32_t* __restrict__ n1, int G,
                   const __half* __restrict__ b_down, int b_period, float* __restrict__ y, int d,
-                  int accumulate, int n_cap, int* clear_after_wait) {
+                  int accumulate, int n_cap, int* next_run_after_wait) {
   __shared__ float4 red[32][kSumCols];
   const int tid = threadIdx.x;
   const int c4 = tid & (kSumCols - 1), gs = tid / kSumCols;
@@ -239,9 +239,9 @@ ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
   }
   pdl_wait();
   pdl_trigger();
-  // every earlier kernel of the step is complete: the predictor's count of written mask words
-  // has no watcher left and is cleared for the next step
-  if (clear_after_wait && blockIdx.x == 0 && tid == 0) *clear_after_wait = 0;
+  // every earlier kernel of the step is complete: the next predictor run gets its number here,
+  // long before it starts (a predictor without a first stage of its own relies on this)
+  if (next_run_after_wait && blockIdx.x == 0 && tid == 0) *next_run_after_wait += 1;
   // counts as the kernels that wrote the partials clamp them: [0, n_cap]
   const int v0 = min(G, max(0, min(*n0, n_cap))), v1 = p1 ? min(G, max(0, min(*n1, n_cap))) : 0;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -464,7 +464,7 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
   e = launch_k(ffn_reduce_kernel, dim3((d / 4 + kSumCols - 1) / kSumCols), dim3(kSumThreads), 0,
                st, L->use_pdl, (const float*)p0, hit.n, (const float*)p1, miss.n, L->ffn_grid,
                (const __half*)D.dev_bias_down, d, y, d, 0, D.capacity,
-               (int*)(L->counts + CNT_TILES_DONE));
+               (int*)(L->counts + CNT_PREDICTOR_RUN));
   if (ev) tm_record(ev[9], st);
   return e;
 }

@@ -31,7 +31,8 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
                    float* __restrict__ gate_val, float* __restrict__ logits,
                    uint32_t* mask_words, int* ticket, int* __restrict__ active_idx,
                    int* __restrict__ n_active, int compact, int nwords,
-                   const int32_t* __restrict__ slot_of, uint32_t* new_mask_words, int* tiles_done) {
+                   const int32_t* __restrict__ slot_of, unsigned long long* new_mask_words,
+                   const int* predictor_run) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* xs = reinterpret_cast<uint4*>(smem_raw);          // [S][d / 8]
   __shared__ int act_flag[kGateTile];     // bit 0: active, bit 1: active and not cached yet
@@ -57,6 +58,7 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
   for (int j = 0; j < kDepth; ++j) load_group(w[j], j);
   pdl_wait();
   pdl_trigger();
+  const int run = tid == 0 ? __ldcg(predictor_run) : 0;
   for (int c = tid; c < S * nvec; c += kThreads) xs[c] = reinterpret_cast<const uint4*>(x)[c];
   __syncthreads();
 
@@ -126,16 +128,16 @@ gate_scores_kernel(const __half* __restrict__ x, const __half* __restrict__ gate
     if (lane == 0) {
       if (kGateTile == 32) {
         mask_words[blockIdx.x] = m;
-        new_mask_words[blockIdx.x] = mn;
       } else if (kGateTile == 16) {
         reinterpret_cast<uint16_t*>(mask_words)[blockIdx.x] = (uint16_t)m;
-        reinterpret_cast<uint16_t*>(new_mask_words)[blockIdx.x] = (uint16_t)mn;
       } else {
         reinterpret_cast<uint8_t*>(mask_words)[blockIdx.x] = (uint8_t)m;
-        reinterpret_cast<uint8_t*>(new_mask_words)[blockIdx.x] = (uint8_t)mn;
       }
-      // count this CTA's mask bits as written (release), for a fetch kernel that watches
-      asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(tiles_done) : "memory");
+      // this CTA's neurons to bring in, with the run's number, in one store (one entry per CTA):
+      // a fetch kernel that is already resident re-reads the entry until the number is the run's
+      const unsigned long long e = (unsigned long long)mn | ((unsigned long long)(unsigned)run << 32);
+      asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(new_mask_words + blockIdx.x), "l"(e)
+                   : "memory");
     }
   }
   if (!compact) return;     // the consumer reads the bit mask itself
@@ -159,12 +161,12 @@ cudaError_t launch_gate_s(lif_layer* L, const __half* x, float* logits, int32_t*
                   D.d_ff, L->gate_val, logits, L->mask_words,
                   (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
                   (D.d_ff + 31) / 32, (const int32_t*)L->slot_of, L->new_mask_words,
-                  (int*)(L->counts + CNT_TILES_DONE));
+                  (int*)(L->counts + CNT_PREDICTOR_RUN));
 }
 
 }  // namespace
 
-int gate_predict_ctas(const lif_layer_desc& D) { return (D.d_ff + kGateTile - 1) / kGateTile; }
+int gate_predict_tile() { return kGateTile; }
 
 cudaError_t launch_gate_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,
                                 int32_t* n_active, cudaStream_t st, cudaEvent_t* ev, int compact) {

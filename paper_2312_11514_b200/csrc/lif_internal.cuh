@@ -13,7 +13,7 @@ namespace lif {
 // Private entries of the counts block (public ones: LIF_CNT_* in lif.h).
 enum {
   CNT_TICKET_PREDICT = 16,  // "last block done" counter of the score kernel
-  CNT_TILES_DONE = 17,      // mask words the score kernel has written so far in this step
+  CNT_PREDICTOR_RUN = 17,   // number of the predictor run whose masks are (being) written
   CNT_TOTALS = 32           // four uint64: bytes_fetched, rows_moved, rows_active, rows_cached
 };
 
@@ -60,7 +60,10 @@ struct lif_layer {
       *active_slots, *hit_slots, *n_tmp;
   float* z_partial;
   uint32_t* mask_words;
-  uint32_t* new_mask_words;   // bit i: neuron i is predicted active and has no cache row yet
+  // Neurons predicted active that have no cache row yet, as 64-bit entries {bits, run}: the low
+  // half holds the bits of 32 consecutive neurons (of one predictor CTA's neurons, where those
+  // are fewer), the high half the number of the predictor run that stored it (one store).
+  unsigned long long* new_mask_words;
   int8_t* keep_tok;   // [d_ff] last kept token per neuron (speculative mode)
   float* y_partial;
   float* h_rows;      // [K slices][d_ff][8] fp32: phase-A output of the multi-stream FFN
@@ -133,7 +136,15 @@ cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
 cudaError_t launch_fetch_staged(lif_layer* L, cudaStream_t st);
 bool fetch_ffn_supported(const lif_layer* L);
 bool fetch_ffn_can_watch(const lif_layer* L);
-int gate_predict_ctas(const lif_layer_desc& D);    // CTAs of the resident-gate predictor
+int gate_predict_tile();                           // neurons per CTA of the resident-gate predictor
+// entries of new_mask_words and the neurons each one covers
+inline int new_mask_entry_bits(const lif_layer_desc& D) {
+  return D.gate_mode == LIF_GATE_RESIDENT ? gate_predict_tile() : 32;
+}
+inline int new_mask_entries(const lif_layer_desc& D) {
+  if (D.gate_mode == LIF_GATE_RESIDENT) return (D.d_ff + gate_predict_tile() - 1) / gate_predict_tile();
+  return (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
+}
 // early: what the kernel may do before its own dependency wait.  kEarlyLists: the lists were
 // final before the kernel ahead of this one passed its wait, so the first bundle's host loads
 // are issued from them; kEarlyMask: the kernel ahead is the window kernel of the same step and

@@ -17,7 +17,7 @@ namespace {
 template <int S>
 __global__ void __launch_bounds__(kThreads)
 predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int d, int r,
-                 int rows_per_cta, float* __restrict__ z_partial, int* tiles_done) {
+                 int rows_per_cta, float* __restrict__ z_partial, int* predictor_run) {
   __shared__ float red[2048];
   const int ncg = r >> 3;            // 8-column groups (16 bytes each)
   const int nrl = kThreads / ncg;    // row lanes
@@ -42,8 +42,9 @@ predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int
   }
   pdl_wait();
   pdl_trigger();
-  // every earlier kernel is complete: nobody still watches the previous step's tile count
-  if (blockIdx.x == 0 && tid == 0) *tiles_done = 0;
+  // every earlier kernel is complete: a new predictor run begins, and its number is settled
+  // before the score kernel, which tags its mask words with it, passes its own wait
+  if (blockIdx.x == 0 && tid == 0) *predictor_run += 1;
   if (rl < nrl) {
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
@@ -97,7 +98,7 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
                       float* __restrict__ logits, uint32_t* mask_words, int* ticket,
                       int* __restrict__ active_idx, int* __restrict__ n_active, int compact,
                       int8_t* __restrict__ keep_tok, int keep, const int32_t* __restrict__ slot_of,
-                      uint32_t* new_mask_words, int* tiles_done) {
+                      unsigned long long* new_mask_words, const int* predictor_run) {
   extern __shared__ float zs[];                 // [S][r]
   __shared__ float red[16][kLogitTile];
   __shared__ int warp_sums[kThreads / 32];
@@ -122,6 +123,7 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
   const int my_row = (tid < kLogitTile && my_col < F) ? slot_of[my_col] : 0;
   pdl_wait();
   pdl_trigger();
+  const int run = (tid < kLogitTile && (tid & 31) == 0) ? __ldcg(predictor_run) : 0;
   if (S == 1) {
     // one stream: every partial of a sum is requested before the first is used (one memory
     // round trip instead of several); the additions keep their order
@@ -209,10 +211,11 @@ predict_logits_kernel(const float* __restrict__ z_partial, int P, const __half* 
     const unsigned mn = __ballot_sync(0xffffffffu, active && my_row < 0);
     if ((tid & 31) == 0) {
       mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = m;
-      new_mask_words[blockIdx.x * (kLogitTile / 32) + (tid >> 5)] = mn;
-      // count the word pair as written (release: whoever sees the count sees the words); no
-      // answer is waited for
-      asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(tiles_done) : "memory");
+      // the bits together with this run's number, in one store: a fetch kernel that is already
+      // resident re-reads the entry until the number is the run's
+      const unsigned long long e = (unsigned long long)mn | ((unsigned long long)(unsigned)run << 32);
+      asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(
+                       new_mask_words + blockIdx.x * (kLogitTile / 32) + (tid >> 5)), "l"(e) : "memory");
     }
   }
 
@@ -228,7 +231,7 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
   cudaError_t e = launch_k(predict_z_kernel<S>, dim3(L->z_ctas), dim3(kThreads), 0, st, L->use_pdl,
                            x, (const __half*)D.dev_pred_A, D.d_model, D.rank,
                            z_rows_per_cta(D.d_model), L->z_partial,
-                           (int*)(L->counts + CNT_TILES_DONE));
+                           (int*)(L->counts + CNT_PREDICTOR_RUN));
   if (e != cudaSuccess) return e;
   if (ev) tm_record(ev[1], st);
   const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
@@ -247,7 +250,7 @@ cudaError_t launch_predict_s(lif_layer* L, const __half* x, float* logits, int32
                D.threshold_logit, D.rank, D.d_ff, logits, L->mask_words,
                (int*)(L->counts + CNT_TICKET_PREDICT), (int*)active_idx, (int*)n_active, compact,
                L->keep_tok, D.spec_keep, (const int32_t*)L->slot_of, L->new_mask_words,
-               (int*)(L->counts + CNT_TILES_DONE));
+               (int*)(L->counts + CNT_PREDICTOR_RUN));
   if (ev) tm_record(ev[2], st);
   return e;
 }
@@ -265,7 +268,7 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
   if (kernel == LIF_KERNEL_PREDICT_Z)
     return launch_k(predict_z_kernel<1>, dim3(L->z_ctas), dim3(kThreads), 0, st, L->use_pdl, x,
                     (const __half*)D.dev_pred_A, D.d_model, D.rank, z_rows_per_cta(D.d_model),
-                    L->z_partial, (int*)(L->counts + CNT_TILES_DONE));
+                    L->z_partial, (int*)(L->counts + CNT_PREDICTOR_RUN));
   const int grid = (D.d_ff + kLogitTile - 1) / kLogitTile;
   return launch_k(L->keep_tok ? predict_logits_kernel<1, true> : predict_logits_kernel<1, false>,
                   dim3(grid), dim3(kThreads),
@@ -274,7 +277,7 @@ cudaError_t launch_predict_one(lif_layer* L, int kernel, const __half* x, cudaSt
                   D.d_ff, (float*)nullptr, L->mask_words, (int*)(L->counts + CNT_TICKET_PREDICT),
                   (int*)L->active_idx, (int*)L->n_tmp, L->fused_plan ? 0 : 1, L->keep_tok,
                   D.spec_keep, (const int32_t*)L->slot_of, L->new_mask_words,
-                  (int*)(L->counts + CNT_TILES_DONE));
+                  (int*)(L->counts + CNT_PREDICTOR_RUN));
 }
 
 cudaError_t launch_predict(lif_layer* L, const __half* x, float* logits, int32_t* active_idx,

@@ -661,19 +661,19 @@ move_rows_kernel(uint4* __restrict__ cache, const int32_t* __restrict__ move_src
 
 __global__ void __launch_bounds__(kThreads)
 reset_kernel(int32_t* counts, int32_t* pointers, int32_t* slot_of, int32_t* last_active,
-             uint32_t* mask_words, uint32_t* new_mask_words, int n_mask, int F, int cap) {
+             uint32_t* mask_words, unsigned long long* new_mask_words, int n_mask, int n_new, int F,
+             int cap) {
   const int i = blockIdx.x * kThreads + threadIdx.x;
   const int stride = gridDim.x * kThreads;
-  for (int j = i; j < LIF_CNT_LEN; j += stride) counts[j] = 0;
+  // predictor runs are numbered from 1: no entry of new_mask_words carries a number in use
+  for (int j = i; j < LIF_CNT_LEN; j += stride) counts[j] = j == CNT_PREDICTOR_RUN ? 1 : 0;
   for (int j = i; j < cap; j += stride) pointers[j] = -1;
   for (int j = i; j < F; j += stride) {
     slot_of[j] = -1;
     last_active[j] = kNever;
   }
-  for (int j = i; j < n_mask; j += stride) {
-    mask_words[j] = 0;
-    new_mask_words[j] = 0;
-  }
+  for (int j = i; j < n_mask; j += stride) mask_words[j] = 0;
+  for (int j = i; j < n_new; j += stride) new_mask_words[j] = 0ull;
 }
 
 }  // namespace
@@ -682,8 +682,8 @@ cudaError_t launch_reset(lif_layer* L, cudaStream_t st) {
   const lif_layer_desc& D = L->desc;
   const int n_mask = (D.d_ff + kLogitTile - 1) / kLogitTile * (kLogitTile / 32);
   reset_kernel<<<64, kThreads, 0, st>>>(L->counts, L->pointers, L->slot_of, L->last_active,
-                                        L->mask_words, L->new_mask_words, n_mask, D.d_ff,
-                                        D.capacity);
+                                        L->mask_words, L->new_mask_words, n_mask,
+                                        new_mask_entries(D), D.d_ff, D.capacity);
   return cudaGetLastError();
 }
 
