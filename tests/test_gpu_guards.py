@@ -175,3 +175,29 @@ def test_guard_row_and_guard_block_survive_a_run_that_fills_the_cache():
         assert gpu.guards_intact()
     assert len(gpu.lists()["hit_slots"]) == cfg.d_ff
     gpu.close()          # raises if a guard was touched
+
+
+@pytest.mark.parametrize("gate_mode", [B.GATE_NONE, B.GATE_RESIDENT])
+def test_predictor_calls_between_steps_do_not_leak_into_the_next_step(gate_mode):
+    # lif_predict with another input leaves the predictor's masks (which the fetch kernel of a
+    # decode step reads while that step's predictor may still be running) describing neurons the
+    # step does not want; every step must still bring in exactly its own
+    cfg = W.LifConfig("between", 1, 520, 4096, 32, 3, 1, 14, 0.08, 1.0, 0.8, 0.6, 41)
+    kw = dict(gate_mode=gate_mode, b_down=True)
+    if gate_mode == B.GATE_RESIDENT:
+        kw.update(activation=B.ACT_FATRELU, act_threshold=0.05)
+    gpu, ora = P.make_layer_pair(cfg, 0, **kw)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(1, cfg.d_model, dtype=torch.float32, device=DEV)
+    idx = torch.empty(cfg.d_ff, dtype=torch.int32, device=DEV)
+    n = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sc, sf = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for t in range(cfg.steps):
+        other = X[(t + 5) % cfg.steps]
+        for _ in range(1 + t % 3):
+            B.lif_predict(gpu.handle, other, None, idx, n, sc)
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
+        P.compare_cache_rows(gpu, ora)
+    gpu.close()
