@@ -854,6 +854,15 @@ def run_floors(args):
     link = {"cudaMemcpyAsync_1GiB_GBs": nb / best / 1e3}
     best = min(timed(lambda: B.lif_probe_host_read(hbuf, dbuf, nb, 16384, st), 1) for _ in range(3))
     link["kernel_read_1GiB_16KiB_chunks_GBs"] = nb / best / 1e3
+    # the same host memory through bulk copies into shared memory (the probe takes any global
+    # address: mapped host memory is one), 16 KiB per copy, 1 and 4 CTAs per SM
+    sink0 = torch.zeros(16, dtype=torch.uint8, device=dev)
+    tmo0 = torch.zeros(1, dtype=torch.int32, device=dev)
+    for ctas, stages in ((1, 4), (4, 3)):
+        best = min(timed(lambda: B.lif_probe_bulk_ring(hbuf, nb, 16384, stages, 1, ctas, 0, sink0, tmo0, st), 1)
+                   for _ in range(3))
+        link[f"bulk_copies_1GiB_16KiB_{ctas}cta_per_sm_GBs"] = nb / best / 1e3
+    link["bulk_copy_waits_that_ran_out"] = int(tmo0.item())
     for mb in (1, 2, 4, 8):
         n = mb << 20
         offs = [(i * 97 % 509) * (2 << 20) for i in range(24)]      # different regions: no reuse
