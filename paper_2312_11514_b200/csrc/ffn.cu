@@ -241,7 +241,8 @@ ffn_reduce_kernel(const float* __restrict__ p0, const int32_t* __restrict__ n0,
   pdl_trigger();
   // every earlier kernel of the step is complete: the next predictor run gets its number here,
   // long before it starts (a predictor without a first stage of its own relies on this)
-  if (next_run_after_wait && blockIdx.x == 0 && tid == 0) *next_run_after_wait += 1;
+  if (next_run_after_wait && blockIdx.x == 0 && tid == 0)
+    *next_run_after_wait = (int)((unsigned)*next_run_after_wait + 1u);   // wraps
   // counts as the kernels that wrote the partials clamp them: [0, n_cap]
   const int v0 = min(G, max(0, min(*n0, n_cap))), v1 = p1 ? min(G, max(0, min(*n1, n_cap))) : 0;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);

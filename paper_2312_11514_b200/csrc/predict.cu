@@ -44,7 +44,7 @@ predict_z_kernel(const __half* __restrict__ x, const __half* __restrict__ A, int
   pdl_trigger();
   // every earlier kernel is complete: a new predictor run begins, and its number is settled
   // before the score kernel, which tags its mask words with it, passes its own wait
-  if (blockIdx.x == 0 && tid == 0) *predictor_run += 1;
+  if (blockIdx.x == 0 && tid == 0) *predictor_run = (int)((unsigned)*predictor_run + 1u);   // wraps
   if (rl < nrl) {
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
