@@ -106,3 +106,32 @@ def test_graph_and_profiling_calls_reject_null_handles():
     assert lib.lif_sparse_ffn_static(None, 1, None, None, None, None, None, None, 256, None) == B.LIF_ERR_INVALID_ARG
     assert lib.lif_sparse_ffn_static_status(None, 0) == B.LIF_ERR_INVALID_ARG
     assert lib.lif_sum_peer_outputs(None, 2, None, 16, None) == B.LIF_ERR_INVALID_ARG
+
+
+def _enumerators():
+    """Every `NAME = integer` enumerator of the headers."""
+    values = {}
+    for header in sorted(os.listdir(INCLUDE)):
+        text = open(os.path.join(INCLUDE, header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        for name, value in re.findall(r"\b(LIF_[A-Z0-9_]+)\s*=\s*(-?\d+)", text):
+            values[name] = int(value)
+    return values
+
+
+def test_binding_constants_equal_the_headers_enumerators():
+    enums = _enumerators()
+    assert len(enums) > 40
+    checked = 0
+    for name, value in enums.items():
+        short = name[4:]                              # the binding drops the LIF_ prefix ...
+        for candidate in (name, short):               # ... except for the status codes
+            if hasattr(B, candidate):
+                assert getattr(B, candidate) == value, name
+                checked += 1
+                break
+    assert checked > 30
+    # tuples indexed by enumerator value
+    for i, kernel in enumerate(B.KERNELS):
+        assert enums["LIF_KERNEL_" + kernel.upper()] == i
+    assert enums["LIF_CNT_LEN"] == B.CNT_LEN
