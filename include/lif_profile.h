@@ -32,12 +32,18 @@ enum {
   LIF_TUNE_FUSED_FETCH_FFN = 8,  /* (1) lif_decode_step, one stream, with LIF_TUNE_SPLIT_FFN: the
                                     fetch kernel also adds the FFN terms of the rows it brings
                                     in (needs fetch CTAs = FFN CTAs, bundles of two vectors) */
-  LIF_TUNE_WAIT_POLLS = 9        /* (2^22) test aid: poll limit of the FIRST wait on each bulk
+  LIF_TUNE_WAIT_POLLS = 9,       /* (2^22) test aid: poll limit of the FIRST wait on each bulk
                                     copy in the sparse-FFN kernels, >= 0 (0: give up without
                                     polling).  When it runs out the CTA sets LIF_ERR_TIMEOUT,
                                     then waits for its copies with the full limit before it
                                     returns, so 0 makes the error path run with nothing left in
                                     flight */
+  LIF_TUNE_EARLY_FETCH = 10      /* (1) lif_decode_step where the fetch is a kernel of its own
+                                    (several input streams, three-vector bundles): it runs on
+                                    the compute stream directly behind the window kernel, is
+                                    resident while the predictor still runs and issues its first
+                                    host loads from the predictor's masks; 0: it waits for the
+                                    window kernel's lists on the fetch stream */
 };
 lif_status lif_set_tuning(lif_layer* layer, int32_t key, int32_t value);
 

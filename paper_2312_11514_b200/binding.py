@@ -33,7 +33,7 @@ KERNELS = ("predict_z", "predict_scores", "fetch", "ffn_active", "ffn_hits", "ff
            "ffn_cache")
 (TUNE_DEPENDENT_LAUNCH, TUNE_SPLIT_FFN, TUNE_FETCH_CTAS, TUNE_FFN_CTAS, TUNE_FFN_STAGES,
  TUNE_BATCHED_COLUMN_PARTS, TUNE_FUSED_PLAN, TUNE_BATCHED_UP_TWO_CTAS, TUNE_FUSED_FETCH_FFN,
- TUNE_WAIT_POLLS) = range(10)
+ TUNE_WAIT_POLLS, TUNE_EARLY_FETCH) = range(11)
 PHASES = ("predict_z", "predict_scores", "window", "moves", "fetch", "ffn", "ffn_sum")
 PHASE_LEN = 8
 

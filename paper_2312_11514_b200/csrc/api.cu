@@ -166,6 +166,7 @@ lif_status lif_create_layer(const lif_layer_desc* desc, lif_layer** out) {
             cudaDeviceGetAttribute(&L->n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
   ok = ok && ffn_configure(L) == cudaSuccess;
   L->fb_up_two_ctas = 0;
+  L->early_fetch = 1;
   ok = ok && ffn_batched_configure(L) == cudaSuccess;
   if (ok) {
     L->z_ctas = z_cta_count(desc->d_model);
@@ -318,9 +319,14 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
   // second stream the moves leave the critical chain (they only precede the cached rows' FFN).
   const bool moves_aside = L->desc.append_first && sf != sc;
   // The fetch kernel can watch the predictor when it directly follows the window kernel (or the
-  // row moves behind it) on the compute stream: two streams, one input stream, fused fetch.
-  L->watch_chain = sf != sc && L->use_pdl && L->split_ffn && L->desc.n_streams == 1 && L->fused_fetch &&
-                   fetch_ffn_supported(L) && fetch_ffn_can_watch(L);
+  // row moves behind it) on the compute stream with dependent launches.  One input stream with
+  // the FFN split around the fetch: two streams (the cached rows' FFN runs on the other).
+  // Otherwise the plain fetch takes that place on the compute stream, and the second stream, if
+  // there is one, carries the row moves.
+  const bool split = L->split_ffn && L->desc.n_streams == 1;
+  // (in speculative mode the load list is a subset of the predictor's mask: no early start)
+  L->watch_chain = L->use_pdl && fetch_ffn_can_watch(L) && L->desc.spec_keep == 0 &&
+                   (split ? sf != sc : L->early_fetch != 0);
   if (L->fused_plan) {
     ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev, 0) == cudaSuccess;
     ok = ok && launch_window_plan(L, sc, ev, !moves_aside) == cudaSuccess;
@@ -328,13 +334,34 @@ lif_status lif_decode_step(lif_layer* L, const void* dev_x, float* dev_y, void* 
     ok = launch_predict(L, x, nullptr, L->active_idx, L->n_tmp, sc, ev) == cudaSuccess;
     ok = ok && launch_window(L, L->active_idx, L->n_tmp, sc, ev, !moves_aside) == cudaSuccess;
   }
-  if (L->split_ffn && L->desc.n_streams == 1) {
+  if (split) {
     ok = ok && launch_fetch_and_ffn_split(L, x, dev_y, sc, sf, ev, moves_aside) == cudaSuccess;
     L->watch_chain = 0;
     if (!ok) cudaGetLastError();
     return ok ? LIF_OK : LIF_ERR_CUDA;
   }
-  L->watch_chain = 0;
+  if (L->watch_chain) {
+    // compute stream: ... window kernel -> (row moves) -> fetch, resident early -> FFN
+    L->watch_chain = 0;
+    if (moves_aside) {                 // the moves touch other rows than the fetch: beside it
+      ok = ok && cudaEventRecord(L->ev_plan, sc) == cudaSuccess;
+      ok = ok && cudaStreamWaitEvent(sf, L->ev_plan, 0) == cudaSuccess;
+      ok = ok && launch_moves(L, sf, ev) == cudaSuccess;
+      ok = ok && cudaEventRecord(L->ev_fetch, sf) == cudaSuccess;
+    }
+    if (ev) tm_record(ev[5], sc);
+    ok = ok && launch_fetch_early(L, sc, kEarlyWatch) == cudaSuccess;
+    if (ev) tm_record(ev[6], sc);
+    if (moves_aside) ok = ok && cudaStreamWaitEvent(sc, L->ev_fetch, 0) == cudaSuccess;
+    if (L->desc.ffn_mode == 0)
+      ok = ok && launch_ffn(L, x, L->active_slots, L->counts + LIF_CNT_N_ACTIVE, nullptr, dev_y,
+                            false, sc, ev) == cudaSuccess;
+    else
+      ok = ok && launch_ffn(L, x, nullptr, L->counts + LIF_CNT_NUM_USED, nullptr, dev_y, false,
+                            sc, ev) == cudaSuccess;
+    if (!ok) cudaGetLastError();
+    return ok ? LIF_OK : LIF_ERR_CUDA;
+  }
   if (sf != sc) {
     ok = ok && cudaEventRecord(L->ev_plan, sc) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(sf, L->ev_plan, 0) == cudaSuccess;
@@ -506,6 +533,7 @@ lif_status lif_set_tuning(lif_layer* L, int32_t key, int32_t value) {
     case LIF_TUNE_BATCHED_UP_TWO_CTAS:
       L->fb_up_two_ctas = value != 0;
       return ffn_batched_configure(L) == cudaSuccess ? LIF_OK : LIF_ERR_CUDA;
+    case LIF_TUNE_EARLY_FETCH: L->early_fetch = value != 0; return LIF_OK;
     case LIF_TUNE_WAIT_POLLS:
       if (value < 0) return LIF_ERR_INVALID_ARG;
       L->wait_polls = (unsigned)value;

@@ -62,6 +62,14 @@ fetch_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
 // final before that kernel passed its own wait, while the cache rows may still be moving.
 constexpr int kFusedChunks = 4;     // 8-column chunks per thread and half row: d_model <= 8192
 
+// The predictor's entries of neurons to bring in, and where the run number lives.
+struct EarlySource {
+  const unsigned long long* entries;   // {bits, run}
+  int nwords, word_bits;               // entries, and the consecutive neurons each one covers
+  const int* predictor_run;            // number of the predictor run of this step
+  const int32_t* counts;
+};
+
 struct FetchFfnArgs {
   const uint4* store;
   uint4* cache;
@@ -74,10 +82,7 @@ struct FetchFfnArgs {
   float* y_partial;          // [gridDim.x][d]
   int d, act;
   float act_thr;
-  const unsigned long long* new_mask_words;   // neurons to bring in: entries {bits, run}
-  int nwords;                       // entries ...
-  int word_bits;                    // ... and the consecutive neurons each one covers
-  const int* predictor_run;         // kEarlyWatch: number of the predictor run of this step
+  EarlySource early;         // what the mask-driven forms read ahead of the dependency wait
 };
 
 // How much of the kernel may run before its dependency wait:
@@ -97,17 +102,21 @@ struct FetchFfnArgs {
 // (the window kernel refused the step, the entries were another run's) starts over from the list.
 constexpr int kWatchPolls = 64;     // about 30 us of polling at most
 
-template <int kGate, int kEarlyT>
-__global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
-  __shared__ float part[kThreads / 32];
-  __shared__ int scan_sums[kThreads / 32];
-  __shared__ int first_id;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int nvec = a.d >> 3;                       // 16-byte chunks per half row
+// What a fetch kernel learned ahead of its dependency wait: the form it ended up in (kEarlyNone:
+// the wait has been passed already; otherwise the caller still has to wait), the count of
+// neurons to bring in (from the entries in kEarlyMask form, else the window kernel's) and, in
+// kEarlyMask form, the id of the want-th of them (-1 if there are fewer).
+struct EarlyPick {
+  int mode, n, id;
+};
+template <int kEarlyT>
+__device__ __forceinline__ EarlyPick early_pick(const EarlySource& src, int want, int* scan_sums,
+                                                int* first_id) {
+  const int tid = threadIdx.x;
   int kEarly = kEarlyT;
   // thread t owns a run of consecutive words of the mask of neurons to bring in
-  const int wpt = (a.nwords + kThreads - 1) / kThreads;
-  const int w0 = min(a.nwords, tid * wpt), w1 = min(a.nwords, w0 + wpt);
+  const int wpt = (src.nwords + kThreads - 1) / kThreads;
+  const int w0 = min(src.nwords, tid * wpt), w1 = min(src.nwords, w0 + wpt);
   uint32_t mw[4] = {0u, 0u, 0u, 0u};               // nwords <= 1024 in the mask-driven forms
   auto read_words = [&](int want_tag, bool check) {
     bool all_mine = true;
@@ -116,7 +125,7 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
       mw[i] = 0u;
       if (w0 + i < w1) {
         unsigned long long v;
-        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(a.new_mask_words + w0 + i)
+        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(src.entries + w0 + i)
                      : "memory");
         mw[i] = (uint32_t)v;
         all_mine = all_mine && (!check || (int)(v >> 32) == want_tag);
@@ -133,7 +142,7 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
     // there and what they hold.  Bounded; if the words do not come the kernel waits for its
     // predecessors like kEarlyNone, and whatever it read is checked against the window kernel's
     // list after the wait, so no result depends on this phase.
-    const int run = __ldcg(a.predictor_run);
+    const int run = __ldcg(src.predictor_run);
     int ok = 0;
     for (int i = 0; i < kWatchPolls && !ok; ++i) ok = __syncthreads_and(read_words(run, true) ? 1 : 0);
     kEarly = ok ? kEarlyMask : kEarlyNone;
@@ -146,13 +155,12 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   }
   int n;
   if (kEarly == kEarlyMask) {
-    // block-wide prefix of the words' bit counts; CTA c takes the c-th set bit
+    // block-wide prefix of the words' bit counts; the caller wants the want-th set bit
     int cnt = 0;
 #pragma unroll
     for (int i = 0; i < 4; ++i) cnt += __popc(mw[i]);
-    if (tid == 0) first_id = -1;
+    if (tid == 0) *first_id = -1;
     int off = block_exclusive_scan_256(cnt, &n, scan_sums);   // also orders the first_id store
-    const int want = blockIdx.x;
     if (want >= off && want < off + cnt) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -160,15 +168,33 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
         if (want >= off && want < off + c) {
           uint32_t m = mw[i];
           for (int s = want - off; s > 0; --s) m &= m - 1;
-          first_id = (w0 + i) * a.word_bits + __ffs(m) - 1;
+          *first_id = (w0 + i) * src.word_bits + __ffs(m) - 1;
         }
         off += c;
       }
     }
     __syncthreads();
   } else {
-    n = __ldcg(a.counts + LIF_CNT_N_LOAD);
+    n = __ldcg(src.counts + LIF_CNT_N_LOAD);
   }
+  EarlyPick pk;
+  pk.mode = kEarly;
+  pk.n = n;
+  pk.id = kEarly == kEarlyMask ? *first_id : -1;
+  return pk;
+}
+
+
+template <int kGate, int kEarlyT>
+__global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
+  __shared__ float part[kThreads / 32];
+  __shared__ int scan_sums[kThreads / 32];
+  __shared__ int first_id;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = a.d >> 3;                       // 16-byte chunks per half row
+  const EarlyPick pk = early_pick<kEarlyT>(a.early, blockIdx.x, scan_sums, &first_id);
+  const int kEarly = pk.mode;
+  int n = pk.n;
   uint4 up[kFusedChunks], down[kFusedChunks];
   auto host_loads = [&](int id) {
     const uint4* src = a.store + (size_t)id * 2 * nvec;
@@ -186,7 +212,7 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
   const bool mine = j < n;                         // this CTA has a first bundle
   if (mine) {
     if (kEarly == kEarlyMask) {
-      id = first_id;
+      id = pk.id;
     } else {
       id = __ldcg(a.load_ids + j);
       slot = __ldcg(a.load_slots + j);
@@ -278,6 +304,76 @@ __global__ void __launch_bounds__(kThreads) fetch_ffn_kernel(FetchFfnArgs a) {
     if (c < nvec) {
       out[2 * c] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
       out[2 * c + 1] = make_float4(acc[k][4], acc[k][5], acc[k][6], acc[k][7]);
+    }
+  }
+}
+
+// The plain fetch with the same early start as fetch_ffn_kernel (used where that kernel does not
+// apply: several input streams, three-vector bundles).  CTA c's first unit is slice c % slices
+// of row c / slices of the load list; its host loads are issued ahead of the dependency wait
+// and held in registers until the window kernel's list says where the row goes.  The units
+// after the first come from the list.
+template <int kEarlyT>
+__global__ void __launch_bounds__(kThreads)
+fetch_early_kernel(const uint4* __restrict__ store, uint4* __restrict__ cache,
+                   const int32_t* __restrict__ load_ids, const int32_t* __restrict__ load_slots,
+                   int row_vec, EarlySource early) {
+  __shared__ int scan_sums[kThreads / 32];
+  __shared__ int first_id;
+  constexpr int kSlice = kThreads * kFetchUnroll;
+  const int slices = (row_vec + kSlice - 1) / kSlice;
+  const int j0 = blockIdx.x / slices;
+  const int v0 = (blockIdx.x % slices) * kSlice + threadIdx.x;
+  const EarlyPick pk = early_pick<kEarlyT>(early, j0, scan_sums, &first_id);
+  uint4 buf[kFetchUnroll];
+  auto host_loads = [&](int id) {
+    const uint4* src = store + (size_t)id * row_vec;
+#pragma unroll
+    for (int i = 0; i < kFetchUnroll; ++i) {
+      const int v = v0 + i * kThreads;
+      if (v < row_vec) buf[i] = ld_stream16(src + v);
+    }
+  };
+  int n = pk.n, id = -1;
+  const bool mine = j0 < n;
+  if (mine) {
+    id = pk.mode == kEarlyMask ? pk.id : __ldcg(load_ids + j0);
+    host_loads(id);
+  }
+  if (pk.mode != kEarlyNone) {
+    pdl_wait();
+    pdl_trigger();
+  }
+  if (pk.mode == kEarlyMask) {
+    // the window kernel's list is the reference (see fetch_ffn_kernel)
+    const int n_plan = __ldcg(early.counts + LIF_CNT_N_LOAD);
+    const bool stale = n_plan != n || (mine && __ldcg(load_ids + j0) != id);
+    n = n_plan;
+    if (j0 < n && stale) host_loads(__ldcg(load_ids + j0));
+  }
+  if (j0 < n) {
+    uint4* dst = cache + (size_t)load_slots[j0] * row_vec;
+#pragma unroll
+    for (int i = 0; i < kFetchUnroll; ++i) {
+      const int v = v0 + i * kThreads;
+      if (v < row_vec) dst[v] = buf[i];
+    }
+  }
+  const long long units = (long long)n * slices;
+  for (long long u = (long long)blockIdx.x + gridDim.x; u < units; u += gridDim.x) {
+    const int j = (int)(u / slices);
+    const int w0 = (int)(u % slices) * kSlice + threadIdx.x;
+    const uint4* src = store + (size_t)load_ids[j] * row_vec;
+    uint4* dst = cache + (size_t)load_slots[j] * row_vec;
+#pragma unroll
+    for (int i = 0; i < kFetchUnroll; ++i) {
+      const int v = w0 + i * kThreads;
+      if (v < row_vec) buf[i] = ld_stream16(src + v);
+    }
+#pragma unroll
+    for (int i = 0; i < kFetchUnroll; ++i) {
+      const int v = w0 + i * kThreads;
+      if (v < row_vec) dst[v] = buf[i];
     }
   }
 }
@@ -411,6 +507,30 @@ cudaError_t launch_fetch(lif_layer* L, cudaStream_t st) {
                   (const int32_t*)L->counts, row_elems(L->desc) / 8);
 }
 
+static EarlySource early_source(const lif_layer* L) {
+  EarlySource e;
+  e.entries = L->new_mask_words;
+  e.nwords = new_mask_entries(L->desc);
+  e.word_bits = new_mask_entry_bits(L->desc);
+  e.predictor_run = L->counts + CNT_PREDICTOR_RUN;
+  e.counts = L->counts;
+  return e;
+}
+
+// The plain fetch behind the window kernel (or the row moves) on the same stream, started early
+// (`early` as for launch_fetch_ffn).
+cudaError_t launch_fetch_early(lif_layer* L, cudaStream_t st, int early) {
+  if (early >= kEarlyMask && !fetch_ffn_can_watch(L)) early = kEarlyNone;
+  if (early == kEarlyNone) return launch_fetch(L, st);
+  auto kernel = early == kEarlyWatch  ? fetch_early_kernel<kEarlyWatch>
+                : early == kEarlyMask ? fetch_early_kernel<kEarlyMask>
+                                      : fetch_early_kernel<kEarlyLists>;
+  return launch_k(kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl,
+                  (const uint4*)L->dev_bundles, (uint4*)L->desc.dev_cache,
+                  (const int32_t*)L->load_ids, (const int32_t*)L->load_slots,
+                  row_elems(L->desc) / 8, early_source(L));
+}
+
 // File-backed store: staging row j (bundle load_ids[j], read by the host) -> cache row load_slots[j].
 cudaError_t launch_fetch_staged(lif_layer* L, cudaStream_t st) {
   return launch_k(fetch_kernel, dim3(L->fetch_grid), dim3(kThreads), 0, st, L->use_pdl,
@@ -447,10 +567,7 @@ cudaError_t launch_fetch_ffn(lif_layer* L, const __half* x, float* partial, cuda
   a.d = D.d_model;
   a.act = D.activation;
   a.act_thr = D.activation_threshold;
-  a.new_mask_words = L->new_mask_words;
-  a.nwords = new_mask_entries(D);
-  a.word_bits = new_mask_entry_bits(D);
-  a.predictor_run = L->counts + CNT_PREDICTOR_RUN;
+  a.early = early_source(L);
   if (early >= kEarlyMask && !fetch_ffn_can_watch(L)) early = kEarlyNone;
   void (*kernel)(FetchFfnArgs);
   if (D.gate_mode == LIF_GATE_RESIDENT)

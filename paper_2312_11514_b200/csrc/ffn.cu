@@ -455,7 +455,8 @@ cudaError_t launch_fetch_and_ffn_split(lif_layer* L, const __half* x, float* y, 
     if ((e = launch_fetch_ffn(L, x, p1, st, L->watch_chain ? kEarlyWatch : (moves_aside ? kEarlyMask : kEarlyLists))) != cudaSuccess) return e;
     if (ev) tm_record(ev[6], st);
   } else {
-    if ((e = launch_fetch(L, st)) != cudaSuccess) return e;
+    e = L->watch_chain ? launch_fetch_early(L, st, kEarlyWatch) : launch_fetch(L, st);
+    if (e != cudaSuccess) return e;
     if (ev) tm_record(ev[6], st);
     e = launch_k(ffn_kernel_for(D.gate_mode), dim3(L->ffn_grid), dim3(kThreads), L->ffn_smem, st,
                  L->use_pdl, miss);

@@ -82,6 +82,7 @@ struct lif_layer {
   int fetch_grid;     // CTAs of the fetch kernel
   int move_grid;
   unsigned wait_polls; // poll limit of the first wait on each bulk copy in the FFN kernels
+  int early_fetch;    // knob: the plain fetch of lif_decode_step starts early behind the window kernel
   int watch_chain;    // set by lif_decode_step while it launches a step whose fetch kernel watches
                       // the predictor: window and row-move kernels release their dependents at entry
   int use_pdl;        // programmatic dependent launch along the compute stream
@@ -134,6 +135,7 @@ cudaError_t launch_moves(lif_layer* L, cudaStream_t st, cudaEvent_t* ev = nullpt
                          bool release_early = false);
 cudaError_t launch_fetch(lif_layer* L, cudaStream_t st);
 cudaError_t launch_fetch_staged(lif_layer* L, cudaStream_t st);
+cudaError_t launch_fetch_early(lif_layer* L, cudaStream_t st, int early);
 bool fetch_ffn_supported(const lif_layer* L);
 bool fetch_ffn_can_watch(const lif_layer* L);
 int gate_predict_tile();                           // neurons per CTA of the resident-gate predictor
