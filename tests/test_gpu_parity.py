@@ -679,3 +679,36 @@ def test_multi_stream_ffn_with_tiny_activations(gate_mode, act):
         B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
         P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
     gpu.close()
+
+
+@pytest.mark.parametrize("early,two_streams,append_first,S,gate_mode", [
+    (1, True, 1, 3, 0), (0, True, 1, 3, 0), (1, True, 0, 3, 0), (1, False, 1, 3, 0), (1, False, 0, 8, 0),
+    (1, True, 1, 1, 1), (0, True, 1, 1, 1), (1, True, 0, 1, 1), (1, True, 1, 4, 1)])
+def test_fetch_as_a_kernel_of_its_own_early_or_after_the_lists(early, two_streams, append_first, S,
+                                                              gate_mode):
+    # several input streams, or three-vector bundles: the fetch is not fused with the FFN; by
+    # default it starts from the predictor's masks while the window kernel runs, with the knob
+    # off it waits for the lists.  A predictor call with another input between the steps leaves
+    # masks that are not the step's.
+    cfg = W.LifConfig("efetch", 1, 512, 4096, 32, 2, S, 12, 0.06, 1.0, 0.8, 0.6, 47)
+    act, thr = (B.ACT_FATRELU, 0.05) if gate_mode else (B.ACT_RELU, 0.0)
+    gpu, ora = P.make_layer_pair(cfg, 0, gate_mode=gate_mode, activation=act, act_threshold=thr,
+                                 b_down=True, append_first=append_first)
+    B.lif_set_tuning(gpu.handle, B.TUNE_EARLY_FETCH, early)
+    X = W.make_inputs(cfg, device=DEV)
+    y = torch.empty(S, cfg.d_model, dtype=torch.float32, device=DEV)
+    idx = torch.empty(cfg.d_ff, dtype=torch.int32, device=DEV)
+    n = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sc, sf = (torch.cuda.Stream(), torch.cuda.Stream()) if two_streams else (None, None)
+    torch.cuda.synchronize()
+    n_load = n_evict = 0
+    for t in range(cfg.steps):
+        if t % 3 == 1:
+            B.lif_predict(gpu.handle, X[(t + 4) % cfg.steps], None, idx, n, sc)
+        B.lif_decode_step(gpu.handle, X[t], y, sc, sf)
+        lists = P.check_decode_step(gpu, ora, X[t].cpu().numpy(), y)
+        P.compare_cache_rows(gpu, ora)
+        n_load += len(lists["load_ids"])
+        n_evict += len(lists["evict_ids"])
+    assert n_load > 148 and n_evict > 0          # more rows than CTAs in some step, and row reuse
+    gpu.close()
